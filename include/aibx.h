@@ -1,0 +1,210 @@
+/*
+ * aibx.h - C ABI of libaibx: the data-parallel hot path behind KV-cache reuse in a
+ * prefix-aware LLM gateway with a distributed KV cache (AIBrix, arXiv 2504.03648).
+ *
+ * The paper describes the system in prose only (Section 3.2.2, routing policies, and
+ * Section 3.2.5, distributed KV cache pool); it prints no algorithm, hash function, block
+ * size or formula.  Each call below cites the passage whose operation it implements and
+ * states the concrete reading this library fixes.
+ *
+ * Conventions
+ *   - Every pointer named d_* is DEVICE memory owned by the caller, naturally aligned for its
+ *     element type.  KV pool and transfer buffer must be 16-byte aligned.  Pointers named
+ *     h_* / plain out-parameters are HOST memory.  No call keeps a caller pointer after it
+ *     returns; the only memory the library owns is the index behind aibx_index_t and one
+ *     small per-device status record.
+ *   - Every call that takes a stream only ENQUEUES work on that stream and returns without
+ *     synchronising, except where noted ("syncs").  `stream` is a cudaStream_t passed as
+ *     void* so that this header needs no CUDA include (0 = the legacy default stream).
+ *   - Return value: an aibx status (0 = AIBX_OK, negative = error) for errors the host can
+ *     see (null pointer, negative size, bad layout).  Errors only the device can see (a block
+ *     id out of range, a full table) are accumulated in the per-device status record and read
+ *     with aibx_status_fetch.  Nothing aborts, throws or traps.
+ *   - All arithmetic is integer; results are defined bit-exactly.
+ */
+#ifndef AIBX_H_
+#define AIBX_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AIBX_OK               0
+#define AIBX_ERR_INVALID     (-1)  /* null pointer, negative count, bad parameter          */
+#define AIBX_ERR_RANGE       (-2)  /* a block id >= num_blocks (item skipped)               */
+#define AIBX_ERR_FULL        (-3)  /* index could not place a key within `capacity` probes  */
+#define AIBX_ERR_CUDA        (-4)  /* a CUDA runtime call failed                            */
+#define AIBX_ERR_UNSUPPORTED (-5)  /* shape outside what the kernels handle                 */
+#define AIBX_ERR_NOMEM       (-6)  /* device allocation failed                              */
+#define AIBX_ERR_TIMEOUT     (-7)  /* a bounded in-kernel wait gave up                      */
+
+#define AIBX_NO_BLOCK 0xFFFFFFFFu   /* "no block id": skipped silently by gather/scatter    */
+#define AIBX_NO_POD   (-1)
+#define AIBX_MAX_PODS 64
+
+typedef struct aibx_index aibx_index_t;   /* opaque; host handle of a device-resident index */
+
+/* ---------------------------------------------------------------------------------------
+ * Prefix keys (Section 3.2.2: the gateway analyses the token pattern of each request to find
+ * reusable prefix cache).  Reading fixed here: request r with tokens t[0..len_r) has
+ * n_r = floor(len_r / block_tokens) keys; key i = XXH64(message, seed) where message is the
+ * 4*block_tokens bytes of t[i*B .. (i+1)*B) written as little-endian int32 and seed is key
+ * i-1 (root_seed for i = 0).  A trailing partial block has no key.
+ *
+ *   d_tokens   [tok_off[R]]      int32 token ids of all requests, concatenated
+ *   d_tok_off  [R+1]             int64 start of each request in d_tokens (tok_off[0] = 0)
+ *   d_blk_off  [R+1]             int64 prefix sum of n_r (blk_off[r+1]-blk_off[r] = n_r)
+ *   d_hashes   [blk_off[R]]      out: uint64 keys, request r at [blk_off[r], blk_off[r+1])
+ *   block_tokens                 positive multiple of 4, at most 1024
+ * Errors: INVALID for null pointers (when R > 0), R < 0 or a bad block_tokens.  R = 0 is a
+ * no-op.  The offsets are trusted (they are the caller's own prefix sums).
+ */
+int32_t aibx_hash_blocks(const int32_t* d_tokens, const int64_t* d_tok_off,
+                         const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
+                         uint64_t root_seed, uint64_t* d_hashes, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Prefix/KV-locality metadata (Sections 3.2.2 and 3.2.5: "prefix cache awareness" and the
+ * cache's metadata updates).  Reading fixed here: a map  key -> (pod_mask != 0, block_id),
+ * where bit p of pod_mask says pod p holds the block and block_id names its slot in the KV
+ * pool.  Keys 0 and ~0 are reserved: inserting them is a no-op, looking them up misses.
+ *
+ * create:  allocates capacity_slots (power of two, >= 8) slots of 32 bytes on the current
+ *          device; num_pods in 1..64.  Syncs.  NOMEM if the allocation fails.
+ * destroy: frees it (syncs the device).     clear: empties it (async on stream).
+ */
+int32_t aibx_index_create(aibx_index_t** out, uint64_t capacity_slots, int32_t num_pods);
+int32_t aibx_index_destroy(aibx_index_t* index);
+int32_t aibx_index_clear(aibx_index_t* index, void* stream);
+
+/* insert: for every i < n (order-free): skip if key reserved or (mask & podmask(P)) == 0;
+ *         absent key -> create (mask & podmask, id); present -> mask |= ..., id = min(id, new).
+ *         AIBX_NO_BLOCK as id means "no id supplied" (identity of min).
+ *         Device status FULL if a key finds no free slot within `capacity` probes; the index
+ *         content is then unspecified until aibx_index_clear.  Slots freed by evict are not
+ *         reused until clear.
+ * evict:  batch-atomic.  First mask &= ~masks[i] for all present keys; then
+ *         freed[i] = id if key i was present and its mask is now 0, else AIBX_NO_BLOCK
+ *         (duplicates of a key all report the same value); then entries with mask 0 vanish.
+ *         d_freed_block_ids may be null.
+ * lookup: d_masks[i], d_block_ids[i] = entry of key i, or (0, AIBX_NO_BLOCK).  Either output
+ *         may be null.
+ * stats:  live entries and capacity.  Syncs the stream.
+ */
+int32_t aibx_index_insert(aibx_index_t* index, const uint64_t* d_keys,
+                          const uint64_t* d_pod_masks, const uint32_t* d_block_ids,
+                          int64_t n, void* stream);
+int32_t aibx_index_evict(aibx_index_t* index, const uint64_t* d_keys,
+                         const uint64_t* d_pod_masks, uint32_t* d_freed_block_ids,
+                         int64_t n, void* stream);
+int32_t aibx_index_lookup(const aibx_index_t* index, const uint64_t* d_keys,
+                          uint64_t* d_masks, uint32_t* d_block_ids, int64_t n, void* stream);
+int32_t aibx_index_stats(const aibx_index_t* index, uint64_t* live, uint64_t* capacity,
+                         void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Longest cached prefix (Section 3.2.2, policy prefix-cache-aware: instances "with reusable
+ * prefix cache").  For request r and pod p:
+ *   match_len[r][p] = max k <= n_r such that every key i < k is in the index with bit p set;
+ *   any_len[r]      = max k <= n_r such that every key i < k is in the index at all;
+ *   block_ids[j]    = id of key j for blk_off[r] <= j < blk_off[r] + any_len[r],
+ *                     AIBX_NO_BLOCK for the rest of the request.
+ * Lengths are in blocks.  A prefix is contiguous from block 0: residency after a hole does
+ * not count.
+ *   d_match_len [R * num_pods] row-major uint32;  d_any_len [R] nullable;
+ *   d_block_ids [blk_off[R]] nullable.
+ */
+int32_t aibx_match_prefix(const aibx_index_t* index, const uint64_t* d_hashes,
+                          const int64_t* d_blk_off, int32_t R, uint32_t* d_match_len,
+                          uint32_t* d_any_len, uint32_t* d_block_ids, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Prefix-and-load route score (Section 3.2.2: prefix-cache-aware prefers instances whose
+ * cache hit exceeds a threshold; least-request prefers the lowest number of admitted
+ * requests).  Integer reading fixed here, with hit = match_len[r][p], n_r from blk_off:
+ *   eff   = hit  if hit > 0 and 100*hit >= threshold_pct*n_r, else 0
+ *   score = w_prefix*eff - w_load*load[p]                      (int64)
+ *   best_pod[r] = argmax of score over pods with their ready_mask bit set, ties to the lowest
+ *   pod; AIBX_NO_POD and INT64_MIN if none is ready.  All requests see the same load snapshot.
+ *   d_scores [R * num_pods] nullable (pods that are not ready still get their score there).
+ * params == NULL means {4, 1, 50}.
+ */
+typedef struct {
+  int32_t w_prefix;
+  int32_t w_load;
+  int32_t threshold_pct;
+} aibx_route_params_t;
+
+int32_t aibx_route_score(const uint32_t* d_match_len, const int64_t* d_blk_off, int32_t R,
+                         int32_t num_pods, const int32_t* d_pod_load, uint64_t ready_mask,
+                         const aibx_route_params_t* params, int32_t* d_best_pod,
+                         int64_t* d_best_score, int64_t* d_scores, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Set of matched blocks (supporting call between match and gather: Section 3.2.5 speaks of
+ * reducing redundant transfers, so a block shared by several requests moves once).
+ *   d_unique_ids [n] = the distinct values of d_block_ids[0..n) that are < num_blocks, in
+ *   ascending order, padded with AIBX_NO_BLOCK;  *d_count (uint32) = how many.
+ *   Values >= num_blocks other than AIBX_NO_BLOCK are dropped and raise device status RANGE.
+ *   d_scratch: caller-owned device scratch of aibx_collect_scratch_bytes(num_blocks) bytes,
+ *   4-byte aligned; contents on entry are irrelevant, contents on exit unspecified.
+ */
+uint64_t aibx_collect_scratch_bytes(uint32_t num_blocks);
+int32_t aibx_collect_blocks(const uint32_t* d_block_ids, int64_t n, uint32_t num_blocks,
+                            void* d_scratch, uint32_t* d_unique_ids, uint32_t* d_count,
+                            void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * Paged-KV data movement (Section 3.2.5: put/get between the engine's paged KV pool and the
+ * cache, with exchange through a contiguous buffer when cache and engine are colocated).
+ *   tile        = 2 (K,V) * num_kv_heads * block_tokens * head_dim * elem_bytes   bytes
+ *   block_bytes = num_layers * tile
+ *   pool offset of (block b, layer l) = (b*num_layers + l)*tile      layout 0, block-major
+ *                                     = (l*num_blocks + b)*tile      layout 1, layer-major
+ *   buffer offset of (item i, layer l) = (i*num_layers + l)*tile     always block-major
+ * gather:  buffer item i <- pool block ids[i]   (ids may repeat)
+ * scatter: pool block ids[i] <- buffer item i   (ids must be distinct; pool != buffer)
+ * Bytes move verbatim.  An id equal to AIBX_NO_BLOCK is skipped silently; any other id
+ * >= num_blocks is skipped and raises device status RANGE (detail counts such items).
+ * tile must be a multiple of 16 bytes (UNSUPPORTED otherwise); pool and buffer 16-byte
+ * aligned (INVALID otherwise).  n = 0 is a no-op.
+ */
+typedef struct {
+  int32_t layout;        /* 0 block-major, 1 layer-major */
+  int32_t num_layers;
+  int32_t num_kv_heads;
+  int32_t block_tokens;
+  int32_t head_dim;
+  int32_t elem_bytes;    /* 1 (fp8) or 2 (bf16/fp16) or 4 */
+  uint32_t num_blocks;
+} aibx_kv_layout_t;
+
+int32_t aibx_kv_gather(const void* d_pool, const aibx_kv_layout_t* layout,
+                       const uint32_t* d_block_ids, int64_t n, void* d_buf, void* stream);
+int32_t aibx_kv_scatter(void* d_pool, const aibx_kv_layout_t* layout,
+                        const uint32_t* d_block_ids, int64_t n, const void* d_buf,
+                        void* stream);
+
+/* Launch shape of gather/scatter, process-wide; for measurement sweeps.  mode 0 = bulk-async
+ * (TMA) ring through shared memory, 1 = 16-byte load/store loop.  chunk_bytes (multiple of 16,
+ * 1 KiB..64 KiB) and stages (2..16) size the ring (chunk*stages <= 200 KiB); ctas_per_sm 1..8.
+ * Any argument <= 0 keeps its current value.  INVALID on an out-of-range value.
+ */
+int32_t aibx_kv_set_tuning(int32_t mode, int32_t chunk_bytes, int32_t stages,
+                           int32_t ctas_per_sm);
+
+/* ---------------------------------------------------------------------------------------
+ * Device status of the current device: the most severe (most negative) code recorded by any
+ * kernel since the last fetch, and how many items raised one.  Syncs `stream`, then resets
+ * the record.  One record per device, shared by all streams.
+ */
+int32_t aibx_status_fetch(void* stream, int32_t* status, int64_t* detail);
+
+const char* aibx_strerror(int32_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AIBX_H_ */

@@ -1,0 +1,88 @@
+"""Pins for paged-KV gather/scatter (CPU only): library index_select, direct indexing,
+round trips, untouched bytes."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+NO_BLOCK = 0xFFFFFFFF
+
+
+def _pool(rng, layout, L, nb, tile):
+    shape = (nb, L, tile) if layout == 0 else (L, nb, tile)
+    return rng.integers(0, 256, shape, dtype=np.uint8)
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_gather_is_index_select(layout):
+    rng = np.random.default_rng(layout)
+    L, H, Bt, D, E, nb = 3, 2, 4, 8, 2, 17
+    tile = 2 * H * Bt * D * E
+    pool = _pool(rng, layout, L, nb, tile)
+    ids = rng.integers(0, nb, 11).astype(np.uint32)          # repeats allowed
+    lay = oracle.kv_layout(layout, L, H, Bt, D, E, nb)
+    buf = np.zeros(11 * L * tile, dtype=np.uint8)
+    rc, bad = oracle.kv_gather(pool.reshape(-1), lay, ids, buf)
+    assert rc == oracle.OK and bad == 0
+    tp = torch.from_numpy(pool)
+    ti = torch.from_numpy(ids.astype(np.int64))
+    if layout == 0:
+        want = torch.index_select(tp, 0, ti)
+    else:
+        want = tp[:, ti].transpose(0, 1).contiguous()
+    assert np.array_equal(buf, want.numpy().reshape(-1))
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_scatter_direct_indexing_and_round_trips(layout):
+    rng = np.random.default_rng(10 + layout)
+    L, H, Bt, D, E, nb = 4, 1, 2, 4, 1, 23
+    tile = 2 * H * Bt * D * E
+    pool = _pool(rng, layout, L, nb, tile)
+    lay = oracle.kv_layout(layout, L, H, Bt, D, E, nb)
+    ids = rng.permutation(nb)[:9].astype(np.uint32)
+    buf = rng.integers(0, 256, 9 * L * tile, dtype=np.uint8)
+    before = pool.copy()
+    flat = pool.reshape(-1)
+    rc, bad = oracle.kv_scatter(flat, lay, ids, buf)
+    assert rc == oracle.OK
+    b3 = buf.reshape(9, L, tile)
+    touched = np.zeros(nb, dtype=bool)
+    for i, b in enumerate(ids):
+        got = pool[b] if layout == 0 else pool[:, b]
+        assert np.array_equal(got, b3[i])
+        touched[b] = True
+    rest = ~touched
+    if layout == 0:
+        assert np.array_equal(pool[rest], before[rest])
+    else:
+        assert np.array_equal(pool[:, rest], before[:, rest])
+    # gather after scatter returns the buffer; scatter after gather leaves the pool alone
+    back = np.zeros_like(buf)
+    oracle.kv_gather(flat, lay, ids, back)
+    assert np.array_equal(back, buf)
+    snap = pool.copy()
+    oracle.kv_scatter(flat, lay, ids, back)
+    assert np.array_equal(pool, snap)
+
+
+def test_skips_and_range_errors():
+    L, H, Bt, D, E, nb = 2, 1, 1, 8, 1, 5
+    tile = 2 * H * Bt * D * E
+    pool = np.arange(nb * L * tile, dtype=np.uint8)
+    lay = oracle.kv_layout(0, L, H, Bt, D, E, nb)
+    ids = np.array([1, NO_BLOCK, 7, 4], dtype=np.uint32)
+    buf = np.full(4 * L * tile, 0xEE, dtype=np.uint8)
+    rc, bad = oracle.kv_gather(pool, lay, ids, buf)
+    assert rc == oracle.ERR_RANGE and bad == 1
+    bb = buf.reshape(4, L * tile)
+    pp = pool.reshape(nb, L * tile)
+    assert np.array_equal(bb[0], pp[1]) and np.array_equal(bb[3], pp[4])
+    assert (bb[1] == 0xEE).all() and (bb[2] == 0xEE).all()
+    snap = pool.copy()
+    rc, bad = oracle.kv_scatter(pool, lay, np.array([NO_BLOCK, 9], dtype=np.uint32),
+                                buf[:2 * L * tile].copy())
+    assert rc == oracle.ERR_RANGE and bad == 1 and np.array_equal(pool, snap)
+    rc, bad = oracle.kv_gather(pool, lay, np.zeros(0, dtype=np.uint32), buf)
+    assert rc == oracle.OK
