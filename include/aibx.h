@@ -57,7 +57,7 @@ typedef struct aibx_index aibx_index_t;   /* opaque; host handle of a device-res
  *   d_tok_off  [R+1]             int64 start of each request in d_tokens (tok_off[0] = 0)
  *   d_blk_off  [R+1]             int64 prefix sum of n_r (blk_off[r+1]-blk_off[r] = n_r)
  *   d_hashes   [blk_off[R]]      out: uint64 keys, request r at [blk_off[r], blk_off[r+1])
- *   block_tokens                 positive multiple of 4, at most 1024
+ *   block_tokens                 positive multiple of 8 (whole 32-byte stripes), at most 1024
  * Errors: INVALID for null pointers (when R > 0), R < 0 or a bad block_tokens.  R = 0 is a
  * no-op.  The offsets are trusted (they are the caller's own prefix sums).
  */
@@ -66,8 +66,8 @@ int32_t aibx_hash_blocks(const int32_t* d_tokens, const int64_t* d_tok_off,
                          uint64_t root_seed, uint64_t* d_hashes, void* stream);
 
 /* ---------------------------------------------------------------------------------------
- * Prefix/KV-locality metadata (Sections 3.2.2 and 3.2.5: "prefix cache awareness" and the
- * cache's metadata updates).  Reading fixed here: a map  key -> (pod_mask != 0, block_id),
+ * Prefix/KV-locality metadata (Sections 3.2.2 and 3.2.5: the gateway knows which instance
+ * caches which prefix, and the cache publishes metadata updates).  Reading fixed here: a map  key -> (pod_mask != 0, block_id),
  * where bit p of pod_mask says pod p holds the block and block_id names its slot in the KV
  * pool.  Keys 0 and ~0 are reserved: inserting them is a no-op, looking them up misses.
  *
@@ -105,8 +105,8 @@ int32_t aibx_index_stats(const aibx_index_t* index, uint64_t* live, uint64_t* ca
                          void* stream);
 
 /* ---------------------------------------------------------------------------------------
- * Longest cached prefix (Section 3.2.2, policy prefix-cache-aware: instances "with reusable
- * prefix cache").  For request r and pod p:
+ * Longest cached prefix (Section 3.2.2, policy prefix-cache-aware: how much of a request's
+ * prefix each instance can reuse).  For request r and pod p:
  *   match_len[r][p] = max k <= n_r such that every key i < k is in the index with bit p set;
  *   any_len[r]      = max k <= n_r such that every key i < k is in the index at all;
  *   block_ids[j]    = id of key j for blk_off[r] <= j < blk_off[r] + any_len[r],

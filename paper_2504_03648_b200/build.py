@@ -1,0 +1,51 @@
+"""Builds the CUDA libraries in-tree with nvcc for sm_100a.
+
+``libaibx.so`` is the product (C ABI of include/aibx.h); ``libaibx_synth.so`` is the device
+twin of the synthetic input generator used by tests and benchmarks.
+"""
+from __future__ import annotations
+
+import os
+import subprocess
+
+PKG = os.path.dirname(os.path.abspath(__file__))
+ROOT = os.path.dirname(PKG)
+CSRC = os.path.join(PKG, "csrc")
+LIB = os.path.join(PKG, "libaibx.so")
+SYNTH_LIB = os.path.join(PKG, "libaibx_synth.so")
+
+NVCC_FLAGS = [
+    "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+    "-shared", "-Xcompiler", "-fPIC",
+]
+
+
+def _stale(target: str, deps) -> bool:
+    if not os.path.exists(target):
+        return True
+    t = os.path.getmtime(target)
+    return any(os.path.getmtime(d) > t for d in deps)
+
+
+def _nvcc(src: str, out: str, verbose: bool):
+    cmd = ["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + [
+        "-I", os.path.join(ROOT, "include"), "-I", CSRC, src, "-o", out + ".tmp"]
+    subprocess.check_call(cmd)
+    os.replace(out + ".tmp", out)
+
+
+def build(force: bool = False, verbose: bool = False) -> None:
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
+    deps.append(os.path.join(ROOT, "include", "aibx.h"))
+    if force or _stale(LIB, deps):
+        _nvcc(os.path.join(CSRC, "libaibx.cu"), LIB, verbose)
+    if force or _stale(SYNTH_LIB, [os.path.join(CSRC, "synth_fill.cu")]):
+        _nvcc(os.path.join(CSRC, "synth_fill.cu"), SYNTH_LIB, verbose)
+
+
+if __name__ == "__main__":
+    import sys
+
+    build(force="--force" in sys.argv, verbose="-v" in sys.argv)
+    print(LIB)
+    print(SYNTH_LIB)

@@ -1,0 +1,54 @@
+// Shared device/host helpers of libaibx: status record, launch checks, small PTX wrappers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "aibx.h"
+
+namespace aibx {
+
+// One status record per device (and per loaded copy of the library).  Kernels never trap:
+// they record the most severe code seen and how many items raised one.
+struct StatusRecord {
+  int code;
+  int pad;
+  unsigned long long detail;
+};
+
+__device__ StatusRecord g_status;
+
+__device__ __forceinline__ void raise_status(int code) {
+  atomicMin(&g_status.code, code);
+  atomicAdd(&g_status.detail, 1ULL);
+}
+
+constexpr uint64_t kKeyEmpty = 0ULL;
+constexpr uint64_t kKeyTomb = ~0ULL;
+
+__host__ __device__ __forceinline__ bool key_reserved(uint64_t k) {
+  return k == kKeyEmpty || k == kKeyTomb;
+}
+
+__host__ __device__ __forceinline__ uint64_t pod_all(int P) {
+  return P >= 64 ? ~0ULL : ((1ULL << P) - 1ULL);
+}
+
+inline int32_t launch_status() {
+  return cudaPeekAtLastError() == cudaSuccess ? AIBX_OK : AIBX_ERR_CUDA;
+}
+
+inline int sm_count() {
+  static int cached[64] = {0};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+}  // namespace aibx

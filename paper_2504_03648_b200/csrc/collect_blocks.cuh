@@ -1,0 +1,75 @@
+// Set of matched blocks: ascending distinct valid ids of a list, padded with AIBX_NO_BLOCK.
+// A bitmap over block ids in caller-provided global scratch is marked by one thread per id,
+// then one CTA turns it into the ascending list with a running popcount scan.
+#pragma once
+
+#include "aibx_common.cuh"
+
+namespace aibx {
+
+constexpr int kCollectThreads = 1024;
+
+__global__ void collect_mark_kernel(const uint32_t* __restrict__ ids, int64_t n,
+                                    uint32_t num_blocks, unsigned int* __restrict__ bitmap) {
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint32_t id = ids[i];
+  if (id < num_blocks) {
+    atomicOr(&bitmap[id >> 5], 1u << (id & 31u));
+  } else if (id != AIBX_NO_BLOCK) {
+    raise_status(AIBX_ERR_RANGE);
+  }
+}
+
+__global__ void __launch_bounds__(kCollectThreads)
+collect_compact_kernel(const unsigned int* __restrict__ bitmap, uint32_t num_blocks, int64_t n,
+                       uint32_t* __restrict__ out, uint32_t* __restrict__ count) {
+  __shared__ unsigned int s_warp[32];
+  __shared__ unsigned int s_base;
+  const int tid = threadIdx.x;
+  const int lane = tid & 31;
+  const int warp = tid >> 5;
+  const uint32_t n_words = (num_blocks + 31u) / 32u;
+  if (tid == 0) s_base = 0;
+  __syncthreads();
+  for (uint32_t w0 = 0; w0 < n_words; w0 += kCollectThreads) {
+    const uint32_t w = w0 + tid;
+    unsigned int bits = (w < n_words) ? bitmap[w] : 0u;
+    const unsigned int c = __popc(bits);
+    // inclusive scan of c inside the warp, then across the 32 warps
+    unsigned int inc = c;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const unsigned int o = __shfl_up_sync(0xffffffffu, inc, d);
+      if (lane >= d) inc += o;
+    }
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+      unsigned int t = s_warp[lane];
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const unsigned int o = __shfl_up_sync(0xffffffffu, t, d);
+        if (lane >= d) t += o;
+      }
+      s_warp[lane] = t;   // inclusive over warps
+    }
+    __syncthreads();
+    const unsigned int before = s_base + (warp ? s_warp[warp - 1] : 0u) + (inc - c);
+    unsigned int pos = before;
+    while (bits) {
+      const int b = __ffs(bits) - 1;
+      bits &= bits - 1;
+      if ((int64_t)pos < n) out[pos] = w * 32u + (uint32_t)b;
+      ++pos;
+    }
+    __syncthreads();
+    if (tid == 0) s_base += s_warp[31];
+    __syncthreads();
+  }
+  const unsigned int total = s_base;
+  for (int64_t i = (int64_t)total + tid; i < n; i += kCollectThreads) out[i] = AIBX_NO_BLOCK;
+  if (tid == 0) *count = total;
+}
+
+}  // namespace aibx

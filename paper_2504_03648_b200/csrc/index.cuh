@@ -1,0 +1,263 @@
+// GPU-resident residency index: open addressing with linear probing over 32-byte slots, so
+// that one probe touches exactly one DRAM sector holding key, pod mask and block id.
+//
+//   insert / evict : one thread per item, atomics only (results are order-free by construction)
+//   lookup         : one thread per key
+//   match_prefix   : a warp probes 32 consecutive blocks of a request at once; ballots find the
+//                    first block each pod misses; warps of one request combine through
+//                    shared-memory minima and stop once an earlier total miss is known.
+#pragma once
+
+#include "aibx_common.cuh"
+
+namespace aibx {
+
+struct __align__(32) Slot {
+  unsigned long long key;    // 0 = never used, ~0 = removed (not reused until clear)
+  unsigned long long mask;   // pod residency bits; an entry with mask 0 is dead
+  unsigned int id;           // block id, min over inserts; AIBX_NO_BLOCK = none supplied
+  unsigned int stamp;        // reserved (recency stamp for eviction policies)
+  unsigned long long pad;
+};
+static_assert(sizeof(Slot) == 32, "one slot per 32-byte sector");
+
+struct IndexView {
+  Slot* slots;
+  unsigned long long cap_mask;   // capacity - 1
+  int shift;                     // 64 - log2(capacity)
+  int num_pods;
+  unsigned long long* counters;  // [0] live entries, [1] removed slots
+};
+
+__device__ __forceinline__ unsigned long long home_slot(const IndexView& ix, uint64_t key) {
+  return (key * 0x9E3779B97F4A7C15ULL) >> ix.shift;
+}
+
+__global__ void index_clear_kernel(IndexView ix) {
+  const unsigned long long n = ix.cap_mask + 1;
+  for (unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; i < n;
+       i += (unsigned long long)gridDim.x * blockDim.x) {
+    uint4* p = reinterpret_cast<uint4*>(ix.slots + i);
+    p[0] = make_uint4(0u, 0u, 0u, 0u);                      // key, mask
+    p[1] = make_uint4(AIBX_NO_BLOCK, 0u, 0u, 0u);           // id, stamp, pad
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    ix.counters[0] = 0;
+    ix.counters[1] = 0;
+  }
+}
+
+// Read-only probe (index not modified while the kernel runs): both halves of the slot are
+// requested together so a hit costs one memory round trip.
+__device__ __forceinline__ bool probe_ro(const IndexView& ix, uint64_t key, uint64_t& mask,
+                                         uint32_t& id) {
+  mask = 0;
+  id = AIBX_NO_BLOCK;
+  if (key_reserved(key)) return false;
+  unsigned long long s = home_slot(ix, key);
+  for (unsigned long long n = 0; n <= ix.cap_mask; ++n) {
+    const uint4* p = reinterpret_cast<const uint4*>(ix.slots + s);
+    const uint4 a = __ldg(p);
+    const uint4 b = __ldg(p + 1);
+    const uint64_t k = (uint64_t)a.x | ((uint64_t)a.y << 32);
+    if (k == key) {
+      const uint64_t m = (uint64_t)a.z | ((uint64_t)a.w << 32);
+      if (m == 0) return false;
+      mask = m;
+      id = b.x;
+      return true;
+    }
+    if (k == kKeyEmpty) return false;
+    s = (s + 1) & ix.cap_mask;
+  }
+  return false;
+}
+
+// Probe while other threads may be claiming slots: returns the slot index or ~0.
+__device__ __forceinline__ unsigned long long find_slot_rw(const IndexView& ix, uint64_t key) {
+  unsigned long long s = home_slot(ix, key);
+  for (unsigned long long n = 0; n <= ix.cap_mask; ++n) {
+    const unsigned long long k = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].key);
+    if (k == key) return s;
+    if (k == kKeyEmpty) return ~0ULL;
+    s = (s + 1) & ix.cap_mask;
+  }
+  return ~0ULL;
+}
+
+__global__ void index_insert_kernel(IndexView ix, const uint64_t* __restrict__ keys,
+                                    const uint64_t* __restrict__ masks,
+                                    const uint32_t* __restrict__ ids, int64_t n) {
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint64_t key = keys[i];
+  const uint64_t m = masks[i] & pod_all(ix.num_pods);
+  if (key_reserved(key) || m == 0) return;
+  unsigned long long s = home_slot(ix, key);
+  bool placed = false;
+  for (unsigned long long probes = 0; probes <= ix.cap_mask; ++probes) {
+    unsigned long long k = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].key);
+    if (k == kKeyEmpty) {
+      k = atomicCAS(&ix.slots[s].key, kKeyEmpty, (unsigned long long)key);
+      if (k == kKeyEmpty) {
+        atomicAdd(&ix.counters[0], 1ULL);
+        placed = true;
+        break;
+      }
+    }
+    if (k == key) {
+      placed = true;
+      break;
+    }
+    s = (s + 1) & ix.cap_mask;
+  }
+  if (!placed) {
+    raise_status(AIBX_ERR_FULL);
+    return;
+  }
+  atomicOr(&ix.slots[s].mask, (unsigned long long)m);
+  atomicMin(&ix.slots[s].id, ids[i]);
+}
+
+// evict, pass 1: clear the named pod bits
+__global__ void index_evict_clear_kernel(IndexView ix, const uint64_t* __restrict__ keys,
+                                         const uint64_t* __restrict__ masks, int64_t n) {
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint64_t key = keys[i];
+  if (key_reserved(key)) return;
+  const unsigned long long s = find_slot_rw(ix, key);
+  if (s == ~0ULL) return;
+  atomicAnd(&ix.slots[s].mask, ~(unsigned long long)masks[i]);
+}
+
+// evict, pass 2: report ids of entries left without a pod (every duplicate sees the same state)
+__global__ void index_evict_report_kernel(IndexView ix, const uint64_t* __restrict__ keys,
+                                          uint32_t* __restrict__ freed, int64_t n) {
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint64_t key = keys[i];
+  uint32_t out = AIBX_NO_BLOCK;
+  if (!key_reserved(key)) {
+    const unsigned long long s = find_slot_rw(ix, key);
+    if (s != ~0ULL) {
+      const unsigned long long m = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].mask);
+      if (m == 0) out = *reinterpret_cast<volatile unsigned int*>(&ix.slots[s].id);
+    }
+  }
+  freed[i] = out;
+}
+
+// evict, pass 3: dead entries leave the table (exactly one thread wins the removal)
+__global__ void index_evict_remove_kernel(IndexView ix, const uint64_t* __restrict__ keys,
+                                          int64_t n) {
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint64_t key = keys[i];
+  if (key_reserved(key)) return;
+  const unsigned long long s = find_slot_rw(ix, key);
+  if (s == ~0ULL) return;
+  const unsigned long long m = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].mask);
+  if (m != 0) return;
+  if (atomicCAS(&ix.slots[s].key, (unsigned long long)key, kKeyTomb) == key) {
+    atomicAdd(&ix.counters[0], ~0ULL);   // live -= 1
+    atomicAdd(&ix.counters[1], 1ULL);
+  }
+}
+
+__global__ void index_lookup_kernel(IndexView ix, const uint64_t* __restrict__ keys,
+                                    uint64_t* __restrict__ out_masks,
+                                    uint32_t* __restrict__ out_ids, int64_t n) {
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  uint64_t m;
+  uint32_t id;
+  probe_ro(ix, keys[i], m, id);
+  if (out_masks) out_masks[i] = m;
+  if (out_ids) out_ids[i] = id;
+}
+
+// ------------------------------------------------------------------------------------------
+// Longest cached prefix.  A group of `wpr` warps serves one request; a CTA holds kMatchWarps
+// warps, i.e. kMatchWarps / wpr requests.
+
+constexpr int kMatchWarpsMin = 4;
+
+struct MatchShared {
+  unsigned int first_miss[AIBX_MAX_PODS];   // per pod: first block whose mask lacks the pod
+  unsigned int first_none;                  // first block with no entry at all
+};
+
+__global__ void match_prefix_kernel(IndexView ix, const uint64_t* __restrict__ hashes,
+                                    const int64_t* __restrict__ blk_off, int R, int wpr,
+                                    uint32_t* __restrict__ match_len,
+                                    uint32_t* __restrict__ any_len,
+                                    uint32_t* __restrict__ block_ids) {
+  extern __shared__ MatchShared s_groups[];
+  const int warps_per_cta = blockDim.x >> 5;
+  const int groups_per_cta = warps_per_cta / wpr;
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int group = warp / wpr;
+  const int warp_in_group = warp % wpr;
+  const int tid_in_group = warp_in_group * 32 + lane;
+  const int group_threads = wpr * 32;
+  const int P = ix.num_pods;
+  const int r = blockIdx.x * groups_per_cta + group;
+  const bool active = r < R;
+
+  MatchShared& sh = s_groups[group];
+  int64_t off = 0;
+  unsigned int n_r = 0;
+  if (active) {
+    off = blk_off[r];
+    n_r = (unsigned int)(blk_off[r + 1] - off);
+    for (int p = tid_in_group; p < P; p += group_threads) sh.first_miss[p] = n_r;
+    if (tid_in_group == 0) sh.first_none = n_r;
+  }
+  __syncthreads();
+
+  if (active) {
+    const uint64_t all = pod_all(P);
+    for (unsigned int base = warp_in_group * 32u; base < n_r; base += wpr * 32u) {
+      // blocks past a known total miss cannot change any result
+      unsigned int known = 0;
+      if (lane == 0) known = *reinterpret_cast<volatile unsigned int*>(&sh.first_none);
+      known = __shfl_sync(0xffffffffu, known, 0);
+      if (base > known) break;
+      const unsigned int i = base + lane;
+      const bool valid = i < n_r;
+      uint64_t mask = 0;
+      uint32_t id = AIBX_NO_BLOCK;
+      if (valid) probe_ro(ix, __ldg(hashes + off + i), mask, id);
+      if (valid && block_ids) block_ids[off + i] = id;
+      const unsigned int none = __ballot_sync(0xffffffffu, valid && mask == 0);
+      if (none && lane == 0) atomicMin(&sh.first_none, base + (unsigned int)__ffs(none) - 1u);
+      // pods missing somewhere in this chunk: complement of the AND over valid lanes
+      const uint64_t mv = valid ? mask : all;
+      const unsigned int lo = __reduce_and_sync(0xffffffffu, (unsigned int)mv);
+      const unsigned int hi = __reduce_and_sync(0xffffffffu, (unsigned int)(mv >> 32));
+      uint64_t todo = ~((uint64_t)lo | ((uint64_t)hi << 32)) & all;
+      while (todo) {
+        const int p = __ffsll((long long)todo) - 1;
+        todo &= todo - 1;
+        const unsigned int lacks = __ballot_sync(0xffffffffu, valid && !((mask >> p) & 1ULL));
+        if (lane == 0) atomicMin(&sh.first_miss[p], base + (unsigned int)__ffs(lacks) - 1u);
+      }
+    }
+  }
+  __syncthreads();
+
+  if (active) {
+    const unsigned int a = sh.first_none;
+    for (int p = tid_in_group; p < P; p += group_threads)
+      match_len[(int64_t)r * P + p] = sh.first_miss[p];
+    if (any_len && tid_in_group == 0) any_len[r] = a;
+    if (block_ids) {
+      for (unsigned int i = a + tid_in_group; i < n_r; i += group_threads)
+        block_ids[off + i] = AIBX_NO_BLOCK;
+    }
+  }
+}
+
+}  // namespace aibx

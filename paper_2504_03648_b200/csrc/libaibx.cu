@@ -1,0 +1,275 @@
+// libaibx: C ABI over the kernels (see include/aibx.h for the contract of every call).
+// One translation unit, so the per-device status record is shared by all kernels.
+#include <cuda_runtime.h>
+
+#include <new>
+
+#include "aibx.h"
+#include "aibx_common.cuh"
+#include "collect_blocks.cuh"
+#include "hash_blocks.cuh"
+#include "index.cuh"
+#include "kv_copy.cuh"
+#include "route_score.cuh"
+
+using namespace aibx;
+
+struct aibx_index {
+  IndexView view;
+  uint64_t capacity;
+  int device;
+};
+
+namespace {
+
+inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+
+inline unsigned int blocks_for(int64_t n, int threads) {
+  return (unsigned int)((n + threads - 1) / threads);
+}
+
+// Device address of the status record of the current device.
+StatusRecord* status_ptr() {
+  static StatusRecord* cached[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cached[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_status) != cudaSuccess) return nullptr;
+    cached[dev] = static_cast<StatusRecord*>(p);
+  }
+  return cached[dev];
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t aibx_hash_blocks(const int32_t* d_tokens, const int64_t* d_tok_off,
+                         const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
+                         uint64_t root_seed, uint64_t* d_hashes, void* stream) {
+  if (R < 0 || block_tokens <= 0 || block_tokens % 8 != 0 || block_tokens > 1024)
+    return AIBX_ERR_INVALID;
+  if (R == 0) return AIBX_OK;
+  if (!d_tokens || !d_tok_off || !d_blk_off || !d_hashes) return AIBX_ERR_INVALID;
+  return launch_hash_blocks(d_tokens, d_tok_off, d_blk_off, R, block_tokens, root_seed, d_hashes,
+                            as_stream(stream));
+}
+
+int32_t aibx_index_create(aibx_index_t** out, uint64_t capacity_slots, int32_t num_pods) {
+  if (!out) return AIBX_ERR_INVALID;
+  *out = nullptr;
+  if (num_pods < 1 || num_pods > AIBX_MAX_PODS) return AIBX_ERR_INVALID;
+  if (capacity_slots < 8 || (capacity_slots & (capacity_slots - 1)) != 0) return AIBX_ERR_INVALID;
+  if (capacity_slots > (1ULL << 40)) return AIBX_ERR_INVALID;
+  aibx_index* ix = new (std::nothrow) aibx_index();
+  if (!ix) return AIBX_ERR_NOMEM;
+  int log2cap = 0;
+  while ((1ULL << log2cap) < capacity_slots) ++log2cap;
+  if (cudaGetDevice(&ix->device) != cudaSuccess) {
+    delete ix;
+    return AIBX_ERR_CUDA;
+  }
+  void* slots = nullptr;
+  void* counters = nullptr;
+  if (cudaMalloc(&slots, capacity_slots * sizeof(Slot)) != cudaSuccess ||
+      cudaMalloc(&counters, 2 * sizeof(unsigned long long)) != cudaSuccess) {
+    cudaGetLastError();   // clear the sticky-free allocation error
+    if (slots) cudaFree(slots);
+    delete ix;
+    return AIBX_ERR_NOMEM;
+  }
+  ix->capacity = capacity_slots;
+  ix->view.slots = static_cast<Slot*>(slots);
+  ix->view.cap_mask = capacity_slots - 1;
+  ix->view.shift = 64 - log2cap;
+  ix->view.num_pods = num_pods;
+  ix->view.counters = static_cast<unsigned long long*>(counters);
+  index_clear_kernel<<<sm_count() * 8, 256>>>(ix->view);
+  if (cudaDeviceSynchronize() != cudaSuccess) {
+    cudaFree(slots);
+    cudaFree(counters);
+    delete ix;
+    return AIBX_ERR_CUDA;
+  }
+  *out = ix;
+  return AIBX_OK;
+}
+
+int32_t aibx_index_destroy(aibx_index_t* ix) {
+  if (!ix) return AIBX_ERR_INVALID;
+  cudaDeviceSynchronize();
+  cudaFree(ix->view.slots);
+  cudaFree(ix->view.counters);
+  delete ix;
+  return AIBX_OK;
+}
+
+int32_t aibx_index_clear(aibx_index_t* ix, void* stream) {
+  if (!ix) return AIBX_ERR_INVALID;
+  index_clear_kernel<<<sm_count() * 8, 256, 0, as_stream(stream)>>>(ix->view);
+  return launch_status();
+}
+
+int32_t aibx_index_insert(aibx_index_t* ix, const uint64_t* d_keys, const uint64_t* d_pod_masks,
+                          const uint32_t* d_block_ids, int64_t n, void* stream) {
+  if (!ix || n < 0) return AIBX_ERR_INVALID;
+  if (n == 0) return AIBX_OK;
+  if (!d_keys || !d_pod_masks || !d_block_ids) return AIBX_ERR_INVALID;
+  index_insert_kernel<<<blocks_for(n, 256), 256, 0, as_stream(stream)>>>(
+      ix->view, d_keys, d_pod_masks, d_block_ids, n);
+  return launch_status();
+}
+
+int32_t aibx_index_evict(aibx_index_t* ix, const uint64_t* d_keys, const uint64_t* d_pod_masks,
+                         uint32_t* d_freed_block_ids, int64_t n, void* stream) {
+  if (!ix || n < 0) return AIBX_ERR_INVALID;
+  if (n == 0) return AIBX_OK;
+  if (!d_keys || !d_pod_masks) return AIBX_ERR_INVALID;
+  cudaStream_t st = as_stream(stream);
+  const unsigned int grid = blocks_for(n, 256);
+  index_evict_clear_kernel<<<grid, 256, 0, st>>>(ix->view, d_keys, d_pod_masks, n);
+  if (d_freed_block_ids)
+    index_evict_report_kernel<<<grid, 256, 0, st>>>(ix->view, d_keys, d_freed_block_ids, n);
+  index_evict_remove_kernel<<<grid, 256, 0, st>>>(ix->view, d_keys, n);
+  return launch_status();
+}
+
+int32_t aibx_index_lookup(const aibx_index_t* ix, const uint64_t* d_keys, uint64_t* d_masks,
+                          uint32_t* d_block_ids, int64_t n, void* stream) {
+  if (!ix || n < 0) return AIBX_ERR_INVALID;
+  if (n == 0) return AIBX_OK;
+  if (!d_keys) return AIBX_ERR_INVALID;
+  index_lookup_kernel<<<blocks_for(n, 256), 256, 0, as_stream(stream)>>>(ix->view, d_keys, d_masks,
+                                                                         d_block_ids, n);
+  return launch_status();
+}
+
+int32_t aibx_index_stats(const aibx_index_t* ix, uint64_t* live, uint64_t* capacity,
+                         void* stream) {
+  if (!ix) return AIBX_ERR_INVALID;
+  unsigned long long c[2] = {0, 0};
+  if (cudaMemcpyAsync(c, ix->view.counters, sizeof(c), cudaMemcpyDeviceToHost,
+                      as_stream(stream)) != cudaSuccess ||
+      cudaStreamSynchronize(as_stream(stream)) != cudaSuccess)
+    return AIBX_ERR_CUDA;
+  if (live) *live = c[0];
+  if (capacity) *capacity = ix->capacity;
+  return AIBX_OK;
+}
+
+int32_t aibx_match_prefix(const aibx_index_t* ix, const uint64_t* d_hashes,
+                          const int64_t* d_blk_off, int32_t R, uint32_t* d_match_len,
+                          uint32_t* d_any_len, uint32_t* d_block_ids, void* stream) {
+  if (!ix || R < 0) return AIBX_ERR_INVALID;
+  if (R == 0) return AIBX_OK;
+  if (!d_hashes || !d_blk_off || !d_match_len) return AIBX_ERR_INVALID;
+  // warps per request: aim at ~32 resident warps per SM; few requests get whole CTAs
+  int wpr = 1;
+  const long long target = (long long)sm_count() * 32;
+  while (wpr < 32 && (long long)R * wpr * 2 <= target) wpr *= 2;
+  const int warps_per_cta = wpr > kMatchWarpsMin ? wpr : kMatchWarpsMin;
+  const int groups = warps_per_cta / wpr;
+  const unsigned int grid = (unsigned int)((R + groups - 1) / groups);
+  const size_t smem = (size_t)groups * sizeof(MatchShared);
+  match_prefix_kernel<<<grid, warps_per_cta * 32, smem, as_stream(stream)>>>(
+      ix->view, d_hashes, d_blk_off, R, wpr, d_match_len, d_any_len, d_block_ids);
+  return launch_status();
+}
+
+int32_t aibx_route_score(const uint32_t* d_match_len, const int64_t* d_blk_off, int32_t R,
+                         int32_t num_pods, const int32_t* d_pod_load, uint64_t ready_mask,
+                         const aibx_route_params_t* params, int32_t* d_best_pod,
+                         int64_t* d_best_score, int64_t* d_scores, void* stream) {
+  if (R < 0 || num_pods < 1 || num_pods > AIBX_MAX_PODS) return AIBX_ERR_INVALID;
+  if (R == 0) return AIBX_OK;
+  if (!d_match_len || !d_blk_off || !d_pod_load || !d_best_pod || !d_best_score)
+    return AIBX_ERR_INVALID;
+  aibx_route_params_t prm = {4, 1, 50};
+  if (params) prm = *params;
+  route_score_kernel<<<blocks_for(R, kRouteWarps), kRouteWarps * 32, 0, as_stream(stream)>>>(
+      d_match_len, d_blk_off, R, num_pods, d_pod_load, ready_mask, prm.w_prefix, prm.w_load,
+      prm.threshold_pct, d_best_pod, d_best_score, d_scores);
+  return launch_status();
+}
+
+uint64_t aibx_collect_scratch_bytes(uint32_t num_blocks) {
+  return 4ULL * (((uint64_t)num_blocks + 31ULL) / 32ULL);
+}
+
+int32_t aibx_collect_blocks(const uint32_t* d_block_ids, int64_t n, uint32_t num_blocks,
+                            void* d_scratch, uint32_t* d_unique_ids, uint32_t* d_count,
+                            void* stream) {
+  if (n < 0 || !d_count) return AIBX_ERR_INVALID;
+  if (n > 0 && (!d_block_ids || !d_unique_ids)) return AIBX_ERR_INVALID;
+  if (num_blocks > 0 && !d_scratch) return AIBX_ERR_INVALID;
+  if (reinterpret_cast<uintptr_t>(d_scratch) & 3) return AIBX_ERR_INVALID;
+  cudaStream_t st = as_stream(stream);
+  unsigned int* bitmap = static_cast<unsigned int*>(d_scratch);
+  if (num_blocks > 0 &&
+      cudaMemsetAsync(bitmap, 0, aibx_collect_scratch_bytes(num_blocks), st) != cudaSuccess)
+    return AIBX_ERR_CUDA;
+  if (n > 0)
+    collect_mark_kernel<<<blocks_for(n, 256), 256, 0, st>>>(d_block_ids, n, num_blocks, bitmap);
+  collect_compact_kernel<<<1, kCollectThreads, 0, st>>>(bitmap, num_blocks, n, d_unique_ids,
+                                                        d_count);
+  return launch_status();
+}
+
+int32_t aibx_kv_gather(const void* d_pool, const aibx_kv_layout_t* layout,
+                       const uint32_t* d_block_ids, int64_t n, void* d_buf, void* stream) {
+  return launch_kv_copy(d_pool, layout, d_block_ids, n, d_buf, 0, as_stream(stream));
+}
+
+int32_t aibx_kv_scatter(void* d_pool, const aibx_kv_layout_t* layout,
+                        const uint32_t* d_block_ids, int64_t n, const void* d_buf,
+                        void* stream) {
+  return launch_kv_copy(d_pool, layout, d_block_ids, n, d_buf, 1, as_stream(stream));
+}
+
+int32_t aibx_kv_set_tuning(int32_t mode, int32_t chunk_bytes, int32_t stages,
+                           int32_t ctas_per_sm) {
+  CopyTuning t = copy_tuning();
+  if (mode >= 0) t.mode = mode;
+  if (chunk_bytes > 0) t.chunk_bytes = chunk_bytes;
+  if (stages > 0) t.stages = stages;
+  if (ctas_per_sm > 0) t.ctas_per_sm = ctas_per_sm;
+  if (t.mode != 0 && t.mode != 1) return AIBX_ERR_INVALID;
+  if (t.chunk_bytes % 16 != 0 || t.chunk_bytes < 1024 || t.chunk_bytes > 65536)
+    return AIBX_ERR_INVALID;
+  if (t.stages < 2 || t.stages > kMaxStages) return AIBX_ERR_INVALID;
+  if (t.ctas_per_sm < 1 || t.ctas_per_sm > 8) return AIBX_ERR_INVALID;
+  if ((long long)t.chunk_bytes * t.stages * t.ctas_per_sm > 200 * 1024) return AIBX_ERR_INVALID;
+  copy_tuning() = t;
+  return AIBX_OK;
+}
+
+int32_t aibx_status_fetch(void* stream, int32_t* status, int64_t* detail) {
+  StatusRecord* dev = status_ptr();
+  if (!dev) return AIBX_ERR_CUDA;
+  cudaStream_t st = as_stream(stream);
+  StatusRecord host = {0, 0, 0};
+  if (cudaMemcpyAsync(&host, dev, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaMemsetAsync(dev, 0, sizeof(host), st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return AIBX_ERR_CUDA;
+  if (status) *status = host.code;
+  if (detail) *detail = (int64_t)host.detail;
+  return AIBX_OK;
+}
+
+const char* aibx_strerror(int32_t status) {
+  switch (status) {
+    case AIBX_OK: return "ok";
+    case AIBX_ERR_INVALID: return "invalid argument";
+    case AIBX_ERR_RANGE: return "block id out of range";
+    case AIBX_ERR_FULL: return "index full";
+    case AIBX_ERR_CUDA: return "CUDA runtime error";
+    case AIBX_ERR_UNSUPPORTED: return "unsupported shape";
+    case AIBX_ERR_NOMEM: return "out of device memory";
+    case AIBX_ERR_TIMEOUT: return "bounded device wait gave up";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

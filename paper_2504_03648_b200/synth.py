@@ -1,0 +1,47 @@
+"""Device-side synthetic KV content (ctypes binding of libaibx_synth.so): the GPU twin of
+``workloads.pool_bytes`` for pools too large to generate on the host.  Input generation only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libaibx_synth.so")
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libaibx_synth.so is missing: run `python -m paper_2504_03648_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        L.aibx_synth_fill_linear.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_void_p]
+        L.aibx_synth_fill_linear.restype = C.c_int32
+        L.aibx_synth_fill_pool.argtypes = [C.c_void_p, C.c_uint64, C.c_int32, C.c_uint64, C.c_uint64,
+                                           C.c_uint64, C.c_void_p]
+        L.aibx_synth_fill_pool.restype = C.c_int32
+        _lib = L
+    return _lib
+
+
+def fill_linear(t: torch.Tensor, seed: int, first_byte: int = 0) -> None:
+    """t (any dtype, contiguous, CUDA) <- bytes [first_byte, first_byte + nbytes) of stream `seed`."""
+    assert t.is_cuda and t.is_contiguous()
+    rc = lib().aibx_synth_fill_linear(t.data_ptr(), t.numel() * t.element_size(), seed, first_byte,
+                                      torch.cuda.current_stream().cuda_stream)
+    if rc != 0:
+        raise RuntimeError("aibx_synth_fill_linear -> %d" % rc)
+
+
+def fill_pool(pool: torch.Tensor, kv) -> None:
+    """Fill a whole pool (KVSpec `kv`) with its logical content in its physical layout."""
+    assert pool.is_cuda and pool.is_contiguous()
+    assert pool.numel() * pool.element_size() == kv.pool_bytes
+    rc = lib().aibx_synth_fill_pool(pool.data_ptr(), kv.seed, kv.layout, kv.num_layers,
+                                    kv.num_blocks, kv.tile_bytes,
+                                    torch.cuda.current_stream().cuda_stream)
+    if rc != 0:
+        raise RuntimeError("aibx_synth_fill_pool -> %d" % rc)

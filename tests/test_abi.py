@@ -1,0 +1,51 @@
+"""The C-ABI library builds for sm_100a, loads without a GPU and exports every symbol the
+public header declares (no compute calls here)."""
+import ctypes
+import os
+import re
+
+from paper_2504_03648_b200 import build as aibx_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    aibx_build.build()
+    header = open(os.path.join(ROOT, "include", "aibx.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(aibx_[a-z_0-9]+)\s*\(", header))
+    assert len(declared) >= 17, declared
+    lib = ctypes.CDLL(aibx_build.LIB)
+    for name in sorted(declared):
+        assert hasattr(lib, name), name
+    lib.aibx_strerror.restype = ctypes.c_char_p
+    assert lib.aibx_strerror(-3) == b"index full"
+    assert lib.aibx_kv_set_tuning(0, 32768, 6, 1) == 0
+    assert lib.aibx_kv_set_tuning(0, 100, 6, 1) == -1          # chunk not a multiple of 16
+    assert lib.aibx_kv_set_tuning(0, 65536, 16, 1) == -1       # ring larger than shared memory
+
+
+def test_binding_has_no_fallback(monkeypatch):
+    from paper_2504_03648_b200 import binding
+
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libaibx.so")
+    try:
+        binding.lib()
+    except RuntimeError as e:
+        assert "missing" in str(e)
+    else:
+        raise AssertionError("loading a missing library must fail loudly")
+
+
+def test_product_package_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2504_03648_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.replace("the CPU oracle's tests", ""), f
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith((".py", ".c", ".h")):
+            text = open(os.path.join(ROOT, "oracle", f)).read()
+            assert "paper_2504_03648_b200" not in text and "aibx.h" not in text, f

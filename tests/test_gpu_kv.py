@@ -1,0 +1,262 @@
+"""GPU parity, data-movement half of the path: paged-KV gather and scatter against the CPU
+oracle, byte for byte, through the C ABI - small pools in full, the large configurations at
+full size on sampled blocks."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import (NO_BLOCK, dev, empty, host, kv_layout_gpu, kv_layout_oracle, read_block)
+from paper_2504_03648_b200 import binding as aibx
+from paper_2504_03648_b200 import synth
+from paper_2504_03648_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+GUARD = 4096
+
+
+@pytest.fixture(autouse=True)
+def _default_tuning():
+    aibx.kv_set_tuning(0, 32768, 6, 1)
+    yield
+    aibx.kv_set_tuning(0, 32768, 6, 1)
+
+
+def guarded(n_bytes, fill):
+    """Device byte buffer with guard bands on both sides; returns (whole, payload view)."""
+    whole = torch.full((n_bytes + 2 * GUARD,), fill, dtype=torch.uint8, device="cuda")
+    return whole, whole[GUARD: GUARD + n_bytes]
+
+
+def guards_intact(whole, n_bytes, fill):
+    h = host(whole)
+    return (h[:GUARD] == fill).all() and (h[GUARD + n_bytes:] == fill).all()
+
+
+def check_gather_scatter(kv, ids_g, ids_s, mode_args):
+    aibx.kv_set_tuning(*mode_args)
+    pool_h = W.host_pool(kv)
+    lay_g, lay_o = kv_layout_gpu(kv), kv_layout_oracle(kv)
+    n = len(ids_g)
+    buf_bytes = n * kv.block_bytes
+    # gather
+    pool_w, pool_d = guarded(kv.pool_bytes, 0xA5)
+    pool_d.copy_(torch.from_numpy(pool_h))
+    buf_w, buf_d = guarded(buf_bytes, 0xEE)
+    aibx.kv_gather(pool_d, lay_g, dev(ids_g), n, buf_d)
+    want = np.full(buf_bytes, 0xEE, dtype=np.uint8)
+    rc, bad = oracle.kv_gather(pool_h, lay_o, ids_g, want)
+    assert np.array_equal(host(buf_d), want)
+    st, detail = aibx.status_fetch()
+    assert (st, detail) == ((aibx.ERR_RANGE, bad) if bad else (0, 0))
+    assert np.array_equal(host(pool_d), pool_h)                    # source untouched
+    assert guards_intact(buf_w, buf_bytes, 0xEE) and guards_intact(pool_w, kv.pool_bytes, 0xA5)
+    # scatter the gathered buffer to another id list
+    ns = len(ids_s)
+    aibx.kv_scatter(pool_d, lay_g, dev(ids_s), ns, buf_d)
+    pool_want = pool_h.copy()
+    rc, bad = oracle.kv_scatter(pool_want, lay_o, ids_s, want)
+    assert np.array_equal(host(pool_d), pool_want)
+    st, detail = aibx.status_fetch()
+    assert (st, detail) == ((aibx.ERR_RANGE, bad) if bad else (0, 0))
+    assert guards_intact(buf_w, buf_bytes, 0xEE) and guards_intact(pool_w, kv.pool_bytes, 0xA5)
+
+
+MODES = [(0, 32768, 6, 1), (0, 4096, 3, 2), (0, 1024, 16, 1), (1, 16384, 2, 1), (0, 49152, 4, 1)]
+
+
+@pytest.mark.parametrize("mode_args", MODES)
+def test_cfg1_tiny(mode_args):
+    kv = W.cfg1_kv()
+    ids_g = W.distinct_ids(0, kv.num_blocks, 64)
+    ids_s = W.distinct_ids(100, kv.num_blocks, 64)
+    assert not np.array_equal(ids_g, ids_s)
+    check_gather_scatter(kv, ids_g, ids_s, mode_args)
+
+
+@pytest.mark.parametrize("mode_args", MODES)
+@pytest.mark.parametrize("layout", [0, 1])
+def test_shapes_with_ragged_chunks(layout, mode_args):
+    # tile = 2*3*5*24*1 = 720 bytes (not a multiple of any chunk size), 7 layers
+    kv = W.KVSpec("ragged", 5, layout, 7, 3, 5, 24, 1, 61)
+    rng = np.random.default_rng(layout)
+    ids_g = rng.integers(0, 61, 200).astype(np.uint32)               # repeats allowed
+    ids_g[[3, 50]] = NO_BLOCK
+    ids_g[[7, 120, 199]] = [61, 1 << 31, 0xFFFFFFFE]                 # out of range
+    ids_s = np.concatenate([rng.permutation(61)[:40], [NO_BLOCK, 77]]).astype(np.uint32)
+    check_gather_scatter(kv, ids_g, ids_s, mode_args)
+    # bigger tiles: 2*2*16*64*2 = 8 KiB and 40 KiB blocks
+    kv = W.KVSpec("mid", 6, layout, 5, 2, 16, 64, 2, 300)
+    ids_g = W.distinct_ids(1, 300, 257)
+    ids_s = W.distinct_ids(2, 300, 257)
+    check_gather_scatter(kv, ids_g, ids_s, mode_args)
+
+
+def test_round_trips_and_single_item():
+    kv = W.KVSpec("rt", 8, 1, 3, 2, 16, 128, 2, 40)                 # 16 KiB tiles, layer-major
+    lay = kv_layout_gpu(kv)
+    pool_h = W.host_pool(kv)
+    pool_d = dev(pool_h)
+    ids = W.distinct_ids(3, 40, 17)
+    buf = empty(17 * kv.block_bytes, torch.uint8)
+    aibx.kv_gather(pool_d, lay, dev(ids), 17, buf)
+    snapshot = host(buf).copy()
+    aibx.kv_scatter(pool_d, lay, dev(ids), 17, buf)                 # scatter after gather: identity
+    assert np.array_equal(host(pool_d), pool_h)
+    buf2 = empty(17 * kv.block_bytes, torch.uint8)
+    aibx.kv_gather(pool_d, lay, dev(ids), 17, buf2)                 # gather after scatter: the buffer
+    assert np.array_equal(host(buf2), snapshot)
+    one = empty(kv.block_bytes, torch.uint8)
+    aibx.kv_gather(pool_d, lay, dev(ids[5:6]), 1, one)
+    assert np.array_equal(host(one), snapshot[5 * kv.block_bytes: 6 * kv.block_bytes])
+    assert aibx.status_fetch() == (0, 0)
+
+
+def test_invalid_arguments():
+    kv = W.cfg1_kv()
+    lay = kv_layout_gpu(kv)
+    pool, buf, ids = empty(kv.pool_bytes, torch.uint8), empty(kv.block_bytes, torch.uint8), dev(np.zeros(1, np.uint32))
+    lib = aibx.lib()
+    import ctypes as C
+    assert lib.aibx_kv_gather(pool.data_ptr(), C.byref(lay), ids.data_ptr(), 0, buf.data_ptr(), None) == 0
+    assert lib.aibx_kv_gather(None, C.byref(lay), ids.data_ptr(), 1, buf.data_ptr(), None) == -1
+    assert lib.aibx_kv_gather(pool.data_ptr(), None, ids.data_ptr(), 1, buf.data_ptr(), None) == -1
+    assert lib.aibx_kv_gather(pool.data_ptr(), C.byref(lay), ids.data_ptr(), -1, buf.data_ptr(), None) == -1
+    assert lib.aibx_kv_gather(pool.data_ptr() + 8, C.byref(lay), ids.data_ptr(), 1, buf.data_ptr(), None) == -1
+    bad = aibx.KVLayout(2, 2, 4, 16, 64, 2, 256)
+    assert lib.aibx_kv_scatter(pool.data_ptr(), C.byref(bad), ids.data_ptr(), 1, buf.data_ptr(), None) == -1
+    odd = aibx.KVLayout(0, 2, 1, 1, 3, 1, 256)                      # 6-byte tiles
+    assert lib.aibx_kv_gather(pool.data_ptr(), C.byref(odd), ids.data_ptr(), 1, buf.data_ptr(), None) == -5
+
+
+# ------------------------------------------------------------------ large configurations
+
+def _fit_blocks(kv, extra_bytes):
+    """Shrink the pool (never the batch) if the device cannot hold the full configuration."""
+    free, _ = torch.cuda.mem_get_info()
+    room = free - extra_bytes - (6 << 30)
+    if kv.pool_bytes <= room:
+        return kv, False
+    nb = int(room // kv.block_bytes)
+    return W.scaled(kv, num_blocks=nb), True
+
+
+def _sample_gather_check(kv, pool_seed_kv, ids, buf_d, sample):
+    """Sampled items of a gathered buffer against the oracle run on a mini pool of those blocks."""
+    lay1 = kv_layout_oracle(kv, layout=0, num_blocks=len(sample))
+    mini = W.logical_blocks(pool_seed_kv, ids[sample])
+    want = np.zeros(len(sample) * kv.block_bytes, dtype=np.uint8)
+    rc, bad = oracle.kv_gather(mini, lay1, np.arange(len(sample), dtype=np.uint32), want)
+    assert rc == oracle.OK
+    want = want.reshape(len(sample), kv.block_bytes)
+    bview = buf_d.view(-1, kv.block_bytes)
+    for j, i in enumerate(sample):
+        assert np.array_equal(host(bview[int(i)]), want[j]), int(i)
+
+
+def test_cfg2_full_size():
+    kv = W.cfg2_kv()
+    n = 1660
+    kv, shrunk = _fit_blocks(kv, n * kv.block_bytes)
+    assert not shrunk, "8 GiB pool must fit"
+    pool = empty(kv.pool_bytes, torch.uint8)
+    synth.fill_pool(pool, kv)
+    ids = np.sort(W.distinct_ids(7, kv.num_blocks, n))            # ascending, like the matched set
+    buf = empty(n * kv.block_bytes, torch.uint8)
+    lay = kv_layout_gpu(kv)
+    aibx.kv_gather(pool, lay, dev(ids), n, buf)
+    assert aibx.status_fetch() == (0, 0)
+    sample = np.concatenate([[0, 1, n - 1], W.Stream(7, 9).randint(0, n, 9)])
+    _sample_gather_check(kv, kv, ids, buf, sample)
+    # whole-buffer property: device-side comparison with the pool rows it names
+    got = buf.view(n, kv.block_bytes)
+    src = pool.view(kv.num_blocks, kv.block_bytes)
+    idx = dev(ids.astype(np.int64))
+    for lo in range(0, n, 256):
+        assert torch.equal(got[lo: lo + 256], src[idx[lo: lo + 256]])
+    # scatter back to the same ids leaves the pool as generated (sampled) ...
+    aibx.kv_scatter(pool, lay, dev(ids), n, buf)
+    for b in ids[sample]:
+        assert np.array_equal(read_block(pool, kv, int(b)), W.logical_blocks(kv, [b]))
+    # ... and scattering fresh content lands where the oracle puts it
+    synth.fill_linear(buf, 1234)
+    aibx.kv_scatter(pool, lay, dev(ids), n, buf)
+    assert aibx.status_fetch() == (0, 0)
+    for i in sample[:6]:
+        mini = np.zeros(kv.block_bytes, dtype=np.uint8)
+        item = W.pool_bytes(1234, int(i) * kv.block_bytes, kv.block_bytes)
+        rc, _ = oracle.kv_scatter(mini, kv_layout_oracle(kv, layout=0, num_blocks=1),
+                                  np.zeros(1, np.uint32), item)
+        assert np.array_equal(read_block(pool, kv, int(ids[int(i)])), mini)
+
+
+def test_cfg4_full_size_layer_major():
+    kv0 = W.cfg4_kv()
+    n = 2048
+    kv, shrunk = _fit_blocks(kv0, n * kv0.block_bytes)
+    pool = empty(kv.pool_bytes, torch.uint8)
+    synth.fill_pool(pool, kv)
+    buf = empty(n * kv.block_bytes, torch.uint8)
+    lay = kv_layout_gpu(kv)
+    touched = {}
+    for it in range(4):                                            # put, get, put, get
+        ids = W.distinct_ids(1000 + it, kv.num_blocks, n)
+        sample = np.concatenate([[0, n - 1], W.Stream(it, 11).randint(0, n, 4)])
+        if it % 2 == 0:
+            aibx.kv_gather(pool, lay, dev(ids), n, buf)
+            lay1 = kv_layout_oracle(kv, layout=0, num_blocks=1)
+            for i in sample:
+                b = int(ids[int(i)])
+                mini = touched.get(b)
+                if mini is None:
+                    mini = W.logical_blocks(kv, [b])
+                want = np.zeros(kv.block_bytes, dtype=np.uint8)
+                oracle.kv_gather(mini, lay1, np.zeros(1, np.uint32), want)
+                assert np.array_equal(host(buf.view(n, kv.block_bytes)[int(i)]), want)
+        else:
+            synth.fill_linear(buf, 5000 + it)
+            aibx.kv_scatter(pool, lay, dev(ids), n, buf)
+            for i in sample:
+                item = W.pool_bytes(5000 + it, int(i) * kv.block_bytes, kv.block_bytes)
+                mini = np.zeros(kv.block_bytes, dtype=np.uint8)
+                oracle.kv_scatter(mini, kv_layout_oracle(kv, layout=0, num_blocks=1),
+                                  np.zeros(1, np.uint32), item)
+                b = int(ids[int(i)])
+                touched[b] = mini
+                assert np.array_equal(read_block(pool, kv, b), mini)
+        assert aibx.status_fetch() == (0, 0)
+    # a block no scatter named still holds its generated content
+    all_scattered = set(W.distinct_ids(1001, kv.num_blocks, n).tolist()) | set(
+        W.distinct_ids(1003, kv.num_blocks, n).tolist())
+    b = next(x for x in range(kv.num_blocks) if x not in all_scattered)
+    assert np.array_equal(read_block(pool, kv, b), W.logical_blocks(kv, [b]))
+    print("cfg4 pool blocks used:", kv.num_blocks, "(shrunk)" if shrunk else "(full)")
+
+
+def test_cfg5_full_size_fp8_mixed():
+    kv0 = W.cfg5_kv()
+    kv, shrunk = _fit_blocks(kv0, 3000 * kv0.block_bytes + 1000 * kv0.block_bytes)
+    per = 4000 if not shrunk else (kv.num_blocks // 32) // 4 * 4
+    n_get, n_put = per * 3 // 4, per // 4
+    pool = empty(kv.pool_bytes, torch.uint8)
+    synth.fill_pool(pool, kv)
+    lay = kv_layout_gpu(kv)
+    get_buf = empty(n_get * kv.block_bytes, torch.uint8)
+    put_buf = empty(n_put * kv.block_bytes, torch.uint8)
+    for r in (0, 13, 31):
+        table = (r * per + W.Stream(4, 100 + r).permutation(per)).astype(np.uint32)
+        ids_get, ids_put = table[:n_get], table[n_get:]
+        aibx.kv_gather(pool, lay, dev(ids_get), n_get, get_buf)
+        synth.fill_linear(put_buf, 900 + r)
+        aibx.kv_scatter(pool, lay, dev(ids_put), n_put, put_buf)
+        assert aibx.status_fetch() == (0, 0)
+        sample = np.array([0, n_get - 1, n_get // 2])
+        _sample_gather_check(kv, kv, ids_get, get_buf, sample)
+        for i in (0, n_put - 1):
+            item = W.pool_bytes(900 + r, i * kv.block_bytes, kv.block_bytes)
+            mini = np.zeros(kv.block_bytes, dtype=np.uint8)
+            oracle.kv_scatter(mini, kv_layout_oracle(kv, layout=0, num_blocks=1),
+                              np.zeros(1, np.uint32), item)
+            assert np.array_equal(read_block(pool, kv, int(ids_put[i])), mini)
+    print("cfg5 pool blocks used:", kv.num_blocks, "(shrunk)" if shrunk else "(full)")

@@ -1,0 +1,326 @@
+"""GPU parity, routing half of the path: prefix keys, index, longest cached prefix, route
+score, matched-block set.  Every comparison is bit-exact against the CPU oracle on the same
+seeded inputs; all calls go through the C ABI."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import (NO_BLOCK, assert_routing_equal, dev, empty, gpu_hash, host, routing_gpu,
+                      routing_oracle)
+from paper_2504_03648_b200 import binding as aibx
+from paper_2504_03648_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+ALL = (1 << 64) - 1
+
+
+# ------------------------------------------------------------------ prefix keys
+
+def test_hash_stored_chains():
+    path = os.path.join(os.path.dirname(__file__), "golden", "hash_chains.txt")
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        head, vals = line.split(":")
+        name, B, root, rule, n = head.split()
+        B, root, n = int(B), int(root), int(n)
+        j = np.arange(n, dtype=np.int64)
+        toks = j.astype(np.int32) if rule == "iota" else ((1000003 * j + 7) % 128256).astype(np.int32)
+        h, _ = gpu_hash(toks, np.array([0, n]), B, root)
+        assert [int(x) for x in h] == [int(v, 16) for v in vals.split()], name
+
+
+@pytest.mark.parametrize("B", [8, 16, 32, 40, 64, 256, 1024])
+def test_hash_ragged_batch(B):
+    rng = np.random.default_rng(B)
+    # lengths around step boundaries (a warp step is 256 tokens), empty and sub-block requests,
+    # odd starts so that requests begin at every alignment inside a 16-byte vector
+    lens = [0, 1, B - 1, B, B + 1, 255, 256, 257, 511, 513, 1027, 2 * B + 3, 4099, 0, 7, 3000]
+    toks = rng.integers(-2**31, 2**31 - 1, sum(lens), dtype=np.int64).astype(np.int32)
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    for root in (0, 0xDEADBEEFCAFEF00D):
+        want, _ = oracle.hash_blocks(toks, off, B, root)
+        got, _ = gpu_hash(toks, off, B, root)
+        assert np.array_equal(got, want)
+
+
+def test_hash_unaligned_token_base():
+    rng = np.random.default_rng(1)
+    toks = rng.integers(0, 32000, 1000).astype(np.int32)
+    big = dev(np.concatenate([np.full(3, -1, np.int32), toks]))
+    for shift in (1, 2, 3):                       # token array starting 4, 8, 12 bytes off
+        view = big[shift:]
+        n = view.numel()
+        sub = host(view)
+        off = np.array([0, 100, 100, 517, n], dtype=np.int64)
+        bo = oracle.block_offsets(off, 16)
+        d_h = empty(int(bo[-1]), torch.uint64)
+        aibx.hash_blocks(view, dev(off), dev(bo), 16, 5, d_h)
+        want, _ = oracle.hash_blocks(sub, off, 16, 5)
+        assert np.array_equal(host(d_h), want)
+
+
+def test_hash_invalid_arguments():
+    t = empty(64, torch.int32)
+    off = dev(np.array([0, 64], dtype=np.int64))
+    bo = dev(np.array([0, 4], dtype=np.int64))
+    h = empty(4, torch.uint64)
+    for B in (0, 12, -16, 2048):
+        with pytest.raises(aibx.AibxError) as e:
+            aibx.hash_blocks(t, off, bo, B, 0, h)
+        assert e.value.code == aibx.ERR_INVALID
+    lib = aibx.lib()
+    assert lib.aibx_hash_blocks(None, None, None, 0, 16, 0, None, None) == 0      # R = 0: no-op
+    assert lib.aibx_hash_blocks(None, off.data_ptr(), bo.data_ptr(), 1, 16, 0, h.data_ptr(), None) == -1
+
+
+# ------------------------------------------------------------------ index
+
+def _rand_ops(rng, universe, P, n_ops, max_batch):
+    ops = []
+    for _ in range(n_ops):
+        kind = "insert" if rng.random() < 0.6 else "evict"
+        n = int(rng.integers(0, max_batch + 1))
+        keys = rng.choice(universe, n).astype(np.uint64)
+        masks = rng.integers(0, 1 << min(P + 1, 63), n).astype(np.uint64)
+        if kind == "evict" and n:
+            masks[rng.random(n) < 0.3] = np.uint64(ALL)
+        ids = rng.integers(0, 1000, n).astype(np.uint32)
+        if n:
+            ids[rng.random(n) < 0.1] = NO_BLOCK
+        ops.append((kind, keys, masks, ids))
+    return ops
+
+
+@pytest.mark.parametrize("capacity,P,n_keys", [(8, 1, 4), (16, 3, 8), (64, 6, 30), (64, 64, 32),
+                                                (4096, 16, 2000)])
+def test_index_random_ops(capacity, P, n_keys):
+    rng = np.random.default_rng(capacity + P)
+    universe = np.concatenate([rng.integers(1, 1 << 63, n_keys).astype(np.uint64),
+                               np.array([0, ALL], dtype=np.uint64)])
+    probe = np.concatenate([universe, rng.integers(1, 1 << 63, 16).astype(np.uint64)])
+    g, o = aibx.Index(capacity, P), oracle.Index(capacity, P)
+    for kind, keys, masks, ids in _rand_ops(rng, universe, P, 25, n_keys):
+        # evicted slots are not reused until clear: keep the table from silting up
+        if kind == "insert":
+            assert o.insert(keys, masks, ids) == oracle.OK
+            g.insert(dev(keys), dev(masks), dev(ids)) if len(keys) else None
+        else:
+            rc, want_freed = o.evict(keys, masks)
+            if len(keys):
+                d_f = empty(len(keys), torch.uint32)
+                g.evict(dev(keys), dev(masks), d_f)
+                assert np.array_equal(host(d_f), want_freed)
+        st = aibx.status_fetch()
+        if st[0] == aibx.ERR_FULL:          # removed slots used up a tiny table: start over
+            g.clear(); o.clear()
+            continue
+        assert st == (0, 0)
+        d_m, d_i = empty(len(probe), torch.uint64), empty(len(probe), torch.uint32)
+        g.lookup(dev(probe), d_m, d_i)
+        wm, wi = o.lookup(probe)
+        assert np.array_equal(host(d_m), wm) and np.array_equal(host(d_i), wi)
+        assert g.stats() == (o.stats()[0], capacity)
+
+
+def test_index_colliding_keys_wrap_around():
+    # brute-force search for keys sharing the last home slot of a 16-slot table is not needed:
+    # with 14 of 16 slots taken every probe sequence wraps
+    rng = np.random.default_rng(0)
+    keys = rng.integers(1, 1 << 63, 14).astype(np.uint64)
+    masks = rng.integers(1, 8, 14).astype(np.uint64)
+    ids = np.arange(14, dtype=np.uint32)
+    g, o = aibx.Index(16, 3), oracle.Index(16, 3)
+    g.insert(dev(keys), dev(masks), dev(ids)); o.insert(keys, masks, ids)
+    probe = np.concatenate([keys, rng.integers(1, 1 << 63, 50).astype(np.uint64)])
+    d_m, d_i = empty(len(probe), torch.uint64), empty(len(probe), torch.uint32)
+    g.lookup(dev(probe), d_m, d_i)
+    wm, wi = o.lookup(probe)
+    assert np.array_equal(host(d_m), wm) and np.array_equal(host(d_i), wi)
+    assert aibx.status_fetch() == (0, 0)
+
+
+def test_index_full_is_reported_not_hung():
+    g, o = aibx.Index(8, 1), oracle.Index(8, 1)
+    keys = np.arange(1, 10, dtype=np.uint64)
+    ones, zeros = np.ones(9, dtype=np.uint64), np.zeros(9, dtype=np.uint32)
+    assert o.insert(keys, ones, zeros) == oracle.ERR_FULL
+    g.insert(dev(keys), dev(ones), dev(zeros))
+    st, detail = aibx.status_fetch()
+    assert st == aibx.ERR_FULL and detail == 1
+    assert aibx.status_fetch() == (0, 0)            # fetch resets the record
+    g.clear()
+    assert g.stats() == (0, 8)
+
+
+def test_index_invalid_arguments():
+    for cap, P in [(12, 4), (4, 4), (16, 0), (16, 65)]:
+        with pytest.raises(aibx.AibxError) as e:
+            aibx.Index(cap, P)
+        assert e.value.code == aibx.ERR_INVALID
+    g = aibx.Index(16, 2)
+    lib = aibx.lib()
+    assert lib.aibx_index_insert(g._h, None, None, None, 0, None) == 0
+    assert lib.aibx_index_insert(g._h, None, None, None, 3, None) == -1
+    assert lib.aibx_index_insert(g._h, None, None, None, -1, None) == -1
+    assert lib.aibx_index_evict(None, None, None, None, 0, None) == -1
+
+
+def test_duplicate_keys_in_one_batch_are_order_free():
+    rng = np.random.default_rng(12)
+    base = rng.integers(1, 1 << 63, 50).astype(np.uint64)
+    keys = np.repeat(base, 40)                      # 40 threads racing on each key
+    masks = rng.integers(0, 1 << 10, len(keys)).astype(np.uint64)
+    ids = rng.integers(0, 1 << 20, len(keys)).astype(np.uint32)
+    perm = rng.permutation(len(keys))
+    g, o = aibx.Index(256, 10), oracle.Index(256, 10)
+    g.insert(dev(keys[perm]), dev(masks[perm]), dev(ids[perm])); o.insert(keys, masks, ids)
+    d_m, d_i = empty(50, torch.uint64), empty(50, torch.uint32)
+    g.lookup(dev(base), d_m, d_i)
+    wm, wi = o.lookup(base)
+    assert np.array_equal(host(d_m), wm) and np.array_equal(host(d_i), wi)
+    assert g.stats()[0] == o.stats()[0]
+    # evict the same key many times in one batch: every duplicate reports the same id
+    ek = np.repeat(base[:5], 7)
+    em = np.full(len(ek), ALL, dtype=np.uint64)
+    d_f = empty(len(ek), torch.uint32)
+    g.evict(dev(ek), dev(em), d_f)
+    rc, wf = o.evict(ek, em)
+    assert np.array_equal(host(d_f), wf) and g.stats()[0] == o.stats()[0]
+
+
+# ------------------------------------------------------------------ whole routing path
+
+def test_routing_cfg1_tiny():
+    w = W.build_routing(W.cfg1_routing())
+    g, o = routing_gpu(w), routing_oracle(w)
+    assert_routing_equal(g, o)
+    assert o["any_len"].max() == 8                  # the shared 128-token prefixes are found
+
+
+def test_match_hand_example():
+    A, B, C, D = 0xA1, 0xB2, 0xC3, 0xD4
+    g = aibx.Index(16, 3)
+    g.insert(dev(np.array([A, B, C], np.uint64)), dev(np.array([3, 1, 6], np.uint64)),
+             dev(np.array([5, 9, 2], np.uint32)))
+    ml, al, ids = empty(3, torch.uint32), empty(1, torch.uint32), empty(4, torch.uint32)
+    g.match_prefix(dev(np.array([A, B, C, D], np.uint64)), dev(np.array([0, 4], np.int64)), ml, al, ids)
+    assert host(ml).tolist() == [2, 1, 0] and host(al).tolist() == [3]
+    assert host(ids).tolist() == [5, 9, 2, NO_BLOCK]
+    bp, bs, sc = empty(1, torch.int32), empty(1, torch.int64), empty(3, torch.int64)
+    aibx.route_score(ml, dev(np.array([0, 4], np.int64)), 3, dev(np.array([10, 3, 0], np.int32)), 7,
+                     (4, 1, 50), bp, bs, sc)
+    assert host(sc).tolist() == [-2, -3, 0] and host(bp).tolist() == [2] and host(bs).tolist() == [0]
+    aibx.route_score(ml, dev(np.array([0, 4], np.int64)), 3, dev(np.array([5, 3, 9], np.int32)), 0,
+                     None, bp, bs, None)
+    assert host(bp).tolist() == [aibx.NO_POD] and host(bs).tolist() == [-(1 << 63)]
+
+
+@pytest.mark.parametrize("R", [1, 3, 40, 200, 700, 1500, 5000])
+def test_match_group_shapes_and_holes(R):
+    """Every warps-per-request choice (R picks it), requests of 0..600 blocks, random holes."""
+    rng = np.random.default_rng(R)
+    P = int(rng.integers(1, 65))
+    lens = rng.integers(0, 600 if R < 100 else 80, R)
+    lens[rng.random(R) < 0.1] = 0
+    bo = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    hashes = rng.integers(1, 1 << 63, int(bo[-1])).astype(np.uint64)
+    allm = ALL if P == 64 else (1 << P) - 1
+    masks = np.full(len(hashes), allm, dtype=np.uint64)
+    # pods drop out at random places; some blocks are absent altogether; a few reserved keys
+    drop = rng.random(len(hashes)) < 0.02
+    masks[drop] &= rng.integers(0, 1 << 62, int(drop.sum())).astype(np.uint64)
+    present = rng.random(len(hashes)) > 0.004
+    hashes[rng.random(len(hashes)) < 0.0005] = 0
+    ids = rng.integers(0, 1 << 20, len(hashes)).astype(np.uint32)
+    cap = 1 << int(np.ceil(np.log2(max(2 * len(hashes), 8))))
+    g, o = aibx.Index(cap, P), oracle.Index(cap, P)
+    sel = present & (masks != 0)
+    o.insert(hashes[sel], masks[sel], ids[sel])
+    if sel.any():
+        g.insert(dev(hashes[sel]), dev(masks[sel]), dev(ids[sel]))
+    nb = max(len(hashes), 1)
+    d_ml, d_al, d_ids = empty(R * P, torch.uint32), empty(R, torch.uint32), empty(nb, torch.uint32)
+    g.match_prefix(dev(hashes) if len(hashes) else empty(1, torch.uint64), dev(bo), d_ml, d_al, d_ids)
+    wml, wal, wids = o.match_prefix(hashes, bo)
+    assert np.array_equal(host(d_ml).reshape(R, P), wml)
+    assert np.array_equal(host(d_al), wal)
+    assert np.array_equal(host(d_ids)[: len(hashes)], wids)
+    # nullable outputs
+    d_ml2 = empty(R * P, torch.uint32)
+    g.match_prefix(dev(hashes) if len(hashes) else empty(1, torch.uint64), dev(bo), d_ml2, None, None)
+    assert np.array_equal(host(d_ml2), host(d_ml))
+    assert aibx.status_fetch() == (0, 0)
+
+
+def test_route_score_parameters_and_ready_masks():
+    rng = np.random.default_rng(77)
+    for P in (1, 7, 32, 33, 64):
+        R = 300
+        n = rng.integers(0, 60, R)
+        bo = np.concatenate([[0], np.cumsum(n)]).astype(np.int64)
+        ml = (rng.random((R, P)) * (n[:, None] + 1)).astype(np.uint32)
+        load = rng.integers(0, 5, P).astype(np.int32)
+        for ready in (ALL, 0, 1 << (P - 1), int(rng.integers(0, 1 << 62)) & ((1 << P) - 1)):
+            for prm in (None, (4, 1, 50), (0, 1, 50), (1, 0, 0), (-3, -2, 120), (2**31 - 1, 2**31 - 1, 100)):
+                d_bp, d_bs, d_sc = empty(R, torch.int32), empty(R, torch.int64), empty(R * P, torch.int64)
+                aibx.route_score(dev(ml.reshape(-1)), dev(bo), P, dev(load), ready, prm, d_bp, d_bs, d_sc)
+                wbp, wbs, wsc = oracle.route_score(ml, bo, load, ready, prm)
+                assert np.array_equal(host(d_bp), wbp), (P, ready, prm)
+                assert np.array_equal(host(d_bs), wbs)
+                assert np.array_equal(host(d_sc).reshape(R, P), wsc)
+
+
+def test_collect_blocks():
+    rng = np.random.default_rng(6)
+    for num_blocks, n in [(1, 5), (31, 100), (32, 100), (33, 1000), (4096, 14000), (100000, 3000),
+                          (1 << 20, 70000)]:
+        ids = rng.integers(0, num_blocks + num_blocks // 8 + 1, n).astype(np.uint32)
+        ids[rng.random(n) < 0.2] = NO_BLOCK
+        scratch = torch.full((aibx.collect_scratch_bytes(num_blocks) // 4 + 1,), 0x5A5A5A5A,
+                             dtype=torch.int32, device="cuda")     # dirty scratch on entry
+        d_un, d_cnt = empty(n, torch.uint32), empty(1, torch.uint32)
+        aibx.collect_blocks(dev(ids), num_blocks, scratch, d_un, d_cnt)
+        rc, wun, wcnt = oracle.collect_blocks(ids, num_blocks)
+        assert int(host(d_cnt)[0]) == wcnt and np.array_equal(host(d_un), wun)
+        st, detail = aibx.status_fetch()
+        n_bad = int(((ids >= num_blocks) & (ids != NO_BLOCK)).sum())
+        assert (st == aibx.ERR_RANGE) == (rc == oracle.ERR_RANGE) and detail == n_bad
+    d_cnt = torch.full((1,), 9, dtype=torch.int32, device="cuda").view(torch.uint32)
+    aibx.collect_blocks(empty(0, torch.uint32), 64, empty(2, torch.uint32), empty(0, torch.uint32), d_cnt)
+    assert int(host(d_cnt)[0]) == 0
+
+
+# ------------------------------------------------------------------ configurations at full size
+
+def test_routing_cfg2_full():
+    w = W.build_routing(W.cfg2_routing())
+    g, o = routing_gpu(w), routing_oracle(w)
+    assert_routing_equal(g, o)
+    assert o["count"] > 1000                        # thousands of distinct matched blocks
+
+
+def test_routing_cfg3_full():
+    w = W.build_routing(W.cfg3_routing())
+    g, o = routing_gpu(w), routing_oracle(w)
+    assert_routing_equal(g, o)
+    for prm in ((4, 1, 0), (4, 1, 25)):
+        P, R = w.spec.num_pods, w.spec.R
+        d_bp, d_bs = empty(R, torch.int32), empty(R, torch.int64)
+        aibx.route_score(dev(o["match_len"].reshape(-1)), dev(o["blk_off"]), P, dev(w.pod_load),
+                         w.ready_mask, prm, d_bp, d_bs, None)
+        wbp, wbs, _ = oracle.route_score(o["match_len"], o["blk_off"], w.pod_load, w.ready_mask, prm)
+        assert np.array_equal(host(d_bp), wbp) and np.array_equal(host(d_bs), wbs)
+
+
+def test_routing_cfg5_full():
+    w = W.build_routing(W.cfg5_routing())
+    g, o = routing_gpu(w), routing_oracle(w)
+    assert_routing_equal(g, o)
+    assert (o["any_len"] == 3000).all()
+    for r in range(w.spec.R):                       # matched ids are the request's block table
+        seg = o["block_ids"][o["blk_off"][r]: o["blk_off"][r] + 3000]
+        assert np.array_equal(seg, w.block_table[r, :3000])
