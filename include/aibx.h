@@ -82,9 +82,9 @@ int32_t aibx_index_clear(aibx_index_t* index, void* stream);
 /* insert: for every i < n (order-free): skip if key reserved or (mask & podmask(P)) == 0;
  *         absent key -> create (mask & podmask, id); present -> mask |= ..., id = min(id, new).
  *         AIBX_NO_BLOCK as id means "no id supplied" (identity of min).
- *         Device status FULL if a key finds no free slot within `capacity` probes; the index
- *         content is then unspecified until aibx_index_clear.  Slots freed by evict are not
- *         reused until clear.
+ *         Device status FULL if a new key finds no free slot within `capacity` probes (all
+ *         slots hold live entries); the index content is then unspecified until
+ *         aibx_index_clear.  Slots freed by evict are reused.
  * evict:  batch-atomic.  First mask &= ~masks[i] for all present keys; then
  *         freed[i] = id if key i was present and its mask is now 0, else AIBX_NO_BLOCK
  *         (duplicates of a key all report the same value); then entries with mask 0 vanish.

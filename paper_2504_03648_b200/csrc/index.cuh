@@ -13,7 +13,7 @@
 namespace aibx {
 
 struct __align__(32) Slot {
-  unsigned long long key;    // 0 = never used, ~0 = removed (not reused until clear)
+  unsigned long long key;    // 0 = never used, ~0 = removed (reusable by insert)
   unsigned long long mask;   // pod residency bits; an entry with mask 0 is dead
   unsigned int id;           // block id, min over inserts; AIBX_NO_BLOCK = none supplied
   unsigned int stamp;        // reserved (recency stamp for eviction policies)
@@ -93,23 +93,41 @@ __global__ void index_insert_kernel(IndexView ix, const uint64_t* __restrict__ k
   const uint64_t key = keys[i];
   const uint64_t m = masks[i] & pod_all(ix.num_pods);
   if (key_reserved(key) || m == 0) return;
+  // pass 1: an existing entry anywhere on the probe path wins (stop at a never-used slot)
   unsigned long long s = home_slot(ix, key);
   bool placed = false;
   for (unsigned long long probes = 0; probes <= ix.cap_mask; ++probes) {
-    unsigned long long k = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].key);
-    if (k == kKeyEmpty) {
-      k = atomicCAS(&ix.slots[s].key, kKeyEmpty, (unsigned long long)key);
-      if (k == kKeyEmpty) {
-        atomicAdd(&ix.counters[0], 1ULL);
-        placed = true;
-        break;
-      }
-    }
+    const unsigned long long k = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].key);
     if (k == key) {
       placed = true;
       break;
     }
+    if (k == kKeyEmpty) break;
     s = (s + 1) & ix.cap_mask;
+  }
+  // pass 2: claim the first never-used or removed slot on the path.  Every thread inserting
+  // this key walks the same path and tries the same slots in the same order, so the losers
+  // of a race find the winner's slot; no slot turns reusable while inserts run.
+  if (!placed) {
+    s = home_slot(ix, key);
+    for (unsigned long long probes = 0; probes <= ix.cap_mask; ++probes) {
+      unsigned long long k = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].key);
+      if (k == kKeyEmpty || k == kKeyTomb) {
+        const unsigned long long seen = atomicCAS(&ix.slots[s].key, k, (unsigned long long)key);
+        if (seen == k) {
+          atomicAdd(&ix.counters[0], 1ULL);
+          if (k == kKeyTomb) atomicAdd(&ix.counters[1], ~0ULL);
+          placed = true;
+          break;
+        }
+        k = seen;
+      }
+      if (k == key) {
+        placed = true;
+        break;
+      }
+      s = (s + 1) & ix.cap_mask;
+    }
   }
   if (!placed) {
     raise_status(AIBX_ERR_FULL);
@@ -160,6 +178,7 @@ __global__ void index_evict_remove_kernel(IndexView ix, const uint64_t* __restri
   const unsigned long long m = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].mask);
   if (m != 0) return;
   if (atomicCAS(&ix.slots[s].key, (unsigned long long)key, kKeyTomb) == key) {
+    ix.slots[s].id = AIBX_NO_BLOCK;      // ready for reuse by a later insert
     atomicAdd(&ix.counters[0], ~0ULL);   // live -= 1
     atomicAdd(&ix.counters[1], 1ULL);
   }

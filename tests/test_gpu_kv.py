@@ -134,6 +134,10 @@ def test_invalid_arguments():
 
 def _fit_blocks(kv, extra_bytes):
     """Shrink the pool (never the batch) if the device cannot hold the full configuration."""
+    import gc
+
+    gc.collect()
+    torch.cuda.empty_cache()                       # earlier tests' pools go back to the driver
     free, _ = torch.cuda.mem_get_info()
     room = free - extra_bytes - (6 << 30)
     if kv.pool_bytes <= room:
@@ -199,7 +203,21 @@ def test_cfg4_full_size_layer_major():
     synth.fill_pool(pool, kv)
     buf = empty(n * kv.block_bytes, torch.uint8)
     lay = kv_layout_gpu(kv)
-    touched = {}
+    history = []                                                   # (ids, content seed) of every scatter
+
+    def block_now(b):
+        """What block b must hold: the newest scatter that named it, else the generated content.
+        The scattered bytes go through the oracle (one-block pool) rather than being retyped."""
+        for ids_h, seed_h in reversed(history):
+            pos = np.nonzero(ids_h == b)[0]
+            if len(pos):
+                item = W.pool_bytes(seed_h, int(pos[0]) * kv.block_bytes, kv.block_bytes)
+                mini = np.zeros(kv.block_bytes, dtype=np.uint8)
+                oracle.kv_scatter(mini, kv_layout_oracle(kv, layout=0, num_blocks=1),
+                                  np.zeros(1, np.uint32), item)
+                return mini
+        return W.logical_blocks(kv, [b])
+
     for it in range(4):                                            # put, get, put, get
         ids = W.distinct_ids(1000 + it, kv.num_blocks, n)
         sample = np.concatenate([[0, n - 1], W.Stream(it, 11).randint(0, n, 4)])
@@ -207,24 +225,16 @@ def test_cfg4_full_size_layer_major():
             aibx.kv_gather(pool, lay, dev(ids), n, buf)
             lay1 = kv_layout_oracle(kv, layout=0, num_blocks=1)
             for i in sample:
-                b = int(ids[int(i)])
-                mini = touched.get(b)
-                if mini is None:
-                    mini = W.logical_blocks(kv, [b])
                 want = np.zeros(kv.block_bytes, dtype=np.uint8)
-                oracle.kv_gather(mini, lay1, np.zeros(1, np.uint32), want)
+                oracle.kv_gather(block_now(int(ids[int(i)])), lay1, np.zeros(1, np.uint32), want)
                 assert np.array_equal(host(buf.view(n, kv.block_bytes)[int(i)]), want)
         else:
             synth.fill_linear(buf, 5000 + it)
             aibx.kv_scatter(pool, lay, dev(ids), n, buf)
+            history.append((ids, 5000 + it))
             for i in sample:
-                item = W.pool_bytes(5000 + it, int(i) * kv.block_bytes, kv.block_bytes)
-                mini = np.zeros(kv.block_bytes, dtype=np.uint8)
-                oracle.kv_scatter(mini, kv_layout_oracle(kv, layout=0, num_blocks=1),
-                                  np.zeros(1, np.uint32), item)
                 b = int(ids[int(i)])
-                touched[b] = mini
-                assert np.array_equal(read_block(pool, kv, b), mini)
+                assert np.array_equal(read_block(pool, kv, b), block_now(b))
         assert aibx.status_fetch() == (0, 0)
     # a block no scatter named still holds its generated content
     all_scattered = set(W.distinct_ids(1001, kv.num_blocks, n).tolist()) | set(
