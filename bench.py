@@ -1,0 +1,514 @@
+#!/usr/bin/env python
+"""Benchmark of the KV-reuse hot path on B200.
+
+One step = one pass of the whole path over one batch of the Llama-3-8B-shaped workload:
+hash the 64 requests -> longest cached prefix against a 200k-entry index -> route score ->
+set of matched blocks -> gather them from the 8 GiB paged pool into the transfer buffer ->
+scatter them back -> publish and expire one batch of new index entries.
+
+`value` is gather+scatter bytes (read + written) per second over the whole step, inputs
+resident in HBM.  `e2e` is the same with host buffers: tokens come from pinned host memory,
+routing results go back to the host, the gathered buffer is copied to pinned host memory (the
+put to a DRAM cache) and copied back before the scatter (the get).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 (under torchrun) runs N independent replicas, one per GPU: the path has no exchange step.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "kv_gather_scatter_GBps_whole_step"
+UNIT = "GB/s"
+WORKLOAD = "cfg2-llama3-8b: 64 requests (1k-8k tokens, 32 Zipf prompts), index 200k/2^19 x 16 pods, " \
+           "pool 4096 x 2 MiB bf16 blocks, gather+scatter of all matched blocks"
+KERNELS_PER_STEP = 11   # hash, match, score, mark, compact, gather, scatter, insert, evict x3
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of kv_copy_bulk_kernel from the ncu
+# capture summarised under profiles/, valid only for the kernel source with this digest.
+NCU_TRAFFIC = {"kv_copy_sha1": None, "bytes_per_launch": None, "launch_algorithmic_bytes": None}
+
+
+def kernel_digest() -> str:
+    path = os.path.join(ROOT, "paper_2504_03648_b200", "csrc", "kv_copy.cuh")
+    return hashlib.sha1(open(path, "rb").read()).hexdigest()[:12]
+
+
+def measured_peak_hbm():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                      "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ---------------------------------------------------------------------------------------------
+# the GPU arm
+
+
+class GpuJob:
+    """Everything resident on one GPU for the cfg2 workload, plus the step functions."""
+
+    def __init__(self, device_index: int):
+        import torch
+
+        from paper_2504_03648_b200 import binding as aibx
+        from paper_2504_03648_b200 import synth
+        from paper_2504_03648_b200 import workloads as W
+
+        self.torch, self.aibx = torch, aibx
+        torch.cuda.set_device(device_index)
+        aibx.lib()          # fails loudly when the CUDA library was not built
+        self.w = w = W.build_routing(W.cfg2_routing())
+        self.kv = kv = W.cfg2_kv()
+        s = w.spec
+        self.B, self.P, self.R = s.block_tokens, s.num_pods, s.R
+
+        def dev(a):
+            return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+        def offsets(tok_off):
+            n = (tok_off[1:] - tok_off[:-1]) // self.B
+            out = np.zeros(len(tok_off), dtype=np.int64)
+            np.cumsum(n, out=out[1:])
+            return out
+
+        # requests: pinned on the host for the end-to-end leg, resident for the device leg
+        self.h_tokens = torch.from_numpy(w.tokens).pin_memory()
+        self.d_tokens = self.h_tokens.cuda()
+        self.d_tok_off = dev(w.tok_off)
+        blk_off = offsets(w.tok_off)
+        self.nb = int(blk_off[-1])
+        self.d_blk_off = dev(blk_off)
+        self.d_hashes = torch.empty(self.nb, dtype=torch.uint64, device="cuda")
+
+        # index content: the prompts' own chains (hashed on the GPU) plus filler entries
+        src_off = offsets(w.src_tok_off)
+        d_src_h = torch.empty(int(src_off[-1]), dtype=torch.uint64, device="cuda")
+        aibx.hash_blocks(dev(w.src_tokens), dev(w.src_tok_off), dev(src_off), self.B, 0, d_src_h)
+        self.index = aibx.Index(s.capacity, self.P)
+        self.index.insert(torch.cat([d_src_h, dev(w.filler_keys)]),
+                          dev(np.concatenate([w.src_masks, w.filler_masks])),
+                          dev(np.concatenate([w.src_ids, w.filler_ids])))
+
+        # one batch of new entries published and expired per step (state returns to the start)
+        st = W.Stream(s.seed, 21)
+        self.d_new_keys = dev(st.keys(self.nb))
+        self.d_new_masks = dev(np.left_shift(np.uint64(1), (np.arange(self.nb) % self.P).astype(np.uint64)))
+        self.d_new_ids = dev(st.randint(0, kv.num_blocks, self.nb).astype(np.uint32))
+        self.d_all_ones = dev(np.full(self.nb, 0xFFFFFFFFFFFFFFFF, dtype=np.uint64))
+        self.d_freed = torch.empty(self.nb, dtype=torch.uint32, device="cuda")
+
+        # routing outputs
+        R, P = self.R, self.P
+        self.d_match_len = torch.empty(R * P, dtype=torch.uint32, device="cuda")
+        self.d_any_len = torch.empty(R, dtype=torch.uint32, device="cuda")
+        self.d_block_ids = torch.empty(self.nb, dtype=torch.uint32, device="cuda")
+        self.d_best_pod = torch.empty(R, dtype=torch.int32, device="cuda")
+        self.d_best_score = torch.empty(R, dtype=torch.int64, device="cuda")
+        self.d_pod_load = dev(w.pod_load)
+        self.d_scratch = torch.empty(aibx.collect_scratch_bytes(kv.num_blocks) // 4 + 1,
+                                     dtype=torch.int32, device="cuda")
+        self.d_unique = torch.empty(self.nb, dtype=torch.uint32, device="cuda")
+        self.d_count = torch.empty(1, dtype=torch.uint32, device="cuda")
+        self.h_count = torch.empty(1, dtype=torch.uint32).pin_memory()
+        self.h_best_pod = torch.empty(R, dtype=torch.int32).pin_memory()
+        self.h_any_len = torch.empty(R, dtype=torch.uint32).pin_memory()
+        self.h_unique = torch.empty(self.nb, dtype=torch.uint32).pin_memory()
+
+        # KV pool and transfer buffer
+        self.layout = aibx.KVLayout(kv.layout, kv.num_layers, kv.num_kv_heads, kv.block_tokens,
+                                    kv.head_dim, kv.elem_bytes, kv.num_blocks)
+        self.d_pool = torch.empty(kv.pool_bytes, dtype=torch.uint8, device="cuda")
+        synth.fill_pool(self.d_pool, kv)
+        self.count = self.routing()                      # how many blocks a step moves
+        self.d_buf = torch.empty(self.count * kv.block_bytes, dtype=torch.uint8, device="cuda")
+        self.h_buf = None
+        self.copy_events = []
+        st_code = aibx.status_fetch()
+        assert st_code == (0, 0), st_code
+
+    # -- pieces of a step ------------------------------------------------------------------
+    def routing(self) -> int:
+        aibx = self.aibx
+        aibx.hash_blocks(self.d_tokens, self.d_tok_off, self.d_blk_off, self.B, 0, self.d_hashes)
+        self.index.match_prefix(self.d_hashes, self.d_blk_off, self.d_match_len, self.d_any_len,
+                                self.d_block_ids)
+        aibx.route_score(self.d_match_len, self.d_blk_off, self.P, self.d_pod_load,
+                         self.w.ready_mask, None, self.d_best_pod, self.d_best_score, None)
+        aibx.collect_blocks(self.d_block_ids, self.kv.num_blocks, self.d_scratch, self.d_unique,
+                            self.d_count)
+        # the host needs the size of the transfer: 4 bytes back, one stream sync
+        self.h_count.copy_(self.d_count, non_blocking=True)
+        self.torch.cuda.current_stream().synchronize()
+        return int(self.h_count.numpy()[0])
+
+    def publish_expire(self):
+        self.index.insert(self.d_new_keys, self.d_new_masks, self.d_new_ids)
+        self.index.evict(self.d_new_keys, self.d_all_ones, self.d_freed)
+
+    def step(self, record_copy_events=False):
+        torch, aibx = self.torch, self.aibx
+        n = self.routing()
+        if record_copy_events:
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            e[0].record()
+        aibx.kv_gather(self.d_pool, self.layout, self.d_unique, n, self.d_buf)
+        if record_copy_events:
+            e[1].record()
+        aibx.kv_scatter(self.d_pool, self.layout, self.d_unique, n, self.d_buf)
+        if record_copy_events:
+            e[2].record()
+            self.copy_events.append(e)
+        self.publish_expire()
+
+    def step_e2e(self):
+        """Same step with host buffers on both sides of every transfer."""
+        torch, aibx = self.torch, self.aibx
+        if self.h_buf is None:
+            self.h_buf = torch.empty(self.d_buf.numel(), dtype=torch.uint8).pin_memory()
+        self.d_tokens.copy_(self.h_tokens, non_blocking=True)
+        n = self.routing()
+        self.h_best_pod.copy_(self.d_best_pod, non_blocking=True)
+        self.h_any_len.copy_(self.d_any_len, non_blocking=True)
+        self.h_unique.copy_(self.d_unique, non_blocking=True)
+        aibx.kv_gather(self.d_pool, self.layout, self.d_unique, n, self.d_buf)
+        nbytes = n * self.kv.block_bytes
+        self.h_buf[:nbytes].copy_(self.d_buf[:nbytes], non_blocking=True)     # put: to the DRAM cache
+        self.d_buf[:nbytes].copy_(self.h_buf[:nbytes], non_blocking=True)     # get: back from it
+        aibx.kv_scatter(self.d_pool, self.layout, self.d_unique, n, self.d_buf)
+        self.publish_expire()
+        torch.cuda.current_stream().synchronize()
+        h2d = self.h_tokens.numel() * 4 + nbytes
+        d2h = 4 + self.R * 8 + self.nb * 4 + nbytes
+        return h2d, d2h
+
+    def stage_breakdown(self, reps=10):
+        """Median device time of every call of the step, in microseconds (outside the timed run)."""
+        torch, aibx = self.torch, self.aibx
+        calls = {
+            "hash_blocks": lambda: aibx.hash_blocks(self.d_tokens, self.d_tok_off, self.d_blk_off,
+                                                    self.B, 0, self.d_hashes),
+            "match_prefix": lambda: self.index.match_prefix(self.d_hashes, self.d_blk_off,
+                                                            self.d_match_len, self.d_any_len,
+                                                            self.d_block_ids),
+            "route_score": lambda: aibx.route_score(self.d_match_len, self.d_blk_off, self.P,
+                                                    self.d_pod_load, self.w.ready_mask, None,
+                                                    self.d_best_pod, self.d_best_score, None),
+            "collect_blocks": lambda: aibx.collect_blocks(self.d_block_ids, self.kv.num_blocks,
+                                                          self.d_scratch, self.d_unique, self.d_count),
+            "kv_gather": lambda: aibx.kv_gather(self.d_pool, self.layout, self.d_unique, self.count,
+                                                self.d_buf),
+            "kv_scatter": lambda: aibx.kv_scatter(self.d_pool, self.layout, self.d_unique,
+                                                  self.count, self.d_buf),
+            "index_insert": lambda: self.index.insert(self.d_new_keys, self.d_new_masks,
+                                                      self.d_new_ids),
+            "index_evict": lambda: self.index.evict(self.d_new_keys, self.d_all_ones, self.d_freed),
+        }
+        out = {}
+        for name, fn in calls.items():
+            ts = []
+            for _ in range(reps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn()
+                b.record()
+                b.synchronize()
+                ts.append(a.elapsed_time(b) * 1e3)
+            out[name] = round(statistics.median(ts), 2)
+        return out
+
+
+def run_gpu(args):
+    import torch
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (no CPU fallback exists)"
+
+    job = GpuJob(local_rank)
+    kv = job.kv
+    step_bytes = 2 * 2 * job.count * kv.block_bytes        # gather + scatter, read + write
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        job.step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        job.step(record_copy_events=True)
+    t1.record()
+    barrier()
+    elapsed_ms = t0.elapsed_time(t1)
+    clocks = sampler.stop() if rank == 0 else None
+    if dist is not None:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    status = job.aibx.status_fetch()
+    assert status == (0, 0), status
+
+    # dominant kernel: the bulk-copy kernel, two launches per step, timed inside the timed region
+    durs = []
+    for e in job.copy_events:
+        durs += [e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2])]
+    launch_ms = sum(durs) / len(durs)
+    launch_bytes = 2 * job.count * kv.block_bytes + 4 * job.count
+    peak, peak_kind = measured_peak_hbm()
+    achieved = launch_bytes / (launch_ms * 1e-3) / 1e9
+    traffic = None
+    if NCU_TRAFFIC["kv_copy_sha1"] == kernel_digest() and NCU_TRAFFIC["bytes_per_launch"]:
+        traffic = NCU_TRAFFIC["bytes_per_launch"] * launch_bytes / NCU_TRAFFIC["launch_algorithmic_bytes"]
+
+    # end-to-end leg (host buffers), fewer steps: PCIe-bound
+    e2e_steps = max(2, min(5, args.steps))
+    job.step_e2e()
+    barrier()
+    w0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        h2d, d2h = job.step_e2e()
+    torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - w0) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+
+    stages = job.stage_breakdown() if rank == 0 else None
+    if dist is not None:
+        dist.barrier()
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = elapsed_ms / args.steps
+    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    cpu = cpu_baseline(budget_s=12.0)
+    line = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 4),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "blocks_moved_per_step": job.count,
+                   "bytes_moved_per_step": step_bytes, "parallelism": "replicas only" if world > 1 else "1 gpu",
+                   "l2": "inputs larger than L2: 6.5 GB of KV traffic per step evicts it between steps",
+                   "kv_tuning": "bulk ring, 16 KiB x 12 stages, 1 CTA/SM"},
+        "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
+        "e2e": {"value": round(world * step_bytes / e2e_s / 1e9, 2), "unit": UNIT,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "roofline": {"bound": "hbm", "kernel": "kv_copy_bulk_kernel", "achieved": round(achieved, 1),
+                     "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": round(achieved / peak, 4), "frac_of_nominal_8000": round(achieved / 8000.0, 4),
+                     "traffic": traffic, "algorithmic_bytes_per_launch": launch_bytes,
+                     "avg_launch_ms": round(launch_ms, 4), "launches_timed": len(durs)},
+        "cpu_baseline": cpu,
+        "match_requests_per_s": round(job.R / (stages["match_prefix"] * 1e-6), 1),
+        "stage_us": stages,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------
+# the CPU oracle: baseline leg and reference arm
+
+
+class OracleSample:
+    """The oracle on a bounded sample of the same workload: the whole routing batch, and
+    gather+scatter of SAMPLE_BLOCKS blocks of the same shape out of a 512-block host pool."""
+
+    SAMPLE_BLOCKS = 128
+    POOL_BLOCKS = 512
+
+    def __init__(self):
+        import oracle
+        from paper_2504_03648_b200 import workloads as W
+
+        self.oracle = oracle
+        self.w = w = W.build_routing(W.cfg2_routing())
+        s = w.spec
+        kv = W.scaled(W.cfg2_kv(), num_blocks=self.POOL_BLOCKS)
+        self.kv = kv
+        sh, _ = oracle.hash_blocks(w.src_tokens, w.src_tok_off, s.block_tokens, 0)
+        self.ix = oracle.Index(s.capacity, s.num_pods)
+        self.ix.insert(np.concatenate([sh, w.filler_keys]),
+                       np.concatenate([w.src_masks, w.filler_masks]),
+                       np.concatenate([w.src_ids, w.filler_ids]))
+        self.pool = W.host_pool(kv)
+        self.lay = oracle.kv_layout(kv.layout, kv.num_layers, kv.num_kv_heads, kv.block_tokens,
+                                    kv.head_dim, kv.elem_bytes, kv.num_blocks)
+        self.ids = W.distinct_ids(5, kv.num_blocks, self.SAMPLE_BLOCKS)
+        self.buf = np.zeros(self.SAMPLE_BLOCKS * kv.block_bytes, dtype=np.uint8)
+        self.step_bytes = 2 * 2 * self.SAMPLE_BLOCKS * kv.block_bytes
+        st = W.Stream(s.seed, 21)
+        nb = int(oracle.block_offsets(w.tok_off, s.block_tokens)[-1])
+        self.new_keys = st.keys(nb)
+        self.new_masks = np.left_shift(np.uint64(1), (np.arange(nb) % s.num_pods).astype(np.uint64))
+        self.new_ids = st.randint(0, 4096, nb).astype(np.uint32)
+        self.all_ones = np.full(nb, 0xFFFFFFFFFFFFFFFF, dtype=np.uint64)
+
+    def step(self):
+        o, w, s = self.oracle, self.w, self.w.spec
+        h, bo = o.hash_blocks(w.tokens, w.tok_off, s.block_tokens, 0)
+        ml, al, ids = self.ix.match_prefix(h, bo)
+        o.route_score(ml, bo, w.pod_load, w.ready_mask, None)
+        o.collect_blocks(ids, 4096)
+        o.kv_gather(self.pool, self.lay, self.ids, self.buf)
+        o.kv_scatter(self.pool, self.lay, self.ids, self.buf)
+        self.ix.insert(self.new_keys, self.new_masks, self.new_ids)
+        self.ix.evict(self.new_keys, self.all_ones)
+
+    describe = ("whole routing batch (64 requests, 200k-entry index) + gather and scatter of 128 of "
+                "the 2 MiB blocks out of a 512-block host pool + one publish/expire batch, per step")
+
+
+def cpu_baseline(budget_s: float):
+    sample = OracleSample()
+    sample.step()
+    n, t0 = 0, time.perf_counter()
+    while True:
+        sample.step()
+        n += 1
+        dt = time.perf_counter() - t0
+        if dt >= budget_s or n >= 2000:
+            break
+    return {"value": round(sample.step_bytes * n / dt / 1e9, 3), "unit": UNIT, "cores": 1,
+            "kind": "oracle", "sample": OracleSample.describe, "steps": n,
+            "seconds": round(dt, 2)}
+
+
+def run_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    sample = OracleSample()
+    for _ in range(max(args.warmup, 1)):
+        sample.step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        sample.step()
+    dt = time.perf_counter() - t0
+    value = round(sample.step_bytes * args.steps / dt / 1e9, 3)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": max(args.warmup, 1),
+        "ms_per_step": round(dt / args.steps * 1e3, 3), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "note": "CPU oracle, one host core, bounded sample per step"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": OracleSample.describe},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -235,8 +235,8 @@ __global__ void __launch_bounds__(kLdstThreads) kv_copy_ldst_kernel(CopyPlan pl)
 
 struct CopyTuning {
   int mode = 0;            // 0 bulk ring, 1 ld/st loop
-  int chunk_bytes = 32768;
-  int stages = 6;
+  int chunk_bytes = 16384;
+  int stages = 12;
   int ctas_per_sm = 1;
 };
 

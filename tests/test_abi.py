@@ -20,7 +20,7 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(lib, name), name
     lib.aibx_strerror.restype = ctypes.c_char_p
     assert lib.aibx_strerror(-3) == b"index full"
-    assert lib.aibx_kv_set_tuning(0, 32768, 6, 1) == 0
+    assert lib.aibx_kv_set_tuning(0, 16384, 12, 1) == 0
     assert lib.aibx_kv_set_tuning(0, 100, 6, 1) == -1          # chunk not a multiple of 16
     assert lib.aibx_kv_set_tuning(0, 65536, 16, 1) == -1       # ring larger than shared memory
 

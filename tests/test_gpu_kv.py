@@ -18,9 +18,9 @@ GUARD = 4096
 
 @pytest.fixture(autouse=True)
 def _default_tuning():
-    aibx.kv_set_tuning(0, 32768, 6, 1)
+    aibx.kv_set_tuning(0, 16384, 12, 1)
     yield
-    aibx.kv_set_tuning(0, 32768, 6, 1)
+    aibx.kv_set_tuning(0, 16384, 12, 1)
 
 
 def guarded(n_bytes, fill):
@@ -63,7 +63,7 @@ def check_gather_scatter(kv, ids_g, ids_s, mode_args):
     assert guards_intact(buf_w, buf_bytes, 0xEE) and guards_intact(pool_w, kv.pool_bytes, 0xA5)
 
 
-MODES = [(0, 32768, 6, 1), (0, 4096, 3, 2), (0, 1024, 16, 1), (1, 16384, 2, 1), (0, 49152, 4, 1)]
+MODES = [(0, 16384, 12, 1), (0, 32768, 6, 1), (0, 4096, 3, 2), (0, 1024, 16, 1), (1, 16384, 2, 1), (0, 49152, 4, 1)]
 
 
 @pytest.mark.parametrize("mode_args", MODES)
