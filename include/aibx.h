@@ -157,6 +157,34 @@ int32_t aibx_collect_blocks(const uint32_t* d_block_ids, int64_t n, uint32_t num
                             void* stream);
 
 /* ---------------------------------------------------------------------------------------
+ * aibx_collect_blocks without any allocation (the paper has no counterpart: this is a
+ * packaging variant of the call above, not an operation of the method).
+ *
+ * For callers that cannot obtain device memory at the moment they need the call: a routing
+ * plug-in living inside an inference engine whose KV pool has already claimed nearly all of
+ * HBM (a cudaMalloc there can fail, or stall the engine because it synchronises the device),
+ * or code running in a callback or latency-critical loop where allocating is forbidden.  Such a
+ * caller still passes its inputs and outputs; only the scratch bitmap comes from the library: a
+ * fixed array of 128 KiB in the library's device image, present on every GPU that loads the
+ * library until the process exits.
+ *
+ *   Same results as aibx_collect_blocks (ascending distinct valid ids, NO_BLOCK padding,
+ *   *d_count, RANGE status for bad ids).  The call itself never calls cudaMalloc, cudaFree
+ *   or any allocating routine.
+ *   num_blocks > aibx_collect_static_max_blocks() (1,048,576)  ->  AIBX_ERR_UNSUPPORTED, nothing
+ *   is enqueued.  Use aibx_collect_blocks with your own scratch for larger pools.
+ *   The first call on each device looks up the array's device address (once, with that device
+ *   current; AIBX_ERR_CUDA if the runtime refuses).  Make that first call before starting any
+ *   stream capture.
+ *   All calls on a device share the one array, which keeps the marks of the previous call; each
+ *   call zeroes the part it uses first.  Two calls whose work overlaps on the GPU (different
+ *   streams, no ordering between them) race on the array and give wrong results: order them.
+ */
+int32_t aibx_collect_blocks_static(const uint32_t* d_block_ids, int64_t n, uint32_t num_blocks,
+                                   uint32_t* d_unique_ids, uint32_t* d_count, void* stream);
+uint32_t aibx_collect_static_max_blocks(void);
+
+/* ---------------------------------------------------------------------------------------
  * Paged-KV data movement (Section 3.2.5: put/get between the engine's paged KV pool and the
  * cache, with exchange through a contiguous buffer when cache and engine are colocated).
  *   tile        = 2 (K,V) * num_kv_heads * block_tokens * head_dim * elem_bytes   bytes

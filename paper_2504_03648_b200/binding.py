@@ -78,6 +78,7 @@ def lib():
             "aibx_match_prefix": [vp, vp, vp, i32, vp, vp, vp, vp],
             "aibx_route_score": [vp, vp, i32, i32, vp, u64, C.POINTER(RouteParams), vp, vp, vp, vp],
             "aibx_collect_blocks": [vp, i64, u32, vp, vp, vp, vp],
+            "aibx_collect_blocks_static": [vp, i64, u32, vp, vp, vp],
             "aibx_kv_gather": [vp, C.POINTER(KVLayout), vp, i64, vp, vp],
             "aibx_kv_scatter": [vp, C.POINTER(KVLayout), vp, i64, vp, vp],
             "aibx_kv_set_tuning": [i32, i32, i32, i32],
@@ -89,6 +90,8 @@ def lib():
             fn.restype = i32
         L.aibx_collect_scratch_bytes.argtypes = [u32]
         L.aibx_collect_scratch_bytes.restype = u64
+        L.aibx_collect_static_max_blocks.argtypes = []
+        L.aibx_collect_static_max_blocks.restype = u32
         L.aibx_strerror.argtypes = [i32]
         L.aibx_strerror.restype = C.c_char_p
         _lib = L
@@ -202,6 +205,21 @@ def collect_blocks(block_ids, num_blocks: int, scratch, unique_ids, count) -> No
     assert unique_ids.numel() >= n
     _check("aibx_collect_blocks", lib().aibx_collect_blocks(
         _ptr(block_ids, torch.uint32), n, num_blocks, _ptr(scratch), _ptr(unique_ids, torch.uint32),
+        _ptr(count, torch.uint32), _stream()))
+
+
+def collect_static_max_blocks() -> int:
+    return int(lib().aibx_collect_static_max_blocks())
+
+
+def collect_blocks_static(block_ids, num_blocks: int, unique_ids, count) -> None:
+    """collect_blocks for callers that must not allocate: the bitmap is the library's own fixed
+    array (pools up to collect_static_max_blocks() blocks).  Calls on one device share that
+    array, so they must not overlap on the GPU."""
+    n = block_ids.numel()
+    assert unique_ids.numel() >= n
+    _check("aibx_collect_blocks_static", lib().aibx_collect_blocks_static(
+        _ptr(block_ids, torch.uint32), n, num_blocks, _ptr(unique_ids, torch.uint32),
         _ptr(count, torch.uint32), _stream()))
 
 

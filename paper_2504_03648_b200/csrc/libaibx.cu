@@ -41,6 +41,30 @@ StatusRecord* status_ptr() {
   return cached[dev];
 }
 
+// Built-in scratch of aibx_collect_blocks_static: a bitmap over block ids that lives in the
+// library image itself, so the call needs no allocation.  128 KiB per GPU that loads the
+// library, held until the process exits.
+constexpr uint32_t kStaticCollectMaxBlocks = 1u << 20;
+static __device__ __align__(256) unsigned int g_collect_bitmap[kStaticCollectMaxBlocks / 32];
+
+// In host code `g_collect_bitmap` is only a handle for the runtime, not a device address, so
+// kernels must be given what cudaGetSymbolAddress returns.  Resolved once per device, with that
+// device current; returns nullptr when the runtime refuses.
+unsigned int* static_bitmap_ptr() {
+  static unsigned int* cached[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!cached[dev]) {
+    unsigned int* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_collect_bitmap) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    cached[dev] = p;
+  }
+  return cached[dev];
+}
+
 }  // namespace
 
 extern "C" {
@@ -215,6 +239,27 @@ int32_t aibx_collect_blocks(const uint32_t* d_block_ids, int64_t n, uint32_t num
                                                         d_count);
   return launch_status();
 }
+
+int32_t aibx_collect_blocks_static(const uint32_t* d_block_ids, int64_t n, uint32_t num_blocks,
+                                   uint32_t* d_unique_ids, uint32_t* d_count, void* stream) {
+  if (n < 0 || !d_count) return AIBX_ERR_INVALID;
+  if (n > 0 && (!d_block_ids || !d_unique_ids)) return AIBX_ERR_INVALID;
+  if (num_blocks > kStaticCollectMaxBlocks) return AIBX_ERR_UNSUPPORTED;
+  unsigned int* bitmap = static_bitmap_ptr();
+  if (!bitmap) return AIBX_ERR_CUDA;
+  cudaStream_t st = as_stream(stream);
+  // the array still holds the previous call's marks: zero the part this call reads
+  if (num_blocks > 0 &&
+      cudaMemsetAsync(bitmap, 0, aibx_collect_scratch_bytes(num_blocks), st) != cudaSuccess)
+    return AIBX_ERR_CUDA;
+  if (n > 0)
+    collect_mark_kernel<<<blocks_for(n, 256), 256, 0, st>>>(d_block_ids, n, num_blocks, bitmap);
+  collect_compact_kernel<<<1, kCollectThreads, 0, st>>>(bitmap, num_blocks, n, d_unique_ids,
+                                                        d_count);
+  return launch_status();
+}
+
+uint32_t aibx_collect_static_max_blocks(void) { return kStaticCollectMaxBlocks; }
 
 int32_t aibx_kv_gather(const void* d_pool, const aibx_kv_layout_t* layout,
                        const uint32_t* d_block_ids, int64_t n, void* d_buf, void* stream) {
