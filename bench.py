@@ -42,7 +42,8 @@ KERNELS_PER_STEP = 11   # hash, match, score, mark, compact, gather, scatter, in
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of kv_copy_bulk_kernel from the ncu
 # capture summarised under profiles/, valid only for the kernel source with this digest.
-NCU_TRAFFIC = {"kv_copy_sha1": None, "bytes_per_launch": None, "launch_algorithmic_bytes": None}
+NCU_TRAFFIC = {"kv_copy_sha1": "286ef8bd7773", "bytes_per_launch": 1018708224,
+               "launch_algorithmic_bytes": 1073742848}
 
 
 def kernel_digest() -> str:
@@ -497,14 +498,192 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ---------------------------------------------------------------------------------------------
+# small single-kernel cases (profiling targets and microbenchmarks; not the bench line)
+
+
+def _event_times(torch, fn, reps, warm):
+    for _ in range(warm):
+        fn()
+    ts = []
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        b.synchronize()
+        ts.append(a.elapsed_time(b))
+    return ts
+
+
+def case_kv_small(args):
+    """Gather then scatter 256 blocks of the cfg2 shape out of a 1 GiB pool (1 GiB of traffic
+    per launch, larger than L2): the capture target for kv_copy_bulk_kernel."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import synth
+    from paper_2504_03648_b200 import workloads as W
+
+    kv = W.scaled(W.cfg2_kv(), num_blocks=512)
+    n = 256
+    pool = torch.empty(kv.pool_bytes, dtype=torch.uint8, device="cuda")
+    synth.fill_pool(pool, kv)
+    ids = torch.from_numpy(np.sort(W.distinct_ids(7, kv.num_blocks, n))).cuda()
+    buf = torch.empty(n * kv.block_bytes, dtype=torch.uint8, device="cuda")
+    lay = aibx.KVLayout(kv.layout, kv.num_layers, kv.num_kv_heads, kv.block_tokens, kv.head_dim,
+                        kv.elem_bytes, kv.num_blocks)
+
+    def both():
+        aibx.kv_gather(pool, lay, ids, n, buf)
+        aibx.kv_scatter(pool, lay, ids, n, buf)
+
+    ts = _event_times(torch, both, max(args.steps, 1), max(args.warmup, 1))
+    nbytes = 2 * (2 * n * kv.block_bytes + 4 * n)
+    peak, kind = measured_peak_hbm()
+    best = nbytes / (min(ts) * 1e-3) / 1e9
+    print(json.dumps({"case": "kv_small", "blocks": n, "algorithmic_bytes_per_launch": nbytes // 2,
+                      "ms_gather_plus_scatter_median": round(statistics.median(ts), 4),
+                      "GBps_median": round(nbytes / (statistics.median(ts) * 1e-3) / 1e9, 1),
+                      "GBps_best": round(best, 1), "peak": peak, "peak_kind": kind,
+                      "status": aibx.status_fetch()}))
+
+
+def _big_index(torch, aibx, W, log2cap, P, seed):
+    """Index of 2^log2cap slots at load 0.5 filled with random keys (all pods resident)."""
+    cap = 1 << log2cap
+    n = cap // 2
+    st = W.Stream(seed, 31)
+    keys = st.keys(n)
+    ix = aibx.Index(cap, P)
+    allm = (1 << P) - 1 if P < 64 else 0xFFFFFFFFFFFFFFFF
+    ix.insert(torch.from_numpy(keys).cuda(),
+              torch.from_numpy(np.full(n, allm, dtype=np.uint64)).cuda(),
+              torch.from_numpy(np.arange(n, dtype=np.uint32)).cuda())
+    return ix, keys
+
+
+def case_match_large(args):
+    """Prefix match at a size where a bandwidth roofline means something: 2^23-slot index
+    (256 MiB, load 0.5, 32 pods), R requests of 64 blocks, every block resident, so all
+    64 lookups of a request are necessary.  Algorithmic bytes: 8 + 32 per lookup,
+    4*P + 4*64 + 4 out per request."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import workloads as W
+
+    P, nblk = 32, 64
+    ix, keys = _big_index(torch, aibx, W, args.log2cap, P, 11)
+    out = []
+    for R in (4096, 32768, 262144):
+        st = W.Stream(12, R)
+        pick = st.randint(0, len(keys), R * nblk)
+        d_h = torch.from_numpy(keys[pick]).cuda()
+        d_bo = torch.arange(0, (R + 1) * nblk, nblk, dtype=torch.int64, device="cuda")
+        d_ml = torch.empty(R * P, dtype=torch.uint32, device="cuda")
+        d_al = torch.empty(R, dtype=torch.uint32, device="cuda")
+        d_ids = torch.empty(R * nblk, dtype=torch.uint32, device="cuda")
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+        def run():
+            flush.fill_(1)                      # evict the table from L2 between repetitions
+            ix.match_prefix(d_h, d_bo, d_ml, d_al, d_ids)
+
+        def only_flush():
+            flush.fill_(1)
+
+        t_both = statistics.median(_event_times(torch, run, max(args.steps, 5), 3))
+        t_flush = statistics.median(_event_times(torch, only_flush, max(args.steps, 5), 3))
+        ms = t_both - t_flush
+        assert int(d_al.cpu().numpy().min()) == nblk
+        nbytes = R * nblk * 40 + R * (4 * P + 4 * nblk + 4)
+        peak, kind = measured_peak_hbm()
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out.append({"R": R, "lookups": R * nblk, "ms": round(ms, 4), "GBps": round(gbs, 1),
+                    "frac": round(gbs / peak, 4), "requests_per_s": round(R / (ms * 1e-3), 0),
+                    "lookups_per_s": round(R * nblk / (ms * 1e-3), 0)})
+    print(json.dumps({"case": "match_large", "index_slots": 1 << args.log2cap, "pods": P,
+                      "blocks_per_request": nblk, "l2": "flushed before every launch (256 MiB fill, "
+                      "its time subtracted)", "peak": peak, "peak_kind": kind, "results": out,
+                      "status": aibx.status_fetch()}))
+
+
+def case_match_cfg(args):
+    """match_prefix alone on the routing-heavy (cfg3) and long-context (cfg5) batches."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import workloads as W
+
+    res = []
+    for mk in (W.cfg3_routing, W.cfg5_routing):
+        w = W.build_routing(mk())
+        s = w.spec
+        B, P, R = s.block_tokens, s.num_pods, s.R
+
+        def dev(a):
+            return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+        def offsets(tok_off):
+            n = (tok_off[1:] - tok_off[:-1]) // B
+            o = np.zeros(len(tok_off), dtype=np.int64)
+            np.cumsum(n, out=o[1:])
+            return o
+
+        bo, sbo = offsets(w.tok_off), offsets(w.src_tok_off)
+        d_tok, d_toff, d_bo = dev(w.tokens), dev(w.tok_off), dev(bo)
+        d_h = torch.empty(int(bo[-1]), dtype=torch.uint64, device="cuda")
+        d_sh = torch.empty(int(sbo[-1]), dtype=torch.uint64, device="cuda")
+        aibx.hash_blocks(dev(w.src_tokens), dev(w.src_tok_off), dev(sbo), B, 0, d_sh)
+        ix = aibx.Index(s.capacity, P)
+        ix.insert(torch.cat([d_sh, dev(w.filler_keys)]),
+                  dev(np.concatenate([w.src_masks, w.filler_masks])),
+                  dev(np.concatenate([w.src_ids, w.filler_ids])))
+        d_ml = torch.empty(R * P, dtype=torch.uint32, device="cuda")
+        d_al = torch.empty(R, dtype=torch.uint32, device="cuda")
+        d_ids = torch.empty(int(bo[-1]), dtype=torch.uint32, device="cuda")
+        d_bp = torch.empty(R, dtype=torch.int32, device="cuda")
+        d_bs = torch.empty(R, dtype=torch.int64, device="cuda")
+        d_load = dev(w.pod_load)
+        t_hash = statistics.median(_event_times(
+            torch, lambda: aibx.hash_blocks(d_tok, d_toff, d_bo, B, 0, d_h), 10, 3))
+        t_match = statistics.median(_event_times(
+            torch, lambda: ix.match_prefix(d_h, d_bo, d_ml, d_al, d_ids), 10, 3))
+        t_score = statistics.median(_event_times(
+            torch, lambda: aibx.route_score(d_ml, d_bo, P, d_load, w.ready_mask, None, d_bp, d_bs,
+                                            None), 10, 3))
+        al = d_al.cpu().numpy().astype(np.int64)
+        n_r = np.diff(bo)
+        lookups = int(np.minimum(al + 1, n_r).sum())
+        nbytes = lookups * 40 + int((4 * P + 4) * R + 4 * al.sum())
+        res.append({"config": s.name, "R": R, "blocks": int(bo[-1]), "necessary_lookups": lookups,
+                    "hash_us": round(t_hash * 1e3, 1), "match_us": round(t_match * 1e3, 1),
+                    "score_us": round(t_score * 1e3, 1),
+                    "hash_tokens_per_s": round(len(w.tokens) / (t_hash * 1e-3), 0),
+                    "hash_ns_per_block_longest_chain": round(t_hash * 1e6 / int(n_r.max()), 1),
+                    "match_requests_per_s": round(R / (t_match * 1e-3), 0),
+                    "match_algorithmic_GBps": round(nbytes / (t_match * 1e-3) / 1e9, 2)})
+        ix.destroy()
+    print(json.dumps({"case": "match_cfg", "results": res, "status": aibx.status_fetch()}))
+
+
+CASES = {"kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg}
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--case", default=None, choices=sorted(CASES),
+                    help="run one small single-kernel case instead of the bench step")
+    ap.add_argument("--log2cap", type=int, default=23)
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.case:
+        CASES[args.case](args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)
