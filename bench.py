@@ -42,7 +42,7 @@ KERNELS_PER_STEP = 11   # hash, match, score, mark, compact, gather, scatter, in
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of kv_copy_bulk_kernel from the ncu
 # capture summarised under profiles/, valid only for the kernel source with this digest.
-NCU_TRAFFIC = {"kv_copy_sha1": "286ef8bd7773", "bytes_per_launch": 1018708224,
+NCU_TRAFFIC = {"kv_copy_sha1": "0f01931bbbc5", "bytes_per_launch": 1023077632,
                "launch_algorithmic_bytes": 1073742848}
 
 
@@ -387,7 +387,7 @@ def run_gpu(args):
         "config": {"workload": WORKLOAD, "blocks_moved_per_step": job.count,
                    "bytes_moved_per_step": step_bytes, "parallelism": "replicas only" if world > 1 else "1 gpu",
                    "l2": "inputs larger than L2: 6.5 GB of KV traffic per step evicts it between steps",
-                   "kv_tuning": "bulk ring, 16 KiB x 12 stages, 1 CTA/SM"},
+                   "kv_tuning": "bulk ring, loader + storer warp, 32 KiB x 3 stages, 1 CTA/SM"},
         "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
         "e2e": {"value": round(world * step_bytes / e2e_s / 1e9, 2), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
@@ -584,14 +584,14 @@ def case_match_large(args):
         d_ml = torch.empty(R * P, dtype=torch.uint32, device="cuda")
         d_al = torch.empty(R, dtype=torch.uint32, device="cuda")
         d_ids = torch.empty(R * nblk, dtype=torch.uint32, device="cuda")
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        flush = torch.empty(64 << 20, dtype=torch.int32, device="cuda")
 
         def run():
-            flush.fill_(1)                      # evict the table from L2 between repetitions
+            flush.sum()                         # a 256 MiB read evicts the table from L2
             ix.match_prefix(d_h, d_bo, d_ml, d_al, d_ids)
 
         def only_flush():
-            flush.fill_(1)
+            flush.sum()
 
         t_both = statistics.median(_event_times(torch, run, max(args.steps, 5), 3))
         t_flush = statistics.median(_event_times(torch, only_flush, max(args.steps, 5), 3))
@@ -604,7 +604,7 @@ def case_match_large(args):
                     "frac": round(gbs / peak, 4), "requests_per_s": round(R / (ms * 1e-3), 0),
                     "lookups_per_s": round(R * nblk / (ms * 1e-3), 0)})
     print(json.dumps({"case": "match_large", "index_slots": 1 << args.log2cap, "pods": P,
-                      "blocks_per_request": nblk, "l2": "flushed before every launch (256 MiB fill, "
+                      "blocks_per_request": nblk, "l2": "evicted before every launch (256 MiB read, "
                       "its time subtracted)", "peak": peak, "peak_kind": kind, "results": out,
                       "status": aibx.status_fetch()}))
 
@@ -668,7 +668,174 @@ def case_match_cfg(args):
     print(json.dumps({"case": "match_cfg", "results": res, "status": aibx.status_fetch()}))
 
 
-CASES = {"kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg}
+def _fit_pool(torch, W, kv, extra_bytes):
+    """Shrink the pool (never the batch) when the device cannot hold the whole configuration."""
+    free, _ = torch.cuda.mem_get_info()
+    room = free - extra_bytes - (6 << 30)
+    if kv.pool_bytes <= room:
+        return kv
+    return W.scaled(kv, num_blocks=int(room // kv.block_bytes))
+
+
+def case_cfg4(args):
+    """Llama-3-70B shape, layer-major pool of 20,000 x 5 MiB blocks: 100 iterations alternating
+    put (gather 2,048 blocks into the block-major buffer) and get (scatter them back out)."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import synth
+    from paper_2504_03648_b200 import workloads as W
+
+    n, iters = 2048, 100
+    kv = _fit_pool(torch, W, W.cfg4_kv(), n * W.cfg4_kv().block_bytes)
+    pool = torch.empty(kv.pool_bytes, dtype=torch.uint8, device="cuda")
+    synth.fill_pool(pool, kv)
+    buf = torch.empty(n * kv.block_bytes, dtype=torch.uint8, device="cuda")
+    synth.fill_linear(buf, 99)
+    lay = aibx.KVLayout(kv.layout, kv.num_layers, kv.num_kv_heads, kv.block_tokens, kv.head_dim,
+                        kv.elem_bytes, kv.num_blocks)
+    ids = [torch.from_numpy(W.distinct_ids(1000 + j, kv.num_blocks, n)).cuda() for j in range(iters)]
+    for j in range(3):
+        aibx.kv_gather(pool, lay, ids[j], n, buf)
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+    ev[0].record()
+    for j in range(iters):
+        if j % 2 == 0:
+            aibx.kv_gather(pool, lay, ids[j], n, buf)
+        else:
+            aibx.kv_scatter(pool, lay, ids[j], n, buf)
+        ev[j + 1].record()
+    torch.cuda.synchronize()
+    ms = [ev[j].elapsed_time(ev[j + 1]) for j in range(iters)]
+    nbytes = 2 * n * kv.block_bytes
+    peak, kind = measured_peak_hbm()
+
+    def gbs(t):
+        return round(nbytes / (t * 1e-3) / 1e9, 1)
+
+    g, sc = ms[0::2], ms[1::2]
+    print(json.dumps({"case": "cfg4", "pool_blocks_effective": kv.num_blocks, "blocks_per_iter": n,
+                      "tile_bytes": kv.tile_bytes, "bytes_per_iter": nbytes,
+                      "gather_GBps_median": gbs(statistics.median(g)), "gather_GBps_best": gbs(min(g)),
+                      "scatter_GBps_median": gbs(statistics.median(sc)), "scatter_GBps_best": gbs(min(sc)),
+                      "all_100_GBps": round(nbytes * iters / (sum(ms) * 1e-3) / 1e9, 1),
+                      "frac_of_measured_median": round(gbs(statistics.median(ms)) / peak, 4),
+                      "frac_of_nominal_8000_median": round(gbs(statistics.median(ms)) / 8000.0, 4),
+                      "peak": peak, "peak_kind": kind, "status": aibx.status_fetch()}))
+
+
+def case_cfg5(args):
+    """Long-context FP8 shape: per request gather its 3,000 cached blocks (get) and scatter its
+    1,000 new blocks (put) in a block-major pool of 128,000 x 896 KiB blocks; 32 requests."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import synth
+    from paper_2504_03648_b200 import workloads as W
+
+    kv0 = W.cfg5_kv()
+    kv = _fit_pool(torch, W, kv0, 4000 * kv0.block_bytes)
+    per = 4000 if kv.num_blocks == kv0.num_blocks else (kv.num_blocks // 32) // 4 * 4
+    n_get, n_put = per * 3 // 4, per // 4
+    pool = torch.empty(kv.pool_bytes, dtype=torch.uint8, device="cuda")
+    synth.fill_pool(pool, kv)
+    get_buf = torch.empty(n_get * kv.block_bytes, dtype=torch.uint8, device="cuda")
+    put_buf = torch.empty(n_put * kv.block_bytes, dtype=torch.uint8, device="cuda")
+    synth.fill_linear(put_buf, 77)
+    lay = aibx.KVLayout(kv.layout, kv.num_layers, kv.num_kv_heads, kv.block_tokens, kv.head_dim,
+                        kv.elem_bytes, kv.num_blocks)
+    tables = [torch.from_numpy((r * per + W.Stream(4, 100 + r).permutation(per)).astype(np.uint32)).cuda()
+              for r in range(32)]
+    for r in range(2):
+        aibx.kv_gather(pool, lay, tables[r][:n_get].contiguous(), n_get, get_buf)
+    torch.cuda.synchronize()
+    t_get, t_put = [], []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for r in range(32):
+        a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        ids_get, ids_put = tables[r][:n_get].contiguous(), tables[r][n_get:].contiguous()
+        a.record()
+        aibx.kv_gather(pool, lay, ids_get, n_get, get_buf)
+        b.record()
+        aibx.kv_scatter(pool, lay, ids_put, n_put, put_buf)
+        c.record()
+        t_get.append((a, b))
+        t_put.append((b, c))
+    t1.record()
+    torch.cuda.synchronize()
+    g = [a.elapsed_time(b) for a, b in t_get]
+    p = [a.elapsed_time(b) for a, b in t_put]
+    gb, pb = 2 * n_get * kv.block_bytes, 2 * n_put * kv.block_bytes
+    peak, kind = measured_peak_hbm()
+    total = (gb + pb) * 32 / (t0.elapsed_time(t1) * 1e-3) / 1e9
+    print(json.dumps({"case": "cfg5", "pool_blocks_effective": kv.num_blocks, "get_blocks": n_get,
+                      "put_blocks": n_put, "block_bytes": kv.block_bytes,
+                      "get_GBps_median": round(gb / (statistics.median(g) * 1e-3) / 1e9, 1),
+                      "put_GBps_median": round(pb / (statistics.median(p) * 1e-3) / 1e9, 1),
+                      "mixed_GBps_all_32_requests": round(total, 1),
+                      "frac_of_measured": round(total / peak, 4),
+                      "frac_of_nominal_8000": round(total / 8000.0, 4), "peak": peak,
+                      "peak_kind": kind, "status": aibx.status_fetch()}))
+
+
+def case_lookup_flat(args):
+    """Flat aibx_index_lookup of 2^24 keys, half of them present, against indexes of the four
+    configured sizes, cold (L2 evicted by a 256 MiB read before each launch) and warm; next to
+    it a plain random gather of 32-byte rows (torch.index_select) as the hardware's own ceiling
+    for this access pattern.  Algorithmic bytes per key: 8 in + 32 (one slot) + 12 out."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import workloads as W
+
+    n = 1 << 24
+    peak, kind = measured_peak_hbm()
+    flush = torch.empty(64 << 20, dtype=torch.int32, device="cuda")
+    out = []
+    for log2cap in (11, 19, 21, 23):
+        ix, keys = _big_index(torch, aibx, W, log2cap, 32, 20 + log2cap)
+        st = W.Stream(40, log2cap)
+        pick = st.randint(0, len(keys), n)
+        q = keys[pick]
+        miss = st.unit(n) < 0.5
+        q[miss] = st.keys(int(miss.sum()))
+        d_q = torch.from_numpy(q).cuda()
+        d_m = torch.empty(n, dtype=torch.uint64, device="cuda")
+        d_i = torch.empty(n, dtype=torch.uint32, device="cuda")
+
+        def cold():
+            flush.sum()
+            ix.lookup(d_q, d_m, d_i)
+
+        t_flush = statistics.median(_event_times(torch, lambda: flush.sum(), 7, 2))
+        t_cold = statistics.median(_event_times(torch, cold, 7, 2)) - t_flush
+        t_warm = statistics.median(_event_times(torch, lambda: ix.lookup(d_q, d_m, d_i), 7, 2))
+        # comparator: gather the home rows of the same table size with a library kernel
+        table = torch.empty(((1 << log2cap), 4), dtype=torch.int64, device="cuda")
+        idx = torch.from_numpy(W.Stream(41, log2cap).randint(0, 1 << log2cap, n)).cuda()
+        dst = torch.empty((n, 4), dtype=torch.int64, device="cuda")
+        t_lib = statistics.median(_event_times(
+            torch, lambda: torch.index_select(table, 0, idx, out=dst), 7, 2))
+        nbytes = n * (8 + 32 + 12)
+        out.append({"slots": 1 << log2cap, "table_MiB": (32 << log2cap) >> 20,
+                    "cold_ms": round(t_cold, 4), "warm_ms": round(t_warm, 4),
+                    "cold_Glookups_per_s": round(n / (t_cold * 1e-3) / 1e9, 2),
+                    "warm_Glookups_per_s": round(n / (t_warm * 1e-3) / 1e9, 2),
+                    "cold_GBps": round(nbytes / (t_cold * 1e-3) / 1e9, 1),
+                    "warm_GBps": round(nbytes / (t_warm * 1e-3) / 1e9, 1),
+                    "cold_frac": round(nbytes / (t_cold * 1e-3) / 1e9 / peak, 4),
+                    "warm_frac": round(nbytes / (t_warm * 1e-3) / 1e9 / peak, 4),
+                    "torch_index_select_32B_rows_Grows_per_s": round(n / (t_lib * 1e-3) / 1e9, 2)})
+        ix.destroy()
+        del table, idx, dst
+    print(json.dumps({"case": "lookup_flat", "keys": n, "present": 0.5, "peak": peak,
+                      "peak_kind": kind, "results": out, "status": aibx.status_fetch()}))
+
+
+CASES = {"kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
+         "cfg4": case_cfg4, "cfg5": case_cfg5, "lookup_flat": case_lookup_flat}
 
 
 def main():

@@ -217,11 +217,17 @@ int32_t aibx_kv_scatter(void* d_pool, const aibx_kv_layout_t* layout,
 
 /* Launch shape of gather/scatter, process-wide; for measurement sweeps.  mode 0 = bulk-async
  * (TMA) ring through shared memory, 1 = 16-byte load/store loop.  chunk_bytes (multiple of 16,
- * 1 KiB..64 KiB) and stages (2..16) size the ring (chunk*stages <= 200 KiB); ctas_per_sm 1..8.
+ * 1 KiB..64 KiB) and stages (2..16) size the ring (chunk*stages <= 200 KiB; the stage count
+ * bounds the loads in flight per CTA); ctas_per_sm 1..8.
  * Any argument <= 0 keeps its current value.  INVALID on an out-of-range value.
  */
 int32_t aibx_kv_set_tuning(int32_t mode, int32_t chunk_bytes, int32_t stages,
                            int32_t ctas_per_sm);
+
+/* Bulk ring only, process-wide: how many store groups may still be reading shared memory
+ * before their stage is handed back to the loader (1..4; default 1).  INVALID otherwise.
+ */
+int32_t aibx_kv_set_store_lag(int32_t lag);
 
 /* ---------------------------------------------------------------------------------------
  * Device status of the current device: the most severe (most negative) code recorded by any

@@ -82,6 +82,7 @@ def lib():
             "aibx_kv_gather": [vp, C.POINTER(KVLayout), vp, i64, vp, vp],
             "aibx_kv_scatter": [vp, C.POINTER(KVLayout), vp, i64, vp, vp],
             "aibx_kv_set_tuning": [i32, i32, i32, i32],
+            "aibx_kv_set_store_lag": [i32],
             "aibx_status_fetch": [vp, C.POINTER(i32), C.POINTER(i64)],
         }
         for name, args in sig.items():
@@ -236,6 +237,10 @@ def kv_scatter(pool, layout: KVLayout, block_ids, n: int, buf) -> None:
 def kv_set_tuning(mode: int = -1, chunk_bytes: int = 0, stages: int = 0,
                   ctas_per_sm: int = 0) -> None:
     _check("aibx_kv_set_tuning", lib().aibx_kv_set_tuning(mode, chunk_bytes, stages, ctas_per_sm))
+
+
+def kv_set_store_lag(lag: int = 1) -> None:
+    _check("aibx_kv_set_store_lag", lib().aibx_kv_set_store_lag(lag))
 
 
 def status_fetch():

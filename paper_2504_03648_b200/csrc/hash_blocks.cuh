@@ -95,8 +95,8 @@ hash_blocks_kernel(const int32_t* __restrict__ tokens, const int64_t* __restrict
   // Groups of 8 stripes: `cur` feeds the chain while `nxt` is in flight.  Whole groups run
   // without per-stripe checks; only the last, partial group of a request is guarded.
   const int n = (int)n_stripes;
-  uint32_t cur_lo[kGroupStripes], cur_hi[kGroupStripes];
-  uint32_t nxt_lo[kGroupStripes], nxt_hi[kGroupStripes];
+  uint32_t cur_lo[kGroupStripes] = {}, cur_hi[kGroupStripes] = {};
+  uint32_t nxt_lo[kGroupStripes] = {}, nxt_hi[kGroupStripes] = {};
   auto fetch = [&](const int32_t* q, int avail, uint32_t* lo, uint32_t* hi) {
     if (avail >= kGroupStripes) {
 #pragma unroll

@@ -1,14 +1,19 @@
-// Paged-KV gather / scatter: whole (item, segment) runs of bytes moved verbatim between a
-// paged pool and a block-major transfer buffer.  A segment is the longest contiguous run both
-// sides share: the whole block for a block-major pool, one (layer, K/V) tile for a layer-major
-// pool.  Segments are cut into chunks; chunk c goes to CTA c mod grid, so at any moment the
-// SMs work on neighbouring addresses.
+// Paged-KV gather / scatter: bytes moved verbatim between a paged pool and a block-major
+// transfer buffer.
+//
+// The buffer side of a call is one contiguous byte stream (item 0 layer 0, item 0 layer 1, ...).
+// It is cut into fixed-size chunks; chunk c goes to CTA c mod grid, so at any moment the SMs
+// work on neighbouring addresses.  On the pool side a chunk is 1..4 "pieces": runs inside one
+// segment, where a segment is the longest contiguous run both sides share (the whole block for
+// a block-major pool, one layer's K/V tile for a layer-major pool).  Cutting the stream rather
+// than the segments keeps every iteration at full size whatever the tile size is.
 //
 // Two copy engines, same chunk schedule:
-//   bulk ring (default): one thread per CTA drives a ring of shared-memory stages with
-//       cp.async.bulk (global -> shared, completion on an mbarrier) and cp.async.bulk
-//       (shared -> global, bulk groups).  No register or L1 traffic, ~S-1 chunks of loads in
-//       flight per SM.  Every wait is bounded and reports AIBX_ERR_TIMEOUT instead of hanging.
+//   bulk ring (default): a loader thread and a storer thread per CTA drive a ring of
+//       shared-memory stages with cp.async.bulk (global -> shared, completion on an mbarrier)
+//       and cp.async.bulk (shared -> global, bulk groups).  No register or L1 traffic.  The
+//       block ids of the next chunk are requested one iteration early so the issue loop never
+//       waits for them.  Every wait is bounded and reports AIBX_ERR_TIMEOUT instead of hanging.
 //   ld/st loop: 16-byte streaming loads and stores, four in flight per thread.
 // Bound: HBM bandwidth, 2 bytes of traffic per byte copied.
 #pragma once
@@ -17,52 +22,69 @@
 
 namespace aibx {
 
+constexpr int kMaxPieces = 4;
+
+// All sizes below are in units of 16 bytes so that they fit 32-bit arithmetic.
 struct CopyPlan {
   const uint32_t* ids;
-  char* pool;                 // paged side
-  char* buf;                  // contiguous side
-  long long n_items;
-  long long segs_per_item;
-  long long seg_bytes;
-  long long pool_item_stride; // bytes between consecutive block ids in the pool
-  long long pool_seg_stride;  // bytes between consecutive segments of one block in the pool
-  long long chunk_bytes;
-  long long chunks_per_seg;
-  long long total_chunks;
+  char* pool;                    // paged side
+  char* buf;                     // contiguous side
+  long long pool_item_stride;    // bytes between consecutive block ids in the pool
+  long long pool_seg_stride;     // bytes between consecutive segments of one block in the pool
+  unsigned int segs_per_item;
+  unsigned int seg_units;        // segment length
+  unsigned int chunk_units;      // chunk length (a whole number of segments when shorter)
+  unsigned int total_units;      // whole stream of this launch (< 2^32 - 2^22)
+  unsigned int total_chunks;
   uint32_t num_blocks;
-  int to_pool;                // 0 gather (pool -> buf), 1 scatter (buf -> pool)
+  int to_pool;                   // 0 gather (pool -> buf), 1 scatter (buf -> pool)
 };
 
-struct ChunkAddr {
-  const char* src;
-  char* dst;
-  unsigned int bytes;         // 0: nothing to copy (skipped item)
+// A chunk before its block ids are known: where its pieces lie in the stream.
+struct ChunkPieces {
+  int np;
+  unsigned int item[kMaxPieces];
+  unsigned int seg[kMaxPieces];
+  unsigned int off[kMaxPieces];        // offset inside the segment
+  unsigned int len[kMaxPieces];
+  unsigned int stream0;                // first unit of the chunk in the stream
 };
 
-__device__ __forceinline__ ChunkAddr chunk_address(const CopyPlan& pl, long long c) {
-  const long long per_item = pl.segs_per_item * pl.chunks_per_seg;
-  const long long item = c / per_item;
-  const long long rem = c - item * per_item;
-  const long long seg = rem / pl.chunks_per_seg;
-  const long long k = rem - seg * pl.chunks_per_seg;
-  const long long off = k * pl.chunk_bytes;
-  const long long len = min(pl.chunk_bytes, pl.seg_bytes - off);
-  ChunkAddr a;
-  a.src = nullptr;
-  a.dst = nullptr;
-  a.bytes = 0;
-  const uint32_t id = __ldg(pl.ids + item);
-  if (id >= pl.num_blocks) {
-    // one report per offending item, from the thread that owns its first chunk
-    if (id != AIBX_NO_BLOCK && rem == 0) raise_status(AIBX_ERR_RANGE);
-    return a;
+__device__ __forceinline__ void chunk_pieces(const CopyPlan& pl, unsigned int c, ChunkPieces& cp) {
+  unsigned int u0 = c * pl.chunk_units;
+  const unsigned int u1 = min(u0 + pl.chunk_units, pl.total_units);
+  unsigned int q = u0 / pl.seg_units;                 // flat segment index
+  unsigned int off = u0 - q * pl.seg_units;
+  cp.stream0 = u0;
+  cp.np = 0;
+#pragma unroll
+  for (int p = 0; p < kMaxPieces; ++p) {
+    cp.len[p] = 0;
+    if (u0 < u1) {
+      const unsigned int len = min(pl.seg_units - off, u1 - u0);
+      const unsigned int item = q / pl.segs_per_item;
+      cp.item[p] = item;
+      cp.seg[p] = q - item * pl.segs_per_item;
+      cp.off[p] = off;
+      cp.len[p] = len;
+      cp.np = p + 1;
+      u0 += len;
+      ++q;
+      off = 0;
+    }
   }
-  char* in_pool = pl.pool + (long long)id * pl.pool_item_stride + seg * pl.pool_seg_stride + off;
-  char* in_buf = pl.buf + (item * pl.segs_per_item + seg) * pl.seg_bytes + off;
-  a.src = pl.to_pool ? in_buf : in_pool;
-  a.dst = pl.to_pool ? in_pool : in_buf;
-  a.bytes = (unsigned int)len;
-  return a;
+}
+
+// Pool-side address of piece p, or nullptr when its block id says "skip".
+__device__ __forceinline__ char* piece_pool_ptr(const CopyPlan& pl, const ChunkPieces& cp, int p,
+                                                uint32_t id) {
+  if (id >= pl.num_blocks) {
+    // one report per offending item, from the piece that starts the item
+    if (id != AIBX_NO_BLOCK && cp.seg[p] == 0 && cp.off[p] == 0) raise_status(AIBX_ERR_RANGE);
+    return nullptr;
+  }
+  return pl.pool + (long long)id * pl.pool_item_stride +
+         (long long)cp.seg[p] * pl.pool_seg_stride + (long long)cp.off[p] * 16;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -121,81 +143,186 @@ __device__ __forceinline__ void bulk_wait_all() {
   asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
-// One thread per CTA runs the whole ring.  Stage s holds chunk j with j mod S == s.
-//   load(j)  : expect_tx + bulk load into stage, or a bare arrive when the chunk is skipped
-//   store(j) : after the stage's barrier flips, bulk store out of it and commit a group
-//   refill   : stage of chunk j-1 is loaded with chunk j-1+S once all groups but the newest
-//              have finished READING shared memory
-__global__ void __launch_bounds__(32, 1) kv_copy_bulk_kernel(CopyPlan pl, int stages) {
+// Two threads per CTA run the ring, one per warp, so that neither waits for the other's
+// instruction latency.  Stage s holds chunk j with j mod S == s.
+//   loader (warp 0): waits until the stage is free (empty barrier), then expect_tx + one bulk
+//       load per piece, or a bare arrive when all pieces are skipped.  It also writes where the
+//       pieces have to go; the arrive on the full barrier publishes that to the storer.
+//   storer (warp 1): waits for the full barrier, issues one bulk store per piece, commits a
+//       group, and once the group of `lag` iterations ago has finished READING shared memory
+//       hands that stage back through its empty barrier.
+// Loads in flight are bounded by the number of stages: that is the knob that keeps the bytes in
+// flight near the bandwidth-delay product (more than that lowers the achieved bandwidth).
+// Every wait is bounded; whoever gives up raises the abort flag so the other side stops too,
+// and the storer waits (bounded) for the loads already issued before the CTA retires.
+constexpr int kRoleThreads = 64;
+
+__device__ __forceinline__ bool bounded_wait(unsigned int bar, unsigned int parity,
+                                             volatile int* abort_flag) {
+  unsigned int spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if (++spins > kWaitSpins || ((spins & 1023u) == 0 && *abort_flag)) return false;
+  }
+  return true;
+}
+
+__global__ void __launch_bounds__(kRoleThreads, 1)
+kv_copy_bulk_kernel(CopyPlan pl, int stages, int lag) {
   extern __shared__ __align__(128) unsigned char s_mem[];
-  __shared__ __align__(8) unsigned long long s_bar[kMaxStages];
-  __shared__ char* s_dst[kMaxStages];
-  __shared__ unsigned int s_len[kMaxStages];
+  __shared__ __align__(8) unsigned long long s_full[kMaxStages];
+  __shared__ __align__(8) unsigned long long s_empty[kMaxStages];
+  __shared__ char* s_out[kMaxStages][kMaxPieces];          // store destination of each piece
+  __shared__ unsigned int s_off[kMaxStages][kMaxPieces];   // its byte offset inside the stage
+  __shared__ unsigned int s_len[kMaxStages][kMaxPieces];   // its bytes (0: skipped)
+  __shared__ int s_abort;
+  __shared__ int s_loader_done;
+  __shared__ long long s_issued;
 
-  if (threadIdx.x != 0) return;
-
-  const long long G = gridDim.x;
-  const long long first = blockIdx.x;
+  const unsigned int G = gridDim.x;
+  const unsigned int first = blockIdx.x;
   if (first >= pl.total_chunks) return;
   const long long n_my = (pl.total_chunks - first + G - 1) / G;
-  const unsigned int stage_bytes = (unsigned int)pl.chunk_bytes;
+  const unsigned int stage_bytes = pl.chunk_units * 16u;
   const unsigned int smem0 = smem_u32(s_mem);
 
-  for (int s = 0; s < stages; ++s) mbar_init(smem_u32(&s_bar[s]), 1u);
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-
-  auto load = [&](long long j) {
-    const int s = (int)(j % stages);
-    const ChunkAddr a = chunk_address(pl, first + j * G);
-    s_dst[s] = a.dst;
-    s_len[s] = a.bytes;
-    const unsigned int bar = smem_u32(&s_bar[s]);
-    if (a.bytes) {
-      mbar_arrive_expect_tx(bar, a.bytes);
-      bulk_load(smem0 + (unsigned int)s * stage_bytes, a.src, a.bytes, bar);
-    } else {
-      mbar_arrive(bar);
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&s_full[s]), 1u);
+      mbar_init(smem_u32(&s_empty[s]), 1u);
     }
-  };
+    s_abort = 0;
+    s_loader_done = 0;
+    s_issued = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  volatile int* abort_flag = &s_abort;
 
-  long long issued = 0;
-  for (; issued < n_my && issued < stages; ++issued) load(issued);
-
-  bool timed_out = false;
-  for (long long j = 0; j < n_my; ++j) {
-    const int s = (int)(j % stages);
-    const unsigned int parity = (unsigned int)((j / stages) & 1);
-    const unsigned int bar = smem_u32(&s_bar[s]);
-    unsigned int spins = 0;
-    while (!mbar_try_wait(bar, parity)) {
-      if (++spins > kWaitSpins) {
-        timed_out = true;
+  if (threadIdx.x < 32) {
+    // ------------------------------------------------------------------ loader warp
+    // A lone thread runs at a fraction of an instruction per cycle, so the address work is
+    // done 32 chunks at a time, one chunk per lane; only the few instructions that arm the
+    // barrier and start the copies are taken in turn, in chunk order.
+    const int lane = threadIdx.x;
+    bool stop = false;
+    for (long long base = 0; base < n_my && !stop; base += 32) {
+      const long long j = base + lane;
+      const char* src[kMaxPieces];
+      char* out[kMaxPieces];
+      unsigned int offs[kMaxPieces], lens[kMaxPieces];
+      unsigned int total = 0;
+      if (j < n_my) {
+        ChunkPieces cp;
+        chunk_pieces(pl, first + (unsigned int)j * G, cp);
+        char* buf_at = pl.buf + (long long)cp.stream0 * 16;
+        unsigned int soff = 0;
+#pragma unroll
+        for (int p = 0; p < kMaxPieces; ++p) {
+          src[p] = nullptr;
+          out[p] = nullptr;
+          offs[p] = soff;
+          lens[p] = 0;
+          if (p < cp.np) {
+            char* in_pool = piece_pool_ptr(pl, cp, p, __ldg(pl.ids + cp.item[p]));
+            if (in_pool) {
+              lens[p] = cp.len[p] * 16u;
+              src[p] = pl.to_pool ? buf_at + soff : in_pool;
+              out[p] = pl.to_pool ? in_pool : buf_at + soff;
+            }
+            soff += cp.len[p] * 16u;
+          }
+          total += lens[p];
+        }
+      }
+      const int turns = (int)min((long long)32, n_my - base);
+      for (int i = 0; i < turns; ++i) {
+        if (lane == i) {
+          const int s = (int)(j % stages);
+          bool ok = !*abort_flag;
+          if (ok && j >= stages) {
+            // the storer frees stage s once the store of chunk j - stages left shared memory
+            ok = bounded_wait(smem_u32(&s_empty[s]), (unsigned int)(((j / stages) - 1) & 1),
+                              abort_flag);
+            if (!ok && !*abort_flag) raise_status(AIBX_ERR_TIMEOUT);
+          }
+          if (ok) {
+            const unsigned int stage0 = smem0 + (unsigned int)s * stage_bytes;
+            const unsigned int bar = smem_u32(&s_full[s]);
+#pragma unroll
+            for (int p = 0; p < kMaxPieces; ++p) {
+              s_out[s][p] = out[p];
+              s_off[s][p] = offs[p];
+              s_len[s][p] = lens[p];
+            }
+            *reinterpret_cast<volatile long long*>(&s_issued) = j + 1;
+            if (total) {
+              mbar_arrive_expect_tx(bar, total);
+#pragma unroll
+              for (int p = 0; p < kMaxPieces; ++p)
+                if (lens[p]) bulk_load(stage0 + offs[p], src[p], lens[p], bar);
+            } else {
+              mbar_arrive(bar);
+            }
+          } else {
+            *abort_flag = 1;
+          }
+        }
+        __syncwarp();
+        if (*abort_flag) {
+          stop = true;
+          break;
+        }
+      }
+    }
+    if (lane == 0) *reinterpret_cast<volatile int*>(&s_loader_done) = 1;
+  } else if (threadIdx.x == 32) {
+    // ------------------------------------------------------------------ storer
+    if (lag < 1) lag = 1;
+    if (lag > stages - 1) lag = stages - 1;
+    if (lag > 4) lag = 4;
+    long long j = 0;
+    bool gave_up = false;
+    for (; j < n_my; ++j) {
+      const int s = (int)(j % stages);
+      if (!bounded_wait(smem_u32(&s_full[s]), (unsigned int)((j / stages) & 1), abort_flag)) {
+        gave_up = true;
         break;
       }
-    }
-    if (timed_out) break;
-    if (s_len[s]) bulk_store(s_dst[s], smem0 + (unsigned int)s * stage_bytes, s_len[s]);
-    bulk_commit();
-    if (j >= 1 && issued < n_my) {
-      bulk_wait_read<1>();        // store of chunk j-1 no longer reads its stage
-      load(issued);
-      ++issued;
-    }
-  }
-  bulk_wait_all();
-  if (timed_out) {
-    // Loads still in flight target this CTA's shared memory: give them a bounded time to
-    // land before the CTA retires, then report.
-    for (long long j = 0; j < issued; ++j) {
-      const int s = (int)(j % stages);
-      if (j + stages < issued) continue;      // only the newest phase of each stage
-      const unsigned int parity = (unsigned int)((j / stages) & 1);
-      unsigned int spins = 0;
-      while (!mbar_try_wait(smem_u32(&s_bar[s]), parity) && ++spins < kWaitSpins) {
+      const unsigned int stage0 = smem0 + (unsigned int)s * stage_bytes;
+#pragma unroll
+      for (int p = 0; p < kMaxPieces; ++p) {
+        const unsigned int bytes = s_len[s][p];
+        if (bytes) bulk_store(s_out[s][p], stage0 + s_off[s][p], bytes);
+      }
+      bulk_commit();
+      if (j >= lag) {
+        // all groups but the newest `lag` have finished reading: chunk j - lag's stage is free
+        if (lag >= 4) bulk_wait_read<4>();
+        else if (lag == 3) bulk_wait_read<3>();
+        else if (lag == 2) bulk_wait_read<2>();
+        else bulk_wait_read<1>();
+        mbar_arrive(smem_u32(&s_empty[(int)((j - lag) % stages)]));
       }
     }
-    raise_status(AIBX_ERR_TIMEOUT);
+    bulk_wait_all();
+    if (gave_up) {
+      if (!*abort_flag) raise_status(AIBX_ERR_TIMEOUT);
+      *abort_flag = 1;
+      // Loads already issued still target this CTA's shared memory: once the loader has
+      // stopped, give them a bounded time to land before the CTA retires.
+      for (unsigned int spins = 0;
+           !*reinterpret_cast<volatile int*>(&s_loader_done) && spins < kWaitSpins; ++spins) {
+      }
+      const long long issued = *reinterpret_cast<volatile long long*>(&s_issued);
+      for (long long i = j; i < issued; ++i) {
+        unsigned int spins = 0;
+        while (!mbar_try_wait(smem_u32(&s_full[(int)(i % stages)]),
+                              (unsigned int)((i / stages) & 1)) &&
+               ++spins < kWaitSpins) {
+        }
+      }
+    }
   }
 }
 
@@ -205,28 +332,49 @@ __global__ void __launch_bounds__(32, 1) kv_copy_bulk_kernel(CopyPlan pl, int st
 constexpr int kLdstThreads = 256;
 
 __global__ void __launch_bounds__(kLdstThreads) kv_copy_ldst_kernel(CopyPlan pl) {
-  __shared__ ChunkAddr s_addr;
-  for (long long c = blockIdx.x; c < pl.total_chunks; c += gridDim.x) {
-    if (threadIdx.x == 0) s_addr = chunk_address(pl, c);
-    __syncthreads();
-    const ChunkAddr a = s_addr;
-    __syncthreads();
-    if (a.bytes == 0) continue;
-    const uint4* src = reinterpret_cast<const uint4*>(a.src);
-    uint4* dst = reinterpret_cast<uint4*>(a.dst);
-    const unsigned int nv = a.bytes >> 4;
-    for (unsigned int v = threadIdx.x; v < nv; v += 4 * kLdstThreads) {
-      uint4 r0, r1, r2, r3;
-      const unsigned int v1 = v + kLdstThreads, v2 = v + 2 * kLdstThreads, v3 = v + 3 * kLdstThreads;
-      r0 = __ldcs(src + v);
-      if (v1 < nv) r1 = __ldcs(src + v1);
-      if (v2 < nv) r2 = __ldcs(src + v2);
-      if (v3 < nv) r3 = __ldcs(src + v3);
-      __stcs(dst + v, r0);
-      if (v1 < nv) __stcs(dst + v1, r1);
-      if (v2 < nv) __stcs(dst + v2, r2);
-      if (v3 < nv) __stcs(dst + v3, r3);
+  __shared__ const char* s_src[kMaxPieces];
+  __shared__ char* s_dst[kMaxPieces];
+  __shared__ unsigned int s_units[kMaxPieces];
+  for (unsigned int c = blockIdx.x; c < pl.total_chunks; c += gridDim.x) {
+    if (threadIdx.x == 0) {
+      ChunkPieces cp;
+      chunk_pieces(pl, c, cp);
+      char* buf_at = pl.buf + (long long)cp.stream0 * 16;
+      unsigned int soff = 0;
+      for (int p = 0; p < kMaxPieces; ++p) {
+        s_units[p] = 0;
+        if (p < cp.np) {
+          char* in_pool = piece_pool_ptr(pl, cp, p, __ldg(pl.ids + cp.item[p]));
+          if (in_pool) {
+            s_units[p] = cp.len[p];
+            s_src[p] = pl.to_pool ? buf_at + soff : in_pool;
+            s_dst[p] = pl.to_pool ? in_pool : buf_at + soff;
+          }
+          soff += cp.len[p] * 16u;
+        }
+      }
     }
+    __syncthreads();
+    for (int p = 0; p < kMaxPieces; ++p) {
+      const unsigned int nv = s_units[p];
+      if (nv == 0) continue;
+      const uint4* src = reinterpret_cast<const uint4*>(s_src[p]);
+      uint4* dst = reinterpret_cast<uint4*>(s_dst[p]);
+      for (unsigned int v = threadIdx.x; v < nv; v += 4 * kLdstThreads) {
+        uint4 r0, r1, r2, r3;
+        const unsigned int v1 = v + kLdstThreads, v2 = v + 2 * kLdstThreads,
+                           v3 = v + 3 * kLdstThreads;
+        r0 = __ldcs(src + v);
+        if (v1 < nv) r1 = __ldcs(src + v1);
+        if (v2 < nv) r2 = __ldcs(src + v2);
+        if (v3 < nv) r3 = __ldcs(src + v3);
+        __stcs(dst + v, r0);
+        if (v1 < nv) __stcs(dst + v1, r1);
+        if (v2 < nv) __stcs(dst + v2, r2);
+        if (v3 < nv) __stcs(dst + v3, r3);
+      }
+    }
+    __syncthreads();
   }
 }
 
@@ -235,9 +383,10 @@ __global__ void __launch_bounds__(kLdstThreads) kv_copy_ldst_kernel(CopyPlan pl)
 
 struct CopyTuning {
   int mode = 0;            // 0 bulk ring, 1 ld/st loop
-  int chunk_bytes = 16384;
-  int stages = 12;
+  int chunk_bytes = 32768;
+  int stages = 3;
   int ctas_per_sm = 1;
+  int lag = 1;             // store groups that may still read shared memory (1..4)
 };
 
 inline CopyTuning& copy_tuning() {
@@ -258,47 +407,58 @@ inline int32_t launch_kv_copy(const void* pool, const aibx_kv_layout_t* L, const
   const long long tile = 2LL * L->num_kv_heads * L->block_tokens * L->head_dim * L->elem_bytes;
   if (tile % 16 != 0) return AIBX_ERR_UNSUPPORTED;
   const long long block_bytes = tile * L->num_layers;
+  const long long seg_bytes = L->layout == 0 ? block_bytes : tile;
+  const long long segs = L->layout == 0 ? 1 : L->num_layers;
+  if (seg_bytes / 16 >= (1LL << 31) || block_bytes / 16 >= (1LL << 31)) return AIBX_ERR_UNSUPPORTED;
 
   const CopyTuning& tn = copy_tuning();
   CopyPlan pl;
-  pl.ids = d_ids;
-  pl.pool = const_cast<char*>(static_cast<const char*>(pool));
-  pl.buf = const_cast<char*>(static_cast<const char*>(buf));
-  pl.n_items = n;
   pl.num_blocks = L->num_blocks;
   pl.to_pool = to_pool;
-  if (L->layout == 0) {
-    pl.segs_per_item = 1;
-    pl.seg_bytes = block_bytes;
-    pl.pool_item_stride = block_bytes;
-    pl.pool_seg_stride = 0;
+  pl.segs_per_item = (unsigned int)segs;
+  pl.seg_units = (unsigned int)(seg_bytes / 16);
+  pl.pool_item_stride = L->layout == 0 ? block_bytes : tile;
+  pl.pool_seg_stride = L->layout == 0 ? 0 : (long long)L->num_blocks * tile;
+  // chunk: the tuned size, or a whole number of segments when segments are shorter than that
+  if (seg_bytes >= tn.chunk_bytes) {
+    pl.chunk_units = (unsigned int)(tn.chunk_bytes / 16);
   } else {
-    pl.segs_per_item = L->num_layers;
-    pl.seg_bytes = tile;
-    pl.pool_item_stride = tile;
-    pl.pool_seg_stride = (long long)L->num_blocks * tile;
+    long long m = tn.chunk_bytes / seg_bytes;
+    if (m > kMaxPieces) m = kMaxPieces;
+    pl.chunk_units = (unsigned int)(m * pl.seg_units);
   }
-  pl.chunk_bytes = tn.chunk_bytes;
-  pl.chunks_per_seg = (pl.seg_bytes + pl.chunk_bytes - 1) / pl.chunk_bytes;
-  pl.total_chunks = pl.n_items * pl.segs_per_item * pl.chunks_per_seg;
 
-  long long grid = (long long)sm_count() * (tn.mode == 0 ? tn.ctas_per_sm : 8);
-  if (grid > pl.total_chunks) grid = pl.total_chunks;
-
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AIBX_ERR_CUDA;
+  const size_t smem = (size_t)tn.stages * tn.chunk_bytes;
   if (tn.mode == 0) {
-    const size_t smem = (size_t)tn.stages * tn.chunk_bytes;
     static size_t configured[64] = {0};   // per device: the attribute lives in the context
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AIBX_ERR_CUDA;
     if (smem > configured[dev]) {
       if (cudaFuncSetAttribute(kv_copy_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                (int)smem) != cudaSuccess)
         return AIBX_ERR_CUDA;
       configured[dev] = smem;
     }
-    kv_copy_bulk_kernel<<<(unsigned int)grid, 32, smem, st>>>(pl, tn.stages);
-  } else {
-    kv_copy_ldst_kernel<<<(unsigned int)grid, kLdstThreads, 0, st>>>(pl);
+  }
+
+  // 32-bit stream offsets: one launch covers at most ~64 GiB; longer lists take several
+  const long long units_per_item = block_bytes / 16;
+  long long max_items = ((1LL << 32) - (1LL << 22)) / units_per_item;
+  if (max_items < 1) max_items = 1;
+  for (int64_t done = 0; done < n; done += max_items) {
+    const long long items = (n - done < max_items) ? (n - done) : max_items;
+    pl.ids = d_ids + done;
+    pl.pool = const_cast<char*>(static_cast<const char*>(pool));
+    pl.buf = const_cast<char*>(static_cast<const char*>(buf)) + done * block_bytes;
+    pl.total_units = (unsigned int)(items * units_per_item);
+    pl.total_chunks = (pl.total_units + pl.chunk_units - 1) / pl.chunk_units;
+    long long grid = (long long)sm_count() * (tn.mode == 0 ? tn.ctas_per_sm : 8);
+    if (grid > pl.total_chunks) grid = pl.total_chunks;
+    if (tn.mode == 0) {
+      kv_copy_bulk_kernel<<<(unsigned int)grid, kRoleThreads, smem, st>>>(pl, tn.stages, tn.lag);
+    } else {
+      kv_copy_ldst_kernel<<<(unsigned int)grid, kLdstThreads, 0, st>>>(pl);
+    }
   }
   return launch_status();
 }

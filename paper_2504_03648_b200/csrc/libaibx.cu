@@ -289,6 +289,12 @@ int32_t aibx_kv_set_tuning(int32_t mode, int32_t chunk_bytes, int32_t stages,
   return AIBX_OK;
 }
 
+int32_t aibx_kv_set_store_lag(int32_t lag) {
+  if (lag < 1 || lag > 4) return AIBX_ERR_INVALID;
+  copy_tuning().lag = lag;
+  return AIBX_OK;
+}
+
 int32_t aibx_status_fetch(void* stream, int32_t* status, int64_t* detail) {
   StatusRecord* dev = status_ptr();
   if (!dev) return AIBX_ERR_CUDA;

@@ -20,9 +20,11 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(lib, name), name
     lib.aibx_strerror.restype = ctypes.c_char_p
     assert lib.aibx_strerror(-3) == b"index full"
-    assert lib.aibx_kv_set_tuning(0, 16384, 12, 1) == 0
+    assert lib.aibx_kv_set_tuning(0, 32768, 3, 1) == 0
     assert lib.aibx_kv_set_tuning(0, 100, 6, 1) == -1          # chunk not a multiple of 16
     assert lib.aibx_kv_set_tuning(0, 65536, 16, 1) == -1       # ring larger than shared memory
+    assert lib.aibx_kv_set_store_lag(0) == -1 and lib.aibx_kv_set_store_lag(5) == -1
+    assert lib.aibx_kv_set_store_lag(1) == 0
 
 
 def test_binding_has_no_fallback(monkeypatch):

@@ -18,9 +18,11 @@ GUARD = 4096
 
 @pytest.fixture(autouse=True)
 def _default_tuning():
-    aibx.kv_set_tuning(0, 16384, 12, 1)
+    aibx.kv_set_tuning(0, 32768, 3, 1)
+    aibx.kv_set_store_lag(1)
     yield
-    aibx.kv_set_tuning(0, 16384, 12, 1)
+    aibx.kv_set_tuning(0, 32768, 3, 1)
+    aibx.kv_set_store_lag(1)
 
 
 def guarded(n_bytes, fill):
@@ -35,7 +37,8 @@ def guards_intact(whole, n_bytes, fill):
 
 
 def check_gather_scatter(kv, ids_g, ids_s, mode_args):
-    aibx.kv_set_tuning(*mode_args)
+    aibx.kv_set_tuning(*mode_args[:4])
+    aibx.kv_set_store_lag(mode_args[4])
     pool_h = W.host_pool(kv)
     lay_g, lay_o = kv_layout_gpu(kv), kv_layout_oracle(kv)
     n = len(ids_g)
@@ -63,7 +66,9 @@ def check_gather_scatter(kv, ids_g, ids_s, mode_args):
     assert guards_intact(buf_w, buf_bytes, 0xEE) and guards_intact(pool_w, kv.pool_bytes, 0xA5)
 
 
-MODES = [(0, 16384, 12, 1), (0, 32768, 6, 1), (0, 4096, 3, 2), (0, 1024, 16, 1), (1, 16384, 2, 1), (0, 49152, 4, 1)]
+# (mode, chunk bytes, stages, CTAs per SM, store lag)
+MODES = [(0, 32768, 3, 1, 1), (0, 16384, 12, 1, 1), (0, 4096, 3, 2, 2), (0, 1024, 16, 1, 4), (1, 16384, 2, 1, 1),
+         (0, 49152, 4, 1, 2), (0, 14848, 5, 1, 1), (0, 2048, 2, 1, 1)]
 
 
 @pytest.mark.parametrize("mode_args", MODES)
@@ -90,6 +95,15 @@ def test_shapes_with_ragged_chunks(layout, mode_args):
     kv = W.KVSpec("mid", 6, layout, 5, 2, 16, 64, 2, 300)
     ids_g = W.distinct_ids(1, 300, 257)
     ids_s = W.distinct_ids(2, 300, 257)
+    check_gather_scatter(kv, ids_g, ids_s, mode_args)
+    # 12,800-byte tiles, 38,400-byte blocks: chunks straddle segments and items, with skipped
+    # and out-of-range ids in the middle of straddling chunks
+    kv = W.KVSpec("straddle", 7, layout, 3, 5, 16, 40, 2, 97)
+    ids_g = rng.integers(0, 97, 333).astype(np.uint32)
+    ids_g[rng.random(333) < 0.15] = NO_BLOCK
+    ids_g[[1, 100, 332]] = [97, 5000, 0xFFFFFFFE]
+    ids_s = np.concatenate([rng.permutation(97)[:90], [NO_BLOCK, 97, NO_BLOCK]]).astype(np.uint32)
+    rng.shuffle(ids_s)
     check_gather_scatter(kv, ids_g, ids_s, mode_args)
 
 
