@@ -296,6 +296,22 @@ class GpuJob:
         return out
 
 
+def max_over_ranks(value: float, dist, device) -> float:
+    """Max of a per-rank scalar over all ranks (the timed interval of a multi-rank run)."""
+    if dist is None:
+        return float(value)
+    import torch
+
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(step_bytes_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Replicas only: every rank moves the same bytes; the job's rate uses the slowest rank."""
+    return world * step_bytes_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
 def run_gpu(args):
     import torch
 
@@ -335,10 +351,7 @@ def run_gpu(args):
     barrier()
     elapsed_ms = t0.elapsed_time(t1)
     clocks = sampler.stop() if rank == 0 else None
-    if dist is not None:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, dist, "cuda")
     status = job.aibx.status_fetch()
     assert status == (0, 0), status
 
@@ -363,10 +376,7 @@ def run_gpu(args):
         h2d, d2h = job.step_e2e()
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - w0) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(e2e_s, dist, "cuda")
 
     stages = job.stage_breakdown() if rank == 0 else None
     if dist is not None:
@@ -377,7 +387,7 @@ def run_gpu(args):
         return
 
     ms_per_step = elapsed_ms / args.steps
-    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_value(step_bytes, world, ms_per_step)
     cpu = cpu_baseline(budget_s=12.0)
     line = {
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world,
@@ -617,7 +627,7 @@ def case_match_cfg(args):
     from paper_2504_03648_b200 import workloads as W
 
     res = []
-    for mk in (W.cfg3_routing, W.cfg5_routing):
+    for mk in (W.cfg2_routing, W.cfg3_routing, W.cfg5_routing):
         w = W.build_routing(mk())
         s = w.spec
         B, P, R = s.block_tokens, s.num_pods, s.R
@@ -637,9 +647,16 @@ def case_match_cfg(args):
         d_sh = torch.empty(int(sbo[-1]), dtype=torch.uint64, device="cuda")
         aibx.hash_blocks(dev(w.src_tokens), dev(w.src_tok_off), dev(sbo), B, 0, d_sh)
         ix = aibx.Index(s.capacity, P)
-        ix.insert(torch.cat([d_sh, dev(w.filler_keys)]),
-                  dev(np.concatenate([w.src_masks, w.filler_masks])),
-                  dev(np.concatenate([w.src_ids, w.filler_ids])))
+        d_keys = torch.cat([d_sh, dev(w.filler_keys)])
+        d_masks = dev(np.concatenate([w.src_masks, w.filler_masks]))
+        d_eids = dev(np.concatenate([w.src_ids, w.filler_ids]))
+
+        def refill():
+            ix.clear()
+            ix.insert(d_keys, d_masks, d_eids)
+
+        t_clear = statistics.median(_event_times(torch, lambda: ix.clear(), 5, 2))
+        t_fill = statistics.median(_event_times(torch, refill, 5, 2)) - t_clear
         d_ml = torch.empty(R * P, dtype=torch.uint32, device="cuda")
         d_al = torch.empty(R, dtype=torch.uint32, device="cuda")
         d_ids = torch.empty(int(bo[-1]), dtype=torch.uint32, device="cuda")
@@ -658,6 +675,9 @@ def case_match_cfg(args):
         lookups = int(np.minimum(al + 1, n_r).sum())
         nbytes = lookups * 40 + int((4 * P + 4) * R + 4 * al.sum())
         res.append({"config": s.name, "R": R, "blocks": int(bo[-1]), "necessary_lookups": lookups,
+                    "index_entries": int(d_keys.numel()),
+                    "insert_us": round(t_fill * 1e3, 1),
+                    "insert_Mkeys_per_s": round(d_keys.numel() / (t_fill * 1e-3) / 1e6, 1),
                     "hash_us": round(t_hash * 1e3, 1), "match_us": round(t_match * 1e3, 1),
                     "score_us": round(t_score * 1e3, 1),
                     "hash_tokens_per_s": round(len(w.tokens) / (t_hash * 1e-3), 0),
@@ -834,7 +854,65 @@ def case_lookup_flat(args):
                       "peak_kind": kind, "results": out, "status": aibx.status_fetch()}))
 
 
-CASES = {"kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
+def case_oracle_cfg(args):
+    """The CPU oracle, one host core, on the routing halves of cfg2 / cfg3 / cfg5 at full size
+    and on gather+scatter of 128 blocks of each KV shape (pool of 256 blocks on the host)."""
+    import oracle
+    from paper_2504_03648_b200 import workloads as W
+
+    def clock(fn, reps=3):
+        ts = []
+        for _ in range(reps):
+            t0 = time.perf_counter()
+            fn()
+            ts.append(time.perf_counter() - t0)
+        return min(ts)
+
+    res = []
+    for mk in (W.cfg2_routing, W.cfg3_routing, W.cfg5_routing):
+        w = W.build_routing(mk())
+        s = w.spec
+        t_hash = clock(lambda: oracle.hash_blocks(w.tokens, w.tok_off, s.block_tokens, 0))
+        h, bo = oracle.hash_blocks(w.tokens, w.tok_off, s.block_tokens, 0)
+        sh, _ = oracle.hash_blocks(w.src_tokens, w.src_tok_off, s.block_tokens, 0)
+        keys = np.concatenate([sh, w.filler_keys])
+        masks = np.concatenate([w.src_masks, w.filler_masks])
+        ids = np.concatenate([w.src_ids, w.filler_ids])
+        ix = oracle.Index(s.capacity, s.num_pods)
+        t0 = time.perf_counter()
+        ix.insert(keys, masks, ids)
+        t_ins = time.perf_counter() - t0
+        t_match = clock(lambda: ix.match_prefix(h, bo))
+        ml, al, _ = ix.match_prefix(h, bo)
+        t_score = clock(lambda: oracle.route_score(ml, bo, w.pod_load, w.ready_mask, None))
+        res.append({"config": s.name, "hash_us": round(t_hash * 1e6, 1),
+                    "insert_us": round(t_ins * 1e6, 1), "match_us": round(t_match * 1e6, 1),
+                    "score_us": round(t_score * 1e6, 1)})
+    for kv0 in (W.cfg2_kv(), W.cfg4_kv(), W.cfg5_kv()):
+        kv = W.scaled(kv0, num_blocks=256)
+        pool = W.host_pool(kv)
+        lay = oracle.kv_layout(kv.layout, kv.num_layers, kv.num_kv_heads, kv.block_tokens,
+                               kv.head_dim, kv.elem_bytes, kv.num_blocks)
+        ids = W.distinct_ids(5, 256, 128)
+        buf = np.zeros(128 * kv.block_bytes, dtype=np.uint8)
+        tg = clock(lambda: oracle.kv_gather(pool, lay, ids, buf))
+        ts = clock(lambda: oracle.kv_scatter(pool, lay, ids, buf))
+        nb = 2 * 128 * kv.block_bytes
+        res.append({"config": kv0.name, "gather_GBps": round(nb / tg / 1e9, 2),
+                    "scatter_GBps": round(nb / ts / 1e9, 2)})
+    cpu = ""
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                cpu = line.split(":", 1)[1].strip()
+                break
+    except OSError:
+        pass
+    print(json.dumps({"case": "oracle_cfg", "cores_used": 1,
+                      "cores_available": len(os.sched_getaffinity(0)), "cpu": cpu, "results": res}))
+
+
+CASES = {"oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
          "cfg4": case_cfg4, "cfg5": case_cfg5, "lookup_flat": case_lookup_flat}
 
 

@@ -3,8 +3,9 @@
 //
 //   insert / evict : one thread per item, atomics only (results are order-free by construction)
 //   lookup         : one thread per key
-//   match_prefix   : a warp probes 32 consecutive blocks of a request at once; ballots find the
-//                    first block each pod misses; warps of one request combine through
+//   match_prefix   : a warp probes 32 consecutive blocks of a request at once; a ballot finds
+//                    the first total miss and a prefix-AND over the lanes finds, per pod, the
+//                    first block that lacks it; warps of one request combine through
 //                    shared-memory minima and stop once an earlier total miss is known.
 #pragma once
 
@@ -252,16 +253,34 @@ __global__ void match_prefix_kernel(IndexView ix, const uint64_t* __restrict__ h
       if (valid && block_ids) block_ids[off + i] = id;
       const unsigned int none = __ballot_sync(0xffffffffu, valid && mask == 0);
       if (none && lane == 0) atomicMin(&sh.first_none, base + (unsigned int)__ffs(none) - 1u);
-      // pods missing somewhere in this chunk: complement of the AND over valid lanes
-      const uint64_t mv = valid ? mask : all;
-      const unsigned int lo = __reduce_and_sync(0xffffffffu, (unsigned int)mv);
-      const unsigned int hi = __reduce_and_sync(0xffffffffu, (unsigned int)(mv >> 32));
-      uint64_t todo = ~((uint64_t)lo | ((uint64_t)hi << 32)) & all;
-      while (todo) {
-        const int p = __ffsll((long long)todo) - 1;
-        todo &= todo - 1;
-        const unsigned int lacks = __ballot_sync(0xffffffffu, valid && !((mask >> p) & 1ULL));
-        if (lane == 0) atomicMin(&sh.first_miss[p], base + (unsigned int)__ffs(lacks) - 1u);
+      // Per pod, the first block whose mask lacks it.  A prefix-AND over the lanes makes pod
+      // bits monotone (set up to the first lacking block), so the pods that drop out exactly at
+      // this lane are the bits its predecessor's prefix still had and its own has lost: every
+      // pod is reported once, by one lane, instead of one ballot per pod.
+      uint64_t pref = valid ? mask : all;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const unsigned int tlo = __shfl_up_sync(0xffffffffu, (unsigned int)pref, d);
+        const unsigned int thi = __shfl_up_sync(0xffffffffu, (unsigned int)(pref >> 32), d);
+        if (lane >= d) pref &= (uint64_t)tlo | ((uint64_t)thi << 32);
+      }
+      // pods already known to drop out BEFORE this chunk are not looked at again (a drop
+      // recorded by a warp working on a later chunk must not hide an earlier one)
+      const volatile unsigned int* fm = sh.first_miss;
+      const unsigned int g_lo = __ballot_sync(0xffffffffu, lane < P && fm[lane] < base);
+      const unsigned int g_hi =
+          __ballot_sync(0xffffffffu, lane + 32 < P && fm[(lane + 32) & 63] < base);
+      const uint64_t gone = (uint64_t)g_lo | ((uint64_t)g_hi << 32);
+      const unsigned int plo = __shfl_up_sync(0xffffffffu, (unsigned int)pref, 1);
+      const unsigned int phi = __shfl_up_sync(0xffffffffu, (unsigned int)(pref >> 32), 1);
+      const uint64_t before = lane == 0 ? (all & ~gone) : ((uint64_t)plo | ((uint64_t)phi << 32));
+      uint64_t drops = before & ~pref & all;
+      if (drops) {
+        while (drops) {
+          const int p = __ffsll((long long)drops) - 1;
+          drops &= drops - 1;
+          atomicMin(&sh.first_miss[p], i);
+        }
       }
     }
   }
