@@ -26,7 +26,13 @@ _lib = None
 
 
 def build(force: bool = False) -> str:
-    """Compile ``aibxo.c`` into ``libaibxo.so`` next to it (no-op when up to date)."""
+    """Compile ``aibxo.c`` into ``libaibxo.so`` next to it (no-op when up to date).
+
+    ``AIBXO_LIB_OVERRIDE`` names another build of the same source to load instead; the tests
+    use it to show that the pins reject deliberately broken copies of the oracle."""
+    override = os.environ.get("AIBXO_LIB_OVERRIDE")
+    if override:
+        return override
     newest = max(os.path.getmtime(_SRC), os.path.getmtime(_HDR))
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < newest:
         tmp = _LIB + ".tmp.%d" % os.getpid()

@@ -61,6 +61,7 @@ def check_gather_scatter(kv, ids_g, ids_s, mode_args):
     pool_want = pool_h.copy()
     rc, bad = oracle.kv_scatter(pool_want, lay_o, ids_s, want)
     assert np.array_equal(host(pool_d), pool_want)
+    assert np.array_equal(host(buf_d), want)                       # source untouched
     st, detail = aibx.status_fetch()
     assert (st, detail) == ((aibx.ERR_RANGE, bad) if bad else (0, 0))
     assert guards_intact(buf_w, buf_bytes, 0xEE) and guards_intact(pool_w, kv.pool_bytes, 0xA5)

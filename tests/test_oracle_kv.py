@@ -23,8 +23,10 @@ def test_gather_is_index_select(layout):
     ids = rng.integers(0, nb, 11).astype(np.uint32)          # repeats allowed
     lay = oracle.kv_layout(layout, L, H, Bt, D, E, nb)
     buf = np.zeros(11 * L * tile, dtype=np.uint8)
+    pool_before = pool.copy()
     rc, bad = oracle.kv_gather(pool.reshape(-1), lay, ids, buf)
     assert rc == oracle.OK and bad == 0
+    assert np.array_equal(pool, pool_before)                # the source side is only read
     tp = torch.from_numpy(pool)
     ti = torch.from_numpy(ids.astype(np.int64))
     if layout == 0:
@@ -44,10 +46,12 @@ def test_scatter_direct_indexing_and_round_trips(layout):
     ids = rng.permutation(nb)[:9].astype(np.uint32)
     buf = rng.integers(0, 256, 9 * L * tile, dtype=np.uint8)
     before = pool.copy()
+    buf_before = buf.copy()
     flat = pool.reshape(-1)
     rc, bad = oracle.kv_scatter(flat, lay, ids, buf)
     assert rc == oracle.OK
-    b3 = buf.reshape(9, L, tile)
+    assert np.array_equal(buf, buf_before)                  # the source side is only read
+    b3 = buf_before.reshape(9, L, tile)
     touched = np.zeros(nb, dtype=bool)
     for i, b in enumerate(ids):
         got = pool[b] if layout == 0 else pool[:, b]

@@ -1,0 +1,115 @@
+"""Do the pins bite?  Each case below plants one plausible mistake in a COPY of the oracle's C
+source (a wrong rotation, a dropped term, a flipped comparison, a transposed layout ...),
+builds it, and runs the matching pin file against it in a subprocess: the pins must fail.
+Everything happens on the CPU; the real oracle is never modified."""
+import os
+import subprocess
+import sys
+from concurrent.futures import ThreadPoolExecutor
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SRC = os.path.join(ROOT, "oracle", "aibxo.c")
+HDR = os.path.join(ROOT, "oracle", "aibxo.h")
+
+# (name, pin file, text to find, replacement, which occurrence)
+MUTANTS = [
+    ("round_rotation", "test_oracle_hash.py", "acc = rotl64(acc, 31);", "acc = rotl64(acc, 30);", 0),
+    ("prime2_digit", "test_oracle_hash.py", "0xC2B2AE3D27D4EB4FULL", "0xC2B2AE3D27D4EB4DULL", 0),
+    ("merge_constant", "test_oracle_hash.py", "acc = acc * PRIME64_1 + PRIME64_4;\n  return acc;",
+     "acc = acc * PRIME64_1 + PRIME64_3;\n  return acc;", 0),
+    ("length_not_added", "test_oracle_hash.py", "acc += (uint64_t)len;", "", 0),
+    ("avalanche_shift", "test_oracle_hash.py", "acc ^= acc >> 29;", "acc ^= acc >> 28;", 0),
+    ("fourth_accumulator_sign", "test_oracle_hash.py", "uint64_t a4 = seed - PRIME64_1;",
+     "uint64_t a4 = seed + PRIME64_1;", 0),
+    ("chain_not_seeded_by_parent", "test_oracle_hash.py",
+     "parent = aibxo_xxh64(msg, (size_t)block_tokens * 4, parent);",
+     "parent = aibxo_xxh64(msg, (size_t)block_tokens * 4, root_seed);", 0),
+    ("big_endian_tokens", "test_oracle_hash.py", "msg[4 * j + 0] = (uint8_t)(v);",
+     "msg[4 * j + 0] = (uint8_t)(v >> 24);", 0),
+    ("tail_word_rotation", "test_oracle_hash.py", "rotl64(acc, 23) * PRIME64_2 + PRIME64_3",
+     "rotl64(acc, 22) * PRIME64_2 + PRIME64_3", 0),
+    ("partial_block_hashed", "test_oracle_hash.py", "int64_t nblk = len / block_tokens;",
+     "int64_t nblk = (len + block_tokens - 1) / block_tokens;", 0),
+    ("insert_overwrites_mask", "test_oracle_index.py", "ix->e[w - 1].mask |= ix->e[i].mask;",
+     "ix->e[w - 1].mask = ix->e[i].mask;", 0),
+    ("insert_keeps_max_id", "test_oracle_index.py", "if (ix->e[i].id < ix->e[w - 1].id)",
+     "if (ix->e[i].id > ix->e[w - 1].id)", 0),
+    ("evict_keeps_named_bits", "test_oracle_index.py", "if (e) e->mask &= ~masks[i];",
+     "if (e) e->mask &= masks[i];", 0),
+    ("evict_reports_live_entries", "test_oracle_index.py",
+     "freed[i] = (e && e->mask == 0) ? e->id : AIBXO_NO_BLOCK;",
+     "freed[i] = (e && e->mask != 0) ? e->id : AIBXO_NO_BLOCK;", 0),
+    ("all_ones_key_not_reserved", "test_oracle_index.py", "return k == 0ULL || k == ~0ULL;",
+     "return k == 0ULL;", 0),
+    ("pods_beyond_P_kept", "test_oracle_index.py", "ix->e[m].mask = masks[i] & all;",
+     "ix->e[m].mask = masks[i];", 0),
+    ("match_tests_wrong_pod", "test_oracle_match.py", "((e->mask >> p) & 1ULL) == 0) break;",
+     "((e->mask >> (p + 1)) & 1ULL) == 0) break;", 0),
+    ("match_ignores_pod_bit", "test_oracle_match.py",
+     "if (!e || ((e->mask >> p) & 1ULL) == 0) break;", "if (!e) break;", 0),
+    ("ids_after_a_hole", "test_oracle_match.py", "if (i < a) {\n          block_ids",
+     "if (!key_reserved(h[i]) && find_entry(ix, h[i])) {\n          block_ids", 0),
+    ("collect_keeps_duplicates", "test_oracle_match.py",
+     "if (w == 0 || unique_ids[w - 1] != unique_ids[i])", "if (1)", 0),
+    ("threshold_exclusive", "test_oracle_score.py", "100 * hit >= (int64_t)prm.threshold_pct * n_r",
+     "100 * hit > (int64_t)prm.threshold_pct * n_r", 0),
+    ("ties_to_highest_pod", "test_oracle_score.py", "arg == AIBXO_NO_POD || score > top",
+     "arg == AIBXO_NO_POD || score >= top", 0),
+    ("load_added", "test_oracle_score.py", "- (int64_t)prm.w_load * (int64_t)pod_load[p]",
+     "+ (int64_t)prm.w_load * (int64_t)pod_load[p]", 0),
+    ("ready_mask_ignored", "test_oracle_score.py", "if (((ready_mask >> p) & 1ULL) == 0) continue;",
+     "", 0),
+    ("threshold_on_tokens_not_blocks", "test_oracle_score.py",
+     "100 * hit >= (int64_t)prm.threshold_pct * n_r", "100 * hit >= (int64_t)prm.threshold_pct * 16 * n_r", 0),
+    ("layer_major_as_block_major", "test_oracle_kv.py",
+     "return ((int64_t)l * L->num_blocks + b) * t;", "return ((int64_t)b * L->num_layers + l) * t;", 0),
+    ("buffer_layer_major", "test_oracle_kv.py",
+     "memcpy((uint8_t*)buf + (i * L->num_layers + l) * t,",
+     "memcpy((uint8_t*)buf + (i + l * n) * t,", 0),
+    ("no_block_counts_as_error", "test_oracle_kv.py",
+     "if (ids[i] == AIBXO_NO_BLOCK) continue;\n    if (ids[i] >= L->num_blocks) { ++nbad; continue; }\n    for (int32_t l = 0; l < L->num_layers; ++l) {\n      memcpy((uint8_t*)buf",
+     "if (ids[i] >= L->num_blocks) { ++nbad; continue; }\n    for (int32_t l = 0; l < L->num_layers; ++l) {\n      memcpy((uint8_t*)buf", 0),
+    ("scatter_copies_wrong_way", "test_oracle_kv.py",
+     "memcpy((uint8_t*)pool + pool_offset(L, ids[i], l),\n             (const uint8_t*)buf + (i * L->num_layers + l) * t, (size_t)t);",
+     "memcpy((uint8_t*)buf + (i * L->num_layers + l) * t,\n             (const uint8_t*)pool + pool_offset(L, ids[i], l), (size_t)t);", 0),
+]
+
+
+def _run_mutant(args):
+    tmp, (name, pin_file, old, new, _) = args
+    text = open(SRC).read()
+    assert text.count(old) >= 1, "mutation site not found: " + name
+    mutated = text.replace(old, new, 1)
+    d = os.path.join(tmp, name)
+    os.makedirs(d)
+    with open(os.path.join(d, "aibxo.c"), "w") as f:
+        f.write(mutated)
+    with open(os.path.join(d, "aibxo.h"), "w") as f:
+        f.write(open(HDR).read())
+    lib = os.path.join(d, "libmutant.so")
+    subprocess.check_call(["gcc", "-std=c99", "-O1", "-w", "-fPIC", "-shared",
+                           os.path.join(d, "aibxo.c"), "-o", lib])
+    env = dict(os.environ, AIBXO_LIB_OVERRIDE=lib, PYTHONDONTWRITEBYTECODE="1")
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
+                        os.path.join(ROOT, "tests", pin_file)],
+                       cwd=ROOT, env=env, stdout=subprocess.PIPE, stderr=subprocess.STDOUT,
+                       timeout=600)
+    return name, r.returncode, r.stdout.decode()[-400:]
+
+
+def test_every_planted_mistake_is_caught(tmp_path):
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 2)) as pool:
+        results = list(pool.map(_run_mutant, [(str(tmp_path), m) for m in MUTANTS]))
+    survivors = [name for name, rc, _ in results if rc == 0]
+    # exit 1 = a pin failed, a negative code = the broken copy crashed (also caught);
+    # 2..5 are pytest's own errors and would mean the harness is not testing anything
+    broken = [(name, rc, tail) for name, rc, tail in results if rc in (2, 3, 4, 5)]
+    assert not broken, broken
+    assert not survivors, "pins did not notice: %s" % survivors
+
+
+def test_unmodified_copy_passes(tmp_path):
+    """The harness itself: an untouched copy of the source passes a pin file."""
+    name, rc, tail = _run_mutant((str(tmp_path), ("identity", "test_oracle_score.py",
+                                                  "acc = rotl64(acc, 31);", "acc = rotl64(acc, 31);", 0)))
+    assert rc == 0, tail
