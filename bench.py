@@ -912,7 +912,33 @@ def case_oracle_cfg(args):
                       "cores_available": len(os.sched_getaffinity(0)), "cpu": cpu, "results": res}))
 
 
-CASES = {"oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
+def case_hash_sweep(args):
+    """hash_blocks alone: R equal-length requests, block sizes 8..64 tokens.  With few requests
+    the time is the serial seed chain of one request, which separates the cost of a 32-byte
+    stripe from the cost of a block end (fold + avalanche + reseed)."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import workloads as W
+
+    out = []
+    for R, L in ((1, 32768), (64, 32768), (4096, 2048)):
+        toks = torch.from_numpy(W.Stream(50, R).randint(0, 128256, R * L).astype(np.int32)).cuda()
+        off = torch.arange(0, (R + 1) * L, L, dtype=torch.int64, device="cuda")
+        for B in (8, 16, 32, 64):
+            nb = L // B
+            bo = torch.arange(0, (R + 1) * nb, nb, dtype=torch.int64, device="cuda")
+            h = torch.empty(R * nb, dtype=torch.uint64, device="cuda")
+            ms = statistics.median(_event_times(
+                torch, lambda: aibx.hash_blocks(toks, off, bo, B, 0, h), 7, 3))
+            out.append({"R": R, "tokens_per_request": L, "block_tokens": B,
+                        "us": round(ms * 1e3, 1), "ns_per_block_of_a_chain": round(ms * 1e6 / nb, 1),
+                        "ns_per_stripe_of_a_chain": round(ms * 1e6 / (nb * B // 8), 1),
+                        "tokens_per_s": round(R * L / (ms * 1e-3), 0)})
+    print(json.dumps({"case": "hash_sweep", "results": out, "status": aibx.status_fetch()}))
+
+
+CASES = {"hash_sweep": case_hash_sweep, "oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
          "cfg4": case_cfg4, "cfg5": case_cfg5, "lookup_flat": case_lookup_flat}
 
 
