@@ -2,7 +2,7 @@
 """Benchmark of the KV-reuse hot path on B200.
 
 One step = one pass of the whole path over one batch of the Llama-3-8B-shaped workload:
-hash the 64 requests -> longest cached prefix against a 200k-entry index -> route score ->
+hash the 64 requests -> longest cached prefix against a 200k-entry index + route score ->
 set of matched blocks -> gather them from the 8 GiB paged pool into the transfer buffer ->
 scatter them back -> publish and expire one batch of new index entries.
 
@@ -38,7 +38,7 @@ METRIC = "kv_gather_scatter_GBps_whole_step"
 UNIT = "GB/s"
 WORKLOAD = "cfg2-llama3-8b: 64 requests (1k-8k tokens, 32 Zipf prompts), index 200k/2^19 x 16 pods, " \
            "pool 4096 x 2 MiB bf16 blocks, gather+scatter of all matched blocks"
-KERNELS_PER_STEP = 11   # hash, match, score, mark, compact, gather, scatter, insert, evict x3
+KERNELS_PER_STEP = 10   # hash, match+score, mark, compact, gather, scatter, insert, evict x3
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of kv_copy_bulk_kernel from the ncu
 # capture summarised under profiles/, valid only for the kernel source with this digest.
@@ -208,11 +208,10 @@ class GpuJob:
     # -- pieces of a step ------------------------------------------------------------------
     def routing(self) -> int:
         aibx = self.aibx
-        aibx.hash_blocks(self.d_tokens, self.d_tok_off, self.d_blk_off, self.B, 0, self.d_hashes)
-        self.index.match_prefix(self.d_hashes, self.d_blk_off, self.d_match_len, self.d_any_len,
-                                self.d_block_ids)
-        aibx.route_score(self.d_match_len, self.d_blk_off, self.P, self.d_pod_load,
-                         self.w.ready_mask, None, self.d_best_pod, self.d_best_score, None)
+        # hash -> match (+ score in the same kernel): one call, two launches
+        aibx.route_batch(self.index, self.d_tokens, self.d_tok_off, self.d_blk_off, self.B, 0,
+                         self.d_pod_load, self.w.ready_mask, None, self.d_hashes, self.d_match_len,
+                         self.d_any_len, self.d_block_ids, self.d_best_pod, self.d_best_score)
         aibx.collect_blocks(self.d_block_ids, self.kv.num_blocks, self.d_scratch, self.d_unique,
                             self.d_count)
         # the host needs the size of the transfer: 4 bytes back, one stream sync

@@ -143,6 +143,34 @@ int32_t aibx_route_score(const uint32_t* d_match_len, const int64_t* d_blk_off, 
                          int64_t* d_best_score, int64_t* d_scores, void* stream);
 
 /* ---------------------------------------------------------------------------------------
+ * Routing in one call (Section 3.2.2: what the gateway does per pending request - token pattern,
+ * cache availability, load - taken for a whole batch).  Same results as aibx_hash_blocks, then
+ * aibx_match_prefix, then aibx_route_score with d_scores = NULL, written to the same outputs;
+ * two launches instead of three (the score is computed by the match kernel while the request's
+ * match lengths are still on chip) and one crossing of this boundary.
+ *   d_hashes [blk_off[R]] out; d_match_len [R * num_pods] out; d_any_len, d_block_ids nullable.
+ */
+int32_t aibx_route_batch(const aibx_index_t* index, const int32_t* d_tokens,
+                         const int64_t* d_tok_off, const int64_t* d_blk_off, int32_t R,
+                         int32_t block_tokens, uint64_t root_seed, const int32_t* d_pod_load,
+                         uint64_t ready_mask, const aibx_route_params_t* params,
+                         uint64_t* d_hashes, uint32_t* d_match_len, uint32_t* d_any_len,
+                         uint32_t* d_block_ids, int32_t* d_best_pod, int64_t* d_best_score,
+                         void* stream);
+
+/* Sequential assignment of a batch (Section 3.2.2, least-request: the count of admitted
+ * requests of an instance grows with every request routed to it).  Requests are taken in
+ * order r = 0..R-1; request r is scored as in aibx_route_score against the CURRENT d_pod_load,
+ * then d_pod_load[best_pod[r]] += load_increment before request r+1 is scored.  d_pod_load is
+ * updated in place (num_pods int32).  load_increment = 0 gives aibx_route_score's results.
+ * One warp walks the batch: the dependence between requests is inherent.
+ */
+int32_t aibx_route_assign(const uint32_t* d_match_len, const int64_t* d_blk_off, int32_t R,
+                          int32_t num_pods, int32_t* d_pod_load, uint64_t ready_mask,
+                          const aibx_route_params_t* params, int32_t load_increment,
+                          int32_t* d_best_pod, int64_t* d_best_score, void* stream);
+
+/* ---------------------------------------------------------------------------------------
  * Set of matched blocks (supporting call between match and gather: Section 3.2.5 speaks of
  * reducing redundant transfers, so a block shared by several requests moves once).
  *   d_unique_ids [n] = the distinct values of d_block_ids[0..n) that are < num_blocks, in

@@ -76,13 +76,14 @@ def lib():
         L.aibxo_index_stats.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
         L.aibxo_match_prefix.argtypes = [vp, vp, vp, i32, vp, vp, vp]
         L.aibxo_route_score.argtypes = [vp, vp, i32, i32, vp, u64, C.POINTER(_Params), vp, vp, vp]
+        L.aibxo_route_assign.argtypes = [vp, vp, i32, i32, vp, u64, C.POINTER(_Params), i32, vp, vp]
         L.aibxo_collect_blocks.argtypes = [vp, i64, u32, vp, C.POINTER(u32)]
         L.aibxo_kv_gather.argtypes = [vp, C.POINTER(_Layout), vp, i64, vp, C.POINTER(i64)]
         L.aibxo_kv_scatter.argtypes = [vp, C.POINTER(_Layout), vp, i64, vp, C.POINTER(i64)]
         for name in (
             "aibxo_hash_blocks aibxo_index_create aibxo_index_destroy aibxo_index_clear "
             "aibxo_index_insert aibxo_index_evict aibxo_index_lookup aibxo_index_stats "
-            "aibxo_match_prefix aibxo_route_score aibxo_collect_blocks aibxo_kv_gather "
+            "aibxo_match_prefix aibxo_route_score aibxo_route_assign aibxo_collect_blocks aibxo_kv_gather "
             "aibxo_kv_scatter"
         ).split():
             getattr(L, name).restype = i32
@@ -195,6 +196,22 @@ def route_score(match_len, blk_off, pod_load, ready_mask, params=None):
                                  _p(scores))
     assert rc == OK, rc
     return best_pod, best_score, scores
+
+
+def route_assign(match_len, blk_off, pod_load, ready_mask, params=None, load_increment=1):
+    """Sequential assignment; returns (best_pod, best_score, loads after the batch)."""
+    match_len = _arr(match_len, np.uint32)
+    R, P = match_len.shape
+    blk_off = _arr(blk_off, np.int64)
+    load = np.array(pod_load, dtype=np.int32, copy=True)
+    best_pod = np.zeros(R, dtype=np.int32)
+    best_score = np.zeros(R, dtype=np.int64)
+    prm = None if params is None else C.byref(_Params(*params))
+    rc = lib().aibxo_route_assign(_p(match_len), _p(blk_off), R, P, _p(load),
+                                  ready_mask & (2**64 - 1), prm, load_increment, _p(best_pod),
+                                  _p(best_score))
+    assert rc == OK, rc
+    return best_pod, best_score, load
 
 
 def collect_blocks(block_ids, num_blocks: int):

@@ -365,6 +365,25 @@ int32_t aibxo_route_score(const uint32_t* match_len, const int64_t* blk_off, int
   return AIBXO_OK;
 }
 
+int32_t aibxo_route_assign(const uint32_t* match_len, const int64_t* blk_off, int32_t R,
+                           int32_t num_pods, int32_t* pod_load, uint64_t ready_mask,
+                           const aibxo_route_params_t* params, int32_t load_increment,
+                           int32_t* best_pod, int64_t* best_score) {
+  if (R < 0 || num_pods < 1 || num_pods > 64) return AIBXO_ERR_INVALID;
+  if (R == 0) return AIBXO_OK;
+  if (!match_len || !blk_off || !pod_load || !best_pod || !best_score) return AIBXO_ERR_INVALID;
+  /* one request at a time, each seeing the loads its predecessors left behind */
+  for (int32_t r = 0; r < R; ++r) {
+    int32_t rc = aibxo_route_score(match_len + (int64_t)r * num_pods, blk_off + r, 1, num_pods,
+                                   pod_load, ready_mask, params, best_pod + r, best_score + r,
+                                   NULL);
+    if (rc != AIBXO_OK) return rc;
+    if (best_pod[r] != AIBXO_NO_POD)
+      pod_load[best_pod[r]] = (int32_t)((uint32_t)pod_load[best_pod[r]] + (uint32_t)load_increment);
+  }
+  return AIBXO_OK;
+}
+
 /* ------------------------------------------------------------------ matched-block set - */
 
 static int cmp_u32(const void* a, const void* b) {

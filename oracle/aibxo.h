@@ -73,6 +73,15 @@ int32_t aibxo_route_score(const uint32_t* match_len, const int64_t* blk_off, int
                           const aibxo_route_params_t* params, int32_t* best_pod,
                           int64_t* best_score, int64_t* scores);
 
+/* Sequential assignment (Section 3.2.2, least-request read over a batch: every admitted request
+ * raises the chosen instance's count before the next one is routed).  Requests are taken in
+ * order; request r is scored against the CURRENT pod_load, and load[best] += load_increment
+ * before request r+1.  pod_load is updated in place.  increment 0 equals aibxo_route_score. */
+int32_t aibxo_route_assign(const uint32_t* match_len, const int64_t* blk_off, int32_t R,
+                           int32_t num_pods, int32_t* pod_load, uint64_t ready_mask,
+                           const aibxo_route_params_t* params, int32_t load_increment,
+                           int32_t* best_pod, int64_t* best_score);
+
 /* Ascending distinct valid block ids, padded with NO_BLOCK; returns RANGE if any id other
  * than NO_BLOCK is >= num_blocks (those are dropped). */
 int32_t aibxo_collect_blocks(const uint32_t* block_ids, int64_t n, uint32_t num_blocks,

@@ -77,6 +77,9 @@ def lib():
             "aibx_index_stats": [vp, C.POINTER(u64), C.POINTER(u64), vp],
             "aibx_match_prefix": [vp, vp, vp, i32, vp, vp, vp, vp],
             "aibx_route_score": [vp, vp, i32, i32, vp, u64, C.POINTER(RouteParams), vp, vp, vp, vp],
+            "aibx_route_batch": [vp, vp, vp, vp, i32, i32, u64, vp, u64, C.POINTER(RouteParams),
+                                 vp, vp, vp, vp, vp, vp, vp],
+            "aibx_route_assign": [vp, vp, i32, i32, vp, u64, C.POINTER(RouteParams), i32, vp, vp, vp],
             "aibx_collect_blocks": [vp, i64, u32, vp, vp, vp, vp],
             "aibx_collect_blocks_static": [vp, i64, u32, vp, vp, vp],
             "aibx_kv_gather": [vp, C.POINTER(KVLayout), vp, i64, vp, vp],
@@ -194,6 +197,29 @@ def route_score(match_len, blk_off, num_pods: int, pod_load, ready_mask: int, pa
         _ptr(match_len, torch.uint32), _ptr(blk_off, torch.int64), R, num_pods,
         _ptr(pod_load, torch.int32), ready_mask & (2**64 - 1), prm, _ptr(best_pod, torch.int32),
         _ptr(best_score, torch.int64), _ptr(scores, torch.int64), _stream()))
+
+
+def route_batch(index: Index, tokens, tok_off, blk_off, block_tokens: int, root_seed: int,
+                pod_load, ready_mask: int, params, hashes, match_len, any_len, block_ids,
+                best_pod, best_score) -> None:
+    R = tok_off.numel() - 1
+    prm = None if params is None else C.byref(RouteParams(*params))
+    _check("aibx_route_batch", lib().aibx_route_batch(
+        index._h, _ptr(tokens, torch.int32), _ptr(tok_off, torch.int64), _ptr(blk_off, torch.int64),
+        R, block_tokens, root_seed & (2**64 - 1), _ptr(pod_load, torch.int32),
+        ready_mask & (2**64 - 1), prm, _ptr(hashes, torch.uint64), _ptr(match_len, torch.uint32),
+        _ptr(any_len, torch.uint32), _ptr(block_ids, torch.uint32), _ptr(best_pod, torch.int32),
+        _ptr(best_score, torch.int64), _stream()))
+
+
+def route_assign(match_len, blk_off, num_pods: int, pod_load, ready_mask: int, params,
+                 load_increment: int, best_pod, best_score) -> None:
+    R = blk_off.numel() - 1
+    prm = None if params is None else C.byref(RouteParams(*params))
+    _check("aibx_route_assign", lib().aibx_route_assign(
+        _ptr(match_len, torch.uint32), _ptr(blk_off, torch.int64), R, num_pods,
+        _ptr(pod_load, torch.int32), ready_mask & (2**64 - 1), prm, load_increment,
+        _ptr(best_pod, torch.int32), _ptr(best_score, torch.int64), _stream()))
 
 
 def collect_scratch_bytes(num_blocks: int) -> int:

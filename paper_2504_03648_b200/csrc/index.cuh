@@ -10,6 +10,7 @@
 #pragma once
 
 #include "aibx_common.cuh"
+#include "route_score.cuh"
 
 namespace aibx {
 
@@ -212,7 +213,9 @@ __global__ void match_prefix_kernel(IndexView ix, const uint64_t* __restrict__ h
                                     const int64_t* __restrict__ blk_off, int R, int wpr,
                                     uint32_t* __restrict__ match_len,
                                     uint32_t* __restrict__ any_len,
-                                    uint32_t* __restrict__ block_ids) {
+                                    uint32_t* __restrict__ block_ids, ScoreParams sp,
+                                    int32_t* __restrict__ best_pod,
+                                    int64_t* __restrict__ best_score) {
   extern __shared__ MatchShared s_groups[];
   const int warps_per_cta = blockDim.x >> 5;
   const int groups_per_cta = warps_per_cta / wpr;
@@ -291,6 +294,23 @@ __global__ void match_prefix_kernel(IndexView ix, const uint64_t* __restrict__ h
     for (int p = tid_in_group; p < P; p += group_threads)
       match_len[(int64_t)r * P + p] = sh.first_miss[p];
     if (any_len && tid_in_group == 0) any_len[r] = a;
+    if (best_pod && warp_in_group == 0) {
+      // fused scoring: the request's match lengths are still in shared memory
+      const long long h0 = lane < P ? (long long)sh.first_miss[lane] : 0;
+      const long long h1 = lane + 32 < P ? (long long)sh.first_miss[lane + 32] : 0;
+      const long long l0 = lane < P ? (long long)sp.pod_load[lane] : 0;
+      const long long l1 = lane + 32 < P ? (long long)sp.pod_load[lane + 32] : 0;
+      long long top;
+      int arg;
+      lane_candidate(lane, P, sp.ready_mask,
+                     pod_score(h0, (long long)n_r, l0, sp.w_prefix, sp.w_load, sp.thr_pct),
+                     pod_score(h1, (long long)n_r, l1, sp.w_prefix, sp.w_load, sp.thr_pct), top, arg);
+      warp_argmax(top, arg);
+      if (lane == 0) {
+        best_pod[r] = arg;
+        best_score[r] = top;
+      }
+    }
     if (block_ids) {
       for (unsigned int i = a + tid_in_group; i < n_r; i += group_threads)
         block_ids[off + i] = AIBX_NO_BLOCK;

@@ -182,12 +182,32 @@ int32_t aibx_index_stats(const aibx_index_t* ix, uint64_t* live, uint64_t* capac
   return AIBX_OK;
 }
 
+namespace {
+
+int32_t launch_match(const aibx_index_t* ix, const uint64_t* d_hashes, const int64_t* d_blk_off,
+                     int32_t R, uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
+                     const ScoreParams& sp, int32_t* d_best_pod, int64_t* d_best_score,
+                     cudaStream_t st);
+
+}  // namespace
+
 int32_t aibx_match_prefix(const aibx_index_t* ix, const uint64_t* d_hashes,
                           const int64_t* d_blk_off, int32_t R, uint32_t* d_match_len,
                           uint32_t* d_any_len, uint32_t* d_block_ids, void* stream) {
   if (!ix || R < 0) return AIBX_ERR_INVALID;
   if (R == 0) return AIBX_OK;
   if (!d_hashes || !d_blk_off || !d_match_len) return AIBX_ERR_INVALID;
+  ScoreParams none = {nullptr, 0, 0, 0, 0};
+  return launch_match(ix, d_hashes, d_blk_off, R, d_match_len, d_any_len, d_block_ids, none,
+                      nullptr, nullptr, as_stream(stream));
+}
+
+namespace {
+
+int32_t launch_match(const aibx_index_t* ix, const uint64_t* d_hashes, const int64_t* d_blk_off,
+                     int32_t R, uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
+                     const ScoreParams& sp, int32_t* d_best_pod, int64_t* d_best_score,
+                     cudaStream_t st) {
   // warps per request: aim at ~32 resident warps per SM; few requests get whole CTAs
   int wpr = 1;
   const long long target = (long long)sm_count() * 32;
@@ -196,8 +216,50 @@ int32_t aibx_match_prefix(const aibx_index_t* ix, const uint64_t* d_hashes,
   const int groups = warps_per_cta / wpr;
   const unsigned int grid = (unsigned int)((R + groups - 1) / groups);
   const size_t smem = (size_t)groups * sizeof(MatchShared);
-  match_prefix_kernel<<<grid, warps_per_cta * 32, smem, as_stream(stream)>>>(
-      ix->view, d_hashes, d_blk_off, R, wpr, d_match_len, d_any_len, d_block_ids);
+  match_prefix_kernel<<<grid, warps_per_cta * 32, smem, st>>>(
+      ix->view, d_hashes, d_blk_off, R, wpr, d_match_len, d_any_len, d_block_ids, sp, d_best_pod,
+      d_best_score);
+  return launch_status();
+}
+
+}  // namespace
+
+int32_t aibx_route_batch(const aibx_index_t* ix, const int32_t* d_tokens, const int64_t* d_tok_off,
+                         const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
+                         uint64_t root_seed, const int32_t* d_pod_load, uint64_t ready_mask,
+                         const aibx_route_params_t* params, uint64_t* d_hashes,
+                         uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
+                         int32_t* d_best_pod, int64_t* d_best_score, void* stream) {
+  if (!ix || R < 0 || block_tokens <= 0 || block_tokens % 8 != 0 || block_tokens > 1024)
+    return AIBX_ERR_INVALID;
+  if (R == 0) return AIBX_OK;
+  if (!d_tokens || !d_tok_off || !d_blk_off || !d_hashes || !d_match_len || !d_pod_load ||
+      !d_best_pod || !d_best_score)
+    return AIBX_ERR_INVALID;
+  aibx_route_params_t prm = {4, 1, 50};
+  if (params) prm = *params;
+  cudaStream_t st = as_stream(stream);
+  const int32_t rc = launch_hash_blocks(d_tokens, d_tok_off, d_blk_off, R, block_tokens, root_seed,
+                                        d_hashes, st);
+  if (rc != AIBX_OK) return rc;
+  ScoreParams sp = {d_pod_load, ready_mask, prm.w_prefix, prm.w_load, prm.threshold_pct};
+  return launch_match(ix, d_hashes, d_blk_off, R, d_match_len, d_any_len, d_block_ids, sp,
+                      d_best_pod, d_best_score, st);
+}
+
+int32_t aibx_route_assign(const uint32_t* d_match_len, const int64_t* d_blk_off, int32_t R,
+                          int32_t num_pods, int32_t* d_pod_load, uint64_t ready_mask,
+                          const aibx_route_params_t* params, int32_t load_increment,
+                          int32_t* d_best_pod, int64_t* d_best_score, void* stream) {
+  if (R < 0 || num_pods < 1 || num_pods > AIBX_MAX_PODS) return AIBX_ERR_INVALID;
+  if (R == 0) return AIBX_OK;
+  if (!d_match_len || !d_blk_off || !d_pod_load || !d_best_pod || !d_best_score)
+    return AIBX_ERR_INVALID;
+  aibx_route_params_t prm = {4, 1, 50};
+  if (params) prm = *params;
+  route_assign_kernel<<<1, 32, 0, as_stream(stream)>>>(
+      d_match_len, d_blk_off, R, num_pods, d_pod_load, ready_mask, prm.w_prefix, prm.w_load,
+      prm.threshold_pct, load_increment, d_best_pod, d_best_score);
   return launch_status();
 }
 
@@ -211,9 +273,9 @@ int32_t aibx_route_score(const uint32_t* d_match_len, const int64_t* d_blk_off, 
     return AIBX_ERR_INVALID;
   aibx_route_params_t prm = {4, 1, 50};
   if (params) prm = *params;
+  ScoreParams sp = {d_pod_load, ready_mask, prm.w_prefix, prm.w_load, prm.threshold_pct};
   route_score_kernel<<<blocks_for(R, kRouteWarps), kRouteWarps * 32, 0, as_stream(stream)>>>(
-      d_match_len, d_blk_off, R, num_pods, d_pod_load, ready_mask, prm.w_prefix, prm.w_load,
-      prm.threshold_pct, d_best_pod, d_best_score, d_scores);
+      d_match_len, d_blk_off, R, num_pods, sp, d_best_pod, d_best_score, d_scores);
   return launch_status();
 }
 

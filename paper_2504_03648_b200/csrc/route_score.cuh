@@ -1,4 +1,6 @@
-// Integer prefix-and-load route score and its argmax: one warp per request, lanes over pods.
+// Integer prefix-and-load route score and its argmax: lanes over pods (two pods per lane), one
+// warp per request.  The same lane code serves the stand-alone score kernel, the scoring tail of
+// the fused match kernel and the sequential assignment kernel.
 #pragma once
 
 #include "aibx_common.cuh"
@@ -7,34 +9,38 @@ namespace aibx {
 
 constexpr int kRouteWarps = 8;
 
-__global__ void __launch_bounds__(kRouteWarps * 32)
-route_score_kernel(const uint32_t* __restrict__ match_len, const int64_t* __restrict__ blk_off,
-                   int R, int P, const int32_t* __restrict__ pod_load, uint64_t ready_mask,
-                   int w_prefix, int w_load, int thr_pct, int32_t* __restrict__ best_pod,
-                   int64_t* __restrict__ best_score, int64_t* __restrict__ scores) {
-  const int lane = threadIdx.x & 31;
-  const int r = blockIdx.x * kRouteWarps + (threadIdx.x >> 5);
-  if (r >= R) return;
-  const long long n_r = blk_off[r + 1] - blk_off[r];
+struct ScoreParams {
+  const int32_t* pod_load;
+  uint64_t ready_mask;
+  int w_prefix, w_load, thr_pct;
+};
 
-  long long top = LLONG_MIN;
-  int arg = AIBX_NO_POD;
-#pragma unroll
-  for (int half = 0; half < 2; ++half) {
-    const int p = lane + 32 * half;
-    if (p < P) {
-      const long long hit = (long long)match_len[(int64_t)r * P + p];
-      const long long eff = (hit > 0 && 100LL * hit >= (long long)thr_pct * n_r) ? hit : 0LL;
-      const long long sc = (long long)w_prefix * eff - (long long)w_load * (long long)pod_load[p];
-      if (scores) scores[(int64_t)r * P + p] = sc;
-      // ascending p within a lane: strict ">" keeps the lower pod on ties
-      if (((ready_mask >> p) & 1ULL) && (arg == AIBX_NO_POD || sc > top)) {
-        top = sc;
-        arg = p;
-      }
-    }
+__device__ __forceinline__ long long pod_score(long long hit, long long n_r, long long load,
+                                               int w_prefix, int w_load, int thr_pct) {
+  const long long eff = (hit > 0 && 100LL * hit >= (long long)thr_pct * n_r) ? hit : 0LL;
+  return (long long)w_prefix * eff - (long long)w_load * load;
+}
+
+// Candidate of one lane: the better of its two pods (ascending pod order, strict ">" keeps the
+// lower pod on ties); pods that are not ready never become candidates.
+__device__ __forceinline__ void lane_candidate(int lane, int P, uint64_t ready_mask, long long sc0,
+                                               long long sc1, long long& top, int& arg) {
+  top = LLONG_MIN;
+  arg = AIBX_NO_POD;
+  if (lane < P && ((ready_mask >> lane) & 1ULL)) {
+    top = sc0;
+    arg = lane;
   }
-  // warp argmax; among equal scores the lower pod index wins; "no pod" loses to any pod
+  const int p1 = lane + 32;
+  if (p1 < P && ((ready_mask >> p1) & 1ULL) && (arg == AIBX_NO_POD || sc1 > top)) {
+    top = sc1;
+    arg = p1;
+  }
+}
+
+// Warp argmax over (score, pod): higher score wins, equal scores go to the lower pod index,
+// "no pod" loses to any pod.  Every lane ends with the winner.
+__device__ __forceinline__ void warp_argmax(long long& top, int& arg) {
 #pragma unroll
   for (int d = 16; d >= 1; d >>= 1) {
     const long long o_top = __shfl_xor_sync(0xffffffffu, top, d);
@@ -46,10 +52,75 @@ route_score_kernel(const uint32_t* __restrict__ match_len, const int64_t* __rest
       arg = o_arg;
     }
   }
+}
+
+__global__ void __launch_bounds__(kRouteWarps * 32)
+route_score_kernel(const uint32_t* __restrict__ match_len, const int64_t* __restrict__ blk_off,
+                   int R, int P, ScoreParams sp, int32_t* __restrict__ best_pod,
+                   int64_t* __restrict__ best_score, int64_t* __restrict__ scores) {
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.x * kRouteWarps + (threadIdx.x >> 5);
+  if (r >= R) return;
+  const long long n_r = blk_off[r + 1] - blk_off[r];
+  long long sc[2] = {0, 0};
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    const int p = lane + 32 * half;
+    if (p < P) {
+      sc[half] = pod_score((long long)match_len[(int64_t)r * P + p], n_r, sp.pod_load[p],
+                           sp.w_prefix, sp.w_load, sp.thr_pct);
+      if (scores) scores[(int64_t)r * P + p] = sc[half];
+    }
+  }
+  long long top;
+  int arg;
+  lane_candidate(lane, P, sp.ready_mask, sc[0], sc[1], top, arg);
+  warp_argmax(top, arg);
   if (lane == 0) {
     best_pod[r] = arg;
     best_score[r] = top;
   }
+}
+
+// Sequential assignment: one warp walks the requests in order; the pod loads live in registers
+// (two per lane) and the winner's lane bumps its own copy before the next request is scored.
+// The next request's match lengths are fetched while the current one is reduced.
+__global__ void __launch_bounds__(32)
+route_assign_kernel(const uint32_t* __restrict__ match_len, const int64_t* __restrict__ blk_off,
+                    int R, int P, int32_t* __restrict__ pod_load, uint64_t ready_mask, int w_prefix,
+                    int w_load, int thr_pct, int increment, int32_t* __restrict__ best_pod,
+                    int64_t* __restrict__ best_score) {
+  const int lane = threadIdx.x;
+  const int p0 = lane, p1 = lane + 32;
+  int32_t load0 = p0 < P ? pod_load[p0] : 0;
+  int32_t load1 = p1 < P ? pod_load[p1] : 0;
+  uint32_t hit0 = 0, hit1 = 0;
+  long long off_lo = 0, off_hi = 0;
+  auto fetch = [&](int r) {
+    if (p0 < P) hit0 = match_len[(int64_t)r * P + p0];
+    if (p1 < P) hit1 = match_len[(int64_t)r * P + p1];
+    off_lo = blk_off[r];
+    off_hi = blk_off[r + 1];
+  };
+  if (R > 0) fetch(0);
+  for (int r = 0; r < R; ++r) {
+    const long long n_r = off_hi - off_lo;
+    const long long sc0 = pod_score(hit0, n_r, load0, w_prefix, w_load, thr_pct);
+    const long long sc1 = pod_score(hit1, n_r, load1, w_prefix, w_load, thr_pct);
+    if (r + 1 < R) fetch(r + 1);
+    long long top;
+    int arg;
+    lane_candidate(lane, P, ready_mask, sc0, sc1, top, arg);
+    warp_argmax(top, arg);
+    if (arg == p0) load0 = (int32_t)((uint32_t)load0 + (uint32_t)increment);
+    if (arg == p1) load1 = (int32_t)((uint32_t)load1 + (uint32_t)increment);
+    if (lane == 0) {
+      best_pod[r] = arg;
+      best_score[r] = top;
+    }
+  }
+  if (p0 < P) pod_load[p0] = load0;
+  if (p1 < P) pod_load[p1] = load1;
 }
 
 }  // namespace aibx

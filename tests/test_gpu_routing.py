@@ -319,3 +319,64 @@ def test_routing_cfg5_full():
     for r in range(w.spec.R):                       # matched ids are the request's block table
         seg = o["block_ids"][o["blk_off"][r]: o["blk_off"][r] + 3000]
         assert np.array_equal(seg, w.block_table[r, :3000])
+
+
+# ------------------------------------------------------------------ fused call, sequential assignment
+
+@pytest.mark.parametrize("mk", [W.cfg1_routing, W.cfg2_routing, W.cfg3_routing])
+def test_route_batch_equals_the_three_calls(mk):
+    w = W.build_routing(mk())
+    s = w.spec
+    B, P, R = s.block_tokens, s.num_pods, s.R
+    o = routing_oracle(w)
+    sh, _ = gpu_hash(w.src_tokens, w.src_tok_off, B)
+    from gpu_util import fill_entries
+    keys, masks, ids = fill_entries(w, sh)
+    ix = aibx.Index(s.capacity, P)
+    ix.insert(dev(keys), dev(masks), dev(ids))
+    bo = o["blk_off"]
+    nb = max(int(bo[-1]), 1)
+    d_h = empty(nb, torch.uint64)
+    d_ml, d_al, d_ids = empty(R * P, torch.uint32), empty(R, torch.uint32), empty(nb, torch.uint32)
+    d_bp, d_bs = empty(R, torch.int32), empty(R, torch.int64)
+    for prm, ready in ((None, w.ready_mask), ((7, 3, 25), w.ready_mask & 0xF0F0F0F0F0F0F0F5)):
+        aibx.route_batch(ix, dev(w.tokens), dev(w.tok_off), dev(bo), B, 0, dev(w.pod_load), ready,
+                         prm, d_h, d_ml, d_al, d_ids, d_bp, d_bs)
+        wbp, wbs, _ = oracle.route_score(o["match_len"], bo, w.pod_load, ready, prm)
+        n = int(bo[-1])
+        assert np.array_equal(host(d_h)[:n], o["hashes"])
+        assert np.array_equal(host(d_ml).reshape(R, P), o["match_len"])
+        assert np.array_equal(host(d_al), o["any_len"])
+        assert np.array_equal(host(d_ids)[:n], o["block_ids"])
+        assert np.array_equal(host(d_bp), wbp) and np.array_equal(host(d_bs), wbs)
+    # nullable outputs
+    aibx.route_batch(ix, dev(w.tokens), dev(w.tok_off), dev(bo), B, 0, dev(w.pod_load),
+                     w.ready_mask, None, d_h, d_ml, None, None, d_bp, d_bs)
+    assert np.array_equal(host(d_bp), o["best_pod"])
+    assert aibx.status_fetch() == (0, 0)
+
+
+def test_route_assign_sequential():
+    rng = np.random.default_rng(55)
+    for P in (1, 5, 32, 33, 64):
+        R = 700
+        n = rng.integers(0, 50, R)
+        bo = np.concatenate([[0], np.cumsum(n)]).astype(np.int64)
+        ml = (rng.random((R, P)) * (n[:, None] + 1)).astype(np.uint32)
+        load0 = rng.integers(0, 9, P).astype(np.int32)
+        for ready in ((1 << 64) - 1, 0, int(rng.integers(1, 1 << 62)) & ((1 << P) - 1)):
+            for prm, inc in ((None, 1), ((4, 1, 50), 0), ((2, 5, 10), 3), ((0, 1, 50), 1),
+                             ((1, 1, 0), 2**31 - 1)):
+                d_load = dev(load0.copy())
+                d_bp, d_bs = empty(R, torch.int32), empty(R, torch.int64)
+                aibx.route_assign(dev(ml.reshape(-1)), dev(bo), P, d_load, ready, prm, inc, d_bp, d_bs)
+                wbp, wbs, wload = oracle.route_assign(ml, bo, load0, ready, prm, inc)
+                assert np.array_equal(host(d_bp), wbp), (P, ready, prm, inc)
+                assert np.array_equal(host(d_bs), wbs)
+                assert np.array_equal(host(d_load), wload)
+    # the three-request hand example: pods 1, 2, then 0
+    d_load = dev(np.array([1, 0, 0], np.int32))
+    d_bp, d_bs = empty(3, torch.int32), empty(3, torch.int64)
+    aibx.route_assign(dev(np.zeros(9, np.uint32)), dev(np.array([0, 4, 8, 12], np.int64)), 3, d_load,
+                      7, (4, 1, 50), 1, d_bp, d_bs)
+    assert host(d_bp).tolist() == [1, 2, 0] and host(d_load).tolist() == [2, 1, 1]

@@ -61,6 +61,8 @@ MUTANTS = [
      "", 0),
     ("threshold_on_tokens_not_blocks", "test_oracle_score.py",
      "100 * hit >= (int64_t)prm.threshold_pct * n_r", "100 * hit >= (int64_t)prm.threshold_pct * 16 * n_r", 0),
+    ("assignment_forgets_the_increment", "test_oracle_score.py",
+     "(uint32_t)pod_load[best_pod[r]] + (uint32_t)load_increment", "(uint32_t)pod_load[best_pod[r]]", 0),
     ("layer_major_as_block_major", "test_oracle_kv.py",
      "return ((int64_t)l * L->num_blocks + b) * t;", "return ((int64_t)b * L->num_layers + l) * t;", 0),
     ("buffer_layer_major", "test_oracle_kv.py",

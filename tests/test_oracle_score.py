@@ -61,3 +61,42 @@ def test_special_cases_and_recompute():
         hit = ml.astype(np.int64)
         eff = np.where((hit > 0) & (100 * hit >= prm[2] * n[:, None]), hit, 0)
         assert np.array_equal(sc, prm[0] * eff - prm[1] * load.astype(np.int64)[None, :])
+
+
+def test_sequential_assignment_hand_example_and_invariants():
+    # three equal requests without any cached prefix, loads [1, 0, 0]: least-request with
+    # ties to the lowest pod sends them to pod 1, pod 2, then pod 0 (all three at load 1)
+    ml = np.zeros((3, 3), dtype=np.uint32)
+    bo = [0, 4, 8, 12]
+    bp, bs, load = oracle.route_assign(ml, bo, [1, 0, 0], 0b111, (4, 1, 50), 1)
+    assert bp.tolist() == [1, 2, 0] and bs.tolist() == [0, 0, -1] and load.tolist() == [2, 1, 1]
+    # a cached prefix outweighs load until the pod has taken enough requests: hit 2 of 4 blocks
+    # on pod 0 is worth 8; each assignment adds 3 to its load
+    ml = np.array([[2, 0]] * 4, dtype=np.uint32)
+    bp, bs, load = oracle.route_assign(ml, [0, 4, 8, 12, 16], [0, 0], 0b11, (4, 1, 50), 3)
+    assert bp.tolist() == [0, 0, 0, 1] and bs.tolist() == [8, 5, 2, 0] and load.tolist() == [9, 3]
+    # increment 0 is the snapshot score; general case against a Python loop over numpy scores
+    rng = np.random.default_rng(31)
+    R, P = 300, 11
+    n = rng.integers(0, 40, R)
+    bo = np.concatenate([[0], np.cumsum(n)]).astype(np.int64)
+    ml = (rng.random((R, P)) * (n[:, None] + 1)).astype(np.uint32)
+    load0 = rng.integers(0, 20, P).astype(np.int32)
+    ready = 0b10111011101
+    bp0, bs0, _ = oracle.route_score(ml, bo, load0, ready, (4, 1, 50))
+    bp, bs, load = oracle.route_assign(ml, bo, load0, ready, (4, 1, 50), 0)
+    assert np.array_equal(bp, bp0) and np.array_equal(bs, bs0) and np.array_equal(load, load0)
+    for inc in (1, 7):
+        bp, bs, load = oracle.route_assign(ml, bo, load0, ready, (3, 2, 25), inc)
+        cur = load0.astype(np.int64).copy()
+        rd = np.array([(ready >> p) & 1 for p in range(P)], dtype=bool)
+        for r in range(R):
+            hit = ml[r].astype(np.int64)
+            eff = np.where((hit > 0) & (100 * hit >= 25 * n[r]), hit, 0)
+            sc = np.where(rd, 3 * eff - 2 * cur, I64_MIN)
+            assert bp[r] == int(np.argmax(sc)) and bs[r] == sc.max()
+            cur[bp[r]] += inc
+        assert np.array_equal(load, cur) and load.sum() - load0.sum() == inc * R
+    # nobody ready: nothing is assigned, loads stay
+    bp, bs, load = oracle.route_assign(ml[:5], bo[:6], load0, 0, None, 1)
+    assert (bp == oracle.NO_POD).all() and np.array_equal(load, load0)
