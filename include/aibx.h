@@ -243,6 +243,18 @@ int32_t aibx_kv_scatter(void* d_pool, const aibx_kv_layout_t* layout,
                         const uint32_t* d_block_ids, int64_t n, const void* d_buf,
                         void* stream);
 
+/* The same with the item count on the device: moves the first min(n_max, *d_count) items of the
+ * list (d_count: one uint32 in device memory, read when the kernel starts).  Lets the output
+ * of aibx_collect_blocks (ids + count) flow into the copy without a host round trip; the buffer
+ * must have room for n_max items only if that many can be valid.  INVALID if d_count is null.
+ */
+int32_t aibx_kv_gather_counted(const void* d_pool, const aibx_kv_layout_t* layout,
+                               const uint32_t* d_block_ids, int64_t n_max, const uint32_t* d_count,
+                               void* d_buf, void* stream);
+int32_t aibx_kv_scatter_counted(void* d_pool, const aibx_kv_layout_t* layout,
+                                const uint32_t* d_block_ids, int64_t n_max,
+                                const uint32_t* d_count, const void* d_buf, void* stream);
+
 /* Launch shape of gather/scatter, process-wide; for measurement sweeps.  mode 0 = bulk-async
  * (TMA) ring through shared memory, 1 = 16-byte load/store loop.  chunk_bytes (multiple of 16,
  * 1 KiB..64 KiB) and stages (2..16) size the ring (chunk*stages <= 200 KiB; the stage count

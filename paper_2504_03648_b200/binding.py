@@ -84,6 +84,8 @@ def lib():
             "aibx_collect_blocks_static": [vp, i64, u32, vp, vp, vp],
             "aibx_kv_gather": [vp, C.POINTER(KVLayout), vp, i64, vp, vp],
             "aibx_kv_scatter": [vp, C.POINTER(KVLayout), vp, i64, vp, vp],
+            "aibx_kv_gather_counted": [vp, C.POINTER(KVLayout), vp, i64, vp, vp, vp],
+            "aibx_kv_scatter_counted": [vp, C.POINTER(KVLayout), vp, i64, vp, vp, vp],
             "aibx_kv_set_tuning": [i32, i32, i32, i32],
             "aibx_kv_set_store_lag": [i32],
             "aibx_status_fetch": [vp, C.POINTER(i32), C.POINTER(i64)],
@@ -258,6 +260,18 @@ def kv_gather(pool, layout: KVLayout, block_ids, n: int, buf) -> None:
 def kv_scatter(pool, layout: KVLayout, block_ids, n: int, buf) -> None:
     _check("aibx_kv_scatter", lib().aibx_kv_scatter(
         _ptr(pool), C.byref(layout), _ptr(block_ids, torch.uint32), n, _ptr(buf), _stream()))
+
+
+def kv_gather_counted(pool, layout: KVLayout, block_ids, n_max: int, count, buf) -> None:
+    _check("aibx_kv_gather_counted", lib().aibx_kv_gather_counted(
+        _ptr(pool), C.byref(layout), _ptr(block_ids, torch.uint32), n_max,
+        _ptr(count, torch.uint32), _ptr(buf), _stream()))
+
+
+def kv_scatter_counted(pool, layout: KVLayout, block_ids, n_max: int, count, buf) -> None:
+    _check("aibx_kv_scatter_counted", lib().aibx_kv_scatter_counted(
+        _ptr(pool), C.byref(layout), _ptr(block_ids, torch.uint32), n_max,
+        _ptr(count, torch.uint32), _ptr(buf), _stream()))
 
 
 def kv_set_tuning(mode: int = -1, chunk_bytes: int = 0, stages: int = 0,

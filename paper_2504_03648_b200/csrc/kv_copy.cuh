@@ -38,7 +38,22 @@ struct CopyPlan {
   unsigned int total_chunks;
   uint32_t num_blocks;
   int to_pool;                   // 0 gather (pool -> buf), 1 scatter (buf -> pool)
+  const uint32_t* d_count;       // optional: number of leading items to move, read on the device
+  unsigned int count_base;       // items of earlier launches of the same call
+  unsigned int units_per_item;
 };
+
+// With a device-side count the stream ends after min(items of this launch, *d_count - base).
+__device__ __forceinline__ void apply_device_count(CopyPlan& pl) {
+  if (pl.d_count == nullptr) return;
+  const unsigned int cnt = __ldg(pl.d_count);
+  const unsigned int mine = cnt > pl.count_base ? cnt - pl.count_base : 0u;
+  const unsigned long long units = (unsigned long long)mine * pl.units_per_item;
+  if (units < pl.total_units) {
+    pl.total_units = (unsigned int)units;
+    pl.total_chunks = (pl.total_units + pl.chunk_units - 1) / pl.chunk_units;
+  }
+}
 
 // A chunk before its block ids are known: where its pieces lie in the stream.
 struct ChunkPieces {
@@ -178,6 +193,7 @@ kv_copy_bulk_kernel(CopyPlan pl, int stages, int lag) {
   __shared__ int s_loader_done;
   __shared__ long long s_issued;
 
+  apply_device_count(pl);
   const unsigned int G = gridDim.x;
   const unsigned int first = blockIdx.x;
   if (first >= pl.total_chunks) return;
@@ -335,6 +351,7 @@ __global__ void __launch_bounds__(kLdstThreads) kv_copy_ldst_kernel(CopyPlan pl)
   __shared__ const char* s_src[kMaxPieces];
   __shared__ char* s_dst[kMaxPieces];
   __shared__ unsigned int s_units[kMaxPieces];
+  apply_device_count(pl);
   for (unsigned int c = blockIdx.x; c < pl.total_chunks; c += gridDim.x) {
     if (threadIdx.x == 0) {
       ChunkPieces cp;
@@ -395,7 +412,8 @@ inline CopyTuning& copy_tuning() {
 }
 
 inline int32_t launch_kv_copy(const void* pool, const aibx_kv_layout_t* L, const uint32_t* d_ids,
-                              int64_t n, const void* buf, int to_pool, cudaStream_t st) {
+                              int64_t n, const void* buf, int to_pool, cudaStream_t st,
+                              const uint32_t* d_count = nullptr) {
   if (!L || n < 0) return AIBX_ERR_INVALID;
   if ((L->layout != 0 && L->layout != 1) || L->num_layers <= 0 || L->num_kv_heads <= 0 ||
       L->block_tokens <= 0 || L->head_dim <= 0 || L->elem_bytes <= 0)
@@ -450,6 +468,9 @@ inline int32_t launch_kv_copy(const void* pool, const aibx_kv_layout_t* L, const
     pl.ids = d_ids + done;
     pl.pool = const_cast<char*>(static_cast<const char*>(pool));
     pl.buf = const_cast<char*>(static_cast<const char*>(buf)) + done * block_bytes;
+    pl.d_count = d_count;
+    pl.count_base = (unsigned int)(done > 0xFFFFFFFFLL ? 0xFFFFFFFFLL : done);
+    pl.units_per_item = (unsigned int)units_per_item;
     pl.total_units = (unsigned int)(items * units_per_item);
     pl.total_chunks = (pl.total_units + pl.chunk_units - 1) / pl.chunk_units;
     long long grid = (long long)sm_count() * (tn.mode == 0 ? tn.ctas_per_sm : 8);

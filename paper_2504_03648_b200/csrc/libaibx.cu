@@ -334,6 +334,20 @@ int32_t aibx_kv_scatter(void* d_pool, const aibx_kv_layout_t* layout,
   return launch_kv_copy(d_pool, layout, d_block_ids, n, d_buf, 1, as_stream(stream));
 }
 
+int32_t aibx_kv_gather_counted(const void* d_pool, const aibx_kv_layout_t* layout,
+                               const uint32_t* d_block_ids, int64_t n_max, const uint32_t* d_count,
+                               void* d_buf, void* stream) {
+  if (!d_count) return AIBX_ERR_INVALID;
+  return launch_kv_copy(d_pool, layout, d_block_ids, n_max, d_buf, 0, as_stream(stream), d_count);
+}
+
+int32_t aibx_kv_scatter_counted(void* d_pool, const aibx_kv_layout_t* layout,
+                                const uint32_t* d_block_ids, int64_t n_max,
+                                const uint32_t* d_count, const void* d_buf, void* stream) {
+  if (!d_count) return AIBX_ERR_INVALID;
+  return launch_kv_copy(d_pool, layout, d_block_ids, n_max, d_buf, 1, as_stream(stream), d_count);
+}
+
 int32_t aibx_kv_set_tuning(int32_t mode, int32_t chunk_bytes, int32_t stages,
                            int32_t ctas_per_sm) {
   CopyTuning t = copy_tuning();

@@ -285,3 +285,32 @@ def test_cfg5_full_size_fp8_mixed():
                               np.zeros(1, np.uint32), item)
             assert np.array_equal(read_block(pool, kv, int(ids_put[i])), mini)
     print("cfg5 pool blocks used:", kv.num_blocks, "(shrunk)" if shrunk else "(full)")
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("layout", [0, 1])
+def test_counted_variants_stop_at_the_device_count(layout, mode):
+    aibx.kv_set_tuning(mode, 16384, 4, 1)
+    kv = W.KVSpec("counted", 9, layout, 3, 5, 16, 40, 2, 97)          # 38,400-byte blocks
+    lay_g, lay_o = kv_layout_gpu(kv), kv_layout_oracle(kv)
+    pool_h = W.host_pool(kv)
+    ids = W.distinct_ids(4, 97, 60)
+    ids[7] = NO_BLOCK
+    for cnt in (0, 1, 33, 60, 1000):
+        m = min(cnt, 60)
+        pool_d = dev(pool_h)
+        buf_w, buf_d = guarded(60 * kv.block_bytes, 0xEE)
+        d_cnt = dev(np.array([cnt], np.uint32))
+        aibx.kv_gather_counted(pool_d, lay_g, dev(ids), 60, d_cnt, buf_d)
+        want = np.full(60 * kv.block_bytes, 0xEE, dtype=np.uint8)
+        oracle.kv_gather(pool_h, lay_o, ids[:m], want[: m * kv.block_bytes])
+        assert np.array_equal(host(buf_d), want), cnt
+        assert guards_intact(buf_w, 60 * kv.block_bytes, 0xEE)
+        # scatter the first `cnt` items of a fresh buffer into a shuffled id list
+        ids_s = W.distinct_ids(5, 97, 60)
+        fresh = W.pool_bytes(77, 0, 60 * kv.block_bytes)
+        aibx.kv_scatter_counted(pool_d, lay_g, dev(ids_s), 60, d_cnt, dev(fresh))
+        pool_want = pool_h.copy()
+        oracle.kv_scatter(pool_want, lay_o, ids_s[:m], fresh[: m * kv.block_bytes].copy())
+        assert np.array_equal(host(pool_d), pool_want), cnt
+        assert aibx.status_fetch() == (0, 0)
