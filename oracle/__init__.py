@@ -80,11 +80,15 @@ def lib():
         L.aibxo_collect_blocks.argtypes = [vp, i64, u32, vp, C.POINTER(u32)]
         L.aibxo_kv_gather.argtypes = [vp, C.POINTER(_Layout), vp, i64, vp, C.POINTER(i64)]
         L.aibxo_kv_scatter.argtypes = [vp, C.POINTER(_Layout), vp, i64, vp, C.POINTER(i64)]
+        L.aibxo_kv_gather_inner.argtypes = [vp, C.POINTER(_Layout), i32, i32, vp, i64, vp,
+                                            C.POINTER(i64)]
+        L.aibxo_kv_scatter_inner.argtypes = [vp, C.POINTER(_Layout), i32, i32, vp, i64, vp,
+                                             C.POINTER(i64)]
         for name in (
             "aibxo_hash_blocks aibxo_index_create aibxo_index_destroy aibxo_index_clear "
             "aibxo_index_insert aibxo_index_evict aibxo_index_lookup aibxo_index_stats "
             "aibxo_match_prefix aibxo_route_score aibxo_route_assign aibxo_collect_blocks aibxo_kv_gather "
-            "aibxo_kv_scatter"
+            "aibxo_kv_scatter aibxo_kv_gather_inner aibxo_kv_scatter_inner"
         ).split():
             getattr(L, name).restype = i32
         _lib = L
@@ -244,4 +248,26 @@ def kv_scatter(pool: np.ndarray, lay: _Layout, ids, buf: np.ndarray):
     assert pool.flags.c_contiguous and buf.flags.c_contiguous
     bad = C.c_int64()
     rc = lib().aibxo_kv_scatter(_p(pool), C.byref(lay), _p(ids), len(ids), _p(buf), C.byref(bad))
+    return rc, bad.value
+
+
+def kv_gather_inner(pool: np.ndarray, lay: _Layout, pool_inner: int, buf_inner: int, ids,
+                    buf: np.ndarray):
+    ids = _arr(ids, np.uint32)
+    assert pool.dtype == np.uint8 and buf.dtype == np.uint8
+    assert pool.flags.c_contiguous and buf.flags.c_contiguous
+    bad = C.c_int64()
+    rc = lib().aibxo_kv_gather_inner(_p(pool), C.byref(lay), pool_inner, buf_inner, _p(ids),
+                                     len(ids), _p(buf), C.byref(bad))
+    return rc, bad.value
+
+
+def kv_scatter_inner(pool: np.ndarray, lay: _Layout, pool_inner: int, buf_inner: int, ids,
+                     buf: np.ndarray):
+    ids = _arr(ids, np.uint32)
+    assert pool.dtype == np.uint8 and buf.dtype == np.uint8
+    assert pool.flags.c_contiguous and buf.flags.c_contiguous
+    bad = C.c_int64()
+    rc = lib().aibxo_kv_scatter_inner(_p(pool), C.byref(lay), pool_inner, buf_inner, _p(ids),
+                                      len(ids), _p(buf), C.byref(bad))
     return rc, bad.value

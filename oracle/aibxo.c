@@ -473,3 +473,58 @@ int32_t aibxo_kv_scatter(void* pool, const aibxo_kv_layout_t* L, const uint32_t*
   if (bad) *bad = nbad;
   return nbad ? AIBXO_ERR_RANGE : AIBXO_OK;
 }
+
+/* ------------------------------------------------------------------ inner-order change - */
+/* Offset of row (kv, head, token) inside a tile stored in the given inner order. */
+
+static int64_t row_offset(const aibxo_kv_layout_t* L, int32_t inner, int32_t kv, int32_t head,
+                          int32_t token) {
+  int64_t row = (int64_t)L->head_dim * L->elem_bytes;
+  int64_t H = L->num_kv_heads, T = L->block_tokens;
+  if (inner == 0) return (((int64_t)kv * H + head) * T + token) * row;
+  return (((int64_t)kv * T + token) * H + head) * row;
+}
+
+static int32_t copy_inner(uint8_t* pool, const aibxo_kv_layout_t* L, int32_t pool_inner,
+                          int32_t buf_inner, const uint32_t* ids, int64_t n, uint8_t* buf,
+                          int to_pool, int64_t* bad) {
+  if (bad) *bad = 0;
+  if (!layout_ok(L) || n < 0) return AIBXO_ERR_INVALID;
+  if ((pool_inner != 0 && pool_inner != 1) || (buf_inner != 0 && buf_inner != 1))
+    return AIBXO_ERR_INVALID;
+  if (n == 0) return AIBXO_OK;
+  if (!pool || !ids || !buf) return AIBXO_ERR_INVALID;
+  int64_t t = tile_bytes(L);
+  int64_t row = (int64_t)L->head_dim * L->elem_bytes;
+  int64_t nbad = 0;
+  for (int64_t i = 0; i < n; ++i) {
+    if (ids[i] == AIBXO_NO_BLOCK) continue;
+    if (ids[i] >= L->num_blocks) { ++nbad; continue; }
+    for (int32_t l = 0; l < L->num_layers; ++l) {
+      uint8_t* ptile = pool + pool_offset(L, ids[i], l);
+      uint8_t* btile = buf + (i * L->num_layers + l) * t;
+      for (int32_t kv = 0; kv < 2; ++kv)
+        for (int32_t h = 0; h < L->num_kv_heads; ++h)
+          for (int32_t tok = 0; tok < L->block_tokens; ++tok) {
+            uint8_t* prow = ptile + row_offset(L, pool_inner, kv, h, tok);
+            uint8_t* brow = btile + row_offset(L, buf_inner, kv, h, tok);
+            if (to_pool) memcpy(prow, brow, (size_t)row);
+            else memcpy(brow, prow, (size_t)row);
+          }
+    }
+  }
+  if (bad) *bad = nbad;
+  return nbad ? AIBXO_ERR_RANGE : AIBXO_OK;
+}
+
+int32_t aibxo_kv_gather_inner(const void* pool, const aibxo_kv_layout_t* L, int32_t pool_inner,
+                              int32_t buf_inner, const uint32_t* ids, int64_t n, void* buf,
+                              int64_t* bad) {
+  return copy_inner((uint8_t*)pool, L, pool_inner, buf_inner, ids, n, (uint8_t*)buf, 0, bad);
+}
+
+int32_t aibxo_kv_scatter_inner(void* pool, const aibxo_kv_layout_t* L, int32_t pool_inner,
+                               int32_t buf_inner, const uint32_t* ids, int64_t n, const void* buf,
+                               int64_t* bad) {
+  return copy_inner((uint8_t*)pool, L, pool_inner, buf_inner, ids, n, (uint8_t*)buf, 1, bad);
+}

@@ -104,4 +104,15 @@ int32_t aibxo_kv_gather(const void* pool, const aibxo_kv_layout_t* lay, const ui
 int32_t aibxo_kv_scatter(void* pool, const aibxo_kv_layout_t* lay, const uint32_t* ids,
                          int64_t n, const void* buf, int64_t* bad);
 
+/* Gather / scatter with a change of the order inside a tile (Section 3.2.5: engines differ in
+ * how they store a block, so the exchange buffer may need another order than the pool).
+ * inner order 0 = [K/V][head][token][dim], 1 = [K/V][token][head][dim]; rows of head_dim elements
+ * move whole.  Equal orders reduce to aibxo_kv_gather / aibxo_kv_scatter. */
+int32_t aibxo_kv_gather_inner(const void* pool, const aibxo_kv_layout_t* lay, int32_t pool_inner,
+                              int32_t buf_inner, const uint32_t* ids, int64_t n, void* buf,
+                              int64_t* bad);
+int32_t aibxo_kv_scatter_inner(void* pool, const aibxo_kv_layout_t* lay, int32_t pool_inner,
+                               int32_t buf_inner, const uint32_t* ids, int64_t n, const void* buf,
+                               int64_t* bad);
+
 #endif /* AIBXO_H_ */

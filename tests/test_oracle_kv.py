@@ -90,3 +90,50 @@ def test_skips_and_range_errors():
     assert rc == oracle.ERR_RANGE and bad == 1 and np.array_equal(pool, snap)
     rc, bad = oracle.kv_gather(pool, lay, np.zeros(0, dtype=np.uint32), buf)
     assert rc == oracle.OK
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_inner_order_change_is_a_numpy_transpose(layout):
+    rng = np.random.default_rng(40 + layout)
+    L, H, Bt, D, E, nb = 3, 4, 6, 8, 2, 13
+    row = D * E
+    tile = 2 * H * Bt * row
+    pool = _pool(rng, layout, L, nb, tile)
+    lay = oracle.kv_layout(layout, L, H, Bt, D, E, nb)
+    ids = rng.integers(0, nb, 9).astype(np.uint32)
+    ids[4] = NO_BLOCK
+    plain = np.full(9 * L * tile, 0xEE, dtype=np.uint8)
+    oracle.kv_gather(pool.reshape(-1), lay, ids, plain)
+    for pi in (0, 1):
+        for bi in (0, 1):
+            got = np.full(9 * L * tile, 0xEE, dtype=np.uint8)
+            rc, bad = oracle.kv_gather_inner(pool.reshape(-1), lay, pi, bi, ids, got)
+            assert rc == oracle.OK
+            # view the plainly gathered tiles in the pool's inner order, reorder with numpy
+            shape_p = (9, L, 2, H, Bt, row) if pi == 0 else (9, L, 2, Bt, H, row)
+            v = plain.reshape(shape_p)
+            want = v if pi == bi else v.transpose(0, 1, 2, 4, 3, 5)
+            want = np.ascontiguousarray(want).reshape(-1)
+            assert np.array_equal(got, want), (pi, bi)
+            # scatter with the same orders brings every named block back
+            pool2 = np.zeros_like(pool)
+            keep = ids != NO_BLOCK
+            oracle.kv_scatter_inner(pool2.reshape(-1), lay, pi, bi, ids, got)
+            for b in set(ids[keep].tolist()):
+                a = pool[b] if layout == 0 else pool[:, b]
+                c = pool2[b] if layout == 0 else pool2[:, b]
+                assert np.array_equal(a, c)
+
+
+def test_inner_order_hand_example():
+    # one block, one layer, 2 heads x 3 tokens, rows of 1 byte: K rows 0..5, V rows 6..11
+    lay = oracle.kv_layout(0, 1, 2, 3, 1, 1, 1)
+    pool = np.arange(12, dtype=np.uint8)                 # [kv][head][token]
+    buf = np.zeros(12, dtype=np.uint8)
+    oracle.kv_gather_inner(pool, lay, 0, 1, np.zeros(1, np.uint32), buf)
+    assert buf.tolist() == [0, 3, 1, 4, 2, 5, 6, 9, 7, 10, 8, 11]   # [kv][token][head]
+    back = np.zeros(12, dtype=np.uint8)
+    oracle.kv_scatter_inner(back, lay, 0, 1, np.zeros(1, np.uint32), buf)
+    assert back.tolist() == list(range(12))
+    rc, _ = oracle.kv_gather_inner(pool, lay, 2, 0, np.zeros(1, np.uint32), buf)
+    assert rc == oracle.ERR_INVALID
