@@ -255,6 +255,24 @@ int32_t aibx_kv_scatter_counted(void* d_pool, const aibx_kv_layout_t* layout,
                                 const uint32_t* d_block_ids, int64_t n_max,
                                 const uint32_t* d_count, const void* d_buf, void* stream);
 
+/* Gather / scatter with a change of the order inside a tile (Section 3.2.5: the cache serves
+ * different engines, and engines differ in how they lay a block out).  Inner order
+ * AIBX_INNER_HEAD_TOKEN (0) = [K/V][head][token][dim], AIBX_INNER_TOKEN_HEAD (1) =
+ * [K/V][token][head][dim]; pool_inner describes the pool's tiles, buf_inner the buffer's.  Rows
+ * of head_dim elements move whole (head_dim * elem_bytes must be a multiple of 16 and at most
+ * 32 KiB: UNSUPPORTED otherwise); everything else - layouts, ids, skipping, errors - is as in
+ * aibx_kv_gather / aibx_kv_scatter, to which equal orders reduce.  The transposition goes
+ * through shared memory so that global reads and writes both stay whole rows.
+ */
+#define AIBX_INNER_HEAD_TOKEN 0
+#define AIBX_INNER_TOKEN_HEAD 1
+int32_t aibx_kv_gather_inner(const void* d_pool, const aibx_kv_layout_t* layout, int32_t pool_inner,
+                             int32_t buf_inner, const uint32_t* d_block_ids, int64_t n,
+                             void* d_buf, void* stream);
+int32_t aibx_kv_scatter_inner(void* d_pool, const aibx_kv_layout_t* layout, int32_t pool_inner,
+                              int32_t buf_inner, const uint32_t* d_block_ids, int64_t n,
+                              const void* d_buf, void* stream);
+
 /* Launch shape of gather/scatter, process-wide; for measurement sweeps.  mode 0 = bulk-async
  * (TMA) ring through shared memory, 1 = 16-byte load/store loop.  chunk_bytes (multiple of 16,
  * 1 KiB..64 KiB) and stages (2..16) size the ring (chunk*stages <= 200 KiB; the stage count

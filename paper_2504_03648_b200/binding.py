@@ -86,6 +86,8 @@ def lib():
             "aibx_kv_scatter": [vp, C.POINTER(KVLayout), vp, i64, vp, vp],
             "aibx_kv_gather_counted": [vp, C.POINTER(KVLayout), vp, i64, vp, vp, vp],
             "aibx_kv_scatter_counted": [vp, C.POINTER(KVLayout), vp, i64, vp, vp, vp],
+            "aibx_kv_gather_inner": [vp, C.POINTER(KVLayout), i32, i32, vp, i64, vp, vp],
+            "aibx_kv_scatter_inner": [vp, C.POINTER(KVLayout), i32, i32, vp, i64, vp, vp],
             "aibx_kv_set_tuning": [i32, i32, i32, i32],
             "aibx_kv_set_store_lag": [i32],
             "aibx_status_fetch": [vp, C.POINTER(i32), C.POINTER(i64)],
@@ -272,6 +274,20 @@ def kv_scatter_counted(pool, layout: KVLayout, block_ids, n_max: int, count, buf
     _check("aibx_kv_scatter_counted", lib().aibx_kv_scatter_counted(
         _ptr(pool), C.byref(layout), _ptr(block_ids, torch.uint32), n_max,
         _ptr(count, torch.uint32), _ptr(buf), _stream()))
+
+
+def kv_gather_inner(pool, layout: KVLayout, pool_inner: int, buf_inner: int, block_ids, n: int,
+                    buf) -> None:
+    _check("aibx_kv_gather_inner", lib().aibx_kv_gather_inner(
+        _ptr(pool), C.byref(layout), pool_inner, buf_inner, _ptr(block_ids, torch.uint32), n,
+        _ptr(buf), _stream()))
+
+
+def kv_scatter_inner(pool, layout: KVLayout, pool_inner: int, buf_inner: int, block_ids, n: int,
+                     buf) -> None:
+    _check("aibx_kv_scatter_inner", lib().aibx_kv_scatter_inner(
+        _ptr(pool), C.byref(layout), pool_inner, buf_inner, _ptr(block_ids, torch.uint32), n,
+        _ptr(buf), _stream()))
 
 
 def kv_set_tuning(mode: int = -1, chunk_bytes: int = 0, stages: int = 0,

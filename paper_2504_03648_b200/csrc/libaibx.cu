@@ -10,6 +10,7 @@
 #include "hash_blocks.cuh"
 #include "index.cuh"
 #include "kv_copy.cuh"
+#include "kv_permute.cuh"
 #include "route_score.cuh"
 
 using namespace aibx;
@@ -346,6 +347,20 @@ int32_t aibx_kv_scatter_counted(void* d_pool, const aibx_kv_layout_t* layout,
                                 const uint32_t* d_count, const void* d_buf, void* stream) {
   if (!d_count) return AIBX_ERR_INVALID;
   return launch_kv_copy(d_pool, layout, d_block_ids, n_max, d_buf, 1, as_stream(stream), d_count);
+}
+
+int32_t aibx_kv_gather_inner(const void* d_pool, const aibx_kv_layout_t* layout, int32_t pool_inner,
+                             int32_t buf_inner, const uint32_t* d_block_ids, int64_t n,
+                             void* d_buf, void* stream) {
+  return launch_kv_permute(d_pool, layout, pool_inner, buf_inner, d_block_ids, n, d_buf, 0,
+                           as_stream(stream));
+}
+
+int32_t aibx_kv_scatter_inner(void* d_pool, const aibx_kv_layout_t* layout, int32_t pool_inner,
+                              int32_t buf_inner, const uint32_t* d_block_ids, int64_t n,
+                              const void* d_buf, void* stream) {
+  return launch_kv_permute(d_pool, layout, pool_inner, buf_inner, d_block_ids, n, d_buf, 1,
+                           as_stream(stream));
 }
 
 int32_t aibx_kv_set_tuning(int32_t mode, int32_t chunk_bytes, int32_t stages,

@@ -1,0 +1,103 @@
+"""GPU parity for gather/scatter with a change of the order inside a tile (head/token
+transposition staged through shared memory), byte for byte against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import NO_BLOCK, dev, empty, host, kv_layout_gpu, kv_layout_oracle
+from paper_2504_03648_b200 import binding as aibx
+from paper_2504_03648_b200 import synth
+from paper_2504_03648_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [
+    # layers, heads, tokens, dim, elem bytes, blocks
+    (2, 4, 16, 64, 2, 50),      # 128-byte rows, 8 KiB planes
+    (3, 8, 16, 128, 2, 40),     # Llama-class: 256-byte rows, 32 KiB planes (one chunk each)
+    (2, 8, 32, 128, 2, 30),     # 64 KiB planes: two chunks per plane
+    (2, 5, 7, 24, 2, 33),       # odd counts, 48-byte rows
+    (1, 4, 32, 128, 1, 64),     # fp8: 128-byte rows
+    (1, 3, 5, 520, 4, 9),       # 2,080-byte rows, 15 rows per chunk of a 15-row plane
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("layout", [0, 1])
+def test_inner_order_gather_and_scatter(layout, shape):
+    L, H, T, D, E, nb = shape
+    kv = W.KVSpec("inner", 21, layout, L, H, T, D, E, nb)
+    lay_g, lay_o = kv_layout_gpu(kv), kv_layout_oracle(kv)
+    pool_h = W.host_pool(kv)
+    rng = np.random.default_rng(L * 100 + H)
+    n = 70
+    ids_g = rng.integers(0, nb, n).astype(np.uint32)
+    ids_g[[2, 40]] = NO_BLOCK
+    ids_g[[5, 69]] = [nb, 0xFFFFFFFE]
+    ids_s = rng.permutation(nb)[: min(nb, n)].astype(np.uint32)
+    ids_s[1] = NO_BLOCK
+    for pi, bi in ((0, 1), (1, 0), (0, 0), (1, 1)):
+        pool_d = dev(pool_h)
+        buf_d = torch.full((n * kv.block_bytes,), 0xEE, dtype=torch.uint8, device="cuda")
+        aibx.kv_gather_inner(pool_d, lay_g, pi, bi, dev(ids_g), n, buf_d)
+        want = np.full(n * kv.block_bytes, 0xEE, dtype=np.uint8)
+        rc, bad = oracle.kv_gather_inner(pool_h, lay_o, pi, bi, ids_g, want)
+        assert np.array_equal(host(buf_d), want), (pi, bi)
+        assert aibx.status_fetch() == (aibx.ERR_RANGE, bad) and bad == 2
+        assert np.array_equal(host(pool_d), pool_h)
+        m = len(ids_s)
+        aibx.kv_scatter_inner(pool_d, lay_g, pi, bi, dev(ids_s), m, buf_d)
+        pool_want = pool_h.copy()
+        oracle.kv_scatter_inner(pool_want, lay_o, pi, bi, ids_s, want[: m * kv.block_bytes].copy())
+        assert np.array_equal(host(pool_d), pool_want), (pi, bi)
+        assert np.array_equal(host(buf_d), want)
+        assert aibx.status_fetch() == (0, 0)
+
+
+def test_inner_order_round_trip_and_invalid():
+    kv = W.KVSpec("rt", 22, 1, 2, 8, 16, 128, 2, 64)
+    lay = kv_layout_gpu(kv)
+    pool_h = W.host_pool(kv)
+    pool_d = dev(pool_h)
+    ids = W.distinct_ids(9, 64, 48)
+    buf = empty(48 * kv.block_bytes, torch.uint8)
+    aibx.kv_gather_inner(pool_d, lay, 0, 1, dev(ids), 48, buf)
+    plain = empty(48 * kv.block_bytes, torch.uint8)
+    aibx.kv_gather(pool_d, lay, dev(ids), 48, plain)
+    # the transposed buffer is the plain one with head and token axes swapped
+    p = host(plain).reshape(48, 2, 2, 8, 16, 256)
+    assert np.array_equal(host(buf).reshape(48, 2, 2, 16, 8, 256), p.transpose(0, 1, 2, 4, 3, 5))
+    pool_d.zero_()
+    aibx.kv_scatter_inner(pool_d, lay, 0, 1, dev(ids), 48, buf)
+    back = empty(48 * kv.block_bytes, torch.uint8)
+    aibx.kv_gather(pool_d, lay, dev(ids), 48, back)
+    assert torch.equal(back, plain)
+    for pi, bi in ((2, 0), (0, -1)):
+        with pytest.raises(aibx.AibxError) as e:
+            aibx.kv_gather_inner(pool_d, lay, pi, bi, dev(ids), 48, buf)
+        assert e.value.code == aibx.ERR_INVALID
+    odd = aibx.KVLayout(0, 1, 2, 4, 12, 2, 8)                 # 24-byte rows, 384-byte tiles
+    with pytest.raises(aibx.AibxError) as e:
+        aibx.kv_gather_inner(pool_d, odd, 0, 1, dev(ids[:2]), 2, buf)
+    assert e.value.code == aibx.ERR_UNSUPPORTED
+    assert aibx.status_fetch() == (0, 0)
+
+
+def test_inner_order_large_launch_bandwidth_shape():
+    """cfg2 block shape, 600 blocks out of a 2 GiB pool: sampled against the oracle."""
+    kv = W.scaled(W.cfg2_kv(), num_blocks=1000)
+    pool = empty(kv.pool_bytes, torch.uint8)
+    synth.fill_pool(pool, kv)
+    n = 600
+    ids = W.distinct_ids(3, kv.num_blocks, n)
+    buf = empty(n * kv.block_bytes, torch.uint8)
+    lay = kv_layout_gpu(kv)
+    aibx.kv_gather_inner(pool, lay, 0, 1, dev(ids), n, buf)
+    assert aibx.status_fetch() == (0, 0)
+    lay1 = kv_layout_oracle(kv, layout=0, num_blocks=1)
+    for i in (0, 1, 299, n - 1):
+        mini = W.logical_blocks(kv, [ids[i]])
+        want = np.zeros(kv.block_bytes, dtype=np.uint8)
+        oracle.kv_gather_inner(mini, lay1, 0, 1, np.zeros(1, np.uint32), want)
+        assert np.array_equal(host(buf.view(n, kv.block_bytes)[i]), want)

@@ -91,11 +91,15 @@ def _run_mutant(args):
     lib = os.path.join(d, "libmutant.so")
     subprocess.check_call(["gcc", "-std=c99", "-O1", "-w", "-fPIC", "-shared",
                            os.path.join(d, "aibxo.c"), "-o", lib])
-    env = dict(os.environ, AIBXO_LIB_OVERRIDE=lib, PYTHONDONTWRITEBYTECODE="1")
-    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
-                        os.path.join(ROOT, "tests", pin_file)],
-                       cwd=ROOT, env=env, stdout=subprocess.PIPE, stderr=subprocess.STDOUT,
-                       timeout=600)
+    env = dict(os.environ, AIBXO_LIB_OVERRIDE=lib, PYTHONDONTWRITEBYTECODE="1",
+               OMP_NUM_THREADS="1", MKL_NUM_THREADS="1")
+    try:
+        r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
+                            os.path.join(ROOT, "tests", pin_file)],
+                           cwd=ROOT, env=env, stdout=subprocess.PIPE, stderr=subprocess.STDOUT,
+                           timeout=240)
+    except subprocess.TimeoutExpired:
+        return name, -9, "timed out (a broken copy that never returns is not a pass either)"
     return name, r.returncode, r.stdout.decode()[-400:]
 
 
