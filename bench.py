@@ -964,7 +964,44 @@ def case_hash_sweep(args):
     print(json.dumps({"case": "hash_sweep", "results": out, "status": aibx.status_fetch()}))
 
 
-CASES = {"hash_sweep": case_hash_sweep, "oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
+def case_kv_inner(args):
+    """Gather/scatter with the head/token order of every tile swapped on the way (cfg2 block
+    shape, 1,600 blocks = 3.4 GB per direction) next to the plain gather of the same blocks."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import synth
+    from paper_2504_03648_b200 import workloads as W
+
+    out = []
+    for name, kv, n in (("cfg2 shape", W.scaled(W.cfg2_kv(), num_blocks=4096), 1600),
+                        ("cfg4 shape", W.scaled(W.cfg4_kv(), num_blocks=2000), 640),
+                        ("cfg5 shape", W.scaled(W.cfg5_kv(), num_blocks=8000), 3000)):
+        pool = torch.empty(kv.pool_bytes, dtype=torch.uint8, device="cuda")
+        synth.fill_pool(pool, kv)
+        ids = torch.from_numpy(W.distinct_ids(7, kv.num_blocks, n)).cuda()
+        buf = torch.empty(n * kv.block_bytes, dtype=torch.uint8, device="cuda")
+        lay = aibx.KVLayout(kv.layout, kv.num_layers, kv.num_kv_heads, kv.block_tokens,
+                            kv.head_dim, kv.elem_bytes, kv.num_blocks)
+        nbytes = 2 * n * kv.block_bytes
+        t_plain = statistics.median(_event_times(
+            torch, lambda: aibx.kv_gather(pool, lay, ids, n, buf), 10, 3))
+        t_g = statistics.median(_event_times(
+            torch, lambda: aibx.kv_gather_inner(pool, lay, 0, 1, ids, n, buf), 10, 3))
+        t_s = statistics.median(_event_times(
+            torch, lambda: aibx.kv_scatter_inner(pool, lay, 0, 1, ids, n, buf), 10, 3))
+        out.append({"shape": name, "blocks": n, "bytes_read_plus_written": nbytes,
+                    "plain_gather_GBps": round(nbytes / (t_plain * 1e-3) / 1e9, 1),
+                    "gather_inner_GBps": round(nbytes / (t_g * 1e-3) / 1e9, 1),
+                    "scatter_inner_GBps": round(nbytes / (t_s * 1e-3) / 1e9, 1)})
+        del pool, buf
+        torch.cuda.empty_cache()
+    peak, kind = measured_peak_hbm()
+    print(json.dumps({"case": "kv_inner", "peak": peak, "peak_kind": kind, "results": out,
+                      "status": aibx.status_fetch()}))
+
+
+CASES = {"kv_inner": case_kv_inner, "hash_sweep": case_hash_sweep, "oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
          "cfg4": case_cfg4, "cfg5": case_cfg5, "lookup_flat": case_lookup_flat}
 
 

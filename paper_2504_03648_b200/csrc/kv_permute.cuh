@@ -185,14 +185,27 @@ kv_permute_kernel(PermPlan pl, int stages, unsigned int stage_bytes) {
         uint4* dst = reinterpret_cast<uint4*>(s_dst[s]);
         const unsigned int row0 = s_row0[s];
         const unsigned int nvec = rows * vpr;
-        for (unsigned int v = tid; v < nvec; v += nthreads) {
-          const unsigned int r_local = v / vpr;
-          const unsigned int col = v - r_local * vpr;
-          const unsigned int rs = row0 + r_local;              // source row [a][b]
-          const unsigned int a = rs / pl.src_inner;
-          const unsigned int b = rs - a * pl.src_inner;
-          const unsigned int rd = b * pl.src_outer + a;        // destination row [b][a]
-          __stcs(dst + (size_t)rd * vpr + col, stage[v]);
+        if (rows == pl.rows_per_plane) {
+          // the whole plane is on chip: walk the DESTINATION in order, so that the CTA's
+          // stores of one pass form one contiguous run
+          for (unsigned int v = tid; v < nvec; v += nthreads) {
+            const unsigned int rd = v / vpr;                     // destination row [b][a]
+            const unsigned int col = v - rd * vpr;
+            const unsigned int b = rd / pl.src_outer;
+            const unsigned int a = rd - b * pl.src_outer;
+            const unsigned int rs = a * pl.src_inner + b;        // source row [a][b]
+            __stcs(dst + v, stage[(size_t)rs * vpr + col]);
+          }
+        } else {
+          for (unsigned int v = tid; v < nvec; v += nthreads) {
+            const unsigned int r_local = v / vpr;
+            const unsigned int col = v - r_local * vpr;
+            const unsigned int rs = row0 + r_local;              // source row [a][b]
+            const unsigned int a = rs / pl.src_inner;
+            const unsigned int b = rs - a * pl.src_inner;
+            const unsigned int rd = b * pl.src_outer + a;        // destination row [b][a]
+            __stcs(dst + (size_t)rd * vpr + col, stage[v]);
+          }
         }
       }
       __syncwarp();
