@@ -104,6 +104,20 @@ int32_t aibx_index_lookup(const aibx_index_t* index, const uint64_t* d_keys,
 int32_t aibx_index_stats(const aibx_index_t* index, uint64_t* live, uint64_t* capacity,
                          void* stream);
 
+/* export: every live entry (key, pod mask, block id) into caller arrays of max_entries
+ *         elements, in no particular order; *d_count (uint64, device) = number of live entries,
+ *         which may exceed max_entries (the surplus is counted, not written).  Arrays may be
+ *         null to only count.  Async on stream.
+ * rehash: move the index into a table of new_capacity slots (power of two >= 8), dropping the
+ *         slots freed by evict on the way; the way out of a FULL table.  FULL (and no change) if
+ *         the live entries do not fit, NOMEM if the new table cannot be allocated.  Syncs the
+ *         device; the handle stays valid.
+ */
+int32_t aibx_index_export(const aibx_index_t* index, uint64_t* d_keys, uint64_t* d_masks,
+                          uint32_t* d_block_ids, uint64_t max_entries, uint64_t* d_count,
+                          void* stream);
+int32_t aibx_index_rehash(aibx_index_t* index, uint64_t new_capacity);
+
 /* ---------------------------------------------------------------------------------------
  * Longest cached prefix (Section 3.2.2, policy prefix-cache-aware: how much of a request's
  * prefix each instance can reuse).  For request r and pod p:

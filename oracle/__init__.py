@@ -74,6 +74,8 @@ def lib():
         L.aibxo_index_evict.argtypes = [vp, vp, vp, vp, i64]
         L.aibxo_index_lookup.argtypes = [vp, vp, vp, vp, i64]
         L.aibxo_index_stats.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
+        L.aibxo_index_export.argtypes = [vp, vp, vp, vp, u64, C.POINTER(u64)]
+        L.aibxo_index_rehash.argtypes = [vp, u64]
         L.aibxo_match_prefix.argtypes = [vp, vp, vp, i32, vp, vp, vp]
         L.aibxo_route_score.argtypes = [vp, vp, i32, i32, vp, u64, C.POINTER(_Params), vp, vp, vp]
         L.aibxo_route_assign.argtypes = [vp, vp, i32, i32, vp, u64, C.POINTER(_Params), i32, vp, vp]
@@ -87,6 +89,7 @@ def lib():
         for name in (
             "aibxo_hash_blocks aibxo_index_create aibxo_index_destroy aibxo_index_clear "
             "aibxo_index_insert aibxo_index_evict aibxo_index_lookup aibxo_index_stats "
+            "aibxo_index_export aibxo_index_rehash "
             "aibxo_match_prefix aibxo_route_score aibxo_route_assign aibxo_collect_blocks aibxo_kv_gather "
             "aibxo_kv_scatter aibxo_kv_gather_inner aibxo_kv_scatter_inner"
         ).split():
@@ -174,6 +177,24 @@ class Index:
         live, cap = C.c_uint64(), C.c_uint64()
         lib().aibxo_index_stats(self._h, C.byref(live), C.byref(cap))
         return live.value, cap.value
+
+    def export(self, max_entries=None):
+        """(keys, masks, ids) of all live entries, ascending by key, and the live count."""
+        live = self.stats()[0]
+        m = live if max_entries is None else max_entries
+        keys = np.zeros(m, dtype=np.uint64)
+        masks = np.zeros(m, dtype=np.uint64)
+        ids = np.zeros(m, dtype=np.uint32)
+        cnt = C.c_uint64()
+        rc = lib().aibxo_index_export(self._h, _p(keys), _p(masks), _p(ids), m, C.byref(cnt))
+        assert rc == OK
+        return keys, masks, ids, cnt.value
+
+    def rehash(self, new_capacity: int) -> int:
+        rc = lib().aibxo_index_rehash(self._h, new_capacity)
+        if rc == OK:
+            self.capacity = new_capacity
+        return rc
 
     def match_prefix(self, hashes, blk_off):
         hashes, blk_off = _arr(hashes, np.uint64), _arr(blk_off, np.int64)

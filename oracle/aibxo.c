@@ -289,6 +289,26 @@ int32_t aibxo_index_stats(const aibxo_index_t* ix, uint64_t* live, uint64_t* cap
   return AIBXO_OK;
 }
 
+int32_t aibxo_index_export(const aibxo_index_t* ix, uint64_t* keys, uint64_t* masks, uint32_t* ids,
+                           uint64_t max_entries, uint64_t* count) {
+  if (!ix || !count) return AIBXO_ERR_INVALID;
+  *count = ix->live;
+  for (uint64_t i = 0; i < ix->live && i < max_entries; ++i) {
+    if (keys) keys[i] = ix->e[i].key;
+    if (masks) masks[i] = ix->e[i].mask;
+    if (ids) ids[i] = ix->e[i].id;
+  }
+  return AIBXO_OK;
+}
+
+int32_t aibxo_index_rehash(aibxo_index_t* ix, uint64_t new_capacity) {
+  if (!ix) return AIBXO_ERR_INVALID;
+  if (new_capacity < 8 || (new_capacity & (new_capacity - 1)) != 0) return AIBXO_ERR_INVALID;
+  if (ix->live > new_capacity) return AIBXO_ERR_FULL;
+  ix->capacity = new_capacity;   /* the content of the map does not depend on its capacity */
+  return AIBXO_OK;
+}
+
 /* ------------------------------------------------------------------ longest prefix ---- */
 /* match_len[r][p] = largest k <= n_r with every key i < k present and holding bit p;
  * any_len[r] the same with "present at all".  Written per pod, straight from that sentence. */

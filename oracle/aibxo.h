@@ -55,6 +55,16 @@ int32_t aibxo_index_lookup(const aibxo_index_t* ix, const uint64_t* keys, uint64
                            uint32_t* ids, int64_t n);
 int32_t aibxo_index_stats(const aibxo_index_t* ix, uint64_t* live, uint64_t* capacity);
 
+/* Operational calls (Section 3.2.5 speaks of metadata that is published and kept up to date;
+ * a table that fills up has to be carried over into a larger one).
+ * export: all live entries, ascending by key; *count = number of live entries, of which at most
+ *         max_entries are written.
+ * rehash: change the capacity, keeping every live entry; FULL (and no change) if the live
+ *         entries do not fit, INVALID for a capacity that is not a power of two >= 8. */
+int32_t aibxo_index_export(const aibxo_index_t* ix, uint64_t* keys, uint64_t* masks, uint32_t* ids,
+                           uint64_t max_entries, uint64_t* count);
+int32_t aibxo_index_rehash(aibxo_index_t* ix, uint64_t new_capacity);
+
 /* Longest cached prefix per request per pod (Section 3.2.2, prefix-cache-aware). */
 int32_t aibxo_match_prefix(const aibxo_index_t* ix, const uint64_t* hashes,
                            const int64_t* blk_off, int32_t R, uint32_t* match_len,

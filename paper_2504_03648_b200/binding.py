@@ -75,6 +75,8 @@ def lib():
             "aibx_index_evict": [vp, vp, vp, vp, i64, vp],
             "aibx_index_lookup": [vp, vp, vp, vp, i64, vp],
             "aibx_index_stats": [vp, C.POINTER(u64), C.POINTER(u64), vp],
+            "aibx_index_export": [vp, vp, vp, vp, u64, vp, vp],
+            "aibx_index_rehash": [vp, u64],
             "aibx_match_prefix": [vp, vp, vp, i32, vp, vp, vp, vp],
             "aibx_route_score": [vp, vp, i32, i32, vp, u64, C.POINTER(RouteParams), vp, vp, vp, vp],
             "aibx_route_batch": [vp, vp, vp, vp, i32, i32, u64, vp, u64, C.POINTER(RouteParams),
@@ -184,6 +186,18 @@ class Index:
         _check("aibx_index_stats",
                lib().aibx_index_stats(self._h, C.byref(live), C.byref(cap), _stream()))
         return live.value, cap.value
+
+    def export(self, keys, masks, block_ids, count) -> None:
+        """Live entries into the given arrays (any of them may be None); count: uint64[1]."""
+        cap = min(t.numel() for t in (keys, masks, block_ids) if t is not None) \
+            if any(t is not None for t in (keys, masks, block_ids)) else 0
+        _check("aibx_index_export", lib().aibx_index_export(
+            self._h, _ptr(keys, torch.uint64), _ptr(masks, torch.uint64),
+            _ptr(block_ids, torch.uint32), cap, _ptr(count, torch.uint64), _stream()))
+
+    def rehash(self, new_capacity: int) -> None:
+        _check("aibx_index_rehash", lib().aibx_index_rehash(self._h, new_capacity))
+        self.capacity = new_capacity
 
     def match_prefix(self, hashes, blk_off, match_len, any_len=None, block_ids=None) -> None:
         R = blk_off.numel() - 1

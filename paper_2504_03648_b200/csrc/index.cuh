@@ -87,14 +87,9 @@ __device__ __forceinline__ unsigned long long find_slot_rw(const IndexView& ix, 
   return ~0ULL;
 }
 
-__global__ void index_insert_kernel(IndexView ix, const uint64_t* __restrict__ keys,
-                                    const uint64_t* __restrict__ masks,
-                                    const uint32_t* __restrict__ ids, int64_t n) {
-  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const uint64_t key = keys[i];
-  const uint64_t m = masks[i] & pod_all(ix.num_pods);
-  if (key_reserved(key) || m == 0) return;
+// Insert or update one entry (mask already restricted to the table's pods, key not reserved).
+__device__ __forceinline__ void insert_entry(const IndexView& ix, uint64_t key, uint64_t m,
+                                             uint32_t id) {
   // pass 1: an existing entry anywhere on the probe path wins (stop at a never-used slot)
   unsigned long long s = home_slot(ix, key);
   bool placed = false;
@@ -136,7 +131,70 @@ __global__ void index_insert_kernel(IndexView ix, const uint64_t* __restrict__ k
     return;
   }
   atomicOr(&ix.slots[s].mask, (unsigned long long)m);
-  atomicMin(&ix.slots[s].id, ids[i]);
+  atomicMin(&ix.slots[s].id, id);
+}
+
+__global__ void index_insert_kernel(IndexView ix, const uint64_t* __restrict__ keys,
+                                    const uint64_t* __restrict__ masks,
+                                    const uint32_t* __restrict__ ids, int64_t n) {
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint64_t key = keys[i];
+  const uint64_t m = masks[i] & pod_all(ix.num_pods);
+  if (key_reserved(key) || m == 0) return;
+  insert_entry(ix, key, m, ids[i]);
+}
+
+// Live entries of the table, in no particular order; *count ends as their number (entries
+// beyond max_entries are counted but not written).
+__global__ void index_export_kernel(IndexView ix, uint64_t* __restrict__ keys,
+                                    uint64_t* __restrict__ masks, uint32_t* __restrict__ ids,
+                                    unsigned long long max_entries,
+                                    unsigned long long* __restrict__ count) {
+  const unsigned long long n = ix.cap_mask + 1;
+  const int lane = threadIdx.x & 31;
+  for (unsigned long long base = (blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x) - lane;
+       base < n; base += (unsigned long long)gridDim.x * blockDim.x) {
+    const unsigned long long i = base + lane;
+    unsigned long long k = 0, m = 0;
+    unsigned int id = AIBX_NO_BLOCK;
+    if (i < n) {
+      const uint4* p = reinterpret_cast<const uint4*>(ix.slots + i);
+      const uint4 a = __ldg(p);
+      const uint4 b = __ldg(p + 1);
+      k = (unsigned long long)a.x | ((unsigned long long)a.y << 32);
+      m = (unsigned long long)a.z | ((unsigned long long)a.w << 32);
+      id = b.x;
+    }
+    const bool live = i < n && !key_reserved(k) && m != 0;
+    // one atomic per warp: the leader reserves room for all live lanes
+    const unsigned int votes = __ballot_sync(0xffffffffu, live);
+    unsigned long long start = 0;
+    if (lane == 0 && votes) start = atomicAdd(count, (unsigned long long)__popc(votes));
+    start = __shfl_sync(0xffffffffu, start, 0);
+    if (live) {
+      const unsigned long long pos = start + __popc(votes & ((1u << lane) - 1u));
+      if (pos < max_entries) {
+        if (keys) keys[pos] = k;
+        if (masks) masks[pos] = m;
+        if (ids) ids[pos] = id;
+      }
+    }
+  }
+}
+
+// Carry every live entry of one table over into another (larger or smaller) one.
+__global__ void index_move_kernel(IndexView from, IndexView to) {
+  const unsigned long long n = from.cap_mask + 1;
+  for (unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; i < n;
+       i += (unsigned long long)gridDim.x * blockDim.x) {
+    const uint4* p = reinterpret_cast<const uint4*>(from.slots + i);
+    const uint4 a = __ldg(p);
+    const uint4 b = __ldg(p + 1);
+    const unsigned long long k = (unsigned long long)a.x | ((unsigned long long)a.y << 32);
+    const unsigned long long m = (unsigned long long)a.z | ((unsigned long long)a.w << 32);
+    if (!key_reserved(k) && m != 0) insert_entry(to, k, m, b.x);
+  }
 }
 
 // evict, pass 1: clear the named pod bits

@@ -183,6 +183,51 @@ int32_t aibx_index_stats(const aibx_index_t* ix, uint64_t* live, uint64_t* capac
   return AIBX_OK;
 }
 
+int32_t aibx_index_export(const aibx_index_t* ix, uint64_t* d_keys, uint64_t* d_masks,
+                          uint32_t* d_block_ids, uint64_t max_entries, uint64_t* d_count,
+                          void* stream) {
+  if (!ix || !d_count) return AIBX_ERR_INVALID;
+  cudaStream_t st = as_stream(stream);
+  if (cudaMemsetAsync(d_count, 0, sizeof(uint64_t), st) != cudaSuccess) return AIBX_ERR_CUDA;
+  index_export_kernel<<<sm_count() * 8, 256, 0, st>>>(
+      ix->view, d_keys, d_masks, d_block_ids, max_entries,
+      reinterpret_cast<unsigned long long*>(d_count));
+  return launch_status();
+}
+
+int32_t aibx_index_rehash(aibx_index_t* ix, uint64_t new_capacity) {
+  if (!ix) return AIBX_ERR_INVALID;
+  if (new_capacity < 8 || (new_capacity & (new_capacity - 1)) != 0 || new_capacity > (1ULL << 40))
+    return AIBX_ERR_INVALID;
+  if (cudaDeviceSynchronize() != cudaSuccess) return AIBX_ERR_CUDA;
+  unsigned long long c[2] = {0, 0};
+  if (cudaMemcpy(c, ix->view.counters, sizeof(c), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return AIBX_ERR_CUDA;
+  if (c[0] > new_capacity) return AIBX_ERR_FULL;
+  void* slots = nullptr;
+  if (cudaMalloc(&slots, new_capacity * sizeof(Slot)) != cudaSuccess) {
+    cudaGetLastError();
+    return AIBX_ERR_NOMEM;
+  }
+  int log2cap = 0;
+  while ((1ULL << log2cap) < new_capacity) ++log2cap;
+  IndexView fresh = ix->view;
+  fresh.slots = static_cast<Slot*>(slots);
+  fresh.cap_mask = new_capacity - 1;
+  fresh.shift = 64 - log2cap;
+  const IndexView old = ix->view;
+  index_clear_kernel<<<sm_count() * 8, 256>>>(fresh);          // also zeroes the shared counters
+  index_move_kernel<<<sm_count() * 8, 256>>>(old, fresh);      // re-counts the live entries
+  if (cudaDeviceSynchronize() != cudaSuccess) {
+    cudaFree(slots);
+    return AIBX_ERR_CUDA;
+  }
+  cudaFree(old.slots);
+  ix->view = fresh;
+  ix->capacity = new_capacity;
+  return AIBX_OK;
+}
+
 namespace {
 
 int32_t launch_match(const aibx_index_t* ix, const uint64_t* d_hashes, const int64_t* d_blk_off,

@@ -380,3 +380,62 @@ def test_route_assign_sequential():
     aibx.route_assign(dev(np.zeros(9, np.uint32)), dev(np.array([0, 4, 8, 12], np.int64)), 3, d_load,
                       7, (4, 1, 50), 1, d_bp, d_bs)
     assert host(d_bp).tolist() == [1, 2, 0] and host(d_load).tolist() == [2, 1, 1]
+
+
+# ------------------------------------------------------------------ export and rehash
+
+def test_index_export_and_rehash():
+    rng = np.random.default_rng(88)
+    P = 12
+    keys = rng.integers(1, 1 << 62, 3000).astype(np.uint64)
+    masks = rng.integers(0, 1 << P, 3000).astype(np.uint64)
+    ids = rng.integers(0, 1 << 20, 3000).astype(np.uint32)
+    g, o = aibx.Index(4096, P), oracle.Index(4096, P)
+    g.insert(dev(keys), dev(masks), dev(ids)); o.insert(keys, masks, ids)
+    ev = np.full(500, ALL, dtype=np.uint64)
+    g.evict(dev(keys[:500]), dev(ev)); o.evict(keys[:500], ev)
+    wk, wm, wi, wcnt = o.export()
+
+    def export_sorted(ix, room):
+        d_k, d_m, d_i = empty(room, torch.uint64), empty(room, torch.uint64), empty(room, torch.uint32)
+        d_c = empty(1, torch.uint64)
+        ix.export(d_k, d_m, d_i, d_c)
+        cnt = int(host(d_c)[0])
+        m = min(cnt, room)
+        k, mm, ii = host(d_k)[:m], host(d_m)[:m], host(d_i)[:m]
+        order = np.argsort(k, kind="stable")
+        return k[order], mm[order], ii[order], cnt
+
+    k, m, i, cnt = export_sorted(g, 4096)
+    assert cnt == wcnt and np.array_equal(k, wk) and np.array_equal(m, wm) and np.array_equal(i, wi)
+    # too little room: the count is still the number of live entries, what is written is valid
+    k2, m2, i2, cnt2 = export_sorted(g, 100)
+    assert cnt2 == wcnt and len(k2) == 100 and np.isin(k2, wk).all()
+    d_c = empty(1, torch.uint64)
+    g.export(None, None, None, d_c)                       # count only
+    assert int(host(d_c)[0]) == wcnt
+    # rehash up and down keeps every lookup and drops the freed slots
+    probe = np.concatenate([keys, rng.integers(1, 1 << 62, 200).astype(np.uint64)])
+    want_m, want_i = o.lookup(probe)
+    for cap in (16384, 4096):
+        g.rehash(cap)
+        assert o.rehash(cap) == oracle.OK
+        d_m, d_i = empty(len(probe), torch.uint64), empty(len(probe), torch.uint32)
+        g.lookup(dev(probe), d_m, d_i)
+        assert np.array_equal(host(d_m), want_m) and np.array_equal(host(d_i), want_i)
+        assert g.stats() == (wcnt, cap)
+    with pytest.raises(aibx.AibxError) as e:
+        g.rehash(1024)                                    # 2,5xx live entries do not fit
+    assert e.value.code == aibx.ERR_FULL and o.rehash(1024) == oracle.ERR_FULL
+    with pytest.raises(aibx.AibxError) as e:
+        g.rehash(5000)
+    assert e.value.code == aibx.ERR_INVALID
+    assert g.stats() == (wcnt, 4096)
+    # a table filled to the brim recovers by growing: FULL before, none after
+    small_g, small_o = aibx.Index(8, 1), oracle.Index(8, 1)
+    k8 = np.arange(1, 9, dtype=np.uint64)
+    small_g.insert(dev(k8), dev(np.ones(8, np.uint64)), dev(np.arange(8, dtype=np.uint32)))
+    small_g.rehash(32)
+    extra = np.arange(100, 110, dtype=np.uint64)
+    small_g.insert(dev(extra), dev(np.ones(10, np.uint64)), dev(np.zeros(10, np.uint32)))
+    assert aibx.status_fetch() == (0, 0) and small_g.stats() == (18, 32)

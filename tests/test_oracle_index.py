@@ -132,3 +132,36 @@ def test_full_and_invalid():
         oracle.Index(12, 4)      # not a power of two
     with pytest.raises(ValueError):
         oracle.Index(16, 65)
+
+
+def test_export_and_rehash():
+    rng = np.random.default_rng(17)
+    keys = rng.integers(1, 1 << 62, 300).astype(np.uint64)
+    masks = rng.integers(1, 1 << 8, 300).astype(np.uint64)
+    ids = rng.integers(0, 5000, 300).astype(np.uint32)
+    ix = oracle.Index(1024, 8)
+    ix.insert(keys, masks, ids)
+    ix.evict(keys[:40], np.full(40, ALL, dtype=np.uint64))
+    ek, em, ei, cnt = ix.export()
+    model = DictModel(8)
+    model.insert(keys.tolist(), masks.tolist(), ids.tolist())
+    model.evict(keys[:40].tolist(), [ALL] * 40)
+    want = sorted(model.d.items())
+    assert cnt == len(want) == ix.stats()[0]
+    assert list(zip(ek.tolist(), zip(em.tolist(), ei.tolist()))) == want
+    # truncated export still reports the full count
+    k2, _, _, cnt2 = ix.export(max_entries=10)
+    assert cnt2 == cnt and k2.tolist() == ek[:10].tolist()
+    # export -> import into a fresh index reproduces every lookup
+    other = oracle.Index(2048, 8)
+    other.insert(ek, em, ei)
+    probe = np.concatenate([keys, rng.integers(1, 1 << 62, 50).astype(np.uint64)])
+    assert all(np.array_equal(a, b) for a, b in zip(ix.lookup(probe), other.lookup(probe)))
+    # rehash keeps the content; too small a table is refused and changes nothing
+    before = ix.lookup(probe)
+    assert ix.rehash(4096) == oracle.OK and ix.stats() == (cnt, 4096)
+    assert all(np.array_equal(a, b) for a, b in zip(before, ix.lookup(probe)))
+    assert ix.rehash(256) == oracle.ERR_FULL and ix.stats() == (cnt, 4096)
+    assert ix.rehash(300) == oracle.ERR_INVALID
+    assert ix.rehash(512) == oracle.OK and ix.stats() == (cnt, 512)
+    assert all(np.array_equal(a, b) for a, b in zip(before, ix.lookup(probe)))

@@ -41,6 +41,11 @@ MUTANTS = [
      "freed[i] = (e && e->mask != 0) ? e->id : AIBXO_NO_BLOCK;", 0),
     ("all_ones_key_not_reserved", "test_oracle_index.py", "return k == 0ULL || k == ~0ULL;",
      "return k == 0ULL;", 0),
+    ("export_drops_the_last_entry", "test_oracle_index.py",
+     "for (uint64_t i = 0; i < ix->live && i < max_entries; ++i) {",
+     "for (uint64_t i = 0; i + 1 < ix->live && i < max_entries; ++i) {", 0),
+    ("rehash_accepts_too_small_a_table", "test_oracle_index.py",
+     "if (ix->live > new_capacity) return AIBXO_ERR_FULL;", "", 0),
     ("pods_beyond_P_kept", "test_oracle_index.py", "ix->e[m].mask = masks[i] & all;",
      "ix->e[m].mask = masks[i];", 0),
     ("match_tests_wrong_pod", "test_oracle_match.py", "((e->mask >> p) & 1ULL) == 0) break;",
