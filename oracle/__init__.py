@@ -74,6 +74,8 @@ def lib():
         L.aibxo_index_evict.argtypes = [vp, vp, vp, vp, i64]
         L.aibxo_index_lookup.argtypes = [vp, vp, vp, vp, i64]
         L.aibxo_index_stats.argtypes = [vp, C.POINTER(u64), C.POINTER(u64)]
+        L.aibxo_index_touch.argtypes = [vp, vp, i64, u32]
+        L.aibxo_index_pick_victims.argtypes = [vp, u64, vp, vp, C.POINTER(u64)]
         L.aibxo_index_export.argtypes = [vp, vp, vp, vp, u64, C.POINTER(u64)]
         L.aibxo_index_rehash.argtypes = [vp, u64]
         L.aibxo_match_prefix.argtypes = [vp, vp, vp, i32, vp, vp, vp]
@@ -89,7 +91,7 @@ def lib():
         for name in (
             "aibxo_hash_blocks aibxo_index_create aibxo_index_destroy aibxo_index_clear "
             "aibxo_index_insert aibxo_index_evict aibxo_index_lookup aibxo_index_stats "
-            "aibxo_index_export aibxo_index_rehash "
+            "aibxo_index_export aibxo_index_rehash aibxo_index_touch aibxo_index_pick_victims "
             "aibxo_match_prefix aibxo_route_score aibxo_route_assign aibxo_collect_blocks aibxo_kv_gather "
             "aibxo_kv_scatter aibxo_kv_gather_inner aibxo_kv_scatter_inner"
         ).split():
@@ -177,6 +179,20 @@ class Index:
         live, cap = C.c_uint64(), C.c_uint64()
         lib().aibxo_index_stats(self._h, C.byref(live), C.byref(cap))
         return live.value, cap.value
+
+    def touch(self, keys, epoch: int) -> int:
+        keys = _arr(keys, np.uint64)
+        return lib().aibxo_index_touch(self._h, _p(keys), len(keys), epoch)
+
+    def pick_victims(self, k: int):
+        """(keys, priorities) of the k entries of lowest priority, ascending (priority, key)."""
+        m = min(k, self.stats()[0])
+        keys = np.zeros(m, dtype=np.uint64)
+        prio = np.zeros(m, dtype=np.uint32)
+        cnt = C.c_uint64()
+        rc = lib().aibxo_index_pick_victims(self._h, k, _p(keys), _p(prio), C.byref(cnt))
+        assert rc == OK and cnt.value == m
+        return keys, prio
 
     def export(self, max_entries=None):
         """(keys, masks, ids) of all live entries, ascending by key, and the live count."""

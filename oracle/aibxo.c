@@ -155,6 +155,8 @@ typedef struct {
   uint64_t mask;
   uint32_t id;
   uint32_t present; /* scratch for evict: 1 if the key existed when the call began */
+  uint32_t touches; /* epochs in which the entry was touched, saturating at 3 */
+  uint32_t epoch;   /* last epoch it was touched in; 0 = never */
 } entry_t;
 
 struct aibxo_index {
@@ -226,6 +228,8 @@ int32_t aibxo_index_insert(aibxo_index_t* ix, const uint64_t* keys, const uint64
     ix->e[m].mask = masks[i] & all;
     ix->e[m].id = ids[i];
     ix->e[m].present = 0;
+    ix->e[m].touches = 0;
+    ix->e[m].epoch = 0;
     ++m;
   }
   qsort(ix->e, (size_t)m, sizeof(entry_t), cmp_entry_key);
@@ -234,6 +238,9 @@ int32_t aibxo_index_insert(aibxo_index_t* ix, const uint64_t* keys, const uint64
     if (w > 0 && ix->e[w - 1].key == ix->e[i].key) {
       ix->e[w - 1].mask |= ix->e[i].mask;
       if (ix->e[i].id < ix->e[w - 1].id) ix->e[w - 1].id = ix->e[i].id;
+      /* an insert never touches: the entry that already existed keeps its history */
+      if (ix->e[i].epoch > ix->e[w - 1].epoch) ix->e[w - 1].epoch = ix->e[i].epoch;
+      if (ix->e[i].touches > ix->e[w - 1].touches) ix->e[w - 1].touches = ix->e[i].touches;
     } else {
       ix->e[w++] = ix->e[i];
     }
@@ -286,6 +293,57 @@ int32_t aibxo_index_stats(const aibxo_index_t* ix, uint64_t* live, uint64_t* cap
   if (!ix) return AIBXO_ERR_INVALID;
   if (live) *live = ix->live;
   if (capacity) *capacity = ix->capacity;
+  return AIBXO_OK;
+}
+
+/* ---- scan-resistant victim choice -------------------------------------------------------
+ * touch: a present key that was not yet touched in `epoch` counts one more touch (at most 3)
+ *        and remembers the epoch.  Several touches in one epoch count once, so a single scan
+ *        over many blocks leaves every one of them at one touch.
+ * priority of an entry = (touches >= 2 ? 2^30 : 0) + epoch: entries seen in fewer than two
+ *        epochs go first, oldest first.  pick_victims returns the k entries of lowest priority
+ *        in ascending (priority, key) order. */
+
+int32_t aibxo_index_touch(aibxo_index_t* ix, const uint64_t* keys, int64_t n, uint32_t epoch) {
+  if (!ix || n < 0 || epoch == 0 || epoch >= (1u << 30)) return AIBXO_ERR_INVALID;
+  if (n == 0) return AIBXO_OK;
+  if (!keys) return AIBXO_ERR_INVALID;
+  for (int64_t i = 0; i < n; ++i) {
+    entry_t* e = key_reserved(keys[i]) ? NULL : find_entry(ix, keys[i]);
+    if (!e || e->epoch == epoch) continue;
+    if (e->touches < 3) e->touches += 1;
+    e->epoch = epoch;
+  }
+  return AIBXO_OK;
+}
+
+static uint32_t entry_priority(const entry_t* e) {
+  return (e->touches >= 2 ? (1u << 30) : 0u) + e->epoch;
+}
+
+static int cmp_entry_priority(const void* a, const void* b) {
+  const entry_t* x = *(const entry_t* const*)a;
+  const entry_t* y = *(const entry_t* const*)b;
+  uint32_t px = entry_priority(x), py = entry_priority(y);
+  if (px != py) return (px > py) - (px < py);
+  return (x->key > y->key) - (x->key < y->key);
+}
+
+int32_t aibxo_index_pick_victims(const aibxo_index_t* ix, uint64_t k, uint64_t* keys,
+                                 uint32_t* priorities, uint64_t* count) {
+  if (!ix || !count) return AIBXO_ERR_INVALID;
+  uint64_t m = ix->live < k ? ix->live : k;
+  *count = m;
+  if (m == 0) return AIBXO_OK;
+  const entry_t** order = (const entry_t**)malloc((size_t)ix->live * sizeof(*order));
+  if (!order) return AIBXO_ERR_NOMEM;
+  for (uint64_t i = 0; i < ix->live; ++i) order[i] = &ix->e[i];
+  qsort(order, (size_t)ix->live, sizeof(*order), cmp_entry_priority);
+  for (uint64_t i = 0; i < m; ++i) {
+    if (keys) keys[i] = order[i]->key;
+    if (priorities) priorities[i] = entry_priority(order[i]);
+  }
+  free(order);
   return AIBXO_OK;
 }
 

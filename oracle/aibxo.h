@@ -61,6 +61,12 @@ int32_t aibxo_index_stats(const aibxo_index_t* ix, uint64_t* live, uint64_t* cap
  *         max_entries are written.
  * rehash: change the capacity, keeping every live entry; FULL (and no change) if the live
  *         entries do not fit, INVALID for a capacity that is not a power of two >= 8. */
+/* Scan-resistant victim choice (Section 3.2.5 names a scan-resistant eviction policy without
+ * giving it; the reading here: an entry touched in fewer than two epochs is "scan-like" and goes
+ * before any entry touched in two or more, oldest last touch first).  See aibxo.c. */
+int32_t aibxo_index_touch(aibxo_index_t* ix, const uint64_t* keys, int64_t n, uint32_t epoch);
+int32_t aibxo_index_pick_victims(const aibxo_index_t* ix, uint64_t k, uint64_t* keys,
+                                 uint32_t* priorities, uint64_t* count);
 int32_t aibxo_index_export(const aibxo_index_t* ix, uint64_t* keys, uint64_t* masks, uint32_t* ids,
                            uint64_t max_entries, uint64_t* count);
 int32_t aibxo_index_rehash(aibxo_index_t* ix, uint64_t new_capacity);

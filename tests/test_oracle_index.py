@@ -165,3 +165,47 @@ def test_export_and_rehash():
     assert ix.rehash(300) == oracle.ERR_INVALID
     assert ix.rehash(512) == oracle.OK and ix.stats() == (cnt, 512)
     assert all(np.array_equal(a, b) for a, b in zip(before, ix.lookup(probe)))
+
+
+def test_scan_resistant_victims_hand_example_and_model():
+    # five entries; epoch 1 touches A B C, epoch 2 touches A (twice: counts once) and D,
+    # epoch 3 is a "scan" touching everything once, epoch 4 touches B
+    A, B, Cc, D, E = 11, 22, 33, 44, 55
+    ix = oracle.Index(16, 2)
+    ix.insert([A, B, Cc, D, E], [1] * 5, [0, 1, 2, 3, 4])
+    assert ix.touch([A, B, Cc, 999], 1) == oracle.OK       # 999 is absent: ignored
+    ix.touch([A, A, D], 2)
+    # touches so far: A 2, B 1, C 1, D 1, E 0 -> cold first (E never, then B, C at epoch 1, D at 2)
+    k, p = ix.pick_victims(5)
+    assert k.tolist() == [E, B, Cc, D, A] and p.tolist() == [0, 1, 1, 2, (1 << 30) + 2]
+    ix.touch([A, B, Cc, D, E], 3)                          # the scan
+    k, p = ix.pick_victims(5)
+    # E has been seen once only: it is still the first to go although it was touched last
+    assert k.tolist() == [E, A, B, Cc, D]
+    assert p.tolist() == [3] + [(1 << 30) + 3] * 4
+    ix.touch([B], 4)
+    k, _ = ix.pick_victims(3)
+    assert k.tolist() == [E, A, Cc]
+    # inserting an existing key again keeps its history; a new key starts cold
+    ix.insert([A, 66], [2, 1], [9, 9])
+    k, p = ix.pick_victims(2)
+    assert k.tolist() == [66, E] and p.tolist() == [0, 3]
+    assert ix.touch([A], 0) == oracle.ERR_INVALID and ix.touch([A], 1 << 30) == oracle.ERR_INVALID
+    # Python model on random traffic
+    rng = np.random.default_rng(23)
+    keys = rng.integers(1, 1 << 60, 400).astype(np.uint64)
+    ix = oracle.Index(1024, 4)
+    ix.insert(keys, np.ones(400, np.uint64), np.zeros(400, np.uint32))
+    model = {int(k): [0, 0] for k in keys}
+    for epoch in range(1, 9):
+        batch = rng.choice(keys, 120)
+        ix.touch(batch, epoch)
+        for kk in batch.tolist():
+            t = model[kk]
+            if t[1] != epoch:
+                t[0], t[1] = min(t[0] + 1, 3), epoch
+    want = sorted(((1 << 30 if t[0] >= 2 else 0) + t[1], kk) for kk, t in model.items())
+    k, p = ix.pick_victims(150)
+    assert list(zip(p.tolist(), k.tolist())) == want[:150]
+    k, p = ix.pick_victims(10**6)
+    assert len(k) == len(model)
