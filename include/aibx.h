@@ -104,6 +104,26 @@ int32_t aibx_index_lookup(const aibx_index_t* index, const uint64_t* d_keys,
 int32_t aibx_index_stats(const aibx_index_t* index, uint64_t* live, uint64_t* capacity,
                          void* stream);
 
+/* Scan-resistant victim choice (Section 3.2.5 names a scan-resistant eviction policy without
+ * describing it; the reading fixed here).  Every entry remembers the last epoch it was touched in
+ * and in how many distinct epochs (saturating at 3); epochs are caller-defined integers in
+ * 1..2^30-1, normally increasing (one per routed batch, say).
+ * touch: marks the present keys among d_keys as used in `epoch`; several touches of a key in
+ *        one epoch count once, so one scan over many blocks leaves each at a single touch.
+ *        New entries start untouched; re-inserting an existing key keeps its history.
+ * pick_victims: the k live entries of lowest priority, priority = (touched in >= 2 epochs ?
+ *        2^30 : 0) + last epoch - entries seen in fewer than two epochs go first, oldest first.
+ *        d_keys [k] and d_priorities [k] (either may be null) receive them in no particular order;
+ *        *d_count (uint64, device) = min(k, live entries).  Every entry below the threshold
+ *        priority is returned; among entries AT the threshold the choice is unspecified.
+ *        The caller removes them with aibx_index_evict (mask of all ones).  The first call
+ *        allocates 384 KiB of scratch that belongs to the index (NOMEM if that fails).
+ */
+int32_t aibx_index_touch(aibx_index_t* index, const uint64_t* d_keys, int64_t n, uint32_t epoch,
+                         void* stream);
+int32_t aibx_index_pick_victims(aibx_index_t* index, uint64_t k, uint64_t* d_keys,
+                                uint32_t* d_priorities, uint64_t* d_count, void* stream);
+
 /* export: every live entry (key, pod mask, block id) into caller arrays of max_entries
  *         elements, in no particular order; *d_count (uint64, device) = number of live entries,
  *         which may exceed max_entries (the surplus is counted, not written).  Arrays may be

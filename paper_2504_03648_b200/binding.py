@@ -75,6 +75,8 @@ def lib():
             "aibx_index_evict": [vp, vp, vp, vp, i64, vp],
             "aibx_index_lookup": [vp, vp, vp, vp, i64, vp],
             "aibx_index_stats": [vp, C.POINTER(u64), C.POINTER(u64), vp],
+            "aibx_index_touch": [vp, vp, i64, u32, vp],
+            "aibx_index_pick_victims": [vp, u64, vp, vp, vp, vp],
             "aibx_index_export": [vp, vp, vp, vp, u64, vp, vp],
             "aibx_index_rehash": [vp, u64],
             "aibx_match_prefix": [vp, vp, vp, i32, vp, vp, vp, vp],
@@ -186,6 +188,15 @@ class Index:
         _check("aibx_index_stats",
                lib().aibx_index_stats(self._h, C.byref(live), C.byref(cap), _stream()))
         return live.value, cap.value
+
+    def touch(self, keys, epoch: int) -> None:
+        _check("aibx_index_touch", lib().aibx_index_touch(
+            self._h, _ptr(keys, torch.uint64), keys.numel(), epoch, _stream()))
+
+    def pick_victims(self, k: int, keys, priorities, count) -> None:
+        _check("aibx_index_pick_victims", lib().aibx_index_pick_victims(
+            self._h, k, _ptr(keys, torch.uint64), _ptr(priorities, torch.uint32),
+            _ptr(count, torch.uint64), _stream()))
 
     def export(self, keys, masks, block_ids, count) -> None:
         """Live entries into the given arrays (any of them may be None); count: uint64[1]."""

@@ -88,8 +88,9 @@ __device__ __forceinline__ unsigned long long find_slot_rw(const IndexView& ix, 
 }
 
 // Insert or update one entry (mask already restricted to the table's pods, key not reserved).
-__device__ __forceinline__ void insert_entry(const IndexView& ix, uint64_t key, uint64_t m,
-                                             uint32_t id) {
+// Returns the slot, or ~0 when the table is full.
+__device__ __forceinline__ unsigned long long insert_entry(const IndexView& ix, uint64_t key,
+                                                           uint64_t m, uint32_t id) {
   // pass 1: an existing entry anywhere on the probe path wins (stop at a never-used slot)
   unsigned long long s = home_slot(ix, key);
   bool placed = false;
@@ -128,10 +129,11 @@ __device__ __forceinline__ void insert_entry(const IndexView& ix, uint64_t key, 
   }
   if (!placed) {
     raise_status(AIBX_ERR_FULL);
-    return;
+    return ~0ULL;
   }
   atomicOr(&ix.slots[s].mask, (unsigned long long)m);
   atomicMin(&ix.slots[s].id, id);
+  return s;
 }
 
 __global__ void index_insert_kernel(IndexView ix, const uint64_t* __restrict__ keys,
@@ -193,7 +195,10 @@ __global__ void index_move_kernel(IndexView from, IndexView to) {
     const uint4 b = __ldg(p + 1);
     const unsigned long long k = (unsigned long long)a.x | ((unsigned long long)a.y << 32);
     const unsigned long long m = (unsigned long long)a.z | ((unsigned long long)a.w << 32);
-    if (!key_reserved(k) && m != 0) insert_entry(to, k, m, b.x);
+    if (!key_reserved(k) && m != 0) {
+      const unsigned long long s = insert_entry(to, k, m, b.x);
+      if (s != ~0ULL) to.slots[s].stamp = b.y;          // the touch history moves along
+    }
   }
 }
 
@@ -239,6 +244,7 @@ __global__ void index_evict_remove_kernel(IndexView ix, const uint64_t* __restri
   if (m != 0) return;
   if (atomicCAS(&ix.slots[s].key, (unsigned long long)key, kKeyTomb) == key) {
     ix.slots[s].id = AIBX_NO_BLOCK;      // ready for reuse by a later insert
+    ix.slots[s].stamp = 0u;
     atomicAdd(&ix.counters[0], ~0ULL);   // live -= 1
     atomicAdd(&ix.counters[1], 1ULL);
   }

@@ -12,6 +12,7 @@
 #include "kv_copy.cuh"
 #include "kv_permute.cuh"
 #include "route_score.cuh"
+#include "victims.cuh"
 
 using namespace aibx;
 
@@ -19,6 +20,7 @@ struct aibx_index {
   IndexView view;
   uint64_t capacity;
   int device;
+  VictimScratch* victim_scratch;   // allocated on first use of aibx_index_pick_victims
 };
 
 namespace {
@@ -126,6 +128,7 @@ int32_t aibx_index_destroy(aibx_index_t* ix) {
   cudaDeviceSynchronize();
   cudaFree(ix->view.slots);
   cudaFree(ix->view.counters);
+  if (ix->victim_scratch) cudaFree(ix->victim_scratch);
   delete ix;
   return AIBX_OK;
 }
@@ -181,6 +184,44 @@ int32_t aibx_index_stats(const aibx_index_t* ix, uint64_t* live, uint64_t* capac
   if (live) *live = c[0];
   if (capacity) *capacity = ix->capacity;
   return AIBX_OK;
+}
+
+int32_t aibx_index_touch(aibx_index_t* ix, const uint64_t* d_keys, int64_t n, uint32_t epoch,
+                         void* stream) {
+  if (!ix || n < 0 || epoch == 0 || epoch >= (1u << 30)) return AIBX_ERR_INVALID;
+  if (n == 0) return AIBX_OK;
+  if (!d_keys) return AIBX_ERR_INVALID;
+  index_touch_kernel<<<blocks_for(n, 256), 256, 0, as_stream(stream)>>>(ix->view, d_keys, n, epoch);
+  return launch_status();
+}
+
+int32_t aibx_index_pick_victims(aibx_index_t* ix, uint64_t k, uint64_t* d_keys,
+                                uint32_t* d_priorities, uint64_t* d_count, void* stream) {
+  if (!ix || !d_count) return AIBX_ERR_INVALID;
+  cudaStream_t st = as_stream(stream);
+  if (!ix->victim_scratch) {
+    void* p = nullptr;
+    if (cudaMalloc(&p, sizeof(VictimScratch)) != cudaSuccess) {
+      cudaGetLastError();
+      return AIBX_ERR_NOMEM;
+    }
+    ix->victim_scratch = static_cast<VictimScratch*>(p);
+  }
+  VictimScratch* sc = ix->victim_scratch;
+  if (cudaMemsetAsync(sc, 0, sizeof(VictimScratch), st) != cudaSuccess ||
+      cudaMemsetAsync(d_count, 0, sizeof(uint64_t), st) != cudaSuccess)
+    return AIBX_ERR_CUDA;
+  if (k == 0) return AIBX_OK;
+  if (cudaMemcpyAsync(&sc->st.k, &k, sizeof(k), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return AIBX_ERR_CUDA;
+  const int grid = sm_count() * 8;
+  unsigned long long* cnt = reinterpret_cast<unsigned long long*>(d_count);
+  victims_hist_kernel<<<grid, 256, 0, st>>>(ix->view, sc, 1);
+  victims_select_kernel<<<1, 1024, 0, st>>>(sc, 1, cnt);
+  victims_hist_kernel<<<grid, 256, 0, st>>>(ix->view, sc, 2);
+  victims_select_kernel<<<1, 1024, 0, st>>>(sc, 2, cnt);
+  victims_collect_kernel<<<grid, 256, 0, st>>>(ix->view, sc, d_keys, d_priorities);
+  return launch_status();
 }
 
 int32_t aibx_index_export(const aibx_index_t* ix, uint64_t* d_keys, uint64_t* d_masks,

@@ -1,0 +1,190 @@
+// Scan-resistant victim choice on the GPU-resident index.
+//
+// Every slot carries a 32-bit stamp: bits 0..29 the last epoch in which the entry was touched
+// (0 = never), bits 30..31 the number of distinct epochs it was touched in, saturating at 3.
+// priority = (touches >= 2 ? 2^30 : 0) + epoch: entries seen in fewer than two epochs - what a
+// single scan leaves behind - go first, oldest first.
+//
+// Picking the k entries of lowest priority is a two-level radix select over the 31-bit
+// priority, all on the device: histogram of the high 16 bits -> the bin holding the k-th entry
+// -> histogram of the low 15 bits inside that bin -> the threshold priority T and how many
+// entries equal to T are still needed -> one pass that appends every entry below T and that
+// many entries equal to T.  Which of the entries AT the threshold are taken is not specified.
+#pragma once
+
+#include "aibx_common.cuh"
+#include "index.cuh"
+
+namespace aibx {
+
+constexpr unsigned int kEpochMask = (1u << 30) - 1u;
+constexpr int kHist1Bins = 1 << 16;
+constexpr int kHist2Bins = 1 << 15;
+
+struct VictimState {
+  unsigned long long k;          // wanted
+  unsigned long long k_rem;      // still wanted inside the chosen high bin
+  unsigned long long need_eq;    // entries equal to the threshold to take
+  unsigned long long eq_taken;
+  unsigned long long out_pos;
+  unsigned int prefix;           // chosen high bin
+  unsigned int threshold;        // entries with priority < threshold are all taken
+};
+
+struct VictimScratch {
+  unsigned int hist1[kHist1Bins];
+  unsigned int hist2[kHist2Bins];
+  VictimState st;
+};
+
+__device__ __forceinline__ unsigned int stamp_priority(unsigned int stamp) {
+  return ((stamp >> 30) >= 2u ? (1u << 30) : 0u) + (stamp & kEpochMask);
+}
+
+__global__ void index_touch_kernel(IndexView ix, const uint64_t* __restrict__ keys, int64_t n,
+                                   unsigned int epoch) {
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const uint64_t key = keys[i];
+  if (key_reserved(key)) return;
+  const unsigned long long s = find_slot_rw(ix, key);
+  if (s == ~0ULL) return;
+  if (*reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].mask) == 0) return;
+  unsigned int* stamp = &ix.slots[s].stamp;
+  unsigned int old = *reinterpret_cast<volatile unsigned int*>(stamp);
+  // several touches of one key in one epoch count once, whoever gets there first
+  for (int tries = 0; tries < 64; ++tries) {
+    if ((old & kEpochMask) == epoch) return;
+    const unsigned int t = old >> 30;
+    const unsigned int fresh = ((t < 3u ? t + 1u : 3u) << 30) | epoch;
+    const unsigned int seen = atomicCAS(stamp, old, fresh);
+    if (seen == old) return;
+    old = seen;
+  }
+}
+
+// Reads one slot; returns whether it holds a live entry.
+__device__ __forceinline__ bool live_slot(const IndexView& ix, unsigned long long i, uint64_t& key,
+                                          unsigned int& prio) {
+  const uint4* p = reinterpret_cast<const uint4*>(ix.slots + i);
+  const uint4 a = __ldg(p);
+  const uint4 b = __ldg(p + 1);
+  key = (uint64_t)a.x | ((uint64_t)a.y << 32);
+  const uint64_t m = (uint64_t)a.z | ((uint64_t)a.w << 32);
+  prio = stamp_priority(b.y);
+  return !key_reserved(key) && m != 0;
+}
+
+__global__ void victims_hist_kernel(IndexView ix, VictimScratch* sc, int level) {
+  const unsigned long long n = ix.cap_mask + 1;
+  const unsigned int prefix = level == 2 ? sc->st.prefix : 0u;
+  if (level == 2 && prefix == 0xFFFFFFFFu) return;       // everything is taken: no second level
+  for (unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; i < n;
+       i += (unsigned long long)gridDim.x * blockDim.x) {
+    uint64_t key;
+    unsigned int p;
+    if (!live_slot(ix, i, key, p)) continue;
+    if (level == 1) {
+      atomicAdd(&sc->hist1[p >> 15], 1u);
+    } else if ((p >> 15) == prefix) {
+      atomicAdd(&sc->hist2[p & 0x7FFFu], 1u);
+    }
+  }
+}
+
+// One CTA finds the bin that holds the `want`-th smallest entry of a histogram.
+__global__ void __launch_bounds__(1024)
+victims_select_kernel(VictimScratch* sc, int level, unsigned long long* __restrict__ d_count) {
+  __shared__ unsigned long long s_warp[32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const unsigned int* hist = level == 1 ? sc->hist1 : sc->hist2;
+  const int nbins = level == 1 ? kHist1Bins : kHist2Bins;
+  const int per = nbins / 1024;
+  if (level == 2 && sc->st.prefix == 0xFFFFFFFFu) return;
+  const unsigned long long want = level == 1 ? sc->st.k : sc->st.k_rem;
+
+  unsigned long long mine = 0;
+  for (int b = 0; b < per; ++b) mine += hist[tid * per + b];
+  unsigned long long inc = mine;                       // inclusive scan over the CTA
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const unsigned long long o = __shfl_up_sync(0xffffffffu, inc, d);
+    if (lane >= d) inc += o;
+  }
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    unsigned long long t = s_warp[lane];
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const unsigned long long o = __shfl_up_sync(0xffffffffu, t, d);
+      if (lane >= d) t += o;
+    }
+    s_warp[lane] = t;
+  }
+  __syncthreads();
+  const unsigned long long before = (warp ? s_warp[warp - 1] : 0ULL) + (inc - mine);
+  const unsigned long long total = s_warp[31];
+
+  if (level == 1 && tid == 0) {
+    *d_count = want < total ? want : total;
+    if (want >= total) {                                // every live entry is a victim
+      sc->st.prefix = 0xFFFFFFFFu;
+      sc->st.threshold = 0x80000000u;
+      sc->st.need_eq = 0;
+    }
+  }
+  if (want == 0 || (level == 1 && want >= total)) return;
+  if (before < want && want <= before + mine) {
+    unsigned long long c = before;
+    for (int b = 0; b < per; ++b) {
+      const unsigned int h = hist[tid * per + b];
+      if (c < want && want <= c + h) {
+        if (level == 1) {
+          sc->st.prefix = (unsigned int)(tid * per + b);
+          sc->st.k_rem = want - c;
+        } else {
+          sc->st.threshold = (sc->st.prefix << 15) | (unsigned int)(tid * per + b);
+          sc->st.need_eq = want - c;
+        }
+        break;
+      }
+      c += h;
+    }
+  }
+}
+
+__global__ void victims_collect_kernel(IndexView ix, VictimScratch* sc,
+                                       uint64_t* __restrict__ out_keys,
+                                       uint32_t* __restrict__ out_prio) {
+  const unsigned long long n = ix.cap_mask + 1;
+  const unsigned int T = sc->st.threshold;
+  const unsigned long long need_eq = sc->st.need_eq;
+  const unsigned long long k = sc->st.k;
+  const int lane = threadIdx.x & 31;
+  for (unsigned long long base = (blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x) - lane;
+       base < n; base += (unsigned long long)gridDim.x * blockDim.x) {
+    const unsigned long long i = base + lane;
+    uint64_t key = 0;
+    unsigned int p = 0;
+    const bool live = i < n && live_slot(ix, i, key, p);
+    bool take = live && p < T;
+    if (live && p == T && need_eq > 0) {
+      // entries at the threshold are interchangeable: the first need_eq tickets win
+      take = atomicAdd(&sc->st.eq_taken, 1ULL) < need_eq;
+    }
+    const unsigned int votes = __ballot_sync(0xffffffffu, take);
+    unsigned long long start = 0;
+    if (lane == 0 && votes) start = atomicAdd(&sc->st.out_pos, (unsigned long long)__popc(votes));
+    start = __shfl_sync(0xffffffffu, start, 0);
+    if (take) {
+      const unsigned long long pos = start + __popc(votes & ((1u << lane) - 1u));
+      if (pos < k) {
+        if (out_keys) out_keys[pos] = key;
+        if (out_prio) out_prio[pos] = p;
+      }
+    }
+  }
+}
+
+}  // namespace aibx

@@ -41,6 +41,11 @@ MUTANTS = [
      "freed[i] = (e && e->mask != 0) ? e->id : AIBXO_NO_BLOCK;", 0),
     ("all_ones_key_not_reserved", "test_oracle_index.py", "return k == 0ULL || k == ~0ULL;",
      "return k == 0ULL;", 0),
+    ("touch_counts_twice_in_one_epoch", "test_oracle_index.py",
+     "if (!e || e->epoch == epoch) continue;", "if (!e) continue;", 0),
+    ("hot_after_one_touch", "test_oracle_index.py", "e->touches >= 2 ? (1u << 30)", "e->touches >= 1 ? (1u << 30)", 0),
+    ("never_touched_looks_recent", "test_oracle_index.py",
+     "ix->e[m].epoch = 0;", "ix->e[m].epoch = 5;", 0),
     ("export_drops_the_last_entry", "test_oracle_index.py",
      "for (uint64_t i = 0; i < ix->live && i < max_entries; ++i) {",
      "for (uint64_t i = 0; i + 1 < ix->live && i < max_entries; ++i) {", 0),
