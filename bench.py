@@ -1031,7 +1031,53 @@ def case_kv_inner(args):
                       "status": aibx.status_fetch()}))
 
 
-CASES = {"kv_inner": case_kv_inner, "hash_sweep": case_hash_sweep, "oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
+def case_index_ops(args):
+    """Operational index calls on the routing-heavy index (2^20 entries in 2^21 slots, 64 pods):
+    touch, pick_victims, export, rehash, and the sequential assignment of 4,096 requests."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import workloads as W
+
+    ix, keys = _big_index(torch, aibx, W, 21, 64, 61)
+    n = len(keys)
+    d_keys = torch.from_numpy(keys).cuda()
+    st = W.Stream(62, 0)
+    res = {}
+    for epoch in range(1, 5):
+        batch = torch.from_numpy(keys[st.randint(0, n, n // 8)]).cuda()
+        ts = _event_times(torch, lambda: ix.touch(batch, epoch), 3, 1)
+        res["touch_%dk_keys_us" % (batch.numel() // 1000)] = round(statistics.median(ts) * 1e3, 1)
+    for k in (1000, 100000):
+        d_k = torch.empty(k, dtype=torch.uint64, device="cuda")
+        d_p = torch.empty(k, dtype=torch.uint32, device="cuda")
+        d_c = torch.empty(1, dtype=torch.uint64, device="cuda")
+        ts = _event_times(torch, lambda: ix.pick_victims(k, d_k, d_p, d_c), 7, 2)
+        res["pick_%d_victims_us" % k] = round(statistics.median(ts) * 1e3, 1)
+        assert int(d_c.cpu().numpy()[0]) == k
+    d_k = torch.empty(n, dtype=torch.uint64, device="cuda")
+    d_m = torch.empty(n, dtype=torch.uint64, device="cuda")
+    d_i = torch.empty(n, dtype=torch.uint32, device="cuda")
+    d_c = torch.empty(1, dtype=torch.uint64, device="cuda")
+    ts = _event_times(torch, lambda: ix.export(d_k, d_m, d_i, d_c), 7, 2)
+    res["export_1M_entries_us"] = round(statistics.median(ts) * 1e3, 1)
+    t0 = time.perf_counter()
+    ix.rehash(1 << 22)
+    torch.cuda.synchronize()
+    res["rehash_2M_to_4M_slots_ms_wall"] = round((time.perf_counter() - t0) * 1e3, 2)
+    R, P = 4096, 64
+    ml = torch.from_numpy(st.randint(0, 100, R * P).astype(np.uint32)).cuda()
+    bo = torch.arange(0, (R + 1) * 128, 128, dtype=torch.int64, device="cuda")
+    load = torch.zeros(P, dtype=torch.int32, device="cuda")
+    bp = torch.empty(R, dtype=torch.int32, device="cuda")
+    bs = torch.empty(R, dtype=torch.int64, device="cuda")
+    ts = _event_times(torch, lambda: aibx.route_assign(ml, bo, P, load, (1 << 64) - 1, None, 1, bp, bs), 7, 2)
+    res["route_assign_4096_requests_64_pods_us"] = round(statistics.median(ts) * 1e3, 1)
+    print(json.dumps({"case": "index_ops", "entries": n, "results": res,
+                      "status": aibx.status_fetch()}))
+
+
+CASES = {"index_ops": case_index_ops, "kv_inner": case_kv_inner, "hash_sweep": case_hash_sweep, "oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
          "cfg4": case_cfg4, "cfg5": case_cfg5, "lookup_flat": case_lookup_flat}
 
 

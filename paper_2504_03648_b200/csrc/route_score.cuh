@@ -39,19 +39,26 @@ __device__ __forceinline__ void lane_candidate(int lane, int P, uint64_t ready_m
 }
 
 // Warp argmax over (score, pod): higher score wins, equal scores go to the lower pod index,
-// "no pod" loses to any pod.  Every lane ends with the winner.
+// "no pod" loses to any pod.  Every lane ends with the winner.  Three warp reductions on
+// 32-bit pieces (high half, low half, pod) instead of a shuffle tree on 64-bit pairs.
 __device__ __forceinline__ void warp_argmax(long long& top, int& arg) {
-#pragma unroll
-  for (int d = 16; d >= 1; d >>= 1) {
-    const long long o_top = __shfl_xor_sync(0xffffffffu, top, d);
-    const int o_arg = __shfl_xor_sync(0xffffffffu, arg, d);
-    const bool take = (o_arg != AIBX_NO_POD) &&
-                      (arg == AIBX_NO_POD || o_top > top || (o_top == top && o_arg < arg));
-    if (take) {
-      top = o_top;
-      arg = o_arg;
-    }
+  const bool valid = arg != AIBX_NO_POD;
+  if (__ballot_sync(0xffffffffu, valid) == 0u) {
+    top = LLONG_MIN;
+    arg = AIBX_NO_POD;
+    return;
   }
+  const unsigned long long u = (unsigned long long)top ^ 0x8000000000000000ULL;   // order-preserving
+  const unsigned int hi = valid ? (unsigned int)(u >> 32) : 0u;
+  const unsigned int max_hi = __reduce_max_sync(0xffffffffu, hi);
+  const bool c1 = valid && hi == max_hi;
+  const unsigned int lo = c1 ? (unsigned int)u : 0u;
+  const unsigned int max_lo = __reduce_max_sync(0xffffffffu, lo);
+  const bool c2 = c1 && lo == max_lo;
+  const unsigned int pod = c2 ? (unsigned int)arg : 0xFFFFFFFFu;
+  const unsigned int best = __reduce_min_sync(0xffffffffu, pod);
+  top = (long long)((((unsigned long long)max_hi << 32) | max_lo) ^ 0x8000000000000000ULL);
+  arg = (int)best;
 }
 
 __global__ void __launch_bounds__(kRouteWarps * 32)

@@ -84,11 +84,13 @@ __global__ void victims_hist_kernel(IndexView ix, VictimScratch* sc, int level) 
     uint64_t key;
     unsigned int p;
     if (!live_slot(ix, i, key, p)) continue;
-    if (level == 1) {
-      atomicAdd(&sc->hist1[p >> 15], 1u);
-    } else if ((p >> 15) == prefix) {
-      atomicAdd(&sc->hist2[p & 0x7FFFu], 1u);
-    }
+    if (level == 2 && (p >> 15) != prefix) continue;
+    // Priorities cluster (few distinct epochs), so lanes that hit the same bin elect one of
+    // them to add their number: one atomic per distinct bin per warp instead of one per entry.
+    unsigned int* bin = level == 1 ? &sc->hist1[p >> 15] : &sc->hist2[p & 0x7FFFu];
+    const unsigned int active = __activemask();
+    const unsigned int same = __match_any_sync(active, (unsigned long long)bin);
+    if ((threadIdx.x & 31) == __ffs(same) - 1) atomicAdd(bin, (unsigned int)__popc(same));
   }
 }
 
@@ -169,9 +171,15 @@ __global__ void victims_collect_kernel(IndexView ix, VictimScratch* sc,
     unsigned int p = 0;
     const bool live = i < n && live_slot(ix, i, key, p);
     bool take = live && p < T;
-    if (live && p == T && need_eq > 0) {
-      // entries at the threshold are interchangeable: the first need_eq tickets win
-      take = atomicAdd(&sc->st.eq_taken, 1ULL) < need_eq;
+    // entries at the threshold are interchangeable: the first need_eq tickets win (one ticket
+    // counter update per warp)
+    const bool at_thr = live && p == T && need_eq > 0;
+    const unsigned int eq = __ballot_sync(0xffffffffu, at_thr);
+    if (eq) {
+      unsigned long long first = 0;
+      if (lane == __ffs(eq) - 1) first = atomicAdd(&sc->st.eq_taken, (unsigned long long)__popc(eq));
+      first = __shfl_sync(0xffffffffu, first, __ffs(eq) - 1);
+      if (at_thr) take = first + __popc(eq & ((1u << lane) - 1u)) < need_eq;
     }
     const unsigned int votes = __ballot_sync(0xffffffffu, take);
     unsigned long long start = 0;

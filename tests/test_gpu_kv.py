@@ -314,3 +314,15 @@ def test_counted_variants_stop_at_the_device_count(layout, mode):
         oracle.kv_scatter(pool_want, lay_o, ids_s[:m], fresh[: m * kv.block_bytes].copy())
         assert np.array_equal(host(pool_d), pool_want), cnt
         assert aibx.status_fetch() == (0, 0)
+
+
+def test_latent_single_stream_shape():
+    """An MLA-style pool keeps one latent vector per token (no separate K and V).  The bytes are
+    opaque to gather/scatter, so such a pool is described by any layout with the same tile size:
+    576 latent dims x 16 tokens x 2 bytes = 18,432 bytes = 2 x 1 head x 16 tokens x 288 dims."""
+    for layout in (0, 1):
+        kv = W.KVSpec("latent", 13, layout, 6, 1, 16, 288, 2, 120)
+        assert kv.tile_bytes == 16 * 576 * 2
+        ids_g = W.distinct_ids(6, 120, 77)
+        ids_s = W.distinct_ids(8, 120, 77)
+        check_gather_scatter(kv, ids_g, ids_s, (0, 32768, 3, 1, 1))
