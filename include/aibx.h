@@ -328,6 +328,13 @@ int32_t aibx_kv_set_store_lag(int32_t lag);
  */
 int32_t aibx_status_fetch(void* stream, int32_t* status, int64_t* detail);
 
+/* Self-test of the bounded waits used by the copy kernels: enqueues one thread that waits on a
+ * barrier nobody completes, gives up after `spins` polls (1..2^20) and records AIBX_ERR_TIMEOUT
+ * in the device status, exactly as a copy kernel would.  Nothing faults or hangs; the device
+ * stays usable.  For health checks and tests of the error path.
+ */
+int32_t aibx_selftest_bounded_wait(uint32_t spins, void* stream);
+
 const char* aibx_strerror(int32_t status);
 
 #ifdef __cplusplus

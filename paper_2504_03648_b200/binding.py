@@ -94,6 +94,7 @@ def lib():
             "aibx_kv_scatter_inner": [vp, C.POINTER(KVLayout), i32, i32, vp, i64, vp, vp],
             "aibx_kv_set_tuning": [i32, i32, i32, i32],
             "aibx_kv_set_store_lag": [i32],
+            "aibx_selftest_bounded_wait": [u32, vp],
             "aibx_status_fetch": [vp, C.POINTER(i32), C.POINTER(i64)],
         }
         for name, args in sig.items():
@@ -322,6 +323,10 @@ def kv_set_tuning(mode: int = -1, chunk_bytes: int = 0, stages: int = 0,
 
 def kv_set_store_lag(lag: int = 1) -> None:
     _check("aibx_kv_set_store_lag", lib().aibx_kv_set_store_lag(lag))
+
+
+def selftest_bounded_wait(spins: int = 1000) -> None:
+    _check("aibx_selftest_bounded_wait", lib().aibx_selftest_bounded_wait(spins, _stream()))
 
 
 def status_fetch():

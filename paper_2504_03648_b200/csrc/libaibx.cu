@@ -11,6 +11,7 @@
 #include "index.cuh"
 #include "kv_copy.cuh"
 #include "kv_permute.cuh"
+#include "selftest.cuh"
 #include "route_score.cuh"
 #include "victims.cuh"
 
@@ -470,6 +471,12 @@ int32_t aibx_kv_set_store_lag(int32_t lag) {
   if (lag < 1 || lag > 4) return AIBX_ERR_INVALID;
   copy_tuning().lag = lag;
   return AIBX_OK;
+}
+
+int32_t aibx_selftest_bounded_wait(uint32_t spins, void* stream) {
+  if (spins == 0 || spins > (1u << 20)) return AIBX_ERR_INVALID;
+  bounded_wait_probe_kernel<<<1, 32, 0, as_stream(stream)>>>(spins);
+  return launch_status();
 }
 
 int32_t aibx_status_fetch(void* stream, int32_t* status, int64_t* detail) {

@@ -326,3 +326,19 @@ def test_latent_single_stream_shape():
         ids_g = W.distinct_ids(6, 120, 77)
         ids_s = W.distinct_ids(8, 120, 77)
         check_gather_scatter(kv, ids_g, ids_s, (0, 32768, 3, 1, 1))
+
+
+def test_a_wait_that_runs_out_becomes_a_status_not_a_hang():
+    """The error path of the bounded waits, exercised without any fault: a probe thread waits
+    on a barrier nobody completes, gives up after 1,000 polls, and the host reads TIMEOUT; the
+    device keeps working."""
+    assert aibx.status_fetch() == (0, 0)
+    aibx.selftest_bounded_wait(1000)
+    st, detail = aibx.status_fetch()
+    assert st == aibx.ERR_TIMEOUT and detail == 1
+    assert aibx.strerror(st) == "bounded device wait gave up"
+    assert aibx.status_fetch() == (0, 0)
+    kv = W.cfg1_kv()
+    check_gather_scatter(kv, W.distinct_ids(0, 256, 64), W.distinct_ids(100, 256, 64), (0, 32768, 3, 1, 1))
+    with pytest.raises(aibx.AibxError):
+        aibx.selftest_bounded_wait(0)
