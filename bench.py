@@ -1077,7 +1077,43 @@ def case_index_ops(args):
                       "status": aibx.status_fetch()}))
 
 
-CASES = {"index_ops": case_index_ops, "kv_inner": case_kv_inner, "hash_sweep": case_hash_sweep, "oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
+def case_kv_comparators(args):
+    """Library comparators for the gather on the same GPU and bytes (cfg2 block shape, 1,600
+    blocks): a plain device-to-device copy of the same size and torch.index_select over rows."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import synth
+    from paper_2504_03648_b200 import workloads as W
+
+    kv = W.cfg2_kv()
+    n = 1600
+    pool = torch.empty(kv.pool_bytes, dtype=torch.uint8, device="cuda")
+    synth.fill_pool(pool, kv)
+    ids_np = np.sort(W.distinct_ids(7, kv.num_blocks, n))
+    ids = torch.from_numpy(ids_np).cuda()
+    idx64 = torch.from_numpy(ids_np.astype(np.int64)).cuda()
+    buf = torch.empty(n * kv.block_bytes, dtype=torch.uint8, device="cuda")
+    lay = aibx.KVLayout(kv.layout, kv.num_layers, kv.num_kv_heads, kv.block_tokens, kv.head_dim,
+                        kv.elem_bytes, kv.num_blocks)
+    nbytes = 2 * n * kv.block_bytes
+    rows = pool.view(torch.int32).view(kv.num_blocks, kv.block_bytes // 4)
+    out_rows = buf.view(torch.int32).view(n, kv.block_bytes // 4)
+    src = pool[: n * kv.block_bytes]
+
+    def rate(fn):
+        return round(nbytes / (statistics.median(_event_times(torch, fn, 10, 3)) * 1e-3) / 1e9, 1)
+
+    res = {"aibx_kv_gather_GBps": rate(lambda: aibx.kv_gather(pool, lay, ids, n, buf)),
+           "device_copy_same_bytes_GBps": rate(lambda: buf.copy_(src)),
+           "torch_index_select_GBps": rate(lambda: torch.index_select(rows, 0, idx64, out=out_rows))}
+    peak, kind = measured_peak_hbm()
+    print(json.dumps({"case": "kv_comparators", "blocks": n, "bytes_read_plus_written": nbytes,
+                      "peak": peak, "peak_kind": kind, "results": res,
+                      "status": aibx.status_fetch()}))
+
+
+CASES = {"kv_comparators": case_kv_comparators, "index_ops": case_index_ops, "kv_inner": case_kv_inner, "hash_sweep": case_hash_sweep, "oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
          "cfg4": case_cfg4, "cfg5": case_cfg5, "lookup_flat": case_lookup_flat}
 
 
