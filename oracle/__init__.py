@@ -81,6 +81,7 @@ def lib():
         L.aibxo_match_prefix.argtypes = [vp, vp, vp, i32, vp, vp, vp]
         L.aibxo_route_score.argtypes = [vp, vp, i32, i32, vp, u64, C.POINTER(_Params), vp, vp, vp]
         L.aibxo_route_assign.argtypes = [vp, vp, i32, i32, vp, u64, C.POINTER(_Params), i32, vp, vp]
+        L.aibxo_route_policy.argtypes = [i32, vp, vp, i32, i32, C.POINTER(_Metrics), vp, u64, i32, vp]
         L.aibxo_collect_blocks.argtypes = [vp, i64, u32, vp, C.POINTER(u32)]
         L.aibxo_kv_gather.argtypes = [vp, C.POINTER(_Layout), vp, i64, vp, C.POINTER(i64)]
         L.aibxo_kv_scatter.argtypes = [vp, C.POINTER(_Layout), vp, i64, vp, C.POINTER(i64)]
@@ -92,7 +93,8 @@ def lib():
             "aibxo_hash_blocks aibxo_index_create aibxo_index_destroy aibxo_index_clear "
             "aibxo_index_insert aibxo_index_evict aibxo_index_lookup aibxo_index_stats "
             "aibxo_index_export aibxo_index_rehash aibxo_index_touch aibxo_index_pick_victims "
-            "aibxo_match_prefix aibxo_route_score aibxo_route_assign aibxo_collect_blocks aibxo_kv_gather "
+            "aibxo_match_prefix aibxo_route_score aibxo_route_assign aibxo_route_policy "
+            "aibxo_collect_blocks aibxo_kv_gather "
             "aibxo_kv_scatter aibxo_kv_gather_inner aibxo_kv_scatter_inner"
         ).split():
             getattr(L, name).restype = i32
@@ -253,6 +255,38 @@ def route_assign(match_len, blk_off, pod_load, ready_mask, params=None, load_inc
                                   _p(best_score))
     assert rc == OK, rc
     return best_pod, best_score, load
+
+
+POLICIES = ("random", "throughput", "least-request", "least-kv-cache", "least-latency",
+            "prefix-cache-aware")
+_METRIC_FIELDS = ("throughput", "requests", "kv_usage", "queue_latency", "serve_latency")
+
+
+class _Metrics(C.Structure):
+    _fields_ = [(f, C.c_void_p) for f in _METRIC_FIELDS]
+
+
+def route_policy(policy, num_pods, R, ready_mask, metrics=None, match_len=None, blk_off=None,
+                 draws=None, threshold_pct=50, expect=OK):
+    """One pod per request under one of the six policies (name or number).  `metrics` maps
+    field names (throughput, requests, kv_usage, queue_latency, serve_latency) to per-pod
+    int32 arrays.  Returns best_pod, or the error code when `expect` is not OK."""
+    pol = POLICIES.index(policy) if isinstance(policy, str) else int(policy)
+    keep = []
+    m = _Metrics()
+    for f in _METRIC_FIELDS:
+        a = None if metrics is None or metrics.get(f) is None else _arr(metrics[f], np.int32)
+        keep.append(a)
+        setattr(m, f, _p(a))
+    match_len = None if match_len is None else _arr(match_len, np.uint32)
+    blk_off = None if blk_off is None else _arr(blk_off, np.int64)
+    draws = None if draws is None else _arr(draws, np.uint64)
+    best_pod = np.full(R, -7, dtype=np.int32)
+    rc = lib().aibxo_route_policy(pol, _p(match_len), _p(blk_off), R, num_pods,
+                                  None if metrics is None else C.byref(m), _p(draws),
+                                  ready_mask & (2**64 - 1), threshold_pct, _p(best_pod))
+    assert rc == expect, rc
+    return best_pod if expect == OK else rc
 
 
 def collect_blocks(block_ids, num_blocks: int):

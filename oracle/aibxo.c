@@ -11,6 +11,8 @@
  *   aibxo_index_*                   : Python dict model, operation-log brute force
  *   aibxo_match_prefix              : brute-force rescan, hand example, monotonicity
  *   aibxo_route_score               : hand example, least-request special case, recompute
+ *   aibxo_route_policy              : numpy argmin, list indexing, sorted tuples, hand example,
+ *                                     equality with aibxo_route_score under a dominating weight
  *   aibxo_collect_blocks            : sorted(set(...))
  *   aibxo_kv_gather / scatter       : index_select, direct indexing, round trips
  */
@@ -458,6 +460,75 @@ int32_t aibxo_route_assign(const uint32_t* match_len, const int64_t* blk_off, in
     if (rc != AIBXO_OK) return rc;
     if (best_pod[r] != AIBXO_NO_POD)
       pod_load[best_pod[r]] = (int32_t)((uint32_t)pod_load[best_pod[r]] + (uint32_t)load_increment);
+  }
+  return AIBXO_OK;
+}
+
+/* ------------------------------------------------------------------ routing policies -- */
+
+/* lowest value[p] over the ready pods, first one on ties; NO_POD if none is ready */
+static int32_t lowest_ready(const int64_t* value, int32_t num_pods, uint64_t ready_mask) {
+  int32_t arg = AIBXO_NO_POD;
+  for (int32_t p = 0; p < num_pods; ++p) {
+    if (((ready_mask >> p) & 1ULL) == 0) continue;
+    if (arg == AIBXO_NO_POD || value[p] < value[arg]) arg = p;
+  }
+  return arg;
+}
+
+int32_t aibxo_route_policy(int32_t policy, const uint32_t* match_len, const int64_t* blk_off,
+                           int32_t R, int32_t num_pods, const aibxo_pod_metrics_t* metrics,
+                           const uint64_t* draws, uint64_t ready_mask, int32_t threshold_pct,
+                           int32_t* best_pod) {
+  if (R < 0 || num_pods < 1 || num_pods > 64 || policy < 0 || policy > 5) return AIBXO_ERR_INVALID;
+  if (R == 0) return AIBXO_OK;
+  if (!best_pod) return AIBXO_ERR_INVALID;
+  const int32_t P = num_pods;
+  int64_t value[64];
+
+  if (policy == 0) { /* random */
+    if (!draws) return AIBXO_ERR_INVALID;
+    int32_t ready[64];
+    int32_t n = 0;
+    for (int32_t p = 0; p < P; ++p)
+      if ((ready_mask >> p) & 1ULL) ready[n++] = p;
+    for (int32_t r = 0; r < R; ++r)
+      best_pod[r] = n == 0 ? AIBXO_NO_POD : ready[draws[r] % (uint64_t)n];
+    return AIBXO_OK;
+  }
+
+  if (!metrics) return AIBXO_ERR_INVALID;
+  if (policy >= 1 && policy <= 4) { /* lowest figure, the same pod for every request */
+    const int32_t* a = policy == 1 ? metrics->throughput
+                     : policy == 2 ? metrics->requests
+                     : policy == 3 ? metrics->kv_usage
+                                   : metrics->queue_latency;
+    const int32_t* b = policy == 4 ? metrics->serve_latency : NULL;
+    if (!a || (policy == 4 && !b)) return AIBXO_ERR_INVALID;
+    for (int32_t p = 0; p < P; ++p) value[p] = (int64_t)a[p] + (b ? (int64_t)b[p] : 0);
+    const int32_t arg = lowest_ready(value, P, ready_mask);
+    for (int32_t r = 0; r < R; ++r) best_pod[r] = arg;
+    return AIBXO_OK;
+  }
+
+  /* prefix-cache-aware */
+  if (!match_len || !blk_off || !metrics->requests) return AIBXO_ERR_INVALID;
+  for (int32_t p = 0; p < P; ++p) value[p] = (int64_t)metrics->requests[p];
+  for (int32_t r = 0; r < R; ++r) {
+    const int64_t n_r = blk_off[r + 1] - blk_off[r];
+    int32_t arg = AIBXO_NO_POD;
+    int64_t arg_hit = 0;
+    for (int32_t p = 0; p < P; ++p) {
+      if (((ready_mask >> p) & 1ULL) == 0) continue;
+      const int64_t hit = (int64_t)match_len[(int64_t)r * P + p];
+      if (!(hit > 0 && 100 * hit >= (int64_t)threshold_pct * n_r)) continue;
+      if (arg == AIBXO_NO_POD || hit > arg_hit || (hit == arg_hit && value[p] < value[arg])) {
+        arg = p;
+        arg_hit = hit;
+      }
+    }
+    if (arg == AIBXO_NO_POD) arg = lowest_ready(value, P, ready_mask);
+    best_pod[r] = arg;
   }
   return AIBXO_OK;
 }

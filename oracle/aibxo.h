@@ -98,6 +98,33 @@ int32_t aibxo_route_assign(const uint32_t* match_len, const int64_t* blk_off, in
                            const aibxo_route_params_t* params, int32_t load_increment,
                            int32_t* best_pod, int64_t* best_score);
 
+/* The six per-request routing policies of Section 3.2.2, one pod per request, all requests of a
+ * call seeing the same snapshot of the per-pod figures.  Only ready pods (ready_mask bit set,
+ * pod < num_pods) can be chosen; with none ready the answer is NO_POD.  Ties go to the lowest
+ * pod index.  Readings fixed here:
+ *   0 random            : the (draws[r] mod n)-th ready pod in ascending order, n = ready pods;
+ *                         the random numbers are an input (draws[R])
+ *   1 throughput        : lowest throughput[p]
+ *   2 least-request     : lowest requests[p]
+ *   3 least-kv-cache    : lowest kv_usage[p]
+ *   4 least-latency     : lowest queue_latency[p] + serve_latency[p] (sum taken in int64)
+ *   5 prefix-cache-aware: among pods whose hit = match_len[r][p] is > 0 and has
+ *                         100*hit >= threshold_pct*n_r, the largest hit, ties to the lowest
+ *                         requests[p]; if no pod qualifies, policy 2.
+ * Arrays a policy does not read may be NULL. */
+typedef struct {
+  const int32_t* throughput;
+  const int32_t* requests;
+  const int32_t* kv_usage;
+  const int32_t* queue_latency;
+  const int32_t* serve_latency;
+} aibxo_pod_metrics_t;
+
+int32_t aibxo_route_policy(int32_t policy, const uint32_t* match_len, const int64_t* blk_off,
+                           int32_t R, int32_t num_pods, const aibxo_pod_metrics_t* metrics,
+                           const uint64_t* draws, uint64_t ready_mask, int32_t threshold_pct,
+                           int32_t* best_pod);
+
 /* Ascending distinct valid block ids, padded with NO_BLOCK; returns RANGE if any id other
  * than NO_BLOCK is >= num_blocks (those are dropped). */
 int32_t aibxo_collect_blocks(const uint32_t* block_ids, int64_t n, uint32_t num_blocks,

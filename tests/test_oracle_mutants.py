@@ -73,6 +73,32 @@ MUTANTS = [
      "100 * hit >= (int64_t)prm.threshold_pct * n_r", "100 * hit >= (int64_t)prm.threshold_pct * 16 * n_r", 0),
     ("assignment_forgets_the_increment", "test_oracle_score.py",
      "(uint32_t)pod_load[best_pod[r]] + (uint32_t)load_increment", "(uint32_t)pod_load[best_pod[r]]", 0),
+    ("policy_picks_the_highest_figure", "test_oracle_policy.py",
+     "if (arg == AIBXO_NO_POD || value[p] < value[arg]) arg = p;",
+     "if (arg == AIBXO_NO_POD || value[p] > value[arg]) arg = p;", 0),
+    ("policy_ties_to_the_last_pod", "test_oracle_policy.py",
+     "if (arg == AIBXO_NO_POD || value[p] < value[arg]) arg = p;",
+     "if (arg == AIBXO_NO_POD || value[p] <= value[arg]) arg = p;", 0),
+    ("latency_ignores_the_queue", "test_oracle_policy.py",
+     "const int32_t* b = policy == 4 ? metrics->serve_latency : NULL;",
+     "const int32_t* b = NULL;", 0),
+    ("latency_sum_wraps_in_32_bits", "test_oracle_policy.py",
+     "value[p] = (int64_t)a[p] + (b ? (int64_t)b[p] : 0);",
+     "value[p] = (int64_t)(int32_t)((uint32_t)a[p] + (b ? (uint32_t)b[p] : 0u));", 0),
+    ("kv_policy_reads_requests", "test_oracle_policy.py",
+     ": policy == 3 ? metrics->kv_usage", ": policy == 3 ? metrics->requests", 0),
+    ("random_indexes_all_pods", "test_oracle_policy.py",
+     "if ((ready_mask >> p) & 1ULL) ready[n++] = p;", "ready[n++] = p;", 0),
+    ("prefix_policy_shortest_hit", "test_oracle_policy.py",
+     "hit > arg_hit || (hit == arg_hit && value[p] < value[arg])",
+     "hit < arg_hit || (hit == arg_hit && value[p] < value[arg])", 0),
+    ("prefix_policy_ignores_requests_on_ties", "test_oracle_policy.py",
+     "hit > arg_hit || (hit == arg_hit && value[p] < value[arg])", "hit > arg_hit", 0),
+    ("prefix_policy_threshold_exclusive", "test_oracle_policy.py",
+     "if (!(hit > 0 && 100 * hit >= (int64_t)threshold_pct * n_r)) continue;",
+     "if (!(hit > 0 && 100 * hit > (int64_t)threshold_pct * n_r)) continue;", 0),
+    ("prefix_policy_no_fallback", "test_oracle_policy.py",
+     "if (arg == AIBXO_NO_POD) arg = lowest_ready(value, P, ready_mask);", "", 0),
     ("layer_major_as_block_major", "test_oracle_kv.py",
      "return ((int64_t)l * L->num_blocks + b) * t;", "return ((int64_t)b * L->num_layers + l) * t;", 0),
     ("buffer_layer_major", "test_oracle_kv.py",
