@@ -192,6 +192,47 @@ int32_t aibx_route_batch(const aibx_index_t* index, const int32_t* d_tokens,
                          uint32_t* d_block_ids, int32_t* d_best_pod, int64_t* d_best_score,
                          void* stream);
 
+/* ---------------------------------------------------------------------------------------
+ * The routing policies the gateway offers per pending request (Section 3.2.2 lists six: random,
+ * throughput, least-request, least-kv-cache, least-latency, prefix-cache-aware), taken for a
+ * batch: one pod per request, every request of the call seeing the same snapshot of the per-pod
+ * figures.  Only ready pods (ready_mask bit set, pod < num_pods) can be chosen; if none is
+ * ready the answer is AIBX_NO_POD.  Ties go to the lowest pod index.  Readings fixed here (the
+ * paper gives one sentence per policy and no units; the figures are the caller's integers):
+ *   RANDOM             the (d_draws[r] mod n)-th ready pod in ascending order, n = ready pods.
+ *                      The random numbers are an input: d_draws [R] uint64.
+ *   THROUGHPUT         lowest d_throughput[p]            (tokens per second being served)
+ *   LEAST_REQUEST      lowest d_requests[p]              (admitted requests)
+ *   LEAST_KV_CACHE     lowest d_kv_usage[p]              (average KV-cache usage)
+ *   LEAST_LATENCY      lowest d_queue_latency[p] + d_serve_latency[p], summed in int64
+ *   PREFIX_CACHE_AWARE among pods with hit = d_match_len[r][p] > 0 and
+ *                      100*hit >= threshold_pct*n_r: the largest hit, ties to the lowest
+ *                      d_requests[p]; if no pod qualifies, LEAST_REQUEST.
+ * Arrays a policy does not read may be NULL (metrics itself may be NULL for RANDOM;
+ * d_match_len / d_blk_off / threshold_pct are read by PREFIX_CACHE_AWARE only).  Each metrics
+ * array is [num_pods] int32 in device memory; the struct itself is host memory, read during
+ * the call.  d_best_pod [R] out.  INVALID for an unknown policy or a missing array.
+ */
+#define AIBX_POLICY_RANDOM             0
+#define AIBX_POLICY_THROUGHPUT         1
+#define AIBX_POLICY_LEAST_REQUEST      2
+#define AIBX_POLICY_LEAST_KV_CACHE     3
+#define AIBX_POLICY_LEAST_LATENCY      4
+#define AIBX_POLICY_PREFIX_CACHE_AWARE 5
+
+typedef struct {
+  const int32_t* d_throughput;
+  const int32_t* d_requests;
+  const int32_t* d_kv_usage;
+  const int32_t* d_queue_latency;
+  const int32_t* d_serve_latency;
+} aibx_pod_metrics_t;
+
+int32_t aibx_route_policy(int32_t policy, const uint32_t* d_match_len, const int64_t* d_blk_off,
+                          int32_t R, int32_t num_pods, const aibx_pod_metrics_t* metrics,
+                          const uint64_t* d_draws, uint64_t ready_mask, int32_t threshold_pct,
+                          int32_t* d_best_pod, void* stream);
+
 /* Sequential assignment of a batch (Section 3.2.2, least-request: the count of admitted
  * requests of an instance grows with every request routed to it).  Requests are taken in
  * order r = 0..R-1; request r is scored as in aibx_route_score against the CURRENT d_pod_load,

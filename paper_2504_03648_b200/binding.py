@@ -53,6 +53,14 @@ class KVLayout(C.Structure):
         return self.num_layers * self.tile_bytes
 
 
+class PodMetrics(C.Structure):
+    _fields_ = [(f, C.c_void_p) for f in ("d_throughput", "d_requests", "d_kv_usage",
+                                          "d_queue_latency", "d_serve_latency")]
+
+
+POLICY_RANDOM, POLICY_THROUGHPUT, POLICY_LEAST_REQUEST, POLICY_LEAST_KV_CACHE, \
+    POLICY_LEAST_LATENCY, POLICY_PREFIX_CACHE_AWARE = range(6)
+
 _lib = None
 
 
@@ -84,6 +92,7 @@ def lib():
             "aibx_route_batch": [vp, vp, vp, vp, i32, i32, u64, vp, u64, C.POINTER(RouteParams),
                                  vp, vp, vp, vp, vp, vp, vp],
             "aibx_route_assign": [vp, vp, i32, i32, vp, u64, C.POINTER(RouteParams), i32, vp, vp, vp],
+            "aibx_route_policy": [i32, vp, vp, i32, i32, C.POINTER(PodMetrics), vp, u64, i32, vp, vp],
             "aibx_collect_blocks": [vp, i64, u32, vp, vp, vp, vp],
             "aibx_collect_blocks_static": [vp, i64, u32, vp, vp, vp],
             "aibx_kv_gather": [vp, C.POINTER(KVLayout), vp, i64, vp, vp],
@@ -250,6 +259,21 @@ def route_assign(match_len, blk_off, num_pods: int, pod_load, ready_mask: int, p
         _ptr(match_len, torch.uint32), _ptr(blk_off, torch.int64), R, num_pods,
         _ptr(pod_load, torch.int32), ready_mask & (2**64 - 1), prm, load_increment,
         _ptr(best_pod, torch.int32), _ptr(best_score, torch.int64), _stream()))
+
+
+def route_policy(policy: int, num_pods: int, R: int, ready_mask: int, best_pod, throughput=None,
+                 requests=None, kv_usage=None, queue_latency=None, serve_latency=None,
+                 match_len=None, blk_off=None, draws=None, threshold_pct: int = 50) -> None:
+    """One pod per request under one of the six policies (POLICY_* numbers); the per-pod
+    figures are int32 device tensors, only those the policy reads are needed."""
+    figs = (throughput, requests, kv_usage, queue_latency, serve_latency)
+    met = None
+    if any(t is not None for t in figs):
+        met = C.byref(PodMetrics(*[_ptr(t, torch.int32) for t in figs]))
+    _check("aibx_route_policy", lib().aibx_route_policy(
+        policy, _ptr(match_len, torch.uint32), _ptr(blk_off, torch.int64), R, num_pods, met,
+        _ptr(draws, torch.uint64), ready_mask & (2**64 - 1), threshold_pct,
+        _ptr(best_pod, torch.int32), _stream()))
 
 
 def collect_scratch_bytes(num_blocks: int) -> int:

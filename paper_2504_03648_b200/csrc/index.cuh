@@ -35,6 +35,17 @@ __device__ __forceinline__ unsigned long long home_slot(const IndexView& ix, uin
   return (key * 0x9E3779B97F4A7C15ULL) >> ix.shift;
 }
 
+// One 32-byte slot in one request: a 256-bit read-only load (slots are 32-byte aligned).
+__device__ __forceinline__ void load_slot(const Slot* p, unsigned long long& k,
+                                          unsigned long long& m, unsigned int& id) {
+  unsigned long long w2, w3;
+  asm volatile("ld.global.nc.v4.u64 {%0,%1,%2,%3}, [%4];"
+               : "=l"(k), "=l"(m), "=l"(w2), "=l"(w3)
+               : "l"(p));
+  (void)w3;
+  id = (unsigned int)w2;
+}
+
 __global__ void index_clear_kernel(IndexView ix) {
   const unsigned long long n = ix.cap_mask + 1;
   for (unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; i < n;
@@ -49,8 +60,8 @@ __global__ void index_clear_kernel(IndexView ix) {
   }
 }
 
-// Read-only probe (index not modified while the kernel runs): both halves of the slot are
-// requested together so a hit costs one memory round trip.
+// Read-only probe (index not modified while the kernel runs): the whole slot arrives with one
+// load, so a hit costs one memory round trip.
 __device__ __forceinline__ bool probe_ro(const IndexView& ix, uint64_t key, uint64_t& mask,
                                          uint32_t& id) {
   mask = 0;
@@ -58,15 +69,13 @@ __device__ __forceinline__ bool probe_ro(const IndexView& ix, uint64_t key, uint
   if (key_reserved(key)) return false;
   unsigned long long s = home_slot(ix, key);
   for (unsigned long long n = 0; n <= ix.cap_mask; ++n) {
-    const uint4* p = reinterpret_cast<const uint4*>(ix.slots + s);
-    const uint4 a = __ldg(p);
-    const uint4 b = __ldg(p + 1);
-    const uint64_t k = (uint64_t)a.x | ((uint64_t)a.y << 32);
+    unsigned long long k, m;
+    unsigned int sid;
+    load_slot(ix.slots + s, k, m, sid);
     if (k == key) {
-      const uint64_t m = (uint64_t)a.z | ((uint64_t)a.w << 32);
       if (m == 0) return false;
       mask = m;
-      id = b.x;
+      id = sid;
       return true;
     }
     if (k == kKeyEmpty) return false;

@@ -367,6 +367,41 @@ int32_t aibx_route_score(const uint32_t* d_match_len, const int64_t* d_blk_off, 
   return launch_status();
 }
 
+int32_t aibx_route_policy(int32_t policy, const uint32_t* d_match_len, const int64_t* d_blk_off,
+                          int32_t R, int32_t num_pods, const aibx_pod_metrics_t* metrics,
+                          const uint64_t* d_draws, uint64_t ready_mask, int32_t threshold_pct,
+                          int32_t* d_best_pod, void* stream) {
+  if (R < 0 || num_pods < 1 || num_pods > AIBX_MAX_PODS || policy < AIBX_POLICY_RANDOM ||
+      policy > AIBX_POLICY_PREFIX_CACHE_AWARE)
+    return AIBX_ERR_INVALID;
+  if (R == 0) return AIBX_OK;
+  if (!d_best_pod) return AIBX_ERR_INVALID;
+  PodMetrics met = {nullptr, nullptr, nullptr, nullptr, nullptr};
+  if (policy == AIBX_POLICY_RANDOM) {
+    if (!d_draws) return AIBX_ERR_INVALID;
+  } else {
+    if (!metrics) return AIBX_ERR_INVALID;
+    met = PodMetrics{metrics->d_throughput, metrics->d_requests, metrics->d_kv_usage,
+                     metrics->d_queue_latency, metrics->d_serve_latency};
+    const bool have =
+        policy == AIBX_POLICY_THROUGHPUT       ? met.throughput != nullptr
+        : policy == AIBX_POLICY_LEAST_KV_CACHE ? met.kv_usage != nullptr
+        : policy == AIBX_POLICY_LEAST_LATENCY  ? met.queue_latency && met.serve_latency
+                                               : met.requests != nullptr;
+    if (!have) return AIBX_ERR_INVALID;
+    if (policy == AIBX_POLICY_PREFIX_CACHE_AWARE && (!d_match_len || !d_blk_off))
+      return AIBX_ERR_INVALID;
+  }
+  // one warp per request up to a few waves of the machine, grid-stride beyond
+  const int64_t want = blocks_for(R, kRouteWarps);
+  const int64_t cap = (int64_t)sm_count() * 16;
+  const unsigned int grid = (unsigned int)(want < cap ? want : cap);
+  route_policy_kernel<<<grid, kRouteWarps * 32, 0, as_stream(stream)>>>(
+      policy, d_match_len, d_blk_off, R, num_pods, met, d_draws, ready_mask, threshold_pct,
+      d_best_pod);
+  return launch_status();
+}
+
 uint64_t aibx_collect_scratch_bytes(uint32_t num_blocks) {
   return 4ULL * (((uint64_t)num_blocks + 31ULL) / 32ULL);
 }

@@ -130,4 +130,91 @@ route_assign_kernel(const uint32_t* __restrict__ match_len, const int64_t* __res
   if (p1 < P) pod_load[p1] = load1;
 }
 
+// The six per-request routing policies.  One warp per request (grid-stride), two pods per lane.
+// A policy is "lowest figure over a candidate set": the candidate set is the ready pods, except
+// for prefix-cache-aware, where a max-reduction over the qualifying hits first narrows it to the
+// pods with the longest qualifying hit (if any).  The random policy picks the k-th ready pod
+// by rank inside the ready mask.
+struct PodMetrics {
+  const int32_t* throughput;
+  const int32_t* requests;
+  const int32_t* kv_usage;
+  const int32_t* queue_latency;
+  const int32_t* serve_latency;
+};
+
+__global__ void __launch_bounds__(kRouteWarps * 32)
+route_policy_kernel(int policy, const uint32_t* __restrict__ match_len,
+                    const int64_t* __restrict__ blk_off, int R, int P, PodMetrics met,
+                    const uint64_t* __restrict__ draws, uint64_t ready_mask, int thr_pct,
+                    int32_t* __restrict__ best_pod) {
+  const int lane = threadIdx.x & 31;
+  const int p0 = lane, p1 = lane + 32;
+  const int warps = gridDim.x * kRouteWarps;
+  const uint64_t ready = ready_mask & pod_all(P);
+
+  if (policy == AIBX_POLICY_RANDOM) {
+    const int n = __popcll(ready);
+    // rank of this lane's pods among the ready ones
+    const int rank0 = __popcll(ready & ((1ULL << p0) - 1ULL));
+    const int rank1 = __popcll(ready & ((1ULL << p1) - 1ULL));
+    const bool in0 = (ready >> p0) & 1ULL, in1 = (ready >> p1) & 1ULL;
+    for (int r = blockIdx.x * kRouteWarps + (threadIdx.x >> 5); r < R; r += warps) {
+      if (n == 0) {
+        if (lane == 0) best_pod[r] = AIBX_NO_POD;
+        continue;
+      }
+      const int k = (int)(draws[r] % (unsigned long long)n);
+      if (in0 && rank0 == k) best_pod[r] = p0;
+      if (in1 && rank1 == k) best_pod[r] = p1;
+    }
+    return;
+  }
+
+  // the figure every remaining policy minimises, negated so that warp_argmax applies
+  const int32_t* a = policy == AIBX_POLICY_THROUGHPUT      ? met.throughput
+                     : policy == AIBX_POLICY_LEAST_KV_CACHE ? met.kv_usage
+                     : policy == AIBX_POLICY_LEAST_LATENCY  ? met.queue_latency
+                                                            : met.requests;
+  const int32_t* b = policy == AIBX_POLICY_LEAST_LATENCY ? met.serve_latency : nullptr;
+  long long sc0 = 0, sc1 = 0;
+  if (p0 < P) sc0 = -((long long)a[p0] + (b ? (long long)b[p0] : 0LL));
+  if (p1 < P) sc1 = -((long long)a[p1] + (b ? (long long)b[p1] : 0LL));
+
+  if (policy != AIBX_POLICY_PREFIX_CACHE_AWARE) {
+    long long top;
+    int arg;
+    lane_candidate(lane, P, ready, sc0, sc1, top, arg);
+    warp_argmax(top, arg);
+    for (int r = blockIdx.x * kRouteWarps * 32 + threadIdx.x; r < R; r += warps * 32)
+      best_pod[r] = arg;                       // the same pod for every request: lanes over r
+    return;
+  }
+
+  for (int r = blockIdx.x * kRouteWarps + (threadIdx.x >> 5); r < R; r += warps) {
+    const long long n_r = blk_off[r + 1] - blk_off[r];
+    unsigned int e0 = 0, e1 = 0;               // qualifying hit of a ready pod, else 0
+    if (p0 < P && ((ready >> p0) & 1ULL)) {
+      const unsigned int hit = match_len[(int64_t)r * P + p0];
+      if (hit > 0 && 100LL * hit >= (long long)thr_pct * n_r) e0 = hit;
+    }
+    if (p1 < P && ((ready >> p1) & 1ULL)) {
+      const unsigned int hit = match_len[(int64_t)r * P + p1];
+      if (hit > 0 && 100LL * hit >= (long long)thr_pct * n_r) e1 = hit;
+    }
+    const unsigned int longest = __reduce_max_sync(0xffffffffu, e0 > e1 ? e0 : e1);
+    uint64_t cand = ready;
+    if (longest > 0) {
+      const unsigned int c_lo = __ballot_sync(0xffffffffu, e0 == longest);
+      const unsigned int c_hi = __ballot_sync(0xffffffffu, e1 == longest);
+      cand = (uint64_t)c_lo | ((uint64_t)c_hi << 32);
+    }
+    long long top;
+    int arg;
+    lane_candidate(lane, P, cand, sc0, sc1, top, arg);
+    warp_argmax(top, arg);
+    if (lane == 0) best_pod[r] = arg;
+  }
+}
+
 }  // namespace aibx

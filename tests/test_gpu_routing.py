@@ -382,6 +382,61 @@ def test_route_assign_sequential():
     assert host(d_bp).tolist() == [1, 2, 0] and host(d_load).tolist() == [2, 1, 1]
 
 
+# ------------------------------------------------------------------ the six routing policies
+
+def test_route_policies():
+    rng = np.random.default_rng(91)
+    fields = ("throughput", "requests", "kv_usage", "queue_latency", "serve_latency")
+    for P in (1, 6, 32, 33, 64):
+        R = 2500 if P == 33 else 400                  # 2,500 requests: several requests per warp slot
+        n = rng.integers(0, 50, R)
+        bo = np.concatenate([[0], np.cumsum(n)]).astype(np.int64)
+        ml = (rng.random((R, P)) * (n[:, None] + 1)).astype(np.uint32)
+        ml[rng.random((R, P)) < 0.3] = 0
+        draws = np.frombuffer(rng.bytes(8 * R), dtype=np.uint64).copy()
+        for wide in (False, True):
+            if wide:                                  # whole int32 range, latency sums past 2^31
+                met = {f: rng.integers(-2**31, 2**31, P).astype(np.int32) for f in fields}
+                met["queue_latency"][: P // 2] = 2**31 - 1
+                met["serve_latency"][: P // 2] = 2**31 - 1 - rng.integers(0, 3, P // 2)
+            else:
+                met = {f: rng.integers(0, 4, P).astype(np.int32) for f in fields}   # many ties
+            d_met = {f: dev(a) for f, a in met.items()}
+            for ready in (ALL, 0, 1 << (P - 1), int(rng.integers(0, 1 << 62)) & ((1 << P) - 1)):
+                for pol, name in enumerate(oracle.POLICIES):
+                    for thr in ((0, 50, 100) if name == "prefix-cache-aware" else (50,)):
+                        d_bp = torch.full((R,), -9, dtype=torch.int32, device="cuda")
+                        aibx.route_policy(pol, P, R, ready, d_bp, match_len=dev(ml.reshape(-1)),
+                                          blk_off=dev(bo), draws=dev(draws), threshold_pct=thr,
+                                          **d_met)
+                        want = oracle.route_policy(name, P, R, ready, met, ml, bo, draws, thr)
+                        assert np.array_equal(host(d_bp), want), (P, wide, ready, name, thr)
+    # the hand example of the oracle's pins
+    met = {"throughput": [900, 400, 650], "requests": [3, 5, 2], "kv_usage": [70, 10, 40],
+           "queue_latency": [5, 50, 20], "serve_latency": [100, 40, 90]}
+    d_met = {f: dev(np.array(a, np.int32)) for f, a in met.items()}
+    ml = np.array([[2, 3, 0], [2, 2, 0], [1, 0, 0], [0, 0, 0]], dtype=np.uint32)
+    bo = np.array([0, 4, 8, 12, 16], np.int64)
+    d_bp = empty(4, torch.int32)
+    aibx.route_policy(aibx.POLICY_PREFIX_CACHE_AWARE, 3, 4, 7, d_bp, match_len=dev(ml.reshape(-1)),
+                      blk_off=dev(bo), **d_met)
+    assert host(d_bp).tolist() == [1, 0, 2, 2]
+    aibx.route_policy(aibx.POLICY_LEAST_LATENCY, 3, 4, 7, d_bp, **d_met)
+    assert host(d_bp).tolist() == [1, 1, 1, 1]
+    # only the arrays a policy reads are needed; a missing one is refused on the host
+    aibx.route_policy(aibx.POLICY_LEAST_KV_CACHE, 3, 4, 0b101, d_bp, kv_usage=d_met["kv_usage"])
+    assert host(d_bp).tolist() == [2] * 4
+    for bad in (dict(policy=6), dict(policy=-1), dict(policy=1, requests=d_met["requests"]),
+                dict(policy=0), dict(policy=5, requests=d_met["requests"]),
+                dict(policy=4, queue_latency=d_met["queue_latency"])):
+        pol = bad.pop("policy")
+        with pytest.raises(aibx.AibxError) as e:
+            aibx.route_policy(pol, 3, 4, 7, d_bp, **bad)
+        assert e.value.code == aibx.ERR_INVALID
+    aibx.route_policy(2, 3, 0, 7, None, requests=d_met["requests"])          # R = 0: no-op
+    assert aibx.status_fetch() == (0, 0)
+
+
 # ------------------------------------------------------------------ export and rehash
 
 def test_index_export_and_rehash():
