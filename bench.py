@@ -1016,19 +1016,60 @@ def case_kv_inner(args):
         nbytes = 2 * n * kv.block_bytes
         t_plain = statistics.median(_event_times(
             torch, lambda: aibx.kv_gather(pool, lay, ids, n, buf), 10, 3))
-        t_g = statistics.median(_event_times(
-            torch, lambda: aibx.kv_gather_inner(pool, lay, 0, 1, ids, n, buf), 10, 3))
-        t_s = statistics.median(_event_times(
-            torch, lambda: aibx.kv_scatter_inner(pool, lay, 0, 1, ids, n, buf), 10, 3))
-        out.append({"shape": name, "blocks": n, "bytes_read_plus_written": nbytes,
-                    "plain_gather_GBps": round(nbytes / (t_plain * 1e-3) / 1e9, 1),
-                    "gather_inner_GBps": round(nbytes / (t_g * 1e-3) / 1e9, 1),
-                    "scatter_inner_GBps": round(nbytes / (t_s * 1e-3) / 1e9, 1)})
+        row = {"shape": name, "blocks": n, "bytes_read_plus_written": nbytes,
+               "plain_gather_GBps": round(nbytes / (t_plain * 1e-3) / 1e9, 1)}
+        for engine, tag in ((2, "tensor_store"), (1, "storer_warps")):
+            aibx.kv_set_inner_engine(engine)
+            for pi, bi, order in ((0, 1, "head_token_to_token_head"),
+                                  (1, 0, "token_head_to_head_token")):
+                t_g = statistics.median(_event_times(
+                    torch, lambda: aibx.kv_gather_inner(pool, lay, pi, bi, ids, n, buf), 10, 3))
+                t_s = statistics.median(_event_times(
+                    torch, lambda: aibx.kv_scatter_inner(pool, lay, pi, bi, ids, n, buf), 10, 3))
+                row["%s_%s_gather_GBps" % (tag, order)] = round(nbytes / (t_g * 1e-3) / 1e9, 1)
+                row["%s_%s_scatter_GBps" % (tag, order)] = round(nbytes / (t_s * 1e-3) / 1e9, 1)
+        aibx.kv_set_inner_engine(0)
+        out.append(row)
         del pool, buf
         torch.cuda.empty_cache()
     peak, kind = measured_peak_hbm()
     print(json.dumps({"case": "kv_inner", "peak": peak, "peak_kind": kind, "results": out,
                       "status": aibx.status_fetch()}))
+
+
+def case_kv_inner_small(args):
+    """Gather then scatter 256 blocks of the cfg2 shape out of a 1 GiB pool with the head/token
+    order swapped (tensor-map store): the capture target for kv_permute_tma_kernel."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import synth
+    from paper_2504_03648_b200 import workloads as W
+
+    kv = W.scaled(W.cfg2_kv(), num_blocks=512)
+    n = 256
+    pool = torch.empty(kv.pool_bytes, dtype=torch.uint8, device="cuda")
+    synth.fill_pool(pool, kv)
+    ids = torch.from_numpy(np.sort(W.distinct_ids(7, kv.num_blocks, n))).cuda()
+    buf = torch.empty(n * kv.block_bytes, dtype=torch.uint8, device="cuda")
+    lay = aibx.KVLayout(kv.layout, kv.num_layers, kv.num_kv_heads, kv.block_tokens, kv.head_dim,
+                        kv.elem_bytes, kv.num_blocks)
+    aibx.kv_set_inner_engine(2)
+
+    def both():
+        aibx.kv_gather_inner(pool, lay, 0, 1, ids, n, buf)
+        aibx.kv_scatter_inner(pool, lay, 0, 1, ids, n, buf)
+
+    ts = _event_times(torch, both, max(args.steps, 1), max(args.warmup, 1))
+    aibx.kv_set_inner_engine(0)
+    nbytes = 2 * (2 * n * kv.block_bytes + 4 * n)
+    peak, kind = measured_peak_hbm()
+    print(json.dumps({"case": "kv_inner_small", "blocks": n,
+                      "algorithmic_bytes_per_launch": nbytes // 2,
+                      "ms_gather_plus_scatter_median": round(statistics.median(ts), 4),
+                      "GBps_median": round(nbytes / (statistics.median(ts) * 1e-3) / 1e9, 1),
+                      "GBps_best": round(nbytes / (min(ts) * 1e-3) / 1e9, 1), "peak": peak,
+                      "peak_kind": kind, "status": aibx.status_fetch()}))
 
 
 def case_index_ops(args):
@@ -1113,7 +1154,7 @@ def case_kv_comparators(args):
                       "status": aibx.status_fetch()}))
 
 
-CASES = {"kv_comparators": case_kv_comparators, "index_ops": case_index_ops, "kv_inner": case_kv_inner, "hash_sweep": case_hash_sweep, "oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
+CASES = {"kv_comparators": case_kv_comparators, "index_ops": case_index_ops, "kv_inner": case_kv_inner, "kv_inner_small": case_kv_inner_small, "hash_sweep": case_hash_sweep, "oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
          "cfg4": case_cfg4, "cfg5": case_cfg5, "lookup_flat": case_lookup_flat}
 
 

@@ -337,7 +337,8 @@ int32_t aibx_kv_scatter_counted(void* d_pool, const aibx_kv_layout_t* layout,
  * of head_dim elements move whole (head_dim * elem_bytes must be a multiple of 16 and at most
  * 32 KiB: UNSUPPORTED otherwise); everything else - layouts, ids, skipping, errors - is as in
  * aibx_kv_gather / aibx_kv_scatter, to which equal orders reduce.  The transposition goes
- * through shared memory so that global reads and writes both stay whole rows.
+ * through shared memory so that global reads and writes both stay whole rows (see
+ * aibx_kv_set_inner_engine for the two engines that write the destination).
  */
 #define AIBX_INNER_HEAD_TOKEN 0
 #define AIBX_INNER_TOKEN_HEAD 1
@@ -356,6 +357,14 @@ int32_t aibx_kv_scatter_inner(void* d_pool, const aibx_kv_layout_t* layout, int3
  */
 int32_t aibx_kv_set_tuning(int32_t mode, int32_t chunk_bytes, int32_t stages,
                            int32_t ctas_per_sm);
+/* Which engine writes the destination of the _inner calls, process-wide; for measurement and
+ * tests.  0 (default) = a tensor-map store (cp.async.bulk.tensor) whose strides are those of the
+ * destination order, falling back to 1 for shapes it cannot take (rows of head_dim*elem_bytes
+ * over 2 KiB); 1 = storer warps (shared memory read back, coalesced streaming stores);
+ * 2 = the tensor-map store or AIBX_ERR_UNSUPPORTED, never the fallback.  INVALID otherwise.
+ */
+int32_t aibx_kv_set_inner_engine(int32_t engine);
+
 
 /* Bulk ring only, process-wide: how many store groups may still be reading shared memory
  * before their stage is handed back to the loader (1..4; default 1).  INVALID otherwise.

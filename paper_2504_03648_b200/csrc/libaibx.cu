@@ -502,6 +502,12 @@ int32_t aibx_kv_set_tuning(int32_t mode, int32_t chunk_bytes, int32_t stages,
   return AIBX_OK;
 }
 
+int32_t aibx_kv_set_inner_engine(int32_t engine) {
+  if (engine < 0 || engine > 2) return AIBX_ERR_INVALID;
+  permute_engine() = engine;
+  return AIBX_OK;
+}
+
 int32_t aibx_kv_set_store_lag(int32_t lag) {
   if (lag < 1 || lag > 4) return AIBX_ERR_INVALID;
   copy_tuning().lag = lag;

@@ -20,13 +20,34 @@ SHAPES = [
     (2, 5, 7, 24, 2, 33),       # odd counts, 48-byte rows
     (1, 4, 32, 128, 1, 64),     # fp8: 128-byte rows
     (1, 3, 5, 520, 4, 9),       # 2,080-byte rows, 15 rows per chunk of a 15-row plane
+    (1, 6, 48, 128, 2, 12),     # boxes of 2 heads x 48 tokens / of 21 tokens x 6 heads (ragged: 21, 21, 6)
+    (1, 2, 200, 128, 2, 6),     # one head's 200 rows overflow a stage: boxes of 128 and 72 rows
 ]
 
+ENGINES = [1, 2]                # storer warps; tensor-map store (no fallback)
 
+
+@pytest.fixture(autouse=True)
+def _default_engine_afterwards():
+    yield
+    aibx.kv_set_inner_engine(0)
+
+
+@pytest.mark.parametrize("engine", ENGINES)
 @pytest.mark.parametrize("shape", SHAPES)
 @pytest.mark.parametrize("layout", [0, 1])
-def test_inner_order_gather_and_scatter(layout, shape):
+def test_inner_order_gather_and_scatter(layout, shape, engine):
     L, H, T, D, E, nb = shape
+    if engine == 2 and D * E > 2048:
+        # rows too long for one box: the tensor-map engine says so, the default falls back
+        aibx.kv_set_inner_engine(2)
+        kv0 = W.KVSpec("inner", 21, layout, L, H, T, D, E, nb)
+        with pytest.raises(aibx.AibxError) as e:
+            aibx.kv_gather_inner(empty(kv0.pool_bytes, torch.uint8), kv_layout_gpu(kv0), 0, 1,
+                                 dev(np.zeros(1, np.uint32)), 1, empty(kv0.block_bytes, torch.uint8))
+        assert e.value.code == aibx.ERR_UNSUPPORTED
+        engine = 0
+    aibx.kv_set_inner_engine(engine)
     kv = W.KVSpec("inner", 21, layout, L, H, T, D, E, nb)
     lay_g, lay_o = kv_layout_gpu(kv), kv_layout_oracle(kv)
     pool_h = W.host_pool(kv)
@@ -91,13 +112,18 @@ def test_inner_order_large_launch_bandwidth_shape():
     synth.fill_pool(pool, kv)
     n = 600
     ids = W.distinct_ids(3, kv.num_blocks, n)
-    buf = empty(n * kv.block_bytes, torch.uint8)
     lay = kv_layout_gpu(kv)
-    aibx.kv_gather_inner(pool, lay, 0, 1, dev(ids), n, buf)
-    assert aibx.status_fetch() == (0, 0)
     lay1 = kv_layout_oracle(kv, layout=0, num_blocks=1)
-    for i in (0, 1, 299, n - 1):
-        mini = W.logical_blocks(kv, [ids[i]])
-        want = np.zeros(kv.block_bytes, dtype=np.uint8)
-        oracle.kv_gather_inner(mini, lay1, 0, 1, np.zeros(1, np.uint32), want)
-        assert np.array_equal(host(buf.view(n, kv.block_bytes)[i]), want)
+    bufs = []
+    for engine in (2, 1):
+        aibx.kv_set_inner_engine(engine)
+        buf = empty(n * kv.block_bytes, torch.uint8)
+        aibx.kv_gather_inner(pool, lay, 0, 1, dev(ids), n, buf)
+        assert aibx.status_fetch() == (0, 0)
+        for i in (0, 1, 299, n - 1):
+            mini = W.logical_blocks(kv, [ids[i]])
+            want = np.zeros(kv.block_bytes, dtype=np.uint8)
+            oracle.kv_gather_inner(mini, lay1, 0, 1, np.zeros(1, np.uint32), want)
+            assert np.array_equal(host(buf.view(n, kv.block_bytes)[i]), want)
+        bufs.append(buf)
+    assert torch.equal(bufs[0], bufs[1])                   # every byte, engine against engine
