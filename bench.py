@@ -38,7 +38,7 @@ METRIC = "kv_gather_scatter_GBps_whole_step"
 UNIT = "GB/s"
 WORKLOAD = "cfg2-llama3-8b: 64 requests (1k-8k tokens, 32 Zipf prompts), index 200k/2^19 x 16 pods, " \
            "pool 4096 x 2 MiB bf16 blocks, gather+scatter of all matched blocks"
-KERNELS_PER_STEP = 10   # hash, match+score, mark, compact, gather, scatter, insert, evict x3
+KERNELS_PER_STEP = 10   # head (hash+match+score), mark, compact, gather, scatter, hash tail, insert, evict x3
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of kv_copy_bulk_kernel from the ncu
 # capture summarised under profiles/, valid only for the kernel source with this digest.
@@ -183,6 +183,8 @@ class GpuJob:
         self.d_block_ids = torch.empty(self.nb, dtype=torch.uint32, device="cuda")
         self.d_best_pod = torch.empty(R, dtype=torch.int32, device="cuda")
         self.d_best_score = torch.empty(R, dtype=torch.int64, device="cuda")
+        self.d_hashed = torch.empty(R, dtype=torch.uint32, device="cuda")
+        self.d_next_seed = torch.empty(R, dtype=torch.uint64, device="cuda")
         self.d_pod_load = dev(w.pod_load)
         self.d_scratch = torch.empty(aibx.collect_scratch_bytes(kv.num_blocks) // 4 + 1,
                                      dtype=torch.int32, device="cuda")
@@ -208,13 +210,21 @@ class GpuJob:
 
     # -- pieces of a step ------------------------------------------------------------------
     def routing_async(self) -> None:
-        """Routing half of a step, enqueued only: the block count stays on the device."""
+        """Routing half of a step, enqueued only: the block count stays on the device.  Only
+        the part of every chain that matching needs is hashed here (aibx_route_head); the rest
+        is hashed by hash_tail() off the critical path."""
         aibx = self.aibx
-        aibx.route_batch(self.index, self.d_tokens, self.d_tok_off, self.d_blk_off, self.B, 0,
-                         self.d_pod_load, self.w.ready_mask, None, self.d_hashes, self.d_match_len,
-                         self.d_any_len, self.d_block_ids, self.d_best_pod, self.d_best_score)
+        aibx.route_head(self.index, self.d_tokens, self.d_tok_off, self.d_blk_off, self.B, 0,
+                        self.d_pod_load, self.w.ready_mask, None, self.d_hashes, self.d_match_len,
+                        self.d_any_len, self.d_block_ids, self.d_best_pod, self.d_best_score,
+                        self.d_hashed, self.d_next_seed)
         aibx.collect_blocks(self.d_block_ids, self.kv.num_blocks, self.d_scratch, self.d_unique,
                             self.d_count)
+
+    def hash_tail(self) -> None:
+        """The rest of every chain (the keys of the blocks that will be published)."""
+        self.aibx.hash_blocks_resume(self.d_tokens, self.d_tok_off, self.d_blk_off, self.B,
+                                     self.d_hashed, self.d_next_seed, self.d_hashes)
 
     def routing(self) -> int:
         aibx = self.aibx
@@ -235,8 +245,9 @@ class GpuJob:
 
     def step(self, record_copy_events=False):
         """One pass of the whole path, enqueued without any host round trip: the number of
-        matched blocks goes from aibx_collect_blocks to the copies on the device, and the index
-        publish/expire batch (independent of the copies) runs beside them on a second stream."""
+        matched blocks goes from aibx_collect_blocks to the copies on the device; the tail of
+        the hash chains and the index publish/expire batch (both independent of the copies) run
+        beside them on a second stream."""
         torch, aibx = self.torch, self.aibx
         main = torch.cuda.current_stream()
         if self.side is None:
@@ -247,6 +258,7 @@ class GpuJob:
         self.ev_routed.record(main)
         self.side.wait_event(self.ev_routed)
         with torch.cuda.stream(self.side):
+            self.hash_tail()
             self.publish_expire()
             self.ev_index.record(self.side)
         cap = self.count                                  # room in the transfer buffer, in blocks
@@ -322,6 +334,12 @@ class GpuJob:
         calls = {
             "hash_blocks": lambda: aibx.hash_blocks(self.d_tokens, self.d_tok_off, self.d_blk_off,
                                                     self.B, 0, self.d_hashes),
+            "route_head": lambda: aibx.route_head(
+                self.index, self.d_tokens, self.d_tok_off, self.d_blk_off, self.B, 0,
+                self.d_pod_load, self.w.ready_mask, None, self.d_hashes, self.d_match_len,
+                self.d_any_len, self.d_block_ids, self.d_best_pod, self.d_best_score,
+                self.d_hashed, self.d_next_seed),
+            "hash_tail": self.hash_tail,
             "match_prefix": lambda: self.index.match_prefix(self.d_hashes, self.d_blk_off,
                                                             self.d_match_len, self.d_any_len,
                                                             self.d_block_ids),
@@ -454,7 +472,7 @@ def run_gpu(args):
         "config": {"workload": WORKLOAD, "blocks_moved_per_step": job.count,
                    "bytes_moved_per_step": step_bytes, "parallelism": "replicas only" if world > 1 else "1 gpu",
                    "l2": "inputs larger than L2: 6.5 GB of KV traffic per step evicts it between steps",
-                   "overlap": "index publish/expire on a second stream beside the copies; no host sync inside a step",
+                   "overlap": "hash chains past the first uncached block and index publish/expire on a second stream beside the copies; no host sync inside a step",
                    "kv_tuning": "bulk ring, loader + storer warp, 32 KiB x 3 stages, 1 CTA/SM"},
         "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
         "e2e": {"value": round(world * step_bytes / e2e_s / 1e9, 2), "unit": UNIT,

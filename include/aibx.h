@@ -193,6 +193,37 @@ int32_t aibx_route_batch(const aibx_index_t* index, const int32_t* d_tokens,
                          void* stream);
 
 /* ---------------------------------------------------------------------------------------
+ * Routing with the critical path cut short (Section 3.2.2: the routing decision depends on the
+ * reusable prefix only; nothing past the first block that no instance caches can change it,
+ * while hashing a chain is serial in its length).  aibx_route_head hashes every request only as
+ * far as matching needs - it probes the index for each key as it is produced and stops soon
+ * after the first block without a live entry - and leaves the rest of the chain to
+ * aibx_hash_blocks_resume, which may run on another stream, e.g. beside the KV copies.
+ *
+ * After aibx_route_head: d_match_len, d_any_len, d_block_ids, d_best_pod, d_best_score hold what
+ * aibx_route_batch would have written (same definitions, bit for bit); d_hashes holds the first
+ * d_hashed[r] keys of every request, with any_len[r] + 1 <= d_hashed[r] <= n_r (or = n_r);
+ * d_next_seed[r] is the key of block d_hashed[r] - 1 (root_seed when d_hashed[r] = 0).  How far
+ * past any_len a request was hashed is not specified.
+ * After aibx_hash_blocks_resume with that state: d_hashes is complete, as from aibx_hash_blocks.
+ *   d_hashed [R] uint32, d_next_seed [R] uint64: out of the first call, in of the second.
+ *   d_any_len, d_block_ids nullable; d_best_pod and d_best_score both given (then d_pod_load is
+ *   required) or both NULL.  Block sizes other than 8, 16, 32, 64 tokens are hashed in full by
+ *   the first call (d_hashed[r] = n_r).
+ */
+int32_t aibx_route_head(const aibx_index_t* index, const int32_t* d_tokens,
+                        const int64_t* d_tok_off, const int64_t* d_blk_off, int32_t R,
+                        int32_t block_tokens, uint64_t root_seed, const int32_t* d_pod_load,
+                        uint64_t ready_mask, const aibx_route_params_t* params,
+                        uint64_t* d_hashes, uint32_t* d_match_len, uint32_t* d_any_len,
+                        uint32_t* d_block_ids, int32_t* d_best_pod, int64_t* d_best_score,
+                        uint32_t* d_hashed, uint64_t* d_next_seed, void* stream);
+int32_t aibx_hash_blocks_resume(const int32_t* d_tokens, const int64_t* d_tok_off,
+                                const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
+                                const uint32_t* d_hashed, const uint64_t* d_next_seed,
+                                uint64_t* d_hashes, void* stream);
+
+/* ---------------------------------------------------------------------------------------
  * The routing policies the gateway offers per pending request (Section 3.2.2 lists six: random,
  * throughput, least-request, least-kv-cache, least-latency, prefix-cache-aware), taken for a
  * batch: one pod per request, every request of the call seeing the same snapshot of the per-pod

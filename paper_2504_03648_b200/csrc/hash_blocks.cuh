@@ -71,7 +71,8 @@ template <int SPB>
 __global__ void __launch_bounds__(32)
 hash_blocks_kernel(const int32_t* __restrict__ tokens, const int64_t* __restrict__ tok_off,
                    const int64_t* __restrict__ blk_off, int R, int spb_rt, uint64_t root_seed,
-                   uint64_t* __restrict__ hashes) {
+                   uint64_t* __restrict__ hashes, const uint32_t* __restrict__ start_blk,
+                   const uint64_t* __restrict__ start_seed) {
   const int lane = threadIdx.x;
   const int k = lane & 3;                              // accumulator of this lane
   const int quad_base = lane & ~3;
@@ -80,11 +81,14 @@ hash_blocks_kernel(const int32_t* __restrict__ tokens, const int64_t* __restrict
   if (r >= R) return;                                  // whole quads leave together
 
   const int spb = SPB > 0 ? SPB : spb_rt;
-  const int64_t out0 = blk_off[r];
+  // a resumed chain starts at block `skip` of the request, seeded with the key of block skip-1
+  const int64_t skip = start_blk ? (int64_t)start_blk[r] : 0;
+  const int64_t out0 = blk_off[r] + skip;
   const int64_t n_stripes = (blk_off[r + 1] - out0) * spb;
   if (n_stripes <= 0) return;
+  if (start_seed) root_seed = start_seed[r];
   // this lane's 8 bytes of stripe s are words [8*s + 2*k, 8*s + 2*k + 2) of the request
-  const int32_t* p = tokens + tok_off[r] + 2 * k;
+  const int32_t* p = tokens + tok_off[r] + skip * spb * 8 + 2 * k;
   uint64_t* out = hashes + out0;
 
   // per-lane constants of the four accumulators
@@ -157,24 +161,26 @@ hash_blocks_kernel(const int32_t* __restrict__ tokens, const int64_t* __restrict
 
 inline int32_t launch_hash_blocks(const int32_t* d_tokens, const int64_t* d_tok_off,
                                   const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
-                                  uint64_t root_seed, uint64_t* d_hashes, cudaStream_t st) {
+                                  uint64_t root_seed, uint64_t* d_hashes, cudaStream_t st,
+                                  const uint32_t* d_start_blk = nullptr,
+                                  const uint64_t* d_start_seed = nullptr) {
   const int spb = block_tokens / 8;
   const int grid = (R + 7) / 8;
   if (spb == 1) {
     hash_blocks_kernel<1><<<grid, 32, 0, st>>>(d_tokens, d_tok_off, d_blk_off, R, spb, root_seed,
-                                               d_hashes);
+                                               d_hashes, d_start_blk, d_start_seed);
   } else if (spb == 2) {
     hash_blocks_kernel<2><<<grid, 32, 0, st>>>(d_tokens, d_tok_off, d_blk_off, R, spb, root_seed,
-                                               d_hashes);
+                                               d_hashes, d_start_blk, d_start_seed);
   } else if (spb == 4) {
     hash_blocks_kernel<4><<<grid, 32, 0, st>>>(d_tokens, d_tok_off, d_blk_off, R, spb, root_seed,
-                                               d_hashes);
+                                               d_hashes, d_start_blk, d_start_seed);
   } else if (spb == 8) {
     hash_blocks_kernel<8><<<grid, 32, 0, st>>>(d_tokens, d_tok_off, d_blk_off, R, spb, root_seed,
-                                               d_hashes);
+                                               d_hashes, d_start_blk, d_start_seed);
   } else {
     hash_blocks_kernel<0><<<grid, 32, 0, st>>>(d_tokens, d_tok_off, d_blk_off, R, spb, root_seed,
-                                               d_hashes);
+                                               d_hashes, d_start_blk, d_start_seed);
   }
   return launch_status();
 }

@@ -38,12 +38,22 @@ __device__ __forceinline__ unsigned long long home_slot(const IndexView& ix, uin
 // One 32-byte slot in one request: a 256-bit read-only load (slots are 32-byte aligned).
 __device__ __forceinline__ void load_slot(const Slot* p, unsigned long long& k,
                                           unsigned long long& m, unsigned int& id) {
-  unsigned long long w2, w3;
+  unsigned long long w2;
+  [[maybe_unused]] unsigned long long w3;       // stamp and padding: not needed by a probe
   asm volatile("ld.global.nc.v4.u64 {%0,%1,%2,%3}, [%4];"
                : "=l"(k), "=l"(m), "=l"(w2), "=l"(w3)
                : "l"(p));
-  (void)w3;
   id = (unsigned int)w2;
+}
+
+// The same load with the third word (block id in its low half, stamp above) left as it arrives:
+// no instruction touches the result, so issuing it never waits for the data.
+__device__ __forceinline__ void load_slot_raw(const Slot* p, unsigned long long& k,
+                                              unsigned long long& m, unsigned long long& id_stamp) {
+  [[maybe_unused]] unsigned long long w3;
+  asm volatile("ld.global.nc.v4.u64 {%0,%1,%2,%3}, [%4];"
+               : "=l"(k), "=l"(m), "=l"(id_stamp), "=l"(w3)
+               : "l"(p));
 }
 
 __global__ void index_clear_kernel(IndexView ix) {

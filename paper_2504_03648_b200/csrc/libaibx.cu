@@ -12,6 +12,7 @@
 #include "kv_copy.cuh"
 #include "kv_permute.cuh"
 #include "selftest.cuh"
+#include "route_head.cuh"
 #include "route_score.cuh"
 #include "victims.cuh"
 
@@ -30,6 +31,29 @@ inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
 
 inline unsigned int blocks_for(int64_t n, int threads) {
   return (unsigned int)((n + threads - 1) / threads);
+}
+
+// The kernels that are meant to run BESIDE the KV copies (on another stream) ask for the same
+// shared-memory carve-out as the copy kernel needs.  An SM cannot host kernels with different
+// carve-outs at once: without this, every SM that runs one of these small kernels would keep the
+// copy kernel's CTA waiting until the small kernel has drained (measured: the gather ended later
+// by the whole duration of whatever ran beside it).  Once per device.
+void prefer_copy_carveout() {
+  static bool done[64] = {false};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || done[dev]) return;
+  done[dev] = true;
+  const void* side_kernels[] = {
+      (const void*)hash_blocks_kernel<0>,      (const void*)hash_blocks_kernel<1>,
+      (const void*)hash_blocks_kernel<2>,      (const void*)hash_blocks_kernel<4>,
+      (const void*)hash_blocks_kernel<8>,      (const void*)index_insert_kernel,
+      (const void*)index_evict_clear_kernel,   (const void*)index_evict_report_kernel,
+      (const void*)index_evict_remove_kernel,  (const void*)index_touch_kernel,
+  };
+  for (const void* f : side_kernels)
+    cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
+                         cudaSharedmemCarveoutMaxShared);
+  cudaGetLastError();   // a refused hint is not an error of the call that follows
 }
 
 // Device address of the status record of the current device.
@@ -80,6 +104,7 @@ int32_t aibx_hash_blocks(const int32_t* d_tokens, const int64_t* d_tok_off,
     return AIBX_ERR_INVALID;
   if (R == 0) return AIBX_OK;
   if (!d_tokens || !d_tok_off || !d_blk_off || !d_hashes) return AIBX_ERR_INVALID;
+  prefer_copy_carveout();
   return launch_hash_blocks(d_tokens, d_tok_off, d_blk_off, R, block_tokens, root_seed, d_hashes,
                             as_stream(stream));
 }
@@ -145,6 +170,7 @@ int32_t aibx_index_insert(aibx_index_t* ix, const uint64_t* d_keys, const uint64
   if (!ix || n < 0) return AIBX_ERR_INVALID;
   if (n == 0) return AIBX_OK;
   if (!d_keys || !d_pod_masks || !d_block_ids) return AIBX_ERR_INVALID;
+  prefer_copy_carveout();
   index_insert_kernel<<<blocks_for(n, 256), 256, 0, as_stream(stream)>>>(
       ix->view, d_keys, d_pod_masks, d_block_ids, n);
   return launch_status();
@@ -155,6 +181,7 @@ int32_t aibx_index_evict(aibx_index_t* ix, const uint64_t* d_keys, const uint64_
   if (!ix || n < 0) return AIBX_ERR_INVALID;
   if (n == 0) return AIBX_OK;
   if (!d_keys || !d_pod_masks) return AIBX_ERR_INVALID;
+  prefer_copy_carveout();
   cudaStream_t st = as_stream(stream);
   const unsigned int grid = blocks_for(n, 256);
   index_evict_clear_kernel<<<grid, 256, 0, st>>>(ix->view, d_keys, d_pod_masks, n);
@@ -333,6 +360,69 @@ int32_t aibx_route_batch(const aibx_index_t* ix, const int32_t* d_tokens, const 
   ScoreParams sp = {d_pod_load, ready_mask, prm.w_prefix, prm.w_load, prm.threshold_pct};
   return launch_match(ix, d_hashes, d_blk_off, R, d_match_len, d_any_len, d_block_ids, sp,
                       d_best_pod, d_best_score, st);
+}
+
+int32_t aibx_route_head(const aibx_index_t* ix, const int32_t* d_tokens, const int64_t* d_tok_off,
+                        const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
+                        uint64_t root_seed, const int32_t* d_pod_load, uint64_t ready_mask,
+                        const aibx_route_params_t* params, uint64_t* d_hashes,
+                        uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
+                        int32_t* d_best_pod, int64_t* d_best_score, uint32_t* d_hashed,
+                        uint64_t* d_next_seed, void* stream) {
+  if (!ix || R < 0 || block_tokens <= 0 || block_tokens % 8 != 0 || block_tokens > 1024)
+    return AIBX_ERR_INVALID;
+  if (R == 0) return AIBX_OK;
+  if (!d_tokens || !d_tok_off || !d_blk_off || !d_hashes || !d_match_len || !d_hashed ||
+      !d_next_seed)
+    return AIBX_ERR_INVALID;
+  if ((d_best_pod == nullptr) != (d_best_score == nullptr)) return AIBX_ERR_INVALID;
+  if (d_best_pod && !d_pod_load) return AIBX_ERR_INVALID;
+  aibx_route_params_t prm = {4, 1, 50};
+  if (params) prm = *params;
+  cudaStream_t st = as_stream(stream);
+  ScoreParams sp = {d_pod_load, ready_mask, prm.w_prefix, prm.w_load, prm.threshold_pct};
+  const int spb = block_tokens / 8;
+  const int grid = (R + 7) / 8;
+#define AIBX_HEAD_LAUNCH(SPB)                                                                   \
+  route_head_kernel<SPB><<<grid, 288, 0, st>>>(ix->view, d_tokens, d_tok_off, d_blk_off, R,      \
+                                              root_seed, d_hashes, d_match_len, d_any_len,      \
+                                              d_block_ids, sp, d_best_pod, d_best_score,        \
+                                              d_hashed, d_next_seed)
+  if (spb == 1) {
+    AIBX_HEAD_LAUNCH(1);
+  } else if (spb == 2) {
+    AIBX_HEAD_LAUNCH(2);
+  } else if (spb == 4) {
+    AIBX_HEAD_LAUNCH(4);
+  } else if (spb == 8) {
+    AIBX_HEAD_LAUNCH(8);
+  } else {
+    // other block sizes: the whole chain, then the match kernel; nothing is left to resume
+    int32_t rc = launch_hash_blocks(d_tokens, d_tok_off, d_blk_off, R, block_tokens, root_seed,
+                                    d_hashes, st);
+    if (rc != AIBX_OK) return rc;
+    rc = launch_match(ix, d_hashes, d_blk_off, R, d_match_len, d_any_len, d_block_ids, sp,
+                      d_best_pod, d_best_score, st);
+    if (rc != AIBX_OK) return rc;
+    route_head_state_full_kernel<<<blocks_for(R, 256), 256, 0, st>>>(d_blk_off, R, root_seed,
+                                                                     d_hashes, d_hashed, d_next_seed);
+  }
+#undef AIBX_HEAD_LAUNCH
+  return launch_status();
+}
+
+int32_t aibx_hash_blocks_resume(const int32_t* d_tokens, const int64_t* d_tok_off,
+                                const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
+                                const uint32_t* d_hashed, const uint64_t* d_next_seed,
+                                uint64_t* d_hashes, void* stream) {
+  if (R < 0 || block_tokens <= 0 || block_tokens % 8 != 0 || block_tokens > 1024)
+    return AIBX_ERR_INVALID;
+  if (R == 0) return AIBX_OK;
+  if (!d_tokens || !d_tok_off || !d_blk_off || !d_hashed || !d_next_seed || !d_hashes)
+    return AIBX_ERR_INVALID;
+  prefer_copy_carveout();
+  return launch_hash_blocks(d_tokens, d_tok_off, d_blk_off, R, block_tokens, 0, d_hashes,
+                            as_stream(stream), d_hashed, d_next_seed);
 }
 
 int32_t aibx_route_assign(const uint32_t* d_match_len, const int64_t* d_blk_off, int32_t R,

@@ -1,6 +1,6 @@
 """The step that bench.py times, at the benchmark's full size and in its launch configuration
-(route_batch, collect, device-counted gather and scatter, index publish/expire on a second
-stream), checked against the oracle: routing outputs element by element, the gathered buffer
+(route_head, collect, device-counted gather and scatter; the tail of the hash chains and the index
+publish/expire on a second stream), checked against the oracle: routing outputs element by element, the gathered buffer
 and the pool on sampled blocks, and the index back in its start state."""
 import os
 import sys
