@@ -746,6 +746,14 @@ def case_match_cfg(args):
         t_score = statistics.median(_event_times(
             torch, lambda: aibx.route_score(d_ml, d_bo, P, d_load, w.ready_mask, None, d_bp, d_bs,
                                             None), 10, 3))
+        d_dn = torch.empty(R, dtype=torch.uint32, device="cuda")
+        d_sd = torch.empty(R, dtype=torch.uint64, device="cuda")
+        t_head = statistics.median(_event_times(
+            torch, lambda: aibx.route_head(ix, d_tok, d_toff, d_bo, B, 0, d_load, w.ready_mask, None,
+                                           d_h, d_ml, d_al, d_ids, d_bp, d_bs, d_dn, d_sd), 10, 3))
+        t_tail = statistics.median(_event_times(
+            torch, lambda: aibx.hash_blocks_resume(d_tok, d_toff, d_bo, B, d_dn, d_sd, d_h), 10, 3))
+        hashed_by_head = int(d_dn.cpu().numpy().astype(np.int64).sum())
         al = d_al.cpu().numpy().astype(np.int64)
         n_r = np.diff(bo)
         lookups = int(np.minimum(al + 1, n_r).sum())
@@ -756,6 +764,8 @@ def case_match_cfg(args):
                     "insert_Mkeys_per_s": round(d_keys.numel() / (t_fill * 1e-3) / 1e6, 1),
                     "hash_us": round(t_hash * 1e3, 1), "match_us": round(t_match * 1e3, 1),
                     "score_us": round(t_score * 1e3, 1),
+                    "route_head_us": round(t_head * 1e3, 1), "hash_tail_us": round(t_tail * 1e3, 1),
+                    "blocks_hashed_by_head": hashed_by_head,
                     "hash_tokens_per_s": round(len(w.tokens) / (t_hash * 1e-3), 0),
                     "hash_ns_per_block_longest_chain": round(t_hash * 1e6 / int(n_r.max()), 1),
                     "match_requests_per_s": round(R / (t_match * 1e-3), 0),

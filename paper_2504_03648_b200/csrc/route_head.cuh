@@ -74,6 +74,17 @@ __device__ __forceinline__ unsigned int ld_relaxed_shared(const unsigned int* p)
 
 constexpr unsigned int kHeadStopBit = 0x80000000u;     // in `consumed`: no more keys needed
 
+// Polls the prober's word until it has consumed at least `need` blocks or says stop; `c` gets
+// the last value seen.  False when the bounded number of polls ran out.
+__device__ __noinline__ bool head_wait_for_room(const unsigned int* word, unsigned int need,
+                                                unsigned int& c) {
+  for (unsigned int polls = 0; polls < kHeadPolls; ++polls) {
+    c = ld_relaxed_shared(word);
+    if ((c & kHeadStopBit) || c >= need) return true;
+  }
+  return false;
+}
+
 template <int SPB>   // stripes of 32 bytes per block: 1, 2, 4 or 8
 __global__ void __launch_bounds__(288)
 route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
@@ -145,42 +156,45 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
     // What the prober says is read once per group and looked at one group LATER: a shared-memory
     // load that is consumed at once would wait together with the token loads in flight around
     // it (measured: +100 ns per block).  A stale count only errs on the safe side.
+    constexpr int kPublishGroups = BPG >= 4 ? 1 : 4 / BPG;
+    int groups_done = 0;
     unsigned int c = 0;
-    while (left > 0) {
-      if (c & kHeadStopBit) break;
-      if (hashed + BPG > c + kHeadRing) {
-        // a whole ring ahead of the prober (rare): wait for it, bounded - it always catches up
-        unsigned int polls = 0;
-        do {
-          c = *v_consumed;
-        } while (!(c & kHeadStopBit) && hashed + BPG > c + kHeadRing && ++polls < kHeadPolls);
-        if (c & kHeadStopBit) break;
-        if (polls >= kHeadPolls) {
-          if (k == 0) raise_status(AIBX_ERR_TIMEOUT);
-          break;
-        }
-      }
-      const unsigned int c_next = ld_relaxed_shared(&sh.consumed[qi]);
-      fetch(p + 8 * kGroupStripes, left - kGroupStripes, nxt_lo, nxt_hi);
-      if (left >= kGroupStripes) {                     // whole group: no per-stripe checks
+    for (;;) {
+      // hot loop: runs while there is work, no stop, and room in the ring (as last seen)
+      while (left > 0 && !(c & kHeadStopBit) && hashed + BPG <= c + kHeadRing) {
+        const unsigned int c_next = ld_relaxed_shared(&sh.consumed[qi]);
+        fetch(p + 8 * kGroupStripes, left - kGroupStripes, nxt_lo, nxt_hi);
+        if (left >= kGroupStripes) {                     // whole group: no per-stripe checks
 #pragma unroll
-        for (int s = 0; s < kGroupStripes; ++s) stripe(s);
-      } else {
+          for (int s = 0; s < kGroupStripes; ++s) stripe(s);
+        } else {
+#pragma unroll
+          for (int s = 0; s < kGroupStripes; ++s) {
+            if (s < left) stripe(s);                     // uniform inside the quad
+          }
+        }
 #pragma unroll
         for (int s = 0; s < kGroupStripes; ++s) {
-          if (s < left) stripe(s);                     // uniform inside the quad
+          cur_lo[s] = nxt_lo[s];
+          cur_hi[s] = nxt_hi[s];
         }
+        p += 8 * kGroupStripes;
+        left -= kGroupStripes;
+        // The keys before the count that announces them (release; the probers acquire).  The
+        // release also waits for the token loads in flight, so with few blocks per group it is
+        // done only every kPublishGroups groups (at least four blocks per release).
+        if (++groups_done % kPublishGroups == 0 || left <= 0) {
+          if (k == 0) st_release_shared(&sh.progress[qi], hashed);
+        }
+        c = c_next;
       }
-#pragma unroll
-      for (int s = 0; s < kGroupStripes; ++s) {
-        cur_lo[s] = nxt_lo[s];
-        cur_hi[s] = nxt_hi[s];
+      if (left <= 0 || (c & kHeadStopBit)) break;
+      // A whole ring ahead of the prober (rare; kept out of the hot loop, whose code the compiler
+      // schedules much worse with a wait inside it): wait for it, bounded - it always catches up.
+      if (!head_wait_for_room(&sh.consumed[qi], hashed + BPG - kHeadRing, c)) {
+        if (k == 0) raise_status(AIBX_ERR_TIMEOUT);
+        break;
       }
-      p += 8 * kGroupStripes;
-      left -= kGroupStripes;
-      // the keys before the count that announces them (release; the probers acquire)
-      if (k == 0) st_release_shared(&sh.progress[qi], hashed);
-      c = c_next;
     }
     return;
   }
