@@ -454,6 +454,11 @@ def run_gpu(args):
     e2e_s = max_over_ranks(e2e_s, dist, "cuda")
 
     stages = job.stage_breakdown() if rank == 0 else None
+    cfg3 = None
+    if rank == 0:
+        # the other half of the metric: prefix match alone on the routing-heavy batch
+        from paper_2504_03648_b200 import workloads as W
+        cfg3 = routing_batch_times(W.cfg3_routing)
     if dist is not None:
         dist.barrier()
     if rank != 0:
@@ -485,6 +490,12 @@ def run_gpu(args):
                      "avg_launch_ms": round(launch_ms, 4), "launches_timed": len(durs)},
         "cpu_baseline": cpu,
         "match_requests_per_s": round(job.R / (stages["match_prefix"] * 1e-6), 1),
+        "prefix_match_routing_heavy": {
+            "workload": "cfg3: 4,096 requests, 527k blocks, index 2^20 entries / 2^21 slots, 64 pods",
+            "match_requests_per_s": cfg3["match_requests_per_s"], "match_us": cfg3["match_us"],
+            "hash_us": cfg3["hash_us"], "route_head_us": cfg3["route_head_us"],
+            "decisions_per_s_via_route_head": round(cfg3["R"] / (cfg3["route_head_us"] * 1e-6), 0),
+            "match_algorithmic_GBps": cfg3["match_algorithmic_GBps"]},
         "stage_us": stages,
     }
     print(json.dumps(line))
@@ -695,82 +706,90 @@ def case_match_large(args):
                       "status": aibx.status_fetch()}))
 
 
-def case_match_cfg(args):
-    """match_prefix alone on the routing-heavy (cfg3) and long-context (cfg5) batches."""
+def routing_batch_times(mk):
+    """Event-timed routing calls (hash, match, score, head, tail, index fill) on one of the
+    routing workloads, each call alone on an otherwise idle GPU."""
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
     from paper_2504_03648_b200 import workloads as W
 
-    res = []
-    for mk in (W.cfg2_routing, W.cfg3_routing, W.cfg5_routing):
-        w = W.build_routing(mk())
-        s = w.spec
-        B, P, R = s.block_tokens, s.num_pods, s.R
+    w = W.build_routing(mk())
+    s = w.spec
+    B, P, R = s.block_tokens, s.num_pods, s.R
 
-        def dev(a):
-            return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    def dev(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
-        def offsets(tok_off):
-            n = (tok_off[1:] - tok_off[:-1]) // B
-            o = np.zeros(len(tok_off), dtype=np.int64)
-            np.cumsum(n, out=o[1:])
-            return o
+    def offsets(tok_off):
+        n = (tok_off[1:] - tok_off[:-1]) // B
+        o = np.zeros(len(tok_off), dtype=np.int64)
+        np.cumsum(n, out=o[1:])
+        return o
 
-        bo, sbo = offsets(w.tok_off), offsets(w.src_tok_off)
-        d_tok, d_toff, d_bo = dev(w.tokens), dev(w.tok_off), dev(bo)
-        d_h = torch.empty(int(bo[-1]), dtype=torch.uint64, device="cuda")
-        d_sh = torch.empty(int(sbo[-1]), dtype=torch.uint64, device="cuda")
-        aibx.hash_blocks(dev(w.src_tokens), dev(w.src_tok_off), dev(sbo), B, 0, d_sh)
-        ix = aibx.Index(s.capacity, P)
-        d_keys = torch.cat([d_sh, dev(w.filler_keys)])
-        d_masks = dev(np.concatenate([w.src_masks, w.filler_masks]))
-        d_eids = dev(np.concatenate([w.src_ids, w.filler_ids]))
+    bo, sbo = offsets(w.tok_off), offsets(w.src_tok_off)
+    d_tok, d_toff, d_bo = dev(w.tokens), dev(w.tok_off), dev(bo)
+    d_h = torch.empty(int(bo[-1]), dtype=torch.uint64, device="cuda")
+    d_sh = torch.empty(int(sbo[-1]), dtype=torch.uint64, device="cuda")
+    aibx.hash_blocks(dev(w.src_tokens), dev(w.src_tok_off), dev(sbo), B, 0, d_sh)
+    ix = aibx.Index(s.capacity, P)
+    d_keys = torch.cat([d_sh, dev(w.filler_keys)])
+    d_masks = dev(np.concatenate([w.src_masks, w.filler_masks]))
+    d_eids = dev(np.concatenate([w.src_ids, w.filler_ids]))
 
-        def refill():
-            ix.clear()
-            ix.insert(d_keys, d_masks, d_eids)
+    def refill():
+        ix.clear()
+        ix.insert(d_keys, d_masks, d_eids)
 
-        t_clear = statistics.median(_event_times(torch, lambda: ix.clear(), 5, 2))
-        t_fill = statistics.median(_event_times(torch, refill, 5, 2)) - t_clear
-        d_ml = torch.empty(R * P, dtype=torch.uint32, device="cuda")
-        d_al = torch.empty(R, dtype=torch.uint32, device="cuda")
-        d_ids = torch.empty(int(bo[-1]), dtype=torch.uint32, device="cuda")
-        d_bp = torch.empty(R, dtype=torch.int32, device="cuda")
-        d_bs = torch.empty(R, dtype=torch.int64, device="cuda")
-        d_load = dev(w.pod_load)
-        t_hash = statistics.median(_event_times(
-            torch, lambda: aibx.hash_blocks(d_tok, d_toff, d_bo, B, 0, d_h), 10, 3))
-        t_match = statistics.median(_event_times(
-            torch, lambda: ix.match_prefix(d_h, d_bo, d_ml, d_al, d_ids), 10, 3))
-        t_score = statistics.median(_event_times(
-            torch, lambda: aibx.route_score(d_ml, d_bo, P, d_load, w.ready_mask, None, d_bp, d_bs,
-                                            None), 10, 3))
-        d_dn = torch.empty(R, dtype=torch.uint32, device="cuda")
-        d_sd = torch.empty(R, dtype=torch.uint64, device="cuda")
-        t_head = statistics.median(_event_times(
-            torch, lambda: aibx.route_head(ix, d_tok, d_toff, d_bo, B, 0, d_load, w.ready_mask, None,
-                                           d_h, d_ml, d_al, d_ids, d_bp, d_bs, d_dn, d_sd), 10, 3))
-        t_tail = statistics.median(_event_times(
-            torch, lambda: aibx.hash_blocks_resume(d_tok, d_toff, d_bo, B, d_dn, d_sd, d_h), 10, 3))
-        hashed_by_head = int(d_dn.cpu().numpy().astype(np.int64).sum())
-        al = d_al.cpu().numpy().astype(np.int64)
-        n_r = np.diff(bo)
-        lookups = int(np.minimum(al + 1, n_r).sum())
-        nbytes = lookups * 40 + int((4 * P + 4) * R + 4 * al.sum())
-        res.append({"config": s.name, "R": R, "blocks": int(bo[-1]), "necessary_lookups": lookups,
-                    "index_entries": int(d_keys.numel()),
-                    "insert_us": round(t_fill * 1e3, 1),
-                    "insert_Mkeys_per_s": round(d_keys.numel() / (t_fill * 1e-3) / 1e6, 1),
-                    "hash_us": round(t_hash * 1e3, 1), "match_us": round(t_match * 1e3, 1),
-                    "score_us": round(t_score * 1e3, 1),
-                    "route_head_us": round(t_head * 1e3, 1), "hash_tail_us": round(t_tail * 1e3, 1),
-                    "blocks_hashed_by_head": hashed_by_head,
-                    "hash_tokens_per_s": round(len(w.tokens) / (t_hash * 1e-3), 0),
-                    "hash_ns_per_block_longest_chain": round(t_hash * 1e6 / int(n_r.max()), 1),
-                    "match_requests_per_s": round(R / (t_match * 1e-3), 0),
-                    "match_algorithmic_GBps": round(nbytes / (t_match * 1e-3) / 1e9, 2)})
-        ix.destroy()
+    t_clear = statistics.median(_event_times(torch, lambda: ix.clear(), 5, 2))
+    t_fill = statistics.median(_event_times(torch, refill, 5, 2)) - t_clear
+    d_ml = torch.empty(R * P, dtype=torch.uint32, device="cuda")
+    d_al = torch.empty(R, dtype=torch.uint32, device="cuda")
+    d_ids = torch.empty(int(bo[-1]), dtype=torch.uint32, device="cuda")
+    d_bp = torch.empty(R, dtype=torch.int32, device="cuda")
+    d_bs = torch.empty(R, dtype=torch.int64, device="cuda")
+    d_load = dev(w.pod_load)
+    t_hash = statistics.median(_event_times(
+        torch, lambda: aibx.hash_blocks(d_tok, d_toff, d_bo, B, 0, d_h), 10, 3))
+    t_match = statistics.median(_event_times(
+        torch, lambda: ix.match_prefix(d_h, d_bo, d_ml, d_al, d_ids), 10, 3))
+    t_score = statistics.median(_event_times(
+        torch, lambda: aibx.route_score(d_ml, d_bo, P, d_load, w.ready_mask, None, d_bp, d_bs,
+                                        None), 10, 3))
+    d_dn = torch.empty(R, dtype=torch.uint32, device="cuda")
+    d_sd = torch.empty(R, dtype=torch.uint64, device="cuda")
+    t_head = statistics.median(_event_times(
+        torch, lambda: aibx.route_head(ix, d_tok, d_toff, d_bo, B, 0, d_load, w.ready_mask, None,
+                                       d_h, d_ml, d_al, d_ids, d_bp, d_bs, d_dn, d_sd), 10, 3))
+    t_tail = statistics.median(_event_times(
+        torch, lambda: aibx.hash_blocks_resume(d_tok, d_toff, d_bo, B, d_dn, d_sd, d_h), 10, 3))
+    hashed_by_head = int(d_dn.cpu().numpy().astype(np.int64).sum())
+    al = d_al.cpu().numpy().astype(np.int64)
+    n_r = np.diff(bo)
+    lookups = int(np.minimum(al + 1, n_r).sum())
+    nbytes = lookups * 40 + int((4 * P + 4) * R + 4 * al.sum())
+    out = {"config": s.name, "R": R, "blocks": int(bo[-1]), "necessary_lookups": lookups,
+           "index_entries": int(d_keys.numel()),
+           "insert_us": round(t_fill * 1e3, 1),
+           "insert_Mkeys_per_s": round(d_keys.numel() / (t_fill * 1e-3) / 1e6, 1),
+           "hash_us": round(t_hash * 1e3, 1), "match_us": round(t_match * 1e3, 1),
+           "score_us": round(t_score * 1e3, 1),
+           "route_head_us": round(t_head * 1e3, 1), "hash_tail_us": round(t_tail * 1e3, 1),
+           "blocks_hashed_by_head": hashed_by_head,
+           "hash_tokens_per_s": round(len(w.tokens) / (t_hash * 1e-3), 0),
+           "hash_ns_per_block_longest_chain": round(t_hash * 1e6 / int(n_r.max()), 1),
+           "match_requests_per_s": round(R / (t_match * 1e-3), 0),
+           "match_algorithmic_GBps": round(nbytes / (t_match * 1e-3) / 1e9, 2)}
+    ix.destroy()
+    return out
+
+
+def case_match_cfg(args):
+    """The routing calls alone on the cfg2, routing-heavy (cfg3) and long-context (cfg5) batches."""
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import workloads as W
+
+    res = [routing_batch_times(mk) for mk in (W.cfg2_routing, W.cfg3_routing, W.cfg5_routing)]
     print(json.dumps({"case": "match_cfg", "results": res, "status": aibx.status_fetch()}))
 
 

@@ -361,12 +361,14 @@ __global__ void match_prefix_kernel(IndexView ix, const uint64_t* __restrict__ h
       const unsigned int phi = __shfl_up_sync(0xffffffffu, (unsigned int)(pref >> 32), 1);
       const uint64_t before = lane == 0 ? (all & ~gone) : ((uint64_t)plo | ((uint64_t)phi << 32));
       uint64_t drops = before & ~pref & all;
-      if (drops) {
-        while (drops) {
-          const int p = __ffsll((long long)drops) - 1;
-          drops &= drops - 1;
-          atomicMin(&sh.first_miss[p], i);
-        }
+      // At the chunk's first block with no entry at all every pod still there drops out at
+      // once: those are not recorded one by one (up to 64 atomics in one lane) - the result is
+      // taken as min(first_miss, first_none) at the end instead.
+      if (none && lane == __ffs(none) - 1) drops = 0;
+      while (drops) {
+        const int p = __ffsll((long long)drops) - 1;
+        drops &= drops - 1;
+        atomicMin(&sh.first_miss[p], i);
       }
     }
   }
@@ -375,12 +377,12 @@ __global__ void match_prefix_kernel(IndexView ix, const uint64_t* __restrict__ h
   if (active) {
     const unsigned int a = sh.first_none;
     for (int p = tid_in_group; p < P; p += group_threads)
-      match_len[(int64_t)r * P + p] = sh.first_miss[p];
+      match_len[(int64_t)r * P + p] = min(sh.first_miss[p], a);
     if (any_len && tid_in_group == 0) any_len[r] = a;
     if (best_pod && warp_in_group == 0) {
       // fused scoring: the request's match lengths are still in shared memory
-      const long long h0 = lane < P ? (long long)sh.first_miss[lane] : 0;
-      const long long h1 = lane + 32 < P ? (long long)sh.first_miss[lane + 32] : 0;
+      const long long h0 = lane < P ? (long long)min(sh.first_miss[lane], a) : 0;
+      const long long h1 = lane + 32 < P ? (long long)min(sh.first_miss[lane + 32], a) : 0;
       const long long l0 = lane < P ? (long long)sp.pod_load[lane] : 0;
       const long long l1 = lane + 32 < P ? (long long)sp.pod_load[lane + 32] : 0;
       long long top;

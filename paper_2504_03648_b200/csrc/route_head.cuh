@@ -249,6 +249,9 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
     const uint64_t prev = shfl_up64(pref, 1);
     const uint64_t before = lane == 0 ? alive : prev;
     uint64_t drops = valid ? (before & ~pref) : 0ULL;  // each pod drops once, at one lane
+    // the pods still there at the first total miss all end at any_len: written at the end, in
+    // parallel, not one by one by this lane
+    if ((unsigned int)lane == f) drops = 0;
     while (drops) {
       const int q = __ffsll((long long)drops) - 1;
       drops &= drops - 1;
@@ -257,6 +260,7 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
     if (valid && block_ids) block_ids[out0 + pos + lane] = (unsigned int)lane < f ? id : AIBX_NO_BLOCK;
     if (f < 32u) {
       ended = true;                                    // any_len = pos + f
+      alive = shfl64(0xffffffffu, before, (int)f);     // the pods that held every block before it
       pos += f;
     } else {
       alive = shfl64(0xffffffffu, pref, (int)m - 1);
@@ -267,9 +271,11 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
 
   // ---- the request's results
   __syncwarp();
-  if (!ended && !timed_out) {                          // every block had a live entry
-    if (lane < P && ((alive >> lane) & 1ULL)) sh.match_len[qi][lane] = n_r;
-    if (lane + 32 < P && ((alive >> (lane + 32)) & 1ULL)) sh.match_len[qi][lane + 32] = n_r;
+  if (!timed_out) {
+    // pods that never dropped out: the whole request, or everything up to the first total miss
+    const unsigned int full = ended ? pos : n_r;
+    if (lane < P && ((alive >> lane) & 1ULL)) sh.match_len[qi][lane] = full;
+    if (lane + 32 < P && ((alive >> (lane + 32)) & 1ULL)) sh.match_len[qi][lane + 32] = full;
   }
   __syncwarp();
   const long long h0 = lane < P ? (long long)sh.match_len[qi][lane] : 0;
