@@ -211,8 +211,8 @@ int32_t aibx_route_batch(const aibx_index_t* index, const int32_t* d_tokens,
  *   required) or both NULL.  Block sizes other than 8, 16, 32, 64 tokens are hashed in full by
  *   the first call (d_hashed[r] = n_r).
  * Worth it when the cached prefix is a small part of a request (a shared prompt in front of a
- * long unique tail); a batch whose requests are cached almost to the end gains nothing, and the
- * hashing inside this call is somewhat slower per block than aibx_hash_blocks.
+ * long unique tail); a batch whose requests are cached almost to the end gains nothing (the
+ * hashing inside this call is a little slower per block than aibx_hash_blocks).
  */
 int32_t aibx_route_head(const aibx_index_t* index, const int32_t* d_tokens,
                         const int64_t* d_tok_off, const int64_t* d_blk_off, int32_t R,
