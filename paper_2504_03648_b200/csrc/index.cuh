@@ -94,65 +94,89 @@ __device__ __forceinline__ bool probe_ro(const IndexView& ix, uint64_t key, uint
   return false;
 }
 
+// Keys of kWalk consecutive slots of a probe run, requested together (they usually share one
+// 128-byte line): a walk advances kWalk slots per memory round trip.  Volatile: other threads
+// may be claiming slots meanwhile.
+constexpr int kWalk = 2;
+__device__ __forceinline__ void load_keys(const IndexView& ix, unsigned long long s,
+                                           unsigned long long (&k)[kWalk]) {
+#pragma unroll
+  for (int j = 0; j < kWalk; ++j)
+    k[j] = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[(s + j) & ix.cap_mask].key);
+}
+
 // Probe while other threads may be claiming slots: returns the slot index or ~0.
 __device__ __forceinline__ unsigned long long find_slot_rw(const IndexView& ix, uint64_t key) {
   unsigned long long s = home_slot(ix, key);
-  for (unsigned long long n = 0; n <= ix.cap_mask; ++n) {
-    const unsigned long long k = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].key);
-    if (k == key) return s;
-    if (k == kKeyEmpty) return ~0ULL;
-    s = (s + 1) & ix.cap_mask;
+  for (unsigned long long n = 0; n <= ix.cap_mask; n += kWalk) {
+    unsigned long long k[kWalk];
+    load_keys(ix, s, k);
+#pragma unroll
+    for (int j = 0; j < kWalk; ++j) {
+      if (k[j] == key) return (s + j) & ix.cap_mask;
+      if (k[j] == kKeyEmpty) return ~0ULL;
+    }
+    s = (s + kWalk) & ix.cap_mask;
   }
   return ~0ULL;
 }
 
 // Insert or update one entry (mask already restricted to the table's pods, key not reserved).
 // Returns the slot, or ~0 when the table is full.
+//
+// One walk from the home slot to the first never-used slot: an existing entry anywhere on the
+// way wins; otherwise the first never-used or removed slot seen on the way is claimed.  An entry
+// may lie BEHIND a removed slot (it was placed when that slot was taken), hence the walk to the
+// end before claiming.  Every thread inserting this key walks the same path and tries the same
+// slots in the same order, and no slot turns reusable while inserts run, so the loser of a race
+// for a slot either finds the key there (another thread of the same key won) or starts over
+// and finds the key, or the next free slot, further on.
 __device__ __forceinline__ unsigned long long insert_entry(const IndexView& ix, uint64_t key,
                                                            uint64_t m, uint32_t id) {
-  // pass 1: an existing entry anywhere on the probe path wins (stop at a never-used slot)
-  unsigned long long s = home_slot(ix, key);
-  bool placed = false;
-  for (unsigned long long probes = 0; probes <= ix.cap_mask; ++probes) {
-    const unsigned long long k = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].key);
-    if (k == key) {
-      placed = true;
-      break;
-    }
-    if (k == kKeyEmpty) break;
-    s = (s + 1) & ix.cap_mask;
-  }
-  // pass 2: claim the first never-used or removed slot on the path.  Every thread inserting
-  // this key walks the same path and tries the same slots in the same order, so the losers
-  // of a race find the winner's slot; no slot turns reusable while inserts run.
-  if (!placed) {
-    s = home_slot(ix, key);
-    for (unsigned long long probes = 0; probes <= ix.cap_mask; ++probes) {
-      unsigned long long k = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].key);
-      if (k == kKeyEmpty || k == kKeyTomb) {
-        const unsigned long long seen = atomicCAS(&ix.slots[s].key, k, (unsigned long long)key);
-        if (seen == k) {
-          atomicAdd(&ix.counters[0], 1ULL);
-          if (k == kKeyTomb) atomicAdd(&ix.counters[1], ~0ULL);
-          placed = true;
-          break;
+  unsigned long long slot = ~0ULL;
+  // a lost race costs one more walk; each one means some slot was taken, so the table bounds them
+  for (unsigned long long attempts = 0; attempts <= ix.cap_mask && slot == ~0ULL; ++attempts) {
+    unsigned long long s = home_slot(ix, key);
+    unsigned long long free_slot = ~0ULL, free_was = kKeyEmpty;
+    bool at_end = false;
+    for (unsigned long long n = 0; n <= ix.cap_mask && slot == ~0ULL && !at_end; n += kWalk) {
+      unsigned long long k[kWalk];
+      load_keys(ix, s, k);
+#pragma unroll
+      for (int j = 0; j < kWalk; ++j) {
+        if (slot != ~0ULL || at_end) continue;
+        const unsigned long long here = (s + j) & ix.cap_mask;
+        if (k[j] == key) {
+          slot = here;
+        } else if (k[j] == kKeyEmpty || k[j] == kKeyTomb) {
+          if (free_slot == ~0ULL) {
+            free_slot = here;
+            free_was = k[j];
+          }
+          at_end = k[j] == kKeyEmpty;
         }
-        k = seen;
       }
-      if (k == key) {
-        placed = true;
-        break;
-      }
-      s = (s + 1) & ix.cap_mask;
+      s = (s + kWalk) & ix.cap_mask;
+    }
+    if (slot != ~0ULL) break;
+    if (free_slot == ~0ULL) break;                      // no room anywhere on the path
+    const unsigned long long seen =
+        atomicCAS(&ix.slots[free_slot].key, free_was, (unsigned long long)key);
+    if (seen == free_was) {
+      atomicAdd(&ix.counters[0], 1ULL);
+      if (free_was == kKeyTomb) atomicAdd(&ix.counters[1], ~0ULL);
+      slot = free_slot;
+    } else if (seen == key) {
+      slot = free_slot;
     }
   }
-  if (!placed) {
+  if (slot == ~0ULL) {
     raise_status(AIBX_ERR_FULL);
     return ~0ULL;
   }
-  atomicOr(&ix.slots[s].mask, (unsigned long long)m);
-  atomicMin(&ix.slots[s].id, id);
-  return s;
+  atomicOr(&ix.slots[slot].mask, (unsigned long long)m);
+  atomicMin(&ix.slots[slot].id, id);
+  return slot;
 }
 
 __global__ void index_insert_kernel(IndexView ix, const uint64_t* __restrict__ keys,
