@@ -259,6 +259,47 @@ def test_cfg4_full_size_layer_major():
     print("cfg4 pool blocks used:", kv.num_blocks, "(shrunk)" if shrunk else "(full)")
 
 
+def test_list_longer_than_one_launch_covers():
+    """A launch addresses its transfer buffer with 32-bit offsets in 16-byte units, i.e. about
+    64 GiB; a longer list is cut into several launches.  13,500 items of the 5 MiB Llama-3-70B
+    block shape (65.9 GiB of buffer, ids repeating over a 64-block layer-major pool) cross that
+    line after item 13,093: items on both sides of it, and the last one, are checked against the
+    oracle, and so is the counted variant, whose device-side count ends inside the second launch."""
+    free, _ = torch.cuda.mem_get_info()
+    kv = W.scaled(W.cfg4_kv(), num_blocks=64)
+    n = 13500
+    if free < n * kv.block_bytes + kv.pool_bytes + (8 << 30):
+        pytest.skip("needs 75 GiB of free device memory")
+    first_launch = ((1 << 32) - (1 << 22)) // (kv.block_bytes // 16)
+    assert first_launch == 13094 and n > first_launch
+    pool = empty(kv.pool_bytes, torch.uint8)
+    synth.fill_pool(pool, kv)
+    ids = W.Stream(77, 3).randint(0, kv.num_blocks, n).astype(np.uint32)
+    ids[first_launch + 5] = NO_BLOCK                                # a skipped item past the line
+    lay, lay1 = kv_layout_gpu(kv), kv_layout_oracle(kv, layout=0, num_blocks=1)
+    buf = empty(n * kv.block_bytes, torch.uint8)
+    d_ids = dev(ids)
+
+    def check(upto):
+        view = buf.view(n, kv.block_bytes)
+        for i in (0, 1, first_launch - 1, first_launch, first_launch + 1, first_launch + 5,
+                  first_launch + 6, n - 2, n - 1):
+            want = np.full(kv.block_bytes, 0xAB, dtype=np.uint8)
+            if i < upto and ids[i] != NO_BLOCK:
+                oracle.kv_gather(W.logical_blocks(kv, [int(ids[i])]), lay1, np.zeros(1, np.uint32), want)
+            assert np.array_equal(host(view[i]), want), i
+
+    buf.fill_(0xAB)
+    aibx.kv_gather(pool, lay, d_ids, n, buf)
+    assert aibx.status_fetch() == (0, 0)
+    check(n)
+    buf.fill_(0xAB)
+    cnt = first_launch + 3                                          # ends inside the second launch
+    aibx.kv_gather_counted(pool, lay, d_ids, n, dev(np.array([cnt], np.uint32)), buf)
+    assert aibx.status_fetch() == (0, 0)
+    check(cnt)
+
+
 def test_cfg5_full_size_fp8_mixed():
     kv0 = W.cfg5_kv()
     kv, shrunk = _fit_blocks(kv0, 3000 * kv0.block_bytes + 1000 * kv0.block_bytes)
