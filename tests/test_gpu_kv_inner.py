@@ -127,3 +127,47 @@ def test_inner_order_large_launch_bandwidth_shape():
             assert np.array_equal(host(buf.view(n, kv.block_bytes)[i]), want)
         bufs.append(buf)
     assert torch.equal(bufs[0], bufs[1])                   # every byte, engine against engine
+
+
+def test_inner_order_on_the_full_cfg4_pool():
+    """The 97.7 GiB layer-major pool of the Llama-3-70B configuration: the tensor map of a
+    scatter spans all 3.2 million planes of the pool, and the blocks picked include the last
+    ones, so the largest plane coordinates are exercised.  Gathered items and scattered blocks
+    are checked against the oracle."""
+    import gc
+
+    gc.collect()
+    torch.cuda.empty_cache()
+    kv = W.cfg4_kv()
+    n = 48
+    free, _ = torch.cuda.mem_get_info()
+    if free < kv.pool_bytes + n * kv.block_bytes + (6 << 30):
+        kv = W.scaled(kv, num_blocks=int((free - n * kv.block_bytes - (6 << 30)) // kv.block_bytes))
+    nb = kv.num_blocks
+    pool = empty(kv.pool_bytes, torch.uint8)
+    synth.fill_pool(pool, kv)
+    middle = W.distinct_ids(5, nb - 3, n - 3) + 1             # distinct ids in [1, nb - 3]
+    ids = np.concatenate([[nb - 1, nb - 2, 0], middle]).astype(np.uint32)
+    lay = kv_layout_gpu(kv)
+    lay1 = kv_layout_oracle(kv, layout=0, num_blocks=1)
+    for engine in (2, 1):
+        aibx.kv_set_inner_engine(engine)
+        buf = torch.full((n * kv.block_bytes,), 0xCD, dtype=torch.uint8, device="cuda")
+        aibx.kv_gather_inner(pool, lay, 0, 1, dev(ids), n, buf)
+        assert aibx.status_fetch() == (0, 0)
+        for i in (0, 1, 2, n // 2, n - 1):
+            want = np.zeros(kv.block_bytes, dtype=np.uint8)
+            oracle.kv_gather_inner(W.logical_blocks(kv, [int(ids[i])]), lay1, 0, 1,
+                                   np.zeros(1, np.uint32), want)
+            assert np.array_equal(host(buf.view(n, kv.block_bytes)[i]), want), (engine, i)
+        # scatter other content into the same blocks, converting back on the way
+        synth.fill_linear(buf, 900 + engine)
+        aibx.kv_scatter_inner(pool, lay, 0, 1, dev(ids), n, buf)
+        assert aibx.status_fetch() == (0, 0)
+        for i in (0, 1, n - 1):
+            item = W.pool_bytes(900 + engine, i * kv.block_bytes, kv.block_bytes)
+            want = np.zeros(kv.block_bytes, dtype=np.uint8)
+            oracle.kv_scatter_inner(want, lay1, 0, 1, np.zeros(1, np.uint32), item)
+            got = host(pool.view(kv.num_layers, nb, kv.tile_bytes)[:, int(ids[i])].contiguous()).reshape(-1)
+            assert np.array_equal(got, want), (engine, i)
+        synth.fill_pool(pool, kv)                             # generated content again
