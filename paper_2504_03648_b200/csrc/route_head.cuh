@@ -271,6 +271,9 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
       alive = shfl64(0xffffffffu, pref, (int)m - 1);
       pos += m;
     }
+    // Lets the hasher reuse the ring slots just read.  The keys read from them have been used
+    // by now (every lane computed its probe address from its key), so the reads are complete
+    // before this store is issued; a plain store is enough.
     if (lane == 0) *v_consumed = ended ? (pos | kHeadStopBit) : pos;
   }
 
