@@ -138,6 +138,21 @@ int32_t aibx_index_export(const aibx_index_t* index, uint64_t* d_keys, uint64_t*
                           void* stream);
 int32_t aibx_index_rehash(aibx_index_t* index, uint64_t new_capacity);
 
+/* The same move without stopping the readers (Section 3.2.5: metadata is updated beside the
+ * traffic, not in its way).  _begin allocates the new table and enqueues the move on `stream`,
+ * waiting only for that stream (to read the live count), then returns; until _finish the handle
+ * keeps answering from the old table, so aibx_index_lookup / aibx_match_prefix / aibx_route_* /
+ * aibx_index_export / aibx_index_stats calls on any stream run beside the move and see the
+ * content as it was.  Calls that would change the index (insert, evict, clear, touch, rehash)
+ * return INVALID between _begin and _finish: nothing is lost, the caller holds them back.
+ * _finish waits for the move, switches the handle to the new table and frees the old one (which
+ * waits for readers still using it).  Updates enqueued before _begin must be ordered before
+ * `stream` by the caller.  Codes of _begin as aibx_index_rehash; INVALID if a move is already
+ * under way, for _finish if none is.
+ */
+int32_t aibx_index_rehash_begin(aibx_index_t* index, uint64_t new_capacity, void* stream);
+int32_t aibx_index_rehash_finish(aibx_index_t* index);
+
 /* ---------------------------------------------------------------------------------------
  * Longest cached prefix (Section 3.2.2, policy prefix-cache-aware: how much of a request's
  * prefix each instance can reuse).  For request r and pod p:

@@ -87,6 +87,8 @@ def lib():
             "aibx_index_pick_victims": [vp, u64, vp, vp, vp, vp],
             "aibx_index_export": [vp, vp, vp, vp, u64, vp, vp],
             "aibx_index_rehash": [vp, u64],
+            "aibx_index_rehash_begin": [vp, u64, vp],
+            "aibx_index_rehash_finish": [vp],
             "aibx_match_prefix": [vp, vp, vp, i32, vp, vp, vp, vp],
             "aibx_route_score": [vp, vp, i32, i32, vp, u64, C.POINTER(RouteParams), vp, vp, vp, vp],
             "aibx_route_batch": [vp, vp, vp, vp, i32, i32, u64, vp, u64, C.POINTER(RouteParams),
@@ -223,6 +225,17 @@ class Index:
     def rehash(self, new_capacity: int) -> None:
         _check("aibx_index_rehash", lib().aibx_index_rehash(self._h, new_capacity))
         self.capacity = new_capacity
+
+    def rehash_begin(self, new_capacity: int) -> None:
+        """Start moving the index into a table of another size on the current stream; readers
+        keep working on the old table until rehash_finish()."""
+        _check("aibx_index_rehash_begin",
+               lib().aibx_index_rehash_begin(self._h, new_capacity, _stream()))
+        self._pending_capacity = new_capacity
+
+    def rehash_finish(self) -> None:
+        _check("aibx_index_rehash_finish", lib().aibx_index_rehash_finish(self._h))
+        self.capacity = self._pending_capacity
 
     def match_prefix(self, hashes, blk_off, match_len, any_len=None, block_ids=None) -> None:
         R = blk_off.numel() - 1

@@ -23,6 +23,12 @@ struct aibx_index {
   uint64_t capacity;
   int device;
   VictimScratch* victim_scratch;   // allocated on first use of aibx_index_pick_victims
+  // a rehash in progress (aibx_index_rehash_begin .. _finish): the table being filled, and the
+  // event that says the move has finished.  Readers keep using `view` meanwhile.
+  bool migrating;
+  IndexView pending;
+  uint64_t pending_capacity;
+  cudaEvent_t moved;
 };
 
 namespace {
@@ -133,6 +139,8 @@ int32_t aibx_index_create(aibx_index_t** out, uint64_t capacity_slots, int32_t n
     return AIBX_ERR_NOMEM;
   }
   ix->capacity = capacity_slots;
+  ix->migrating = false;
+  ix->moved = nullptr;
   ix->view.slots = static_cast<Slot*>(slots);
   ix->view.cap_mask = capacity_slots - 1;
   ix->view.shift = 64 - log2cap;
@@ -152,6 +160,11 @@ int32_t aibx_index_create(aibx_index_t** out, uint64_t capacity_slots, int32_t n
 int32_t aibx_index_destroy(aibx_index_t* ix) {
   if (!ix) return AIBX_ERR_INVALID;
   cudaDeviceSynchronize();
+  if (ix->migrating) {
+    cudaFree(ix->pending.slots);
+    cudaFree(ix->pending.counters);
+  }
+  if (ix->moved) cudaEventDestroy(ix->moved);
   cudaFree(ix->view.slots);
   cudaFree(ix->view.counters);
   if (ix->victim_scratch) cudaFree(ix->victim_scratch);
@@ -160,14 +173,14 @@ int32_t aibx_index_destroy(aibx_index_t* ix) {
 }
 
 int32_t aibx_index_clear(aibx_index_t* ix, void* stream) {
-  if (!ix) return AIBX_ERR_INVALID;
+  if (!ix || ix->migrating) return AIBX_ERR_INVALID;
   index_clear_kernel<<<sm_count() * 8, 256, 0, as_stream(stream)>>>(ix->view);
   return launch_status();
 }
 
 int32_t aibx_index_insert(aibx_index_t* ix, const uint64_t* d_keys, const uint64_t* d_pod_masks,
                           const uint32_t* d_block_ids, int64_t n, void* stream) {
-  if (!ix || n < 0) return AIBX_ERR_INVALID;
+  if (!ix || n < 0 || ix->migrating) return AIBX_ERR_INVALID;
   if (n == 0) return AIBX_OK;
   if (!d_keys || !d_pod_masks || !d_block_ids) return AIBX_ERR_INVALID;
   prefer_copy_carveout();
@@ -178,7 +191,7 @@ int32_t aibx_index_insert(aibx_index_t* ix, const uint64_t* d_keys, const uint64
 
 int32_t aibx_index_evict(aibx_index_t* ix, const uint64_t* d_keys, const uint64_t* d_pod_masks,
                          uint32_t* d_freed_block_ids, int64_t n, void* stream) {
-  if (!ix || n < 0) return AIBX_ERR_INVALID;
+  if (!ix || n < 0 || ix->migrating) return AIBX_ERR_INVALID;
   if (n == 0) return AIBX_OK;
   if (!d_keys || !d_pod_masks) return AIBX_ERR_INVALID;
   prefer_copy_carveout();
@@ -216,7 +229,7 @@ int32_t aibx_index_stats(const aibx_index_t* ix, uint64_t* live, uint64_t* capac
 
 int32_t aibx_index_touch(aibx_index_t* ix, const uint64_t* d_keys, int64_t n, uint32_t epoch,
                          void* stream) {
-  if (!ix || n < 0 || epoch == 0 || epoch >= (1u << 30)) return AIBX_ERR_INVALID;
+  if (!ix || n < 0 || epoch == 0 || epoch >= (1u << 30) || ix->migrating) return AIBX_ERR_INVALID;
   if (n == 0) return AIBX_OK;
   if (!d_keys) return AIBX_ERR_INVALID;
   index_touch_kernel<<<blocks_for(n, 256), 256, 0, as_stream(stream)>>>(ix->view, d_keys, n, epoch);
@@ -265,7 +278,7 @@ int32_t aibx_index_export(const aibx_index_t* ix, uint64_t* d_keys, uint64_t* d_
 }
 
 int32_t aibx_index_rehash(aibx_index_t* ix, uint64_t new_capacity) {
-  if (!ix) return AIBX_ERR_INVALID;
+  if (!ix || ix->migrating) return AIBX_ERR_INVALID;
   if (new_capacity < 8 || (new_capacity & (new_capacity - 1)) != 0 || new_capacity > (1ULL << 40))
     return AIBX_ERR_INVALID;
   if (cudaDeviceSynchronize() != cudaSuccess) return AIBX_ERR_CUDA;
@@ -294,6 +307,64 @@ int32_t aibx_index_rehash(aibx_index_t* ix, uint64_t new_capacity) {
   cudaFree(old.slots);
   ix->view = fresh;
   ix->capacity = new_capacity;
+  return AIBX_OK;
+}
+
+int32_t aibx_index_rehash_begin(aibx_index_t* ix, uint64_t new_capacity, void* stream) {
+  if (!ix || ix->migrating) return AIBX_ERR_INVALID;
+  if (new_capacity < 8 || (new_capacity & (new_capacity - 1)) != 0 || new_capacity > (1ULL << 40))
+    return AIBX_ERR_INVALID;
+  cudaStream_t st = as_stream(stream);
+  // the live count as of `stream` (only this stream is waited for, not the device)
+  unsigned long long c[2] = {0, 0};
+  if (cudaMemcpyAsync(c, ix->view.counters, sizeof(c), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return AIBX_ERR_CUDA;
+  if (c[0] > new_capacity) return AIBX_ERR_FULL;
+  if (!ix->moved &&
+      cudaEventCreateWithFlags(&ix->moved, cudaEventDisableTiming) != cudaSuccess) {
+    ix->moved = nullptr;
+    return AIBX_ERR_CUDA;
+  }
+  void* slots = nullptr;
+  void* counters = nullptr;
+  if (cudaMalloc(&slots, new_capacity * sizeof(Slot)) != cudaSuccess ||
+      cudaMalloc(&counters, 2 * sizeof(unsigned long long)) != cudaSuccess) {
+    cudaGetLastError();
+    if (slots) cudaFree(slots);
+    return AIBX_ERR_NOMEM;
+  }
+  int log2cap = 0;
+  while ((1ULL << log2cap) < new_capacity) ++log2cap;
+  IndexView fresh = ix->view;
+  fresh.slots = static_cast<Slot*>(slots);
+  fresh.counters = static_cast<unsigned long long*>(counters);   // its own: `view` stays intact
+  fresh.cap_mask = new_capacity - 1;
+  fresh.shift = 64 - log2cap;
+  index_clear_kernel<<<sm_count() * 8, 256, 0, st>>>(fresh);
+  index_move_kernel<<<sm_count() * 8, 256, 0, st>>>(ix->view, fresh);
+  if (cudaEventRecord(ix->moved, st) != cudaSuccess || launch_status() != AIBX_OK) {
+    cudaStreamSynchronize(st);
+    cudaFree(slots);
+    cudaFree(counters);
+    return AIBX_ERR_CUDA;
+  }
+  ix->pending = fresh;
+  ix->pending_capacity = new_capacity;
+  ix->migrating = true;
+  return AIBX_OK;
+}
+
+int32_t aibx_index_rehash_finish(aibx_index_t* ix) {
+  if (!ix || !ix->migrating) return AIBX_ERR_INVALID;
+  if (cudaEventSynchronize(ix->moved) != cudaSuccess) return AIBX_ERR_CUDA;
+  const IndexView old = ix->view;
+  ix->view = ix->pending;
+  ix->capacity = ix->pending_capacity;
+  ix->migrating = false;
+  // cudaFree waits for the work still using the old table (readers launched before the switch)
+  cudaFree(old.slots);
+  cudaFree(old.counters);
   return AIBX_OK;
 }
 

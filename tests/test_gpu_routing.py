@@ -494,3 +494,72 @@ def test_index_export_and_rehash():
     extra = np.arange(100, 110, dtype=np.uint64)
     small_g.insert(dev(extra), dev(np.ones(10, np.uint64)), dev(np.zeros(10, np.uint32)))
     assert aibx.status_fetch() == (0, 0) and small_g.stats() == (18, 32)
+
+
+def test_rehash_beside_the_readers():
+    """rehash_begin .. rehash_finish: lookups and matches issued on another stream while the move
+    runs answer from the old table (same results as before and after), calls that would change
+    the index are refused meanwhile, and afterwards the larger table holds the same content."""
+    rng = np.random.default_rng(99)
+    P, n = 20, 300000
+    keys = np.unique(rng.integers(1, 1 << 62, n).astype(np.uint64))
+    n = len(keys)
+    masks = (rng.integers(0, 1 << P, n) | 1).astype(np.uint64)
+    ids = rng.integers(0, 1 << 20, n).astype(np.uint32)
+    g, o = aibx.Index(1 << 19, P), oracle.Index(1 << 19, P)
+    g.insert(dev(keys), dev(masks), dev(ids)); assert o.insert(keys, masks, ids) == oracle.OK
+    gone = keys[::7]
+    g.evict(dev(gone), dev(np.full(len(gone), ALL, np.uint64))); o.evict(gone, np.full(len(gone), ALL, np.uint64))
+    live = o.stats()[0]
+    probe = np.concatenate([keys[:50000], rng.integers(1, 1 << 62, 5000).astype(np.uint64)])
+    want_m, want_i = o.lookup(probe)
+    # requests made of resident keys, with holes where keys were evicted
+    bo = np.arange(0, 50001, 50, dtype=np.int64)
+    wml, wal, wids = o.match_prefix(keys[:50000], bo)
+    d_probe, d_req, d_bo = dev(probe), dev(keys[:50000]), dev(bo)
+    R = len(bo) - 1
+
+    def read_all():
+        d_m, d_i = empty(len(probe), torch.uint64), empty(len(probe), torch.uint32)
+        g.lookup(d_probe, d_m, d_i)
+        d_ml, d_al, d_ids = empty(R * P, torch.uint32), empty(R, torch.uint32), empty(50000, torch.uint32)
+        g.match_prefix(d_req, d_bo, d_ml, d_al, d_ids)
+        return d_m, d_i, d_ml, d_al, d_ids
+
+    def check(res):
+        d_m, d_i, d_ml, d_al, d_ids = res
+        assert np.array_equal(host(d_m), want_m) and np.array_equal(host(d_i), want_i)
+        assert np.array_equal(host(d_ml).reshape(R, P), wml) and np.array_equal(host(d_al), wal)
+        assert np.array_equal(host(d_ids), wids)
+
+    check(read_all())
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        g.rehash_begin(1 << 21)                          # the move runs on the side stream
+    during = [read_all() for _ in range(4)]              # readers on the main stream, beside it
+    for call in (lambda: g.insert(dev(keys[:4]), dev(masks[:4]), dev(ids[:4])),
+                 lambda: g.evict(dev(keys[:4]), dev(masks[:4])),
+                 lambda: g.clear(), lambda: g.rehash(1 << 20),
+                 lambda: g.rehash_begin(1 << 20)):
+        with pytest.raises(aibx.AibxError) as e:
+            call()
+        assert e.value.code == aibx.ERR_INVALID
+    assert g.stats() == (live, 1 << 19)                  # still the old table
+    g.rehash_finish()
+    for res in during:
+        check(res)
+    check(read_all())
+    assert g.stats() == (live, 1 << 21)
+    with pytest.raises(aibx.AibxError) as e:
+        g.rehash_finish()                                # nothing under way
+    assert e.value.code == aibx.ERR_INVALID
+    # the index takes updates again, in step with the oracle
+    more = rng.integers(1, 1 << 62, 1000).astype(np.uint64)
+    g.insert(dev(more), dev(np.ones(1000, np.uint64)), dev(np.zeros(1000, np.uint32)))
+    o.rehash(1 << 21); o.insert(more, np.ones(1000, np.uint64), np.zeros(1000, np.uint32))
+    assert g.stats() == (o.stats()[0], 1 << 21)
+    with pytest.raises(aibx.AibxError) as e:
+        g.rehash_begin(1 << 17)                          # the live entries do not fit
+    assert e.value.code == aibx.ERR_FULL
+    assert aibx.status_fetch() == (0, 0)
