@@ -575,6 +575,12 @@ int32_t aibx_collect_blocks(const uint32_t* d_block_ids, int64_t n, uint32_t num
   if (num_blocks > 0 && !d_scratch) return AIBX_ERR_INVALID;
   if (reinterpret_cast<uintptr_t>(d_scratch) & 3) return AIBX_ERR_INVALID;
   cudaStream_t st = as_stream(stream);
+  if (n <= kCollectSmallIds && (num_blocks + 31u) / 32u <= kCollectSmallWords) {
+    // a list one CTA gets through in a few microseconds: one launch, bitmap in shared memory
+    collect_small_kernel<<<1, kCollectThreads, 0, st>>>(d_block_ids, n, num_blocks, d_unique_ids,
+                                                        d_count);
+    return launch_status();
+  }
   unsigned int* bitmap = static_cast<unsigned int*>(d_scratch);
   if (num_blocks > 0 &&
       cudaMemsetAsync(bitmap, 0, aibx_collect_scratch_bytes(num_blocks), st) != cudaSuccess)

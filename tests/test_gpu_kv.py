@@ -265,6 +265,10 @@ def test_list_longer_than_one_launch_covers():
     block shape (65.9 GiB of buffer, ids repeating over a 64-block layer-major pool) cross that
     line after item 13,093: items on both sides of it, and the last one, are checked against the
     oracle, and so is the counted variant, whose device-side count ends inside the second launch."""
+    import gc
+
+    gc.collect()
+    torch.cuda.empty_cache()                       # earlier tests' pools go back to the driver
     free, _ = torch.cuda.mem_get_info()
     kv = W.scaled(W.cfg4_kv(), num_blocks=64)
     n = 13500
