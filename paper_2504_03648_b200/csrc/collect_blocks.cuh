@@ -91,12 +91,21 @@ collect_small_kernel(const uint32_t* __restrict__ ids, int64_t n, uint32_t num_b
   for (uint32_t w = tid; w < n_words; w += kCollectThreads) s_bits[w] = 0u;
   if (tid == 0) s_base = 0;
   __syncthreads();
-  for (int64_t i = tid; i < n; i += kCollectThreads) {
-    const uint32_t id = ids[i];
-    if (id < num_blocks) {
-      atomicOr(&s_bits[id >> 5], 1u << (id & 31u));
-    } else if (id != AIBX_NO_BLOCK) {
-      raise_status(AIBX_ERR_RANGE);
+  // eight ids per thread in flight: the list is read in a couple of memory round trips
+  for (int64_t i0 = tid; i0 < n; i0 += 8 * kCollectThreads) {
+    uint32_t id[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int64_t i = i0 + (int64_t)u * kCollectThreads;
+      id[u] = i < n ? __ldg(ids + i) : AIBX_NO_BLOCK;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      if (id[u] < num_blocks) {
+        atomicOr(&s_bits[id[u] >> 5], 1u << (id[u] & 31u));
+      } else if (id[u] != AIBX_NO_BLOCK) {
+        raise_status(AIBX_ERR_RANGE);
+      }
     }
   }
   __syncthreads();
