@@ -34,6 +34,25 @@ __host__ __device__ __forceinline__ uint64_t pod_all(int P) {
   return P >= 64 ? ~0ULL : ((1ULL << P) - 1ULL);
 }
 
+// 64-bit warp shuffles (two 32-bit shuffles each).
+__device__ __forceinline__ uint64_t shfl64(unsigned int mask, uint64_t v, int src_lane) {
+  const unsigned int lo = __shfl_sync(mask, (unsigned int)v, src_lane);
+  const unsigned int hi = __shfl_sync(mask, (unsigned int)(v >> 32), src_lane);
+  return (uint64_t)lo | ((uint64_t)hi << 32);
+}
+
+__device__ __forceinline__ uint64_t shfl_xor64(unsigned int mask, uint64_t v, int lane_mask) {
+  const unsigned int lo = __shfl_xor_sync(mask, (unsigned int)v, lane_mask);
+  const unsigned int hi = __shfl_xor_sync(mask, (unsigned int)(v >> 32), lane_mask);
+  return (uint64_t)lo | ((uint64_t)hi << 32);
+}
+
+__device__ __forceinline__ uint64_t shfl_up64(uint64_t v, int d) {
+  const unsigned int lo = __shfl_up_sync(0xffffffffu, (unsigned int)v, d);
+  const unsigned int hi = __shfl_up_sync(0xffffffffu, (unsigned int)(v >> 32), d);
+  return (uint64_t)lo | ((uint64_t)hi << 32);
+}
+
 inline int32_t launch_status() {
   return cudaPeekAtLastError() == cudaSuccess ? AIBX_OK : AIBX_ERR_CUDA;
 }

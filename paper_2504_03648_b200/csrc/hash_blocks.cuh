@@ -30,18 +30,6 @@ __device__ __forceinline__ uint64_t rotl64(uint64_t x, int r) {
   return (x << r) | (x >> (64 - r));
 }
 
-__device__ __forceinline__ uint64_t shfl64(unsigned int mask, uint64_t v, int src_lane) {
-  const unsigned int lo = __shfl_sync(mask, (unsigned int)v, src_lane);
-  const unsigned int hi = __shfl_sync(mask, (unsigned int)(v >> 32), src_lane);
-  return (uint64_t)lo | ((uint64_t)hi << 32);
-}
-
-__device__ __forceinline__ uint64_t shfl_xor64(unsigned int mask, uint64_t v, int lane_mask) {
-  const unsigned int lo = __shfl_xor_sync(mask, (unsigned int)v, lane_mask);
-  const unsigned int hi = __shfl_xor_sync(mask, (unsigned int)(v >> 32), lane_mask);
-  return (uint64_t)lo | ((uint64_t)hi << 32);
-}
-
 // End of a block: `v` is this lane's accumulator.  Returns the block's key in all four lanes.
 __device__ __forceinline__ uint64_t finish_block_quad(unsigned int qmask, int quad_base, uint64_t v,
                                                       int rot, uint64_t len_bytes) {

@@ -306,6 +306,126 @@ __global__ void index_lookup_kernel(IndexView ix, const uint64_t* __restrict__ k
 }
 
 // ------------------------------------------------------------------------------------------
+// Longest cached prefix, folded chunk by chunk by ONE warp that walks a request in order.
+// State between chunks: the pods that hold every block so far, how many blocks are folded, and
+// whether a block without any live entry has ended the request.
+
+struct PrefixFold {
+  uint64_t alive;
+  unsigned int pos;
+  bool ended;
+};
+
+// One chunk: lane t holds the probe result (mask, id) of block pos + t, valid for t < m.  A
+// ballot finds the first block with no live entry; a prefix-AND over the lanes, seeded with
+// `alive`, makes pod bits monotone, so each lane sees exactly the pods that drop out at its
+// block and records them in ml[pod] (each pod at most once over the whole request).  The pods
+// still there at the first total miss, or at the end of the request, are NOT recorded here:
+// they all get the same value (any_len, or the request's length) from fold_finish, in parallel.
+__device__ __forceinline__ void fold_chunk(PrefixFold& st, int lane, unsigned int m, uint64_t mask,
+                                           uint32_t id, uint64_t all, unsigned int* ml,
+                                           uint32_t* block_ids_at) {
+  const bool valid = (unsigned int)lane < m;
+  const unsigned int none = __ballot_sync(0xffffffffu, valid && mask == 0);
+  const unsigned int f = none ? (unsigned int)__ffs(none) - 1u : 32u;   // first total miss
+  uint64_t pref = valid ? mask : all;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint64_t o = shfl_up64(pref, d);
+    if (lane >= d) pref &= o;
+  }
+  pref &= st.alive;
+  const uint64_t prev = shfl_up64(pref, 1);
+  const uint64_t before = lane == 0 ? st.alive : prev;
+  uint64_t drops = valid ? (before & ~pref) : 0ULL;
+  if ((unsigned int)lane == f) drops = 0;
+  while (drops) {
+    const int q = __ffsll((long long)drops) - 1;
+    drops &= drops - 1;
+    ml[q] = st.pos + lane;
+  }
+  if (valid && block_ids_at)
+    block_ids_at[st.pos + lane] = (unsigned int)lane < f ? id : AIBX_NO_BLOCK;
+  if (f < 32u) {
+    st.ended = true;                                   // any_len = pos + f
+    st.alive = shfl64(0xffffffffu, before, (int)f);    // the pods that held every block before it
+    st.pos += f;
+  } else {
+    st.alive = shfl64(0xffffffffu, pref, (int)m - 1);
+    st.pos += m;
+  }
+}
+
+// After the last chunk: the pods that never dropped out, the results, the score.  `ml` is the
+// warp's scratch of AIBX_MAX_PODS words (shared memory); lanes cover pods lane and lane + 32.
+__device__ __forceinline__ void fold_finish(const PrefixFold& st, int lane, int P, int r,
+                                            unsigned int n_r, int64_t off, unsigned int* ml,
+                                            uint32_t* __restrict__ match_len,
+                                            uint32_t* __restrict__ any_len,
+                                            uint32_t* __restrict__ block_ids, const ScoreParams& sp,
+                                            int32_t* __restrict__ best_pod,
+                                            int64_t* __restrict__ best_score) {
+  __syncwarp();
+  const unsigned int full = st.ended ? st.pos : n_r;
+  if (lane < P && ((st.alive >> lane) & 1ULL)) ml[lane] = full;
+  if (lane + 32 < P && ((st.alive >> (lane + 32)) & 1ULL)) ml[lane + 32] = full;
+  __syncwarp();
+  const long long h0 = lane < P ? (long long)ml[lane] : 0;
+  const long long h1 = lane + 32 < P ? (long long)ml[lane + 32] : 0;
+  if (lane < P) match_len[(int64_t)r * P + lane] = (uint32_t)h0;
+  if (lane + 32 < P) match_len[(int64_t)r * P + lane + 32] = (uint32_t)h1;
+  if (lane == 0 && any_len) any_len[r] = st.pos;
+  if (block_ids) {
+    for (unsigned int i = st.pos + lane; i < n_r; i += 32) block_ids[off + i] = AIBX_NO_BLOCK;
+  }
+  if (best_pod) {
+    const long long l0 = lane < P ? (long long)sp.pod_load[lane] : 0;
+    const long long l1 = lane + 32 < P ? (long long)sp.pod_load[lane + 32] : 0;
+    long long top;
+    int arg;
+    lane_candidate(lane, P, sp.ready_mask,
+                   pod_score(h0, (long long)n_r, l0, sp.w_prefix, sp.w_load, sp.thr_pct),
+                   pod_score(h1, (long long)n_r, l1, sp.w_prefix, sp.w_load, sp.thr_pct), top, arg);
+    warp_argmax(top, arg);
+    if (lane == 0) {
+      best_pod[r] = arg;
+      best_score[r] = top;
+    }
+  }
+}
+
+// One warp per request, chunks of 32 blocks in order: the shape for large batches, where there
+// are warps enough without splitting a request.  No barrier, no shared-memory atomics.
+constexpr int kMatchWarpKernelWarps = 4;
+
+__global__ void __launch_bounds__(kMatchWarpKernelWarps * 32)
+match_prefix_warp_kernel(IndexView ix, const uint64_t* __restrict__ hashes,
+                         const int64_t* __restrict__ blk_off, int R,
+                         uint32_t* __restrict__ match_len, uint32_t* __restrict__ any_len,
+                         uint32_t* __restrict__ block_ids, ScoreParams sp,
+                         int32_t* __restrict__ best_pod, int64_t* __restrict__ best_score) {
+  __shared__ unsigned int s_ml[kMatchWarpKernelWarps][AIBX_MAX_PODS];
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int r = blockIdx.x * kMatchWarpKernelWarps + warp;
+  if (r >= R) return;
+  const int P = ix.num_pods;
+  const uint64_t all = pod_all(P);
+  const int64_t off = blk_off[r];
+  const unsigned int n_r = (unsigned int)(blk_off[r + 1] - off);
+  PrefixFold st = {all, 0u, false};
+  while (!st.ended && st.pos < n_r) {
+    const unsigned int m = min(32u, n_r - st.pos);
+    uint64_t mask = 0;
+    uint32_t id = AIBX_NO_BLOCK;
+    if ((unsigned int)lane < m) probe_ro(ix, __ldg(hashes + off + st.pos + lane), mask, id);
+    fold_chunk(st, lane, m, mask, id, all, s_ml[warp], block_ids ? block_ids + off : nullptr);
+  }
+  fold_finish(st, lane, P, r, n_r, off, s_ml[warp], match_len, any_len, block_ids, sp, best_pod,
+              best_score);
+}
+
+// ------------------------------------------------------------------------------------------
 // Longest cached prefix.  A group of `wpr` warps serves one request; a CTA holds kMatchWarps
 // warps, i.e. kMatchWarps / wpr requests.
 

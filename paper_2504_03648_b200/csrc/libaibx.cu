@@ -398,6 +398,13 @@ int32_t launch_match(const aibx_index_t* ix, const uint64_t* d_hashes, const int
   int wpr = 1;
   const long long target = (long long)sm_count() * 32;
   while (wpr < 32 && (long long)R * wpr * 2 <= target) wpr *= 2;
+  if (wpr == 1) {
+    // warps enough with one per request: the shape without barriers and shared-memory atomics
+    match_prefix_warp_kernel<<<blocks_for(R, kMatchWarpKernelWarps), kMatchWarpKernelWarps * 32, 0,
+                               st>>>(ix->view, d_hashes, d_blk_off, R, d_match_len, d_any_len,
+                                     d_block_ids, sp, d_best_pod, d_best_score);
+    return launch_status();
+  }
   const int warps_per_cta = wpr > kMatchWarpsMin ? wpr : kMatchWarpsMin;
   const int groups = warps_per_cta / wpr;
   const unsigned int grid = (unsigned int)((R + groups - 1) / groups);

@@ -47,12 +47,6 @@ struct HeadShared {
   unsigned int match_len[8][AIBX_MAX_PODS];
 };
 
-__device__ __forceinline__ uint64_t shfl_up64(uint64_t v, int d) {
-  const unsigned int lo = __shfl_up_sync(0xffffffffu, (unsigned int)v, d);
-  const unsigned int hi = __shfl_up_sync(0xffffffffu, (unsigned int)(v >> 32), d);
-  return (uint64_t)lo | ((uint64_t)hi << 32);
-}
-
 // Release / acquire on a shared-memory word at CTA scope: the light way to hand data written
 // before the store to whoever reads the word (a full fence would also drain unrelated traffic).
 __device__ __forceinline__ void st_release_shared(unsigned int* p, unsigned int v) {
@@ -208,20 +202,16 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
   if (!live) return;
   const int P = ix.num_pods;
   const uint64_t all = pod_all(P);
-  uint64_t alive = all;                                // pods that hold every block so far
-  unsigned int pos = 0;                                // blocks folded so far, in order
-  bool ended = false;                                  // a block with no live entry was seen
-  bool timed_out = false;
+  PrefixFold st = {all, 0u, false};                    // see index.cuh
   unsigned int idle = 0;
   unsigned int written = 0;                            // keys of this request written to `hashes`
   uint64_t last_key = root_seed;                       // the last of them: the seed to resume from
-  while (!ended && pos < n_r) {
+  while (!st.ended && st.pos < n_r) {
     const unsigned int avail = ld_acquire_shared(&sh.progress[qi]);   // same word for all lanes
-    if (avail == pos) {
+    if (avail == st.pos) {
       if (++idle >= kHeadPolls) {                      // the hasher never delivered: give up
-        timed_out = true;
         if (lane == 0) {
-          *v_consumed = pos | kHeadStopBit;
+          *v_consumed = st.pos | kHeadStopBit;
           raise_status(AIBX_ERR_TIMEOUT);
         }
         break;
@@ -230,87 +220,30 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
       continue;
     }
     idle = 0;
-    const unsigned int m = min(32u, avail - pos);
-    const bool valid = (unsigned int)lane < m;
+    const unsigned int m = min(32u, avail - st.pos);
     uint64_t mask = 0, key = 0;
     uint32_t id = AIBX_NO_BLOCK;
-    if (valid) {
-      key = *reinterpret_cast<volatile unsigned long long*>(&sh.ring[qi][(pos + lane) % kHeadRing]);
-      hashes[out0 + pos + lane] = key;                 // the keys leave the CTA through the prober
+    if ((unsigned int)lane < m) {
+      key = *reinterpret_cast<volatile unsigned long long*>(
+          &sh.ring[qi][(st.pos + lane) % kHeadRing]);
+      hashes[out0 + st.pos + lane] = key;              // the keys leave the CTA through the prober
       probe_ro(ix, key, mask, id);
     }
-    written = pos + m;
+    written = st.pos + m;
     last_key = shfl64(0xffffffffu, key, (int)m - 1);
-    const unsigned int none = __ballot_sync(0xffffffffu, valid && mask == 0);
-    const unsigned int f = none ? (unsigned int)__ffs(none) - 1u : 32u;   // first total miss
-    // pods still there after this lane's block: AND of the masks up to it, and of `alive`
-    uint64_t pref = valid ? mask : all;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const uint64_t o = shfl_up64(pref, d);
-      if (lane >= d) pref &= o;
-    }
-    pref &= alive;
-    const uint64_t prev = shfl_up64(pref, 1);
-    const uint64_t before = lane == 0 ? alive : prev;
-    uint64_t drops = valid ? (before & ~pref) : 0ULL;  // each pod drops once, at one lane
-    // the pods still there at the first total miss all end at any_len: written at the end, in
-    // parallel, not one by one by this lane
-    if ((unsigned int)lane == f) drops = 0;
-    while (drops) {
-      const int q = __ffsll((long long)drops) - 1;
-      drops &= drops - 1;
-      sh.match_len[qi][q] = pos + lane;
-    }
-    if (valid && block_ids) block_ids[out0 + pos + lane] = (unsigned int)lane < f ? id : AIBX_NO_BLOCK;
-    if (f < 32u) {
-      ended = true;                                    // any_len = pos + f
-      alive = shfl64(0xffffffffu, before, (int)f);     // the pods that held every block before it
-      pos += f;
-    } else {
-      alive = shfl64(0xffffffffu, pref, (int)m - 1);
-      pos += m;
-    }
+    fold_chunk(st, lane, m, mask, id, all, sh.match_len[qi], block_ids ? block_ids + out0 : nullptr);
     // Lets the hasher reuse the ring slots just read.  The keys read from them have been used
     // by now (every lane computed its probe address from its key), so the reads are complete
     // before this store is issued; a plain store is enough.
-    if (lane == 0) *v_consumed = ended ? (pos | kHeadStopBit) : pos;
+    if (lane == 0) *v_consumed = st.ended ? (st.pos | kHeadStopBit) : st.pos;
   }
 
-  // ---- the request's results
-  __syncwarp();
-  if (!timed_out) {
-    // pods that never dropped out: the whole request, or everything up to the first total miss
-    const unsigned int full = ended ? pos : n_r;
-    if (lane < P && ((alive >> lane) & 1ULL)) sh.match_len[qi][lane] = full;
-    if (lane + 32 < P && ((alive >> (lane + 32)) & 1ULL)) sh.match_len[qi][lane + 32] = full;
-  }
-  __syncwarp();
-  const long long h0 = lane < P ? (long long)sh.match_len[qi][lane] : 0;
-  const long long h1 = lane + 32 < P ? (long long)sh.match_len[qi][lane + 32] : 0;
-  if (lane < P) match_len[(int64_t)r * P + lane] = (uint32_t)h0;
-  if (lane + 32 < P) match_len[(int64_t)r * P + lane + 32] = (uint32_t)h1;
+  // ---- the request's results (after a time-out they are unspecified; the status says so)
+  fold_finish(st, lane, P, r, n_r, out0, sh.match_len[qi], match_len, any_len, block_ids, sp,
+              best_pod, best_score);
   if (lane == 0) {
-    if (any_len) any_len[r] = pos;
     hashed_out[r] = written;                           // keys the hasher made beyond these are dropped
     seed_out[r] = last_key;
-  }
-  if (block_ids) {
-    for (unsigned int i = pos + lane; i < n_r; i += 32) block_ids[out0 + i] = AIBX_NO_BLOCK;
-  }
-  if (best_pod) {
-    const long long l0 = lane < P ? (long long)sp.pod_load[lane] : 0;
-    const long long l1 = lane + 32 < P ? (long long)sp.pod_load[lane + 32] : 0;
-    long long top;
-    int arg;
-    lane_candidate(lane, P, sp.ready_mask,
-                   pod_score(h0, (long long)n_r, l0, sp.w_prefix, sp.w_load, sp.thr_pct),
-                   pod_score(h1, (long long)n_r, l1, sp.w_prefix, sp.w_load, sp.thr_pct), top, arg);
-    warp_argmax(top, arg);
-    if (lane == 0) {
-      best_pod[r] = arg;
-      best_score[r] = top;
-    }
   }
 }
 
