@@ -398,7 +398,7 @@ __device__ __forceinline__ void fold_finish(const PrefixFold& st, int lane, int 
 // are warps enough without splitting a request.  No barrier, no shared-memory atomics.
 constexpr int kMatchWarpKernelWarps = 4;
 
-__global__ void __launch_bounds__(kMatchWarpKernelWarps * 32)
+__global__ void __launch_bounds__(kMatchWarpKernelWarps * 32, 16)
 match_prefix_warp_kernel(IndexView ix, const uint64_t* __restrict__ hashes,
                          const int64_t* __restrict__ blk_off, int R,
                          uint32_t* __restrict__ match_len, uint32_t* __restrict__ any_len,
