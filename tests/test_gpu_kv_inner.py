@@ -98,6 +98,10 @@ def test_inner_order_round_trip_and_invalid():
         with pytest.raises(aibx.AibxError) as e:
             aibx.kv_gather_inner(pool_d, lay, pi, bi, dev(ids), 48, buf)
         assert e.value.code == aibx.ERR_INVALID
+    for bad_engine in (-1, 3):
+        with pytest.raises(aibx.AibxError) as e:
+            aibx.kv_set_inner_engine(bad_engine)
+        assert e.value.code == aibx.ERR_INVALID
     odd = aibx.KVLayout(0, 1, 2, 4, 12, 2, 8)                 # 24-byte rows, 384-byte tiles
     with pytest.raises(aibx.AibxError) as e:
         aibx.kv_gather_inner(pool_d, odd, 0, 1, dev(ids[:2]), 2, buf)
