@@ -38,7 +38,7 @@ typedef struct aibxo_index aibxo_index_t;
 /* XXH64 of `len` bytes with `seed`, all input lengths (xxHash specification, 64-bit variant). */
 uint64_t aibxo_xxh64(const void* data, size_t len, uint64_t seed);
 
-/* Chained per-block prefix keys (Section 3.2.2; hash and block size are this build's
+/* Chained per-block prefix keys (Section 3.2.2; hash and block size are this library's
  * reading since the paper fixes neither). */
 int32_t aibxo_hash_blocks(const int32_t* tokens, const int64_t* tok_off, const int64_t* blk_off,
                           int32_t R, int32_t block_tokens, uint64_t root_seed, uint64_t* hashes);
