@@ -1131,6 +1131,55 @@ def case_kv_inner_small(args):
                       "peak_kind": kind, "status": aibx.status_fetch()}))
 
 
+def case_kv_sweep(args):
+    """Gather and scatter of n blocks, n = 1 ... 4,096, on the three KV shapes: where the
+    bandwidth saturates (CUDA events around single calls, median of 15; L2 is evicted by a
+    256 MiB read before every call and that read's time is subtracted)."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from paper_2504_03648_b200 import synth
+    from paper_2504_03648_b200 import workloads as W
+
+    out = []
+    flush = torch.empty(64 << 20, dtype=torch.int32, device="cuda")
+    t_flush = statistics.median(_event_times(torch, lambda: flush.sum(), 15, 3))
+    for name, kv in (("cfg2 shape (2 MiB blocks, block-major)", W.scaled(W.cfg2_kv(), num_blocks=4096)),
+                     ("cfg4 shape (5 MiB blocks, layer-major)", W.scaled(W.cfg4_kv(), num_blocks=4096)),
+                     ("cfg5 shape (896 KiB blocks, block-major)", W.scaled(W.cfg5_kv(), num_blocks=4096))):
+        pool = torch.empty(kv.pool_bytes, dtype=torch.uint8, device="cuda")
+        synth.fill_pool(pool, kv)
+        buf = torch.empty(4096 * kv.block_bytes, dtype=torch.uint8, device="cuda")
+        lay = aibx.KVLayout(kv.layout, kv.num_layers, kv.num_kv_heads, kv.block_tokens,
+                            kv.head_dim, kv.elem_bytes, kv.num_blocks)
+        all_ids = torch.from_numpy(W.distinct_ids(7, kv.num_blocks, 4096)).cuda()
+        rows = []
+        for n in (1, 2, 4, 8, 16, 32, 64, 128, 256, 512, 1024, 2048, 4096):
+            ids = all_ids[:n].contiguous()
+
+            def g():
+                flush.sum()
+                aibx.kv_gather(pool, lay, ids, n, buf)
+
+            def sc():
+                flush.sum()
+                aibx.kv_scatter(pool, lay, ids, n, buf)
+
+            tg = statistics.median(_event_times(torch, g, 15, 3)) - t_flush
+            ts = statistics.median(_event_times(torch, sc, 15, 3)) - t_flush
+            nbytes = 2 * n * kv.block_bytes
+            rows.append({"n": n, "MB_moved": round(nbytes / 1e6, 1),
+                         "gather_us": round(tg * 1e3, 1), "scatter_us": round(ts * 1e3, 1),
+                         "gather_GBps": round(nbytes / (tg * 1e-3) / 1e9, 1),
+                         "scatter_GBps": round(nbytes / (ts * 1e-3) / 1e9, 1)})
+        out.append({"shape": name, "rows": rows})
+        del pool, buf
+        torch.cuda.empty_cache()
+    peak, kind = measured_peak_hbm()
+    print(json.dumps({"case": "kv_sweep", "peak": peak, "peak_kind": kind, "results": out,
+                      "status": aibx.status_fetch()}))
+
+
 def case_index_ops(args):
     """Operational index calls on the routing-heavy index (2^20 entries in 2^21 slots, 64 pods):
     touch, pick_victims, export, rehash, and the sequential assignment of 4,096 requests."""
@@ -1213,7 +1262,7 @@ def case_kv_comparators(args):
                       "status": aibx.status_fetch()}))
 
 
-CASES = {"kv_comparators": case_kv_comparators, "index_ops": case_index_ops, "kv_inner": case_kv_inner, "kv_inner_small": case_kv_inner_small, "hash_sweep": case_hash_sweep, "oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
+CASES = {"kv_comparators": case_kv_comparators, "index_ops": case_index_ops, "kv_inner": case_kv_inner, "kv_inner_small": case_kv_inner_small, "kv_sweep": case_kv_sweep, "hash_sweep": case_hash_sweep, "oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
          "cfg4": case_cfg4, "cfg5": case_cfg5, "lookup_flat": case_lookup_flat}
 
 
