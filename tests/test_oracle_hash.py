@@ -41,6 +41,20 @@ def test_published_values():
         assert oracle.xxh64(stream[:n], seed) == expect, (n, seed)
 
 
+def test_block_sized_vectors():
+    """The sizes the path hashes (whole 32-byte stripes, no tail), values from the build plan."""
+    n_rows = 0
+    for line in open(os.path.join(GOLDEN, "xxh64_block_sized.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        what, seed, hx = line.split()
+        kind, n = what.split(":")
+        data = bytes(int(n)) if kind == "zeros" else bytes(range(int(n)))
+        assert oracle.xxh64(data, int(seed)) == int(hx, 16), what
+        n_rows += 1
+    assert n_rows == 3
+
+
 def test_against_independent_library():
     xxhash = pytest.importorskip("xxhash")
     rng = np.random.default_rng(7)
