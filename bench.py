@@ -277,51 +277,51 @@ class GpuJob:
 
     def step_e2e(self, pieces=32):
         """Same step with host buffers on both sides of every transfer: tokens come from pinned
-        host memory, results go back to it, the gathered blocks are copied to pinned host
-        memory (put) and copied back from there before they are scattered (get).  The block list
-        is cut into `pieces` so that gather, device->host, host->device and scatter of
-        different pieces overlap (the two PCIe directions run at the same time).  With 32 pieces
-        a step runs at the rate the link gives with both directions busy (measured 47.6 GB/s
-        each way, against 57 / 56 GB/s for one direction alone)."""
+        host memory, results go back to it, and the matched blocks go to pinned host memory (put:
+        aibx_kv_gather_to_host) and come back from there (get: aibx_kv_scatter_from_host).  The
+        block list is cut into `pieces`, consecutive pieces alternating between two streams per
+        direction, so that gather, device->host, host->device and scatter of different pieces
+        overlap and the two PCIe directions run at the same time.  With 32 pieces a step runs at
+        the rate the link gives with both directions busy (measured 47.6 GB/s each way, against
+        57 / 56 GB/s for one direction alone)."""
         torch, aibx = self.torch, self.aibx
         main = torch.cuda.current_stream()
         if self.h_buf is None:
             self.h_buf = torch.empty(self.d_buf.numel(), dtype=torch.uint8).pin_memory()
             self.d_buf_back = torch.empty_like(self.d_buf)
-            self.s_put, self.s_get, self.s_scatter = (torch.cuda.Stream() for _ in range(3))
+            self.s_put = [torch.cuda.Stream() for _ in range(2)]
+            self.s_get = [torch.cuda.Stream() for _ in range(2)]
         self.d_tokens.copy_(self.h_tokens, non_blocking=True)
         n = self.routing()
         self.h_best_pod.copy_(self.d_best_pod, non_blocking=True)
         self.h_any_len.copy_(self.d_any_len, non_blocking=True)
         self.h_unique.copy_(self.d_unique, non_blocking=True)
+        routed = torch.cuda.Event()
+        routed.record(main)
         bb = self.kv.block_bytes
         per = (n + pieces - 1) // pieces
-        last = None
-        for c0 in range(0, n, per):
+        done = []
+        for k, c0 in enumerate(range(0, n, per)):
             m = min(per, n - c0)
             ids = self.d_unique[c0: c0 + m]
             lo, hi = c0 * bb, (c0 + m) * bb
-            aibx.kv_gather(self.d_pool, self.layout, ids, m, self.d_buf[lo:hi])
-            e_g = torch.cuda.Event()
-            e_g.record(main)
-            self.s_put.wait_event(e_g)
-            with torch.cuda.stream(self.s_put):
-                self.h_buf[lo:hi].copy_(self.d_buf[lo:hi], non_blocking=True)      # put
+            sp, sg = self.s_put[k % 2], self.s_get[k % 2]
+            sp.wait_event(routed)
+            with torch.cuda.stream(sp):
+                aibx.kv_gather_to_host(self.d_pool, self.layout, ids, m, self.d_buf[lo:hi],
+                                       self.h_buf[lo:hi])                       # put
                 e_p = torch.cuda.Event()
-                e_p.record(self.s_put)
-            self.s_get.wait_event(e_p)
-            with torch.cuda.stream(self.s_get):
-                self.d_buf_back[lo:hi].copy_(self.h_buf[lo:hi], non_blocking=True)  # get
-                e_h = torch.cuda.Event()
-                e_h.record(self.s_get)
-            self.s_scatter.wait_event(e_h)
-            with torch.cuda.stream(self.s_scatter):
-                aibx.kv_scatter(self.d_pool, self.layout, ids, m, self.d_buf_back[lo:hi])
-                last = torch.cuda.Event()
-                last.record(self.s_scatter)
+                e_p.record(sp)
+            sg.wait_event(e_p)
+            with torch.cuda.stream(sg):
+                aibx.kv_scatter_from_host(self.d_pool, self.layout, ids, m, self.d_buf_back[lo:hi],
+                                          self.h_buf[lo:hi])                    # get
+                e_g = torch.cuda.Event()
+                e_g.record(sg)
+            done.append(e_g)
         self.publish_expire()
-        if last is not None:
-            main.wait_event(last)
+        for e in done[-2:]:
+            main.wait_event(e)
         main.synchronize()
         nbytes = n * bb
         h2d = self.h_tokens.numel() * 4 + nbytes

@@ -367,6 +367,25 @@ int32_t aibx_kv_scatter(void* d_pool, const aibx_kv_layout_t* layout,
                         const uint32_t* d_block_ids, int64_t n, const void* d_buf,
                         void* stream);
 
+/* The same two movements with the far end in HOST memory (Section 3.2.5: the cache pool lives in
+ * host DRAM; put = engine pool -> cache, get = cache -> engine pool).  d_staging is a device
+ * buffer of n * block_bytes owned by the caller; h_buf is host memory of the same size (pinned
+ * memory makes the copy asynchronous; pageable memory works but blocks the calling thread).
+ *   gather_to_host   : aibx_kv_gather into d_staging, then d_staging -> h_buf, both on `stream`.
+ *                      Items the gather skips leave their part of h_buf as d_staging had it.
+ *   scatter_from_host: h_buf -> d_staging, then aibx_kv_scatter from d_staging, both on `stream`.
+ * Both only enqueue.  To keep both directions of the link busy, cut a list into pieces and give
+ * consecutive pieces to different streams: the copy of one piece then runs beside the kernel of
+ * the next.  Arguments and codes as aibx_kv_gather / aibx_kv_scatter; CUDA if a copy cannot be
+ * enqueued.
+ */
+int32_t aibx_kv_gather_to_host(const void* d_pool, const aibx_kv_layout_t* layout,
+                               const uint32_t* d_block_ids, int64_t n, void* d_staging,
+                               void* h_buf, void* stream);
+int32_t aibx_kv_scatter_from_host(void* d_pool, const aibx_kv_layout_t* layout,
+                                  const uint32_t* d_block_ids, int64_t n, void* d_staging,
+                                  const void* h_buf, void* stream);
+
 /* The same with the item count on the device: moves the first min(n_max, *d_count) items of the
  * list (d_count: one uint32 in device memory, read when the kernel starts).  Lets the output
  * of aibx_collect_blocks (ids + count) flow into the copy without a host round trip; the buffer

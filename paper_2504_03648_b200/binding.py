@@ -102,6 +102,8 @@ def lib():
             "aibx_collect_blocks_static": [vp, i64, u32, vp, vp, vp],
             "aibx_kv_gather": [vp, C.POINTER(KVLayout), vp, i64, vp, vp],
             "aibx_kv_scatter": [vp, C.POINTER(KVLayout), vp, i64, vp, vp],
+            "aibx_kv_gather_to_host": [vp, C.POINTER(KVLayout), vp, i64, vp, vp, vp],
+            "aibx_kv_scatter_from_host": [vp, C.POINTER(KVLayout), vp, i64, vp, vp, vp],
             "aibx_kv_gather_counted": [vp, C.POINTER(KVLayout), vp, i64, vp, vp, vp],
             "aibx_kv_scatter_counted": [vp, C.POINTER(KVLayout), vp, i64, vp, vp, vp],
             "aibx_kv_gather_inner": [vp, C.POINTER(KVLayout), i32, i32, vp, i64, vp, vp],
@@ -354,6 +356,23 @@ def kv_gather(pool, layout: KVLayout, block_ids, n: int, buf) -> None:
 def kv_scatter(pool, layout: KVLayout, block_ids, n: int, buf) -> None:
     _check("aibx_kv_scatter", lib().aibx_kv_scatter(
         _ptr(pool), C.byref(layout), _ptr(block_ids, torch.uint32), n, _ptr(buf), _stream()))
+
+
+def kv_gather_to_host(pool, layout: KVLayout, block_ids, n: int, staging, host_buf) -> None:
+    """Gather into the device staging buffer, then on to `host_buf` (a CPU tensor, pinned for an
+    asynchronous copy), all on the current stream."""
+    assert not host_buf.is_cuda and host_buf.is_contiguous()
+    _check("aibx_kv_gather_to_host", lib().aibx_kv_gather_to_host(
+        _ptr(pool), C.byref(layout), _ptr(block_ids, torch.uint32), n, _ptr(staging),
+        host_buf.data_ptr(), _stream()))
+
+
+def kv_scatter_from_host(pool, layout: KVLayout, block_ids, n: int, staging, host_buf) -> None:
+    """`host_buf` (CPU tensor) into the device staging buffer, then scatter, on the current stream."""
+    assert not host_buf.is_cuda and host_buf.is_contiguous()
+    _check("aibx_kv_scatter_from_host", lib().aibx_kv_scatter_from_host(
+        _ptr(pool), C.byref(layout), _ptr(block_ids, torch.uint32), n, _ptr(staging),
+        host_buf.data_ptr(), _stream()))
 
 
 def kv_gather_counted(pool, layout: KVLayout, block_ids, n_max: int, count, buf) -> None:

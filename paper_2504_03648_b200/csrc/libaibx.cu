@@ -631,6 +631,37 @@ int32_t aibx_kv_scatter(void* d_pool, const aibx_kv_layout_t* layout,
   return launch_kv_copy(d_pool, layout, d_block_ids, n, d_buf, 1, as_stream(stream));
 }
 
+int32_t aibx_kv_gather_to_host(const void* d_pool, const aibx_kv_layout_t* layout,
+                               const uint32_t* d_block_ids, int64_t n, void* d_staging,
+                               void* h_buf, void* stream) {
+  if (n > 0 && !h_buf) return AIBX_ERR_INVALID;
+  const int32_t rc = launch_kv_copy(d_pool, layout, d_block_ids, n, d_staging, 0, as_stream(stream));
+  if (rc != AIBX_OK || n == 0) return rc;
+  const size_t bytes = (size_t)n * 2u * layout->num_kv_heads * layout->block_tokens *
+                       layout->head_dim * layout->elem_bytes * layout->num_layers;
+  if (cudaMemcpyAsync(h_buf, d_staging, bytes, cudaMemcpyDeviceToHost, as_stream(stream)) !=
+      cudaSuccess)
+    return AIBX_ERR_CUDA;
+  return AIBX_OK;
+}
+
+int32_t aibx_kv_scatter_from_host(void* d_pool, const aibx_kv_layout_t* layout,
+                                  const uint32_t* d_block_ids, int64_t n, void* d_staging,
+                                  const void* h_buf, void* stream) {
+  if (!layout || n < 0) return AIBX_ERR_INVALID;
+  if (n == 0) return AIBX_OK;
+  if (!h_buf || !d_staging) return AIBX_ERR_INVALID;
+  if (layout->num_layers <= 0 || layout->num_kv_heads <= 0 || layout->block_tokens <= 0 ||
+      layout->head_dim <= 0 || layout->elem_bytes <= 0)
+    return AIBX_ERR_INVALID;
+  const size_t bytes = (size_t)n * 2u * layout->num_kv_heads * layout->block_tokens *
+                       layout->head_dim * layout->elem_bytes * layout->num_layers;
+  if (cudaMemcpyAsync(d_staging, h_buf, bytes, cudaMemcpyHostToDevice, as_stream(stream)) !=
+      cudaSuccess)
+    return AIBX_ERR_CUDA;
+  return launch_kv_copy(d_pool, layout, d_block_ids, n, d_staging, 1, as_stream(stream));
+}
+
 int32_t aibx_kv_gather_counted(const void* d_pool, const aibx_kv_layout_t* layout,
                                const uint32_t* d_block_ids, int64_t n_max, const uint32_t* d_count,
                                void* d_buf, void* stream) {

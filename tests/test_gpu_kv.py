@@ -259,6 +259,53 @@ def test_cfg4_full_size_layer_major():
     print("cfg4 pool blocks used:", kv.num_blocks, "(shrunk)" if shrunk else "(full)")
 
 
+@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("layout", [0, 1])
+def test_host_side_put_and_get(layout, pinned):
+    """gather_to_host / scatter_from_host: the far end of the transfer in host memory (pinned or
+    pageable), byte for byte against the oracle's gather and scatter."""
+    kv = W.KVSpec("host", 31, layout, 3, 4, 16, 64, 2, 90)
+    lay_g, lay_o = kv_layout_gpu(kv), kv_layout_oracle(kv)
+    pool_h = W.host_pool(kv)
+    rng = np.random.default_rng(layout + 5)
+    n = 57
+    ids_g = rng.integers(0, kv.num_blocks, n).astype(np.uint32)
+    ids_g[[4, 30]] = NO_BLOCK
+    ids_g[9] = kv.num_blocks + 3                                  # out of range: skipped, RANGE
+    pool_d = dev(pool_h)
+    staging = torch.full((n * kv.block_bytes,), 0x5A, dtype=torch.uint8, device="cuda")
+    h_buf = torch.zeros(n * kv.block_bytes, dtype=torch.uint8)
+    if pinned:
+        h_buf = h_buf.pin_memory()
+    aibx.kv_gather_to_host(pool_d, lay_g, dev(ids_g), n, staging, h_buf)
+    assert aibx.status_fetch() == (aibx.ERR_RANGE, 1)             # syncs the stream
+    want = np.full(n * kv.block_bytes, 0x5A, dtype=np.uint8)      # skipped items: staging as it was
+    oracle.kv_gather(pool_h, lay_o, ids_g, want)
+    assert np.array_equal(h_buf.numpy(), want) and np.array_equal(host(staging), want)
+    assert np.array_equal(host(pool_d), pool_h)
+    # get: other content from the host into a distinct set of blocks
+    ids_s = rng.permutation(kv.num_blocks)[:n].astype(np.uint32)
+    ids_s[3] = NO_BLOCK
+    src = torch.from_numpy(rng.integers(0, 256, n * kv.block_bytes, dtype=np.uint8))
+    if pinned:
+        src = src.pin_memory()
+    aibx.kv_scatter_from_host(pool_d, lay_g, dev(ids_s), n, staging, src)
+    assert aibx.status_fetch() == (0, 0)
+    pool_want = pool_h.copy()
+    oracle.kv_scatter(pool_want, lay_o, ids_s, src.numpy().copy())
+    assert np.array_equal(host(pool_d), pool_want)
+    # nothing to do, and what the host can refuse
+    aibx.kv_gather_to_host(pool_d, lay_g, dev(ids_g), 0, staging, h_buf)
+    aibx.kv_scatter_from_host(pool_d, lay_g, dev(ids_s), 0, staging, src)
+    lib = aibx.lib()
+    import ctypes as C
+    assert lib.aibx_kv_gather_to_host(pool_d.data_ptr(), C.byref(lay_g), dev(ids_g).data_ptr(), n,
+                                      staging.data_ptr(), None, None) == aibx.ERR_INVALID
+    assert lib.aibx_kv_scatter_from_host(pool_d.data_ptr(), C.byref(lay_g), dev(ids_s).data_ptr(), n,
+                                         None, src.data_ptr(), None) == aibx.ERR_INVALID
+    assert aibx.status_fetch() == (0, 0)
+
+
 def test_list_longer_than_one_launch_covers():
     """A launch addresses its transfer buffer with 32-bit offsets in 16-byte units, i.e. about
     64 GiB; a longer list is cut into several launches.  13,500 items of the 5 MiB Llama-3-70B
