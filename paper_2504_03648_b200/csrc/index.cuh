@@ -414,12 +414,18 @@ match_prefix_warp_kernel(IndexView ix, const uint64_t* __restrict__ hashes,
   const int64_t off = blk_off[r];
   const unsigned int n_r = (unsigned int)(blk_off[r + 1] - off);
   PrefixFold st = {all, 0u, false};
+  // the keys of the next chunk are requested before this chunk is probed: if the request goes
+  // on, they are there by then (one memory round trip less per further chunk)
+  uint64_t key = (unsigned int)lane < n_r ? __ldg(hashes + off + lane) : 0ULL;
   while (!st.ended && st.pos < n_r) {
     const unsigned int m = min(32u, n_r - st.pos);
+    const unsigned int nxt = st.pos + 32u + (unsigned int)lane;
+    const uint64_t key_next = nxt < n_r ? __ldg(hashes + off + nxt) : 0ULL;
     uint64_t mask = 0;
     uint32_t id = AIBX_NO_BLOCK;
-    if ((unsigned int)lane < m) probe_ro(ix, __ldg(hashes + off + st.pos + lane), mask, id);
+    if ((unsigned int)lane < m) probe_ro(ix, key, mask, id);
     fold_chunk(st, lane, m, mask, id, all, s_ml[warp], block_ids ? block_ids + off : nullptr);
+    key = key_next;
   }
   fold_finish(st, lane, P, r, n_r, off, s_ml[warp], match_len, any_len, block_ids, sp, best_pod,
               best_score);
