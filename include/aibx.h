@@ -21,6 +21,10 @@
  *     id out of range, a full table) are accumulated in the per-device status record and read
  *     with aibx_status_fetch.  Nothing aborts, throws or traps.
  *   - All arithmetic is integer; results are defined bit-exactly.
+ *   - Threads: calls on different indexes, pools and streams may come from different host
+ *     threads, except that the FIRST call of any kind on a device performs a few one-time
+ *     per-device settings (kernel attributes, the address of the status record) without locking:
+ *     make it from one thread.  Calls on one index are ordered by the caller.
  */
 #ifndef AIBX_H_
 #define AIBX_H_
