@@ -131,8 +131,13 @@ __device__ __forceinline__ unsigned long long find_slot_rw(const IndexView& ix, 
 // slots in the same order, and no slot turns reusable while inserts run, so the loser of a race
 // for a slot either finds the key there (another thread of the same key won) or starts over
 // and finds the key, or the next free slot, further on.
+// `added` / `reused` are raised when a slot was claimed / when that slot was a removed one: the
+// caller folds them into the table's counters once per CTA (one atomic per thread on the same
+// two words would serialise the whole kernel behind them).
 __device__ __forceinline__ unsigned long long insert_entry(const IndexView& ix, uint64_t key,
-                                                           uint64_t m, uint32_t id) {
+                                                           uint64_t m, uint32_t id,
+                                                           unsigned int& added,
+                                                           unsigned int& reused) {
   unsigned long long slot = ~0ULL;
   // a lost race costs one more walk; each one means some slot was taken, so the table bounds them
   for (unsigned long long attempts = 0; attempts <= ix.cap_mask && slot == ~0ULL; ++attempts) {
@@ -163,8 +168,8 @@ __device__ __forceinline__ unsigned long long insert_entry(const IndexView& ix, 
     const unsigned long long seen =
         atomicCAS(&ix.slots[free_slot].key, free_was, (unsigned long long)key);
     if (seen == free_was) {
-      atomicAdd(&ix.counters[0], 1ULL);
-      if (free_was == kKeyTomb) atomicAdd(&ix.counters[1], ~0ULL);
+      added += 1u;
+      if (free_was == kKeyTomb) reused += 1u;
       slot = free_slot;
     } else if (seen == key) {
       slot = free_slot;
@@ -179,15 +184,41 @@ __device__ __forceinline__ unsigned long long insert_entry(const IndexView& ix, 
   return slot;
 }
 
+// live += added - removed, freed-slot count += removed - reused: summed over the CTA in shared
+// memory, then one pair of atomics per CTA.  Every thread of the CTA must call it.
+__device__ __forceinline__ void fold_counters(const IndexView& ix, unsigned int added,
+                                              unsigned int reused, unsigned int removed) {
+  __shared__ unsigned int s_cnt[3];
+  if (threadIdx.x < 3) s_cnt[threadIdx.x] = 0u;
+  __syncthreads();
+  const unsigned int a = __reduce_add_sync(0xffffffffu, added);
+  const unsigned int u = __reduce_add_sync(0xffffffffu, reused);
+  const unsigned int d = __reduce_add_sync(0xffffffffu, removed);
+  if ((threadIdx.x & 31) == 0 && (a | u | d)) {
+    if (a) atomicAdd(&s_cnt[0], a);
+    if (u) atomicAdd(&s_cnt[1], u);
+    if (d) atomicAdd(&s_cnt[2], d);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned long long live = (unsigned long long)s_cnt[0] - (unsigned long long)s_cnt[2];
+    const unsigned long long tomb = (unsigned long long)s_cnt[2] - (unsigned long long)s_cnt[1];
+    if (live) atomicAdd(&ix.counters[0], live);       // two's complement: may be a decrease
+    if (tomb) atomicAdd(&ix.counters[1], tomb);
+  }
+}
+
 __global__ void index_insert_kernel(IndexView ix, const uint64_t* __restrict__ keys,
                                     const uint64_t* __restrict__ masks,
                                     const uint32_t* __restrict__ ids, int64_t n) {
   const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const uint64_t key = keys[i];
-  const uint64_t m = masks[i] & pod_all(ix.num_pods);
-  if (key_reserved(key) || m == 0) return;
-  insert_entry(ix, key, m, ids[i]);
+  unsigned int added = 0, reused = 0;
+  if (i < n) {
+    const uint64_t key = keys[i];
+    const uint64_t m = masks[i] & pod_all(ix.num_pods);
+    if (!key_reserved(key) && m != 0) insert_entry(ix, key, m, ids[i], added, reused);
+  }
+  fold_counters(ix, added, reused, 0u);
 }
 
 // Live entries of the table, in no particular order; *count ends as their number (entries
@@ -231,6 +262,7 @@ __global__ void index_export_kernel(IndexView ix, uint64_t* __restrict__ keys,
 // Carry every live entry of one table over into another (larger or smaller) one.
 __global__ void index_move_kernel(IndexView from, IndexView to) {
   const unsigned long long n = from.cap_mask + 1;
+  unsigned int added = 0, reused = 0;
   for (unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; i < n;
        i += (unsigned long long)gridDim.x * blockDim.x) {
     const uint4* p = reinterpret_cast<const uint4*>(from.slots + i);
@@ -239,10 +271,11 @@ __global__ void index_move_kernel(IndexView from, IndexView to) {
     const unsigned long long k = (unsigned long long)a.x | ((unsigned long long)a.y << 32);
     const unsigned long long m = (unsigned long long)a.z | ((unsigned long long)a.w << 32);
     if (!key_reserved(k) && m != 0) {
-      const unsigned long long s = insert_entry(to, k, m, b.x);
+      const unsigned long long s = insert_entry(to, k, m, b.x, added, reused);
       if (s != ~0ULL) to.slots[s].stamp = b.y;          // the touch history moves along
     }
   }
+  fold_counters(to, added, reused, 0u);
 }
 
 // evict, pass 1: clear the named pod bits
@@ -278,19 +311,19 @@ __global__ void index_evict_report_kernel(IndexView ix, const uint64_t* __restri
 __global__ void index_evict_remove_kernel(IndexView ix, const uint64_t* __restrict__ keys,
                                           int64_t n) {
   const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const uint64_t key = keys[i];
-  if (key_reserved(key)) return;
-  const unsigned long long s = find_slot_rw(ix, key);
-  if (s == ~0ULL) return;
-  const unsigned long long m = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].mask);
-  if (m != 0) return;
-  if (atomicCAS(&ix.slots[s].key, (unsigned long long)key, kKeyTomb) == key) {
-    ix.slots[s].id = AIBX_NO_BLOCK;      // ready for reuse by a later insert
-    ix.slots[s].stamp = 0u;
-    atomicAdd(&ix.counters[0], ~0ULL);   // live -= 1
-    atomicAdd(&ix.counters[1], 1ULL);
+  unsigned int removed = 0;
+  const uint64_t key = i < n ? keys[i] : kKeyEmpty;
+  if (!key_reserved(key)) {
+    const unsigned long long s = find_slot_rw(ix, key);
+    if (s != ~0ULL &&
+        *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].mask) == 0 &&
+        atomicCAS(&ix.slots[s].key, (unsigned long long)key, kKeyTomb) == key) {
+      ix.slots[s].id = AIBX_NO_BLOCK;      // ready for reuse by a later insert
+      ix.slots[s].stamp = 0u;
+      removed = 1u;
+    }
   }
+  fold_counters(ix, 0u, 0u, removed);     // live -= removed, freed slots += removed
 }
 
 __global__ void index_lookup_kernel(IndexView ix, const uint64_t* __restrict__ keys,
