@@ -222,16 +222,22 @@ __global__ void index_insert_kernel(IndexView ix, const uint64_t* __restrict__ k
 }
 
 // Live entries of the table, in no particular order; *count ends as their number (entries
-// beyond max_entries are counted but not written).
+// beyond max_entries are counted but not written).  Room is reserved once per CTA and turn of
+// the loop (warp ballots, a sum over the warps in shared memory, one atomic): one atomic per
+// warp on the single counter was what bounded the kernel.
 __global__ void index_export_kernel(IndexView ix, uint64_t* __restrict__ keys,
                                     uint64_t* __restrict__ masks, uint32_t* __restrict__ ids,
                                     unsigned long long max_entries,
                                     unsigned long long* __restrict__ count) {
+  __shared__ unsigned int s_warp[32];
+  __shared__ unsigned long long s_base;
   const unsigned long long n = ix.cap_mask + 1;
   const int lane = threadIdx.x & 31;
-  for (unsigned long long base = (blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x) - lane;
-       base < n; base += (unsigned long long)gridDim.x * blockDim.x) {
-    const unsigned long long i = base + lane;
+  const int warp = threadIdx.x >> 5;
+  const int n_warps = blockDim.x >> 5;
+  for (unsigned long long cta0 = blockIdx.x * (unsigned long long)blockDim.x; cta0 < n;
+       cta0 += (unsigned long long)gridDim.x * blockDim.x) {
+    const unsigned long long i = cta0 + threadIdx.x;
     unsigned long long k = 0, m = 0;
     unsigned int id = AIBX_NO_BLOCK;
     if (i < n) {
@@ -243,19 +249,28 @@ __global__ void index_export_kernel(IndexView ix, uint64_t* __restrict__ keys,
       id = b.x;
     }
     const bool live = i < n && !key_reserved(k) && m != 0;
-    // one atomic per warp: the leader reserves room for all live lanes
     const unsigned int votes = __ballot_sync(0xffffffffu, live);
-    unsigned long long start = 0;
-    if (lane == 0 && votes) start = atomicAdd(count, (unsigned long long)__popc(votes));
-    start = __shfl_sync(0xffffffffu, start, 0);
+    if (lane == 0) s_warp[warp] = __popc(votes);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      unsigned int total = 0;
+      for (int w = 0; w < n_warps; ++w) {
+        const unsigned int c = s_warp[w];
+        s_warp[w] = total;                               // exclusive prefix over the warps
+        total += c;
+      }
+      s_base = total ? atomicAdd(count, (unsigned long long)total) : 0ULL;
+    }
+    __syncthreads();
     if (live) {
-      const unsigned long long pos = start + __popc(votes & ((1u << lane) - 1u));
+      const unsigned long long pos = s_base + s_warp[warp] + __popc(votes & ((1u << lane) - 1u));
       if (pos < max_entries) {
         if (keys) keys[pos] = k;
         if (masks) masks[pos] = m;
         if (ids) ids[pos] = id;
       }
     }
+    __syncthreads();                                     // s_warp / s_base are reused next turn
   }
 }
 
