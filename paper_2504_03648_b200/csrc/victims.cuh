@@ -75,22 +75,49 @@ __device__ __forceinline__ bool live_slot(const IndexView& ix, unsigned long lon
   return !key_reserved(key) && m != 0;
 }
 
-__global__ void victims_hist_kernel(IndexView ix, VictimScratch* sc, int level) {
+// Histogram pass.  Priorities cluster (few distinct epochs), so (1) lanes of a warp that hit the
+// same bin elect one of them to add their number, and (2) a CTA collects its counts in a small
+// direct-mapped table in shared memory and adds each hot bin to the global histogram once, at
+// the end; only bins that collide in that table go to global memory at once.  Without (2) every
+// warp of the grid queued up on the same few words of the global histogram.
+constexpr int kHistCache = 256;
+
+__global__ void __launch_bounds__(256)
+victims_hist_kernel(IndexView ix, VictimScratch* sc, int level) {
+  __shared__ unsigned int s_bin[kHistCache];
+  __shared__ unsigned int s_cnt[kHistCache];
   const unsigned long long n = ix.cap_mask + 1;
   const unsigned int prefix = level == 2 ? sc->st.prefix : 0u;
   if (level == 2 && prefix == 0xFFFFFFFFu) return;       // everything is taken: no second level
+  unsigned int* hist = level == 1 ? sc->hist1 : sc->hist2;
+  for (int j = threadIdx.x; j < kHistCache; j += blockDim.x) {
+    s_bin[j] = 0xFFFFFFFFu;
+    s_cnt[j] = 0u;
+  }
+  __syncthreads();
   for (unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; i < n;
        i += (unsigned long long)gridDim.x * blockDim.x) {
     uint64_t key;
     unsigned int p;
     if (!live_slot(ix, i, key, p)) continue;
     if (level == 2 && (p >> 15) != prefix) continue;
-    // Priorities cluster (few distinct epochs), so lanes that hit the same bin elect one of
-    // them to add their number: one atomic per distinct bin per warp instead of one per entry.
-    unsigned int* bin = level == 1 ? &sc->hist1[p >> 15] : &sc->hist2[p & 0x7FFFu];
+    const unsigned int bin = level == 1 ? p >> 15 : p & 0x7FFFu;
     const unsigned int active = __activemask();
-    const unsigned int same = __match_any_sync(active, (unsigned long long)bin);
-    if ((threadIdx.x & 31) == __ffs(same) - 1) atomicAdd(bin, (unsigned int)__popc(same));
+    const unsigned int same = __match_any_sync(active, bin);
+    if ((threadIdx.x & 31) == __ffs(same) - 1) {
+      const unsigned int c = (unsigned int)__popc(same);
+      const unsigned int slot = bin & (kHistCache - 1);
+      const unsigned int seen = atomicCAS(&s_bin[slot], 0xFFFFFFFFu, bin);
+      if (seen == 0xFFFFFFFFu || seen == bin) {
+        atomicAdd(&s_cnt[slot], c);
+      } else {
+        atomicAdd(&hist[bin], c);                        // the table's slot belongs to another bin
+      }
+    }
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < kHistCache; j += blockDim.x) {
+    if (s_bin[j] != 0xFFFFFFFFu && s_cnt[j]) atomicAdd(&hist[s_bin[j]], s_cnt[j]);
   }
 }
 
@@ -156,42 +183,65 @@ victims_select_kernel(VictimScratch* sc, int level, unsigned long long* __restri
   }
 }
 
-__global__ void victims_collect_kernel(IndexView ix, VictimScratch* sc,
-                                       uint64_t* __restrict__ out_keys,
-                                       uint32_t* __restrict__ out_prio) {
+// Collect pass.  Tickets for the entries at the threshold and room in the output are reserved
+// once per CTA and turn of the loop (ballots, a sum over the warps in shared memory, one atomic
+// each), not once per warp: with clustered priorities nearly every warp holds threshold entries.
+__global__ void __launch_bounds__(256)
+victims_collect_kernel(IndexView ix, VictimScratch* sc, uint64_t* __restrict__ out_keys,
+                       uint32_t* __restrict__ out_prio) {
+  __shared__ unsigned int s_eq[8], s_take[8];
+  __shared__ unsigned long long s_eq_base, s_out_base;
   const unsigned long long n = ix.cap_mask + 1;
   const unsigned int T = sc->st.threshold;
   const unsigned long long need_eq = sc->st.need_eq;
   const unsigned long long k = sc->st.k;
   const int lane = threadIdx.x & 31;
-  for (unsigned long long base = (blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x) - lane;
-       base < n; base += (unsigned long long)gridDim.x * blockDim.x) {
-    const unsigned long long i = base + lane;
+  const int warp = threadIdx.x >> 5;
+  const int n_warps = blockDim.x >> 5;
+  for (unsigned long long cta0 = blockIdx.x * (unsigned long long)blockDim.x; cta0 < n;
+       cta0 += (unsigned long long)gridDim.x * blockDim.x) {
+    const unsigned long long i = cta0 + threadIdx.x;
     uint64_t key = 0;
     unsigned int p = 0;
     const bool live = i < n && live_slot(ix, i, key, p);
     bool take = live && p < T;
-    // entries at the threshold are interchangeable: the first need_eq tickets win (one ticket
-    // counter update per warp)
+    // entries at the threshold are interchangeable: the first need_eq tickets win
     const bool at_thr = live && p == T && need_eq > 0;
     const unsigned int eq = __ballot_sync(0xffffffffu, at_thr);
-    if (eq) {
-      unsigned long long first = 0;
-      if (lane == __ffs(eq) - 1) first = atomicAdd(&sc->st.eq_taken, (unsigned long long)__popc(eq));
-      first = __shfl_sync(0xffffffffu, first, __ffs(eq) - 1);
-      if (at_thr) take = first + __popc(eq & ((1u << lane) - 1u)) < need_eq;
+    if (lane == 0) s_eq[warp] = __popc(eq);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      unsigned int total = 0;
+      for (int w = 0; w < n_warps; ++w) {
+        const unsigned int c = s_eq[w];
+        s_eq[w] = total;
+        total += c;
+      }
+      s_eq_base = total ? atomicAdd(&sc->st.eq_taken, (unsigned long long)total) : 0ULL;
     }
+    __syncthreads();
+    if (at_thr) take = s_eq_base + s_eq[warp] + __popc(eq & ((1u << lane) - 1u)) < need_eq;
     const unsigned int votes = __ballot_sync(0xffffffffu, take);
-    unsigned long long start = 0;
-    if (lane == 0 && votes) start = atomicAdd(&sc->st.out_pos, (unsigned long long)__popc(votes));
-    start = __shfl_sync(0xffffffffu, start, 0);
+    if (lane == 0) s_take[warp] = __popc(votes);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      unsigned int total = 0;
+      for (int w = 0; w < n_warps; ++w) {
+        const unsigned int c = s_take[w];
+        s_take[w] = total;
+        total += c;
+      }
+      s_out_base = total ? atomicAdd(&sc->st.out_pos, (unsigned long long)total) : 0ULL;
+    }
+    __syncthreads();
     if (take) {
-      const unsigned long long pos = start + __popc(votes & ((1u << lane) - 1u));
+      const unsigned long long pos = s_out_base + s_take[warp] + __popc(votes & ((1u << lane) - 1u));
       if (pos < k) {
         if (out_keys) out_keys[pos] = key;
         if (out_prio) out_prio[pos] = p;
       }
     }
+    __syncthreads();                                     // the shared words are reused next turn
   }
 }
 
