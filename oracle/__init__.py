@@ -151,8 +151,9 @@ class Index:
         self.capacity = capacity
 
     def __del__(self):
-        if getattr(self, "_h", None):
-            lib().aibxo_index_destroy(self._h)
+        # at interpreter shutdown the module globals may already be gone: then leave it
+        if getattr(self, "_h", None) and _lib is not None:
+            _lib.aibxo_index_destroy(self._h)
             self._h = None
 
     def clear(self):
