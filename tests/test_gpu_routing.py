@@ -563,3 +563,44 @@ def test_rehash_beside_the_readers():
         g.rehash_begin(1 << 17)                          # the live entries do not fit
     assert e.value.code == aibx.ERR_FULL
     assert aibx.status_fetch() == (0, 0)
+
+
+def test_index_duplicate_heavy_random_batches():
+    """Many short op sequences on small and mid-sized tables, every batch drawing its keys with
+    heavy repetition from a small universe (so that threads race for the same slots), checked
+    after every call against the oracle: evict's freed ids, every lookup, the live count."""
+    checked = 0
+    for seed in range(120):
+        rng = np.random.default_rng(5000 + seed)
+        cap = int(rng.choice([8, 16, 64, 1024, 65536]))
+        P = int(rng.integers(1, 65))
+        universe = rng.integers(1, 1 << 62, max(4, int(cap * rng.choice([0.3, 0.6, 0.9])))).astype(np.uint64)
+        g, o = aibx.Index(cap, P), oracle.Index(cap, P)
+        for step in range(8):
+            n = int(rng.integers(1, 4 * len(universe)))
+            ks = universe[rng.integers(0, len(universe), n)]
+            if rng.random() < 0.1:
+                ks[rng.integers(0, n)] = 0                       # a reserved key in the batch
+            ms = (rng.integers(0, 1 << 63, n).astype(np.uint64) * 2
+                  + rng.integers(0, 2, n).astype(np.uint64))
+            if rng.random() < 0.6:
+                ids = rng.integers(0, 1 << 20, n).astype(np.uint32)
+                assert o.insert(ks, ms, ids) == oracle.OK
+                g.insert(dev(ks), dev(ms), dev(ids))
+            else:
+                if rng.random() < 0.5:
+                    ms[:] = ALL
+                _, wf = o.evict(ks, ms)
+                d_f = empty(n, torch.uint32)
+                g.evict(dev(ks), dev(ms), d_f)
+                assert np.array_equal(host(d_f), wf), (seed, step)
+            assert aibx.status_fetch() == (0, 0), (seed, step)
+            probe = np.concatenate([universe, rng.integers(1, 1 << 62, 8).astype(np.uint64)])
+            wm, wi = o.lookup(probe)
+            d_m, d_i = empty(len(probe), torch.uint64), empty(len(probe), torch.uint32)
+            g.lookup(dev(probe), d_m, d_i)
+            assert np.array_equal(host(d_m), wm) and np.array_equal(host(d_i), wi), (seed, step)
+            assert g.stats()[0] == o.stats()[0], (seed, step)
+            checked += 1
+        g.destroy()
+    assert checked == 960
