@@ -175,3 +175,47 @@ def test_inner_order_on_the_full_cfg4_pool():
             got = host(pool.view(kv.num_layers, nb, kv.tile_bytes)[:, int(ids[i])].contiguous()).reshape(-1)
             assert np.array_equal(got, want), (engine, i)
         synth.fill_pool(pool, kv)                             # generated content again
+
+
+def test_inner_order_random_shapes():
+    """Sixty random shapes (element size, row length, heads, tokens, layers, layout; planes from
+    a few rows to several stages, ragged boxes): the tensor-map engine against the oracle, and
+    against the storer-warp engine byte for byte, gather and scatter, both directions of the swap."""
+    done = 0
+    for seed in range(60):
+        rng = np.random.default_rng(900 + seed)
+        E = int(rng.choice([1, 2, 4]))
+        D = int(rng.choice([16, 32, 64, 128, 256]))
+        H = int(rng.integers(1, 20))
+        T = int(rng.integers(1, 300 if rng.random() < 0.2 else 40))
+        L, layout = int(rng.integers(1, 4)), int(rng.integers(0, 2))
+        nb = int(rng.integers(2, 10))
+        kv = W.KVSpec("rnd", seed, layout, L, H, T, D, E, nb)
+        if kv.pool_bytes > (256 << 20):
+            continue
+        lay_g, lay_o = kv_layout_gpu(kv), kv_layout_oracle(kv)
+        pool_h = W.host_pool(kv)
+        n = int(rng.integers(1, 2 * nb))
+        ids = rng.integers(0, nb, n).astype(np.uint32)
+        ids_s = rng.permutation(nb)[: min(nb, n)].astype(np.uint32)
+        for pi, bi in ((0, 1), (1, 0)):
+            want = np.zeros(n * kv.block_bytes, dtype=np.uint8)
+            oracle.kv_gather_inner(pool_h, lay_o, pi, bi, ids, want)
+            bufs = []
+            for engine in (2, 1):
+                aibx.kv_set_inner_engine(engine)
+                buf = empty(n * kv.block_bytes, torch.uint8)
+                aibx.kv_gather_inner(dev(pool_h), lay_g, pi, bi, dev(ids), n, buf)
+                bufs.append(buf)
+            assert np.array_equal(host(bufs[0]), want), (seed, pi, bi)
+            assert torch.equal(bufs[0], bufs[1]), (seed, pi, bi)
+            m = len(ids_s)
+            pool_want = pool_h.copy()
+            oracle.kv_scatter_inner(pool_want, lay_o, pi, bi, ids_s, want[: m * kv.block_bytes].copy())
+            for engine in (2, 1):
+                aibx.kv_set_inner_engine(engine)
+                pool_d = dev(pool_h)
+                aibx.kv_scatter_inner(pool_d, lay_g, pi, bi, dev(ids_s), m, bufs[0])
+                assert np.array_equal(host(pool_d), pool_want), (seed, pi, bi, engine)
+            done += 1
+    assert done >= 100 and aibx.status_fetch() == (0, 0)
