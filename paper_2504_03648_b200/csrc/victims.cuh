@@ -132,8 +132,19 @@ victims_select_kernel(VictimScratch* sc, int level, unsigned long long* __restri
   if (level == 2 && sc->st.prefix == 0xFFFFFFFFu) return;
   const unsigned long long want = level == 1 ? sc->st.k : sc->st.k_rem;
 
+  // this thread's `per` consecutive bins (a multiple of 8), read as 16-byte vectors, eight
+  // loads in flight at a time: one bin per dependent load made this one-CTA kernel the longest
+  // of the whole selection
   unsigned long long mine = 0;
-  for (int b = 0; b < per; ++b) mine += hist[tid * per + b];
+  const uint4* h4 = reinterpret_cast<const uint4*>(hist + (size_t)tid * per);
+  for (int v0 = 0; v0 < per / 4; v0 += 8) {
+    uint4 q[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) q[u] = __ldcg(h4 + v0 + u);
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      mine += (unsigned long long)q[u].x + q[u].y + q[u].z + q[u].w;
+  }
   unsigned long long inc = mine;                       // inclusive scan over the CTA
 #pragma unroll
   for (int d = 1; d < 32; d <<= 1) {
