@@ -170,3 +170,31 @@ def test_route_head_invalid_arguments_and_empty_batch():
     assert host(al).tolist() == [0] and host(ml).tolist() == [0] * 4
     assert host(ids).tolist() == [NO_BLOCK, NO_BLOCK] and 1 <= int(host(dn)[0]) <= 2
     assert aibx.status_fetch() == (0, 0)
+
+
+@pytest.mark.parametrize("B", [8, 16, 32, 40, 1024])
+def test_resume_from_any_block(B):
+    """aibx_hash_blocks_resume on its own: every request resumed at a random block (0, the last
+    one and past-the-end included) with the key before it as seed gives the oracle's keys from
+    there on and leaves the earlier part of the output alone."""
+    rng = np.random.default_rng(B)
+    R = 37
+    nblk = rng.integers(0, 60 if B < 1024 else 5, R)
+    lens = nblk * B + rng.integers(0, B, R)
+    tok_off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    tokens = rng.integers(-5, 128256, int(tok_off[-1])).astype(np.int32)
+    root = 0x1234ABCD
+    want, bo = oracle.hash_blocks(tokens, tok_off, B, root)
+    start = np.array([rng.integers(0, n + 1) for n in nblk], dtype=np.uint32)
+    start[:3] = [0, nblk[1], nblk[2]]
+    seed = np.array([want[bo[r] + start[r] - 1] if start[r] else root for r in range(R)], dtype=np.uint64)
+    nb = max(int(bo[-1]), 1)
+    d_h = torch.full((nb,), 0x7E7E7E7E7E7E7E7E, dtype=torch.uint64, device="cuda")
+    aibx.hash_blocks_resume(dev(tokens) if len(tokens) else empty(4, torch.int32), dev(tok_off),
+                            dev(bo), B, dev(start), dev(seed), d_h)
+    got = host(d_h)
+    for r in range(R):
+        lo, hi = int(bo[r]), int(bo[r + 1])
+        assert (got[lo: lo + start[r]] == 0x7E7E7E7E7E7E7E7E).all(), r
+        assert np.array_equal(got[lo + start[r]: hi], want[lo + start[r]: hi]), r
+    assert aibx.status_fetch() == (0, 0)
