@@ -2,14 +2,17 @@
 """Benchmark of the KV-reuse hot path on B200.
 
 One step = one pass of the whole path over one batch of the Llama-3-8B-shaped workload:
-hash the 64 requests -> longest cached prefix against a 200k-entry index + route score ->
-set of matched blocks -> gather them from the 8 GiB paged pool into the transfer buffer ->
-scatter them back -> publish and expire one batch of new index entries.
+hash the 64 requests as far as matching needs, longest cached prefix against a 200k-entry index
+and route score (one kernel) -> set of matched blocks -> gather them from the 8 GiB paged pool
+into the transfer buffer -> scatter them back; beside the copies, on a second stream: the rest
+of the hash chains, then publish and expire one batch of new index entries.
 
 `value` is gather+scatter bytes (read + written) per second over the whole step, inputs
 resident in HBM.  `e2e` is the same with host buffers: tokens come from pinned host memory,
-routing results go back to the host, the gathered buffer is copied to pinned host memory (the
-put to a DRAM cache) and copied back before the scatter (the get).
+routing results go back to the host, the matched blocks are put to pinned host memory
+(aibx_kv_gather_to_host, the put to a DRAM cache) and got back from it
+(aibx_kv_scatter_from_host).  The line also carries the prefix-match figures of the
+routing-heavy batch (`prefix_match_routing_heavy`).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
