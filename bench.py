@@ -973,10 +973,27 @@ def case_lookup_flat(args):
 
 
 def case_oracle_cfg(args):
-    """The CPU oracle, one host core, on the routing halves of cfg2 / cfg3 / cfg5 at full size
-    and on gather+scatter of 128 blocks of each KV shape (pool of 256 blocks on the host)."""
+    """The CPU oracle on the routing halves of cfg2 / cfg3 / cfg5 at full size and on
+    gather+scatter of 128 blocks of each KV shape (pool of 256 blocks on the host): on one host
+    core, and the same oracle functions called from one thread per available core over disjoint
+    request ranges (hash, match, score; the index is only read) or disjoint id ranges (gather,
+    scatter).  The calls are ctypes calls, which release the interpreter lock."""
     import oracle
+    from concurrent.futures import ThreadPoolExecutor
     from paper_2504_03648_b200 import workloads as W
+
+    T = len(os.sched_getaffinity(0))
+    pool_t = ThreadPoolExecutor(max_workers=T)
+
+    def ranges(n):
+        cuts = [n * i // T for i in range(T + 1)]
+        return [(a, b) for a, b in zip(cuts[:-1], cuts[1:]) if b > a]
+
+    def fan(fn, n):
+        list(pool_t.map(lambda ab: fn(*ab), ranges(n)))
+
+    def sub_off(off, a, b):
+        return np.ascontiguousarray(off[a:b + 1] - off[a])
 
     def clock(fn, reps=3):
         ts = []
@@ -1003,9 +1020,22 @@ def case_oracle_cfg(args):
         t_match = clock(lambda: ix.match_prefix(h, bo))
         ml, al, _ = ix.match_prefix(h, bo)
         t_score = clock(lambda: oracle.route_score(ml, bo, w.pod_load, w.ready_mask, None))
+        R = len(w.tok_off) - 1
+        tok_parts = {ab: (np.ascontiguousarray(w.tokens[w.tok_off[ab[0]]:w.tok_off[ab[1]]]),
+                          sub_off(w.tok_off, *ab)) for ab in ranges(R)}
+        h_parts = {ab: (np.ascontiguousarray(h[bo[ab[0]]:bo[ab[1]]]), sub_off(bo, *ab),
+                        np.ascontiguousarray(ml[ab[0]:ab[1]])) for ab in ranges(R)}
+        tt_hash = clock(lambda: fan(lambda a, b: oracle.hash_blocks(
+            *tok_parts[(a, b)], s.block_tokens, 0), R))
+        tt_match = clock(lambda: fan(lambda a, b: ix.match_prefix(*h_parts[(a, b)][:2]), R))
+        tt_score = clock(lambda: fan(lambda a, b: oracle.route_score(
+            h_parts[(a, b)][2], h_parts[(a, b)][1], w.pod_load, w.ready_mask, None), R))
         res.append({"config": s.name, "hash_us": round(t_hash * 1e6, 1),
                     "insert_us": round(t_ins * 1e6, 1), "match_us": round(t_match * 1e6, 1),
-                    "score_us": round(t_score * 1e6, 1)})
+                    "score_us": round(t_score * 1e6, 1),
+                    "threads": {"hash_us": round(tt_hash * 1e6, 1),
+                                "match_us": round(tt_match * 1e6, 1),
+                                "score_us": round(tt_score * 1e6, 1)}})
     for kv0 in (W.cfg2_kv(), W.cfg4_kv(), W.cfg5_kv()):
         kv = W.scaled(kv0, num_blocks=256)
         pool = W.host_pool(kv)
@@ -1016,8 +1046,15 @@ def case_oracle_cfg(args):
         tg = clock(lambda: oracle.kv_gather(pool, lay, ids, buf))
         ts = clock(lambda: oracle.kv_scatter(pool, lay, ids, buf))
         nb = 2 * 128 * kv.block_bytes
+        bb = kv.block_bytes
+        ttg = clock(lambda: fan(lambda a, b: oracle.kv_gather(
+            pool, lay, ids[a:b], buf[a * bb:b * bb]), 128))
+        tts = clock(lambda: fan(lambda a, b: oracle.kv_scatter(
+            pool, lay, ids[a:b], buf[a * bb:b * bb]), 128))
         res.append({"config": kv0.name, "gather_GBps": round(nb / tg / 1e9, 2),
-                    "scatter_GBps": round(nb / ts / 1e9, 2)})
+                    "scatter_GBps": round(nb / ts / 1e9, 2),
+                    "threads": {"gather_GBps": round(nb / ttg / 1e9, 2),
+                                "scatter_GBps": round(nb / tts / 1e9, 2)}})
     cpu = ""
     try:
         for line in open("/proc/cpuinfo"):
@@ -1026,8 +1063,9 @@ def case_oracle_cfg(args):
                 break
     except OSError:
         pass
-    print(json.dumps({"case": "oracle_cfg", "cores_used": 1,
-                      "cores_available": len(os.sched_getaffinity(0)), "cpu": cpu, "results": res}))
+    pool_t.shutdown()
+    print(json.dumps({"case": "oracle_cfg", "cores_used": 1, "threads_used": T,
+                      "cores_available": T, "cpu": cpu, "results": res}))
 
 
 def case_hash_sweep(args):
