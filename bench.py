@@ -133,8 +133,8 @@ class GpuJob:
         import torch
 
         from paper_2504_03648_b200 import binding as aibx
-        from paper_2504_03648_b200 import synth
-        from paper_2504_03648_b200 import workloads as W
+        from workloads import synth
+        import workloads as W
 
         self.torch, self.aibx = torch, aibx
         torch.cuda.set_device(device_index)
@@ -460,7 +460,7 @@ def run_gpu(args):
     cfg3 = None
     if rank == 0:
         # the other half of the metric: prefix match alone on the routing-heavy batch
-        from paper_2504_03648_b200 import workloads as W
+        import workloads as W
         cfg3 = routing_batch_times(W.cfg3_routing)
     if dist is not None:
         dist.barrier()
@@ -521,7 +521,7 @@ class OracleSample:
 
     def __init__(self):
         import oracle
-        from paper_2504_03648_b200 import workloads as W
+        import workloads as W
 
         self.oracle = oracle
         self.w = w = W.build_routing(W.cfg2_routing())
@@ -624,8 +624,8 @@ def case_kv_small(args):
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import synth
-    from paper_2504_03648_b200 import workloads as W
+    from workloads import synth
+    import workloads as W
 
     kv = W.scaled(W.cfg2_kv(), num_blocks=512)
     n = 256
@@ -673,7 +673,7 @@ def case_match_large(args):
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import workloads as W
+    import workloads as W
 
     P, nblk = 32, 64
     ix, keys = _big_index(torch, aibx, W, args.log2cap, P, 11)
@@ -717,7 +717,7 @@ def routing_batch_times(mk):
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import workloads as W
+    import workloads as W
 
     w = W.build_routing(mk())
     s = w.spec
@@ -800,7 +800,7 @@ def routing_batch_times(mk):
 def case_match_cfg(args):
     """The routing calls alone on the cfg2, routing-heavy (cfg3) and long-context (cfg5) batches."""
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import workloads as W
+    import workloads as W
 
     res = [routing_batch_times(mk) for mk in (W.cfg2_routing, W.cfg3_routing, W.cfg5_routing)]
     print(json.dumps({"case": "match_cfg", "results": res, "status": aibx.status_fetch()}))
@@ -821,8 +821,8 @@ def case_cfg4(args):
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import synth
-    from paper_2504_03648_b200 import workloads as W
+    from workloads import synth
+    import workloads as W
 
     n, iters = 2048, 100
     kv = _fit_pool(torch, W, W.cfg4_kv(), n * W.cfg4_kv().block_bytes)
@@ -869,8 +869,8 @@ def case_cfg5(args):
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import synth
-    from paper_2504_03648_b200 import workloads as W
+    from workloads import synth
+    import workloads as W
 
     kv0 = W.cfg5_kv()
     kv = _fit_pool(torch, W, kv0, 4000 * kv0.block_bytes)
@@ -926,7 +926,7 @@ def case_lookup_flat(args):
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import workloads as W
+    import workloads as W
 
     n = 1 << 24
     peak, kind = measured_peak_hbm()
@@ -980,7 +980,7 @@ def case_oracle_cfg(args):
     scatter).  The calls are ctypes calls, which release the interpreter lock."""
     import oracle
     from concurrent.futures import ThreadPoolExecutor
-    from paper_2504_03648_b200 import workloads as W
+    import workloads as W
 
     T = len(os.sched_getaffinity(0))
     pool_t = ThreadPoolExecutor(max_workers=T)
@@ -1075,7 +1075,7 @@ def case_hash_sweep(args):
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import workloads as W
+    import workloads as W
 
     out = []
     for R, L in ((1, 32768), (64, 32768), (4096, 2048)):
@@ -1100,8 +1100,8 @@ def case_kv_inner(args):
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import synth
-    from paper_2504_03648_b200 import workloads as W
+    from workloads import synth
+    import workloads as W
 
     out = []
     for name, kv, n in (("cfg2 shape", W.scaled(W.cfg2_kv(), num_blocks=4096), 1600),
@@ -1143,8 +1143,8 @@ def case_kv_inner_small(args):
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import synth
-    from paper_2504_03648_b200 import workloads as W
+    from workloads import synth
+    import workloads as W
 
     kv = W.scaled(W.cfg2_kv(), num_blocks=512)
     n = 256
@@ -1179,8 +1179,8 @@ def case_kv_sweep(args):
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import synth
-    from paper_2504_03648_b200 import workloads as W
+    from workloads import synth
+    import workloads as W
 
     out = []
     flush = torch.empty(64 << 20, dtype=torch.int32, device="cuda")
@@ -1227,7 +1227,7 @@ def case_index_ops(args):
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import workloads as W
+    import workloads as W
 
     ix, keys = _big_index(torch, aibx, W, 21, 64, 61)
     n = len(keys)
@@ -1273,8 +1273,8 @@ def case_kv_comparators(args):
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
-    from paper_2504_03648_b200 import synth
-    from paper_2504_03648_b200 import workloads as W
+    from workloads import synth
+    import workloads as W
 
     kv = W.cfg2_kv()
     n = 1600

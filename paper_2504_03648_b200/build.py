@@ -1,7 +1,6 @@
 """Builds the CUDA libraries in-tree with nvcc for sm_100a.
 
-``libaibx.so`` is the product (C ABI of include/aibx.h); ``libaibx_synth.so`` is the device
-twin of the synthetic input generator used by tests and benchmarks.
+``libaibx.so`` is the product (C ABI of include/aibx.h).
 """
 from __future__ import annotations
 
@@ -12,7 +11,6 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libaibx.so")
-SYNTH_LIB = os.path.join(PKG, "libaibx_synth.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -39,8 +37,6 @@ def build(force: bool = False, verbose: bool = False) -> None:
     deps.append(os.path.join(ROOT, "include", "aibx.h"))
     if force or _stale(LIB, deps):
         _nvcc(os.path.join(CSRC, "libaibx.cu"), LIB, verbose)
-    if force or _stale(SYNTH_LIB, [os.path.join(CSRC, "synth_fill.cu")]):
-        _nvcc(os.path.join(CSRC, "synth_fill.cu"), SYNTH_LIB, verbose)
 
 
 if __name__ == "__main__":
@@ -48,4 +44,3 @@ if __name__ == "__main__":
 
     build(force="--force" in sys.argv, verbose="-v" in sys.argv)
     print(LIB)
-    print(SYNTH_LIB)

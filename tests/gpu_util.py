@@ -5,7 +5,7 @@ import torch
 
 import oracle
 from paper_2504_03648_b200 import binding as aibx
-from paper_2504_03648_b200 import workloads as W
+import workloads as W
 
 NO_BLOCK = 0xFFFFFFFF
 
@@ -105,3 +105,145 @@ def read_block(pool_t: torch.Tensor, kv: W.KVSpec, b: int) -> np.ndarray:
     if kv.layout == 0:
         return host(pool_t.view(kv.num_blocks, kv.block_bytes)[b])
     return host(pool_t.view(kv.num_layers, kv.num_blocks, kv.tile_bytes)[:, b].contiguous()).reshape(-1)
+
+
+# ------------------------------------------------------------------------------------------
+# whole-buffer / whole-pool comparison of pools far larger than host memory
+
+
+class PoolModel:
+    """What a device pool must hold at any moment: its generated content, then every scatter in
+    order.  Nothing is kept but the id lists: content is regenerated for the blocks asked for,
+    and the scattered bytes are put in place by the oracle's scatter."""
+
+    def __init__(self, kv: W.KVSpec):
+        self.kv = kv
+        self.history = []                    # (position of each block in the id list or -1, seed)
+
+    def scattered(self, ids: np.ndarray, seed: int) -> None:
+        """A transfer buffer holding stream `seed` (item i = bytes [i, i+1) * block_bytes) was
+        scattered to `ids`."""
+        where = np.full(self.kv.num_blocks, -1, dtype=np.int64)
+        ok = np.nonzero(ids < self.kv.num_blocks)[0]
+        where[ids[ok]] = ok
+        self.history.append((where, seed))
+
+    def mini_pool(self, blocks: np.ndarray):
+        """(bytes, oracle layout) of a pool of len(blocks) blocks, in the real pool's physical
+        layout, holding what those blocks must hold now."""
+        from workloads import synth
+
+        kv, k = self.kv, len(blocks)
+        bb = kv.block_bytes
+        if k and int(blocks[-1]) - int(blocks[0]) == k - 1 and (np.diff(blocks) == 1).all():
+            mini = W.physical_blocks(kv, int(blocks[0]), int(blocks[0]) + k)
+        else:
+            mini = W.logical_blocks(kv, blocks)
+            if kv.layout == 1:
+                t = mini.reshape(k, kv.num_layers, kv.tile_bytes)
+                mini = np.ascontiguousarray(t.transpose(1, 0, 2)).reshape(-1)
+        lay = kv_layout_oracle(kv, num_blocks=k)
+        for where, seed in self.history:
+            pos = where[blocks]
+            sel = np.nonzero(pos >= 0)[0]
+            if len(sel) == 0:
+                continue
+            items = np.empty((len(sel), bb), dtype=np.uint8)
+            for j, p in enumerate(pos[sel]):
+                synth.fill_host(items[j], seed, int(p) * bb)
+            rc, bad = oracle.kv_scatter(mini, lay, sel.astype(np.uint32), items.reshape(-1))
+            assert rc == oracle.OK and bad == 0
+        return mini, lay
+
+
+def _same_bytes(a: np.ndarray, b: np.ndarray) -> bool:
+    if a.size != b.size:
+        return False
+    if a.size % 8 == 0 and a.ctypes.data % 8 == 0 and b.ctypes.data % 8 == 0:
+        return bool(np.array_equal(a.view(np.uint64), b.view(np.uint64)))
+    return bool(np.array_equal(a, b))
+
+
+class _ChunkedCompare:
+    """Device bytes come back chunk by chunk through a ring of pinned host buffers (main
+    thread) while worker threads regenerate what each chunk must hold and compare; the native
+    generator, the oracle and numpy all release the interpreter lock."""
+
+    def __init__(self, chunk_bytes: int, workers=None):
+        import concurrent.futures
+        import os
+        import queue
+
+        self.workers = workers or max(2, min(12, (os.cpu_count() or 4) - 2))
+        self.pool = concurrent.futures.ThreadPoolExecutor(self.workers)
+        self.free = queue.Queue()
+        for _ in range(self.workers + 2):
+            stage = torch.empty(chunk_bytes, dtype=torch.uint8)
+            self.free.put(stage.pin_memory() if torch.cuda.is_available() else stage)
+        self.pending = []
+        self.bad = []
+
+    def submit(self, dev_bytes: torch.Tensor, expect, tag):
+        """expect() -> the bytes this chunk must hold (runs in a worker thread)."""
+        stage = self.free.get()
+        n = dev_bytes.numel()
+        stage[:n].copy_(dev_bytes)                        # pinned: a plain synchronous copy
+
+        def work():
+            try:
+                if not _same_bytes(stage[:n].numpy(), expect()):
+                    self.bad.append(tag)
+            finally:
+                self.free.put(stage)
+
+        self.pending.append(self.pool.submit(work))
+
+    def finish(self):
+        for f in self.pending:
+            f.result()
+        self.pool.shutdown()
+        return self.bad
+
+
+def check_gather_full(model: PoolModel, ids: np.ndarray, buf_d: torch.Tensor, chunk_bytes=160 << 20):
+    """EVERY byte of a gathered transfer buffer against the oracle's gather from a regenerated
+    mini pool of the blocks each chunk names.  Returns the list of failing chunks (empty = ok)."""
+    kv = model.kv
+    bb = kv.block_bytes
+    per = max(1, chunk_bytes // bb)
+    cmp = _ChunkedCompare(per * bb)
+
+    def expect_for(sub):
+        def expect():
+            want = np.zeros(len(sub) * bb, dtype=np.uint8)
+            valid = sub < kv.num_blocks
+            mini, lay = model.mini_pool(sub[valid])
+            local = np.full(len(sub), NO_BLOCK, dtype=np.uint32)
+            local[valid] = np.arange(int(valid.sum()), dtype=np.uint32)
+            rc, bad = oracle.kv_gather(mini, lay, local, want)
+            assert rc == oracle.OK
+            return want
+        return expect
+
+    for i0 in range(0, len(ids), per):
+        i1 = min(i0 + per, len(ids))
+        cmp.submit(buf_d[i0 * bb: i1 * bb], expect_for(ids[i0:i1]), ("items", i0, i1))
+    return cmp.finish()
+
+
+def check_pool_full(model: PoolModel, pool_d: torch.Tensor, chunk_bytes=160 << 20):
+    """EVERY byte of a device pool against the model: generated content where nothing was
+    scattered, the oracle's scatter of the regenerated buffers elsewhere."""
+    kv = model.kv
+    bb = kv.block_bytes
+    per = max(1, chunk_bytes // bb)
+    cmp = _ChunkedCompare(per * bb)
+    for b0 in range(0, kv.num_blocks, per):
+        b1 = min(b0 + per, kv.num_blocks)
+        if kv.layout == 0:
+            part = pool_d[b0 * bb: b1 * bb]
+        else:
+            part = pool_d.view(kv.num_layers, kv.num_blocks, kv.tile_bytes)[:, b0:b1].contiguous().view(-1)
+        blocks = np.arange(b0, b1, dtype=np.int64)
+        cmp.submit(part, (lambda bl: (lambda: model.mini_pool(bl)[0]))(blocks), ("blocks", b0, b1))
+    return cmp.finish()

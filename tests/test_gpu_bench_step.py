@@ -1,7 +1,7 @@
 """The step that bench.py times, at the benchmark's full size and in its launch configuration
 (route_head, collect, device-counted gather and scatter; the tail of the hash chains and the index
 publish/expire on a second stream), checked against the oracle: routing outputs element by element, the gathered buffer
-and the pool on sampled blocks, and the index back in its start state."""
+and the pool byte for byte, and the index back in its start state."""
 import os
 import sys
 
@@ -10,8 +10,8 @@ import pytest
 import torch
 
 import oracle
-from gpu_util import fill_entries, host
-from paper_2504_03648_b200 import workloads as W
+from gpu_util import PoolModel, check_gather_full, check_pool_full, fill_entries, host
+import workloads as W
 
 pytestmark = pytest.mark.gpu
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -58,6 +58,12 @@ def test_bench_step_matches_oracle():
         oracle.kv_gather(mini, lay1, np.zeros(1, np.uint32), want)
         assert np.array_equal(host(buf[i]), want)
         assert np.array_equal(host(pool[int(uniq[i])]), mini)
+
+    # every byte of the gathered buffer and of the pool (the scatter wrote the gathered bytes
+    # back where they came from, so the pool must hold its generated content everywhere)
+    model = PoolModel(kv)
+    assert check_gather_full(model, uniq[:cnt], job.d_buf[: cnt * kv.block_bytes]) == []
+    assert check_pool_full(model, job.d_pool) == []
 
     # the published batch was expired again: index as at the start
     assert job.index.stats()[0] == live0 == ox.stats()[0]

@@ -1,15 +1,17 @@
 """GPU parity, data-movement half of the path: paged-KV gather and scatter against the CPU
-oracle, byte for byte, through the C ABI - small pools in full, the large configurations at
-full size on sampled blocks."""
+oracle, byte for byte, through the C ABI - small pools in full, and the large configurations at
+full size: every byte of a gathered buffer and of the whole pool (regenerated on the host chunk
+by chunk and passed through the oracle), plus sampled blocks after every other call."""
 import numpy as np
 import pytest
 import torch
 
 import oracle
-from gpu_util import (NO_BLOCK, dev, empty, host, kv_layout_gpu, kv_layout_oracle, read_block)
+from gpu_util import (NO_BLOCK, PoolModel, check_gather_full, check_pool_full, dev, empty, host,
+                      kv_layout_gpu, kv_layout_oracle, read_block)
 from paper_2504_03648_b200 import binding as aibx
-from paper_2504_03648_b200 import synth
-from paper_2504_03648_b200 import workloads as W
+from workloads import synth
+import workloads as W
 
 pytestmark = pytest.mark.gpu
 
@@ -188,7 +190,9 @@ def test_cfg2_full_size():
     assert aibx.status_fetch() == (0, 0)
     sample = np.concatenate([[0, 1, n - 1], W.Stream(7, 9).randint(0, n, 9)])
     _sample_gather_check(kv, kv, ids, buf, sample)
-    # whole-buffer property: device-side comparison with the pool rows it names
+    model = PoolModel(kv)
+    assert check_gather_full(model, ids, buf) == []                # every byte, against the oracle
+    # and the same property on the device: the buffer rows equal the pool rows they name
     got = buf.view(n, kv.block_bytes)
     src = pool.view(kv.num_blocks, kv.block_bytes)
     idx = dev(ids.astype(np.int64))
@@ -202,6 +206,8 @@ def test_cfg2_full_size():
     synth.fill_linear(buf, 1234)
     aibx.kv_scatter(pool, lay, dev(ids), n, buf)
     assert aibx.status_fetch() == (0, 0)
+    model.scattered(ids, 1234)
+    assert check_pool_full(model, pool) == []                      # all 8 GiB
     for i in sample[:6]:
         mini = np.zeros(kv.block_bytes, dtype=np.uint8)
         item = W.pool_bytes(1234, int(i) * kv.block_bytes, kv.block_bytes)
@@ -218,44 +224,37 @@ def test_cfg4_full_size_layer_major():
     synth.fill_pool(pool, kv)
     buf = empty(n * kv.block_bytes, torch.uint8)
     lay = kv_layout_gpu(kv)
-    history = []                                                   # (ids, content seed) of every scatter
-
-    def block_now(b):
-        """What block b must hold: the newest scatter that named it, else the generated content.
-        The scattered bytes go through the oracle (one-block pool) rather than being retyped."""
-        for ids_h, seed_h in reversed(history):
-            pos = np.nonzero(ids_h == b)[0]
-            if len(pos):
-                item = W.pool_bytes(seed_h, int(pos[0]) * kv.block_bytes, kv.block_bytes)
-                mini = np.zeros(kv.block_bytes, dtype=np.uint8)
-                oracle.kv_scatter(mini, kv_layout_oracle(kv, layout=0, num_blocks=1),
-                                  np.zeros(1, np.uint32), item)
-                return mini
-        return W.logical_blocks(kv, [b])
+    model = PoolModel(kv)                                          # generated content + scatters
 
     for it in range(4):                                            # put, get, put, get
         ids = W.distinct_ids(1000 + it, kv.num_blocks, n)
         sample = np.concatenate([[0, n - 1], W.Stream(it, 11).randint(0, n, 4)])
         if it % 2 == 0:
             aibx.kv_gather(pool, lay, dev(ids), n, buf)
-            lay1 = kv_layout_oracle(kv, layout=0, num_blocks=1)
-            for i in sample:
-                want = np.zeros(kv.block_bytes, dtype=np.uint8)
-                oracle.kv_gather(block_now(int(ids[int(i)])), lay1, np.zeros(1, np.uint32), want)
-                assert np.array_equal(host(buf.view(n, kv.block_bytes)[int(i)]), want)
+            if it == 2:
+                # every byte of this buffer (by now 2,048 blocks of the pool hold scattered
+                # content, about a tenth of which this gather names)
+                assert check_gather_full(model, ids, buf) == []
+            else:
+                picked = ids[sample]
+                mini, lay_m = model.mini_pool(picked)
+                want = np.zeros(len(sample) * kv.block_bytes, dtype=np.uint8)
+                oracle.kv_gather(mini, lay_m, np.arange(len(sample), dtype=np.uint32), want)
+                want = want.reshape(len(sample), kv.block_bytes)
+                for j, i in enumerate(sample):
+                    assert np.array_equal(host(buf.view(n, kv.block_bytes)[int(i)]), want[j])
         else:
             synth.fill_linear(buf, 5000 + it)
             aibx.kv_scatter(pool, lay, dev(ids), n, buf)
-            history.append((ids, 5000 + it))
+            model.scattered(ids, 5000 + it)
             for i in sample:
                 b = int(ids[int(i)])
-                assert np.array_equal(read_block(pool, kv, b), block_now(b))
+                mini, _ = model.mini_pool(np.array([b]))           # one block: layouts coincide
+                assert np.array_equal(read_block(pool, kv, b), mini)
         assert aibx.status_fetch() == (0, 0)
-    # a block no scatter named still holds its generated content
-    all_scattered = set(W.distinct_ids(1001, kv.num_blocks, n).tolist()) | set(
-        W.distinct_ids(1003, kv.num_blocks, n).tolist())
-    b = next(x for x in range(kv.num_blocks) if x not in all_scattered)
-    assert np.array_equal(read_block(pool, kv, b), W.logical_blocks(kv, [b]))
+    # every byte of the pool: scattered blocks hold what the oracle's scatter puts there, all
+    # others their generated content
+    assert check_pool_full(model, pool) == []
     print("cfg4 pool blocks used:", kv.num_blocks, "(shrunk)" if shrunk else "(full)")
 
 
@@ -361,6 +360,7 @@ def test_cfg5_full_size_fp8_mixed():
     lay = kv_layout_gpu(kv)
     get_buf = empty(n_get * kv.block_bytes, torch.uint8)
     put_buf = empty(n_put * kv.block_bytes, torch.uint8)
+    model = PoolModel(kv)
     for r in (0, 13, 31):
         table = (r * per + W.Stream(4, 100 + r).permutation(per)).astype(np.uint32)
         ids_get, ids_put = table[:n_get], table[n_get:]
@@ -368,14 +368,15 @@ def test_cfg5_full_size_fp8_mixed():
         synth.fill_linear(put_buf, 900 + r)
         aibx.kv_scatter(pool, lay, dev(ids_put), n_put, put_buf)
         assert aibx.status_fetch() == (0, 0)
-        sample = np.array([0, n_get - 1, n_get // 2])
-        _sample_gather_check(kv, kv, ids_get, get_buf, sample)
+        if r == 13:
+            assert check_gather_full(model, ids_get, get_buf) == []      # every byte
+        else:
+            _sample_gather_check(kv, kv, ids_get, get_buf, np.array([0, n_get - 1, n_get // 2]))
+        model.scattered(ids_put, 900 + r)
         for i in (0, n_put - 1):
-            item = W.pool_bytes(900 + r, i * kv.block_bytes, kv.block_bytes)
-            mini = np.zeros(kv.block_bytes, dtype=np.uint8)
-            oracle.kv_scatter(mini, kv_layout_oracle(kv, layout=0, num_blocks=1),
-                              np.zeros(1, np.uint32), item)
-            assert np.array_equal(read_block(pool, kv, int(ids_put[i])), mini)
+            b = int(ids_put[i])
+            assert np.array_equal(read_block(pool, kv, b), model.mini_pool(np.array([b]))[0])
+    assert check_pool_full(model, pool) == []                            # every byte of the pool
     print("cfg5 pool blocks used:", kv.num_blocks, "(shrunk)" if shrunk else "(full)")
 
 

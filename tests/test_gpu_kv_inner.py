@@ -7,8 +7,8 @@ import torch
 import oracle
 from gpu_util import NO_BLOCK, dev, empty, host, kv_layout_gpu, kv_layout_oracle
 from paper_2504_03648_b200 import binding as aibx
-from paper_2504_03648_b200 import synth
-from paper_2504_03648_b200 import workloads as W
+from workloads import synth
+import workloads as W
 
 pytestmark = pytest.mark.gpu
 

@@ -9,7 +9,7 @@ import torch
 import oracle
 from gpu_util import NO_BLOCK, dev, empty, fill_entries, gpu_hash, host, routing_oracle
 from paper_2504_03648_b200 import binding as aibx
-from paper_2504_03648_b200 import workloads as W
+import workloads as W
 
 pytestmark = pytest.mark.gpu
 ALL = (1 << 64) - 1

@@ -11,7 +11,7 @@ import oracle
 from gpu_util import (NO_BLOCK, assert_routing_equal, dev, empty, gpu_hash, host, routing_gpu,
                       routing_oracle)
 from paper_2504_03648_b200 import binding as aibx
-from paper_2504_03648_b200 import workloads as W
+import workloads as W
 
 pytestmark = pytest.mark.gpu
 ALL = (1 << 64) - 1

@@ -1,7 +1,11 @@
 """The synthetic input generator: determinism and the structure the configurations state."""
+import os
+
 import numpy as np
 
-from paper_2504_03648_b200 import workloads as W
+import workloads as W
+from workloads import build as synth_build
+from workloads import synth
 
 
 def test_mix64_is_stateless_and_sliceable():
@@ -74,3 +78,29 @@ def test_kv_specs_and_host_pool_layouts():
     bits = W.bf16_normal_bits(0, 10000).astype(np.uint32) << 16
     x = bits.view(np.float32)
     assert abs(x.mean()) < 0.05 and abs(x.std() - 1.0) < 0.05
+
+
+def test_native_host_twin_equals_the_numpy_generator():
+    synth_build.build()
+    for seed, first, n in [(3, 0, 4096), (5003, 8 * 12345, 8 * 777), (2 ** 40 + 1, 5 << 33, 64)]:
+        out = np.zeros(n, dtype=np.uint8)
+        synth.fill_host(out, seed, first)
+        assert np.array_equal(out, W.pool_bytes(seed, first, n))
+    kv = W.KVSpec("t", 9, 1, 3, 1, 2, 8, 1, 5)
+    p = W.physical_blocks(kv, 1, 4).reshape(3, 3, kv.tile_bytes)          # [layer][block][tile]
+    whole = W.host_pool(kv).reshape(3, 5, kv.tile_bytes)
+    assert np.array_equal(p, whole[:, 1:4])
+    kv0 = W.scaled(kv, layout=0)
+    assert np.array_equal(W.physical_blocks(kv0, 1, 4), W.host_pool(kv0)[kv.block_bytes: 4 * kv.block_bytes])
+
+
+def test_generators_hold_no_method_code():
+    """The generator package is shared by the CPU checker's tests and the GPU tests, so it must
+    name neither side."""
+    pkg = os.path.dirname(os.path.abspath(W.__file__))
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "aibxo" not in text and "import oracle" not in text, f
+                assert "paper_2504_03648_b200" not in text and "aibx.h" not in text, f

@@ -311,10 +311,27 @@ def host_pool(kv: KVSpec) -> np.ndarray:
 def logical_blocks(kv: KVSpec, ids) -> np.ndarray:
     """Content of the given blocks as a block-major mini-pool [len(ids) * block_bytes]."""
     assert kv.content == "mix64"
+    from . import synth
+
     out = np.empty((len(ids), kv.block_bytes), dtype=np.uint8)
     for j, b in enumerate(ids):
-        out[j] = pool_bytes(kv.seed, int(b) * kv.block_bytes, kv.block_bytes)
+        synth.fill_host(out[j], kv.seed, int(b) * kv.block_bytes)   # == pool_bytes(...), natively
     return out.reshape(-1)
+
+
+def physical_blocks(kv: KVSpec, b0: int, b1: int) -> np.ndarray:
+    """Generated content of blocks [b0, b1) laid out as a pool of b1 - b0 blocks in kv's
+    PHYSICAL layout (what a slice of the real pool holds before anything is scattered)."""
+    assert kv.content == "mix64"
+    from . import synth
+
+    n = b1 - b0
+    logical = np.empty(n * kv.block_bytes, dtype=np.uint8)
+    synth.fill_host(logical, kv.seed, b0 * kv.block_bytes)
+    if kv.layout == 0:
+        return logical
+    t = logical.reshape(n, kv.num_layers, kv.tile_bytes)
+    return np.ascontiguousarray(t.transpose(1, 0, 2)).reshape(-1)
 
 
 def distinct_ids(seed: int, num_blocks: int, n: int) -> np.ndarray:

@@ -1,6 +1,8 @@
-// Device-side twin of the synthetic input generator (workloads.py): fills KV pools and
-// transfer buffers far too large to generate on the host.  Input generation only - none of
-// the library's own operations is implemented here, and libaibx does not link this file.
+// Native twins of the synthetic input generator (the Python module beside this folder): a
+// device kernel that fills KV pools and transfer buffers far too large to generate on the host,
+// and a plain host loop for tests that regenerate such content chunk by chunk.  Input
+// generation only - none of the library's own operations is implemented here, and libaibx does
+// not link this file.
 //
 // Logical content: 64-bit word w of the block-major byte stream [block][layer][tile] equals
 // splitmix64's output function of (w + 1) * GOLD + seed * SEEDMUL, stored little-endian.  A
@@ -10,7 +12,7 @@
 
 namespace {
 
-__device__ __forceinline__ unsigned long long mix64(unsigned long long seed,
+__host__ __device__ __forceinline__ unsigned long long mix64(unsigned long long seed,
                                                     unsigned long long counter) {
   unsigned long long z = (counter + 1ULL) * 0x9E3779B97F4A7C15ULL + seed * 0xD1B54A32D192ED03ULL;
   z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
@@ -52,6 +54,18 @@ int32_t aibx_synth_fill_linear(void* d_dst, uint64_t n_bytes, uint64_t seed, uin
   fill_kernel<<<148 * 16, 256, 0, static_cast<cudaStream_t>(stream)>>>(
       static_cast<unsigned long long*>(d_dst), n_bytes / 8, seed, first_byte / 8, 0, 1, 1, 1);
   return cudaPeekAtLastError() == cudaSuccess ? 0 : -4;
+}
+
+// The same stream written by the calling host thread: h_dst (host memory, 8-byte aligned) <-
+// bytes [first_byte, first_byte + n_bytes) of stream `seed`.  No CUDA call is made.
+int32_t aibx_synth_fill_host(void* h_dst, uint64_t n_bytes, uint64_t seed, uint64_t first_byte) {
+  if (!h_dst || (n_bytes & 7) || (first_byte & 7) || (reinterpret_cast<uintptr_t>(h_dst) & 7))
+    return -1;
+  unsigned long long* dst = static_cast<unsigned long long*>(h_dst);
+  const unsigned long long first_word = first_byte / 8;
+  const unsigned long long n_words = n_bytes / 8;
+  for (unsigned long long w = 0; w < n_words; ++w) dst[w] = mix64(seed, first_word + w);
+  return 0;
 }
 
 // Whole pool in its physical layout (0 block-major, 1 layer-major); tile_bytes multiple of 8.

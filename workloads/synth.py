@@ -1,11 +1,12 @@
-"""Device-side synthetic KV content (ctypes binding of libaibx_synth.so): the GPU twin of
-``workloads.pool_bytes`` for pools too large to generate on the host.  Input generation only."""
+"""Native synthetic KV content (ctypes binding of libaibx_synth.so): the GPU twin of
+``workloads.pool_bytes`` for pools too large to generate on the host, and a native host twin
+for tests that regenerate such pools chunk by chunk.  Input generation only."""
 from __future__ import annotations
 
 import ctypes as C
 import os
 
-import torch
+import numpy as np
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libaibx_synth.so")
@@ -16,19 +17,33 @@ def lib():
     global _lib
     if _lib is None:
         if not os.path.exists(LIB_PATH):
-            raise RuntimeError("libaibx_synth.so is missing: run `python -m paper_2504_03648_b200.build`")
+            raise RuntimeError("libaibx_synth.so is missing: run `python -m workloads.build`")
         L = C.CDLL(LIB_PATH)
         L.aibx_synth_fill_linear.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_void_p]
         L.aibx_synth_fill_linear.restype = C.c_int32
         L.aibx_synth_fill_pool.argtypes = [C.c_void_p, C.c_uint64, C.c_int32, C.c_uint64, C.c_uint64,
                                            C.c_uint64, C.c_void_p]
         L.aibx_synth_fill_pool.restype = C.c_int32
+        L.aibx_synth_fill_host.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64]
+        L.aibx_synth_fill_host.restype = C.c_int32
         _lib = L
     return _lib
 
 
-def fill_linear(t: torch.Tensor, seed: int, first_byte: int = 0) -> None:
+def fill_host(out: np.ndarray, seed: int, first_byte: int = 0) -> None:
+    """out (contiguous uint8 host array) <- bytes [first_byte, first_byte + out.size) of stream
+    `seed`: what ``workloads.pool_bytes`` returns, about fifty times faster.  The call releases
+    the interpreter lock, so several threads can fill disjoint arrays at once."""
+    assert out.dtype == np.uint8 and out.flags.c_contiguous and out.flags.writeable
+    rc = lib().aibx_synth_fill_host(out.ctypes.data, out.size, seed, first_byte)
+    if rc != 0:
+        raise RuntimeError("aibx_synth_fill_host -> %d" % rc)
+
+
+def fill_linear(t, seed: int, first_byte: int = 0) -> None:
     """t (any dtype, contiguous, CUDA) <- bytes [first_byte, first_byte + nbytes) of stream `seed`."""
+    import torch
+
     assert t.is_cuda and t.is_contiguous()
     rc = lib().aibx_synth_fill_linear(t.data_ptr(), t.numel() * t.element_size(), seed, first_byte,
                                       torch.cuda.current_stream().cuda_stream)
@@ -36,8 +51,10 @@ def fill_linear(t: torch.Tensor, seed: int, first_byte: int = 0) -> None:
         raise RuntimeError("aibx_synth_fill_linear -> %d" % rc)
 
 
-def fill_pool(pool: torch.Tensor, kv) -> None:
+def fill_pool(pool, kv) -> None:
     """Fill a whole pool (KVSpec `kv`) with its logical content in its physical layout."""
+    import torch
+
     assert pool.is_cuda and pool.is_contiguous()
     assert pool.numel() * pool.element_size() == kv.pool_bytes
     rc = lib().aibx_synth_fill_pool(pool.data_ptr(), kv.seed, kv.layout, kv.num_layers,
