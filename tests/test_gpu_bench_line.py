@@ -41,4 +41,24 @@ def test_bench_line_contract():
     assert d["gpu_launches"] == 9 * d["steps"]
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and c["unit"] == d["unit"]
+    assert c["cpu"] and c["all_cores"]["cores"] == c["cores_available"] >= 1
+    assert c["all_cores"]["value"] > 0 and c["all_cores"]["unit"] == d["unit"]
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"} and d["clocks"]["sm_max_mhz"] > 0
+    # sibling records: the largest KV configurations, each with a roofline of its own
+    for key, kernel_launches in (("kv_cfg4", 100), ("kv_cfg5", 64)):
+        k = d[key]
+        assert k["status"] == [0, 0] and "workload" in k
+        assert k["pool_blocks_effective"] <= k["pool_blocks_configured"]
+        r = k["roofline"]
+        assert r["bound"] == "hbm" and r["launches_timed"] == kernel_launches
+        assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-3 and 0.3 < r["frac"] < 1.2
+        assert abs(r["achieved"] - r["algorithmic_bytes_per_launch"] / (r["avg_launch_ms"] * 1e-3) / 1e9) \
+            < 0.01 * r["achieved"]
+    big = d["prefix_match_large_index"]
+    assert [b["index_slots"] for b in big] == [1 << 19, 1 << 21, 1 << 23]
+    for b in big:
+        row = b["results"][-1]
+        assert row["lookups"] == row["R"] * 64 and 0 < row["frac"] < 1.2
+        assert b["random_32B_read_ceiling_Greads_per_s"] > 1
+        assert 0 < row["frac_of_random_read_ceiling"] < 1.5
+    assert len(d["index_lookup_flat"]["results"]) == 4

@@ -231,18 +231,9 @@ def test_cfg4_full_size_layer_major():
         sample = np.concatenate([[0, n - 1], W.Stream(it, 11).randint(0, n, 4)])
         if it % 2 == 0:
             aibx.kv_gather(pool, lay, dev(ids), n, buf)
-            if it == 2:
-                # every byte of this buffer (by now 2,048 blocks of the pool hold scattered
-                # content, about a tenth of which this gather names)
-                assert check_gather_full(model, ids, buf) == []
-            else:
-                picked = ids[sample]
-                mini, lay_m = model.mini_pool(picked)
-                want = np.zeros(len(sample) * kv.block_bytes, dtype=np.uint8)
-                oracle.kv_gather(mini, lay_m, np.arange(len(sample), dtype=np.uint32), want)
-                want = want.reshape(len(sample), kv.block_bytes)
-                for j, i in enumerate(sample):
-                    assert np.array_equal(host(buf.view(n, kv.block_bytes)[int(i)]), want[j])
+            # every byte of the buffer (from the second put on, a tenth of the ids name blocks
+            # that hold scattered content)
+            assert check_gather_full(model, ids, buf) == []
         else:
             synth.fill_linear(buf, 5000 + it)
             aibx.kv_scatter(pool, lay, dev(ids), n, buf)
@@ -368,10 +359,7 @@ def test_cfg5_full_size_fp8_mixed():
         synth.fill_linear(put_buf, 900 + r)
         aibx.kv_scatter(pool, lay, dev(ids_put), n_put, put_buf)
         assert aibx.status_fetch() == (0, 0)
-        if r == 13:
-            assert check_gather_full(model, ids_get, get_buf) == []      # every byte
-        else:
-            _sample_gather_check(kv, kv, ids_get, get_buf, np.array([0, n_get - 1, n_get // 2]))
+        assert check_gather_full(model, ids_get, get_buf) == []          # every byte
         model.scattered(ids_put, 900 + r)
         for i in (0, n_put - 1):
             b = int(ids_put[i])

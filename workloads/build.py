@@ -6,7 +6,7 @@ import os
 import subprocess
 
 PKG = os.path.dirname(os.path.abspath(__file__))
-SRC = os.path.join(PKG, "csrc", "synth_fill.cu")
+SRCS = [os.path.join(PKG, "csrc", f) for f in ("synth_fill.cu", "mem_probe.cu")]
 SYNTH_LIB = os.path.join(PKG, "libaibx_synth.so")
 
 NVCC_FLAGS = [
@@ -17,9 +17,9 @@ NVCC_FLAGS = [
 
 def build(force: bool = False) -> None:
     if (not force and os.path.exists(SYNTH_LIB)
-            and os.path.getmtime(SYNTH_LIB) >= os.path.getmtime(SRC)):
+            and os.path.getmtime(SYNTH_LIB) >= max(os.path.getmtime(f) for f in SRCS)):
         return
-    subprocess.check_call(["nvcc"] + NVCC_FLAGS + [SRC, "-o", SYNTH_LIB + ".tmp"])
+    subprocess.check_call(["nvcc"] + NVCC_FLAGS + SRCS + ["-o", SYNTH_LIB + ".tmp"])
     os.replace(SYNTH_LIB + ".tmp", SYNTH_LIB)
 
 

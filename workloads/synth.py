@@ -26,6 +26,9 @@ def lib():
         L.aibx_synth_fill_pool.restype = C.c_int32
         L.aibx_synth_fill_host.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64]
         L.aibx_synth_fill_host.restype = C.c_int32
+        L.aibx_probe_random_reads.argtypes = [C.c_void_p, C.c_uint64, C.c_int32, C.c_int32,
+                                              C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
+        L.aibx_probe_random_reads.restype = C.c_int32
         _lib = L
     return _lib
 
@@ -62,3 +65,18 @@ def fill_pool(pool, kv) -> None:
                                     torch.cuda.current_stream().cuda_stream)
     if rc != 0:
         raise RuntimeError("aibx_synth_fill_pool -> %d" % rc)
+
+
+def probe_random_reads(base, ws_bytes: int, gran: int, per: int, n_reads: int, seed, sink) -> None:
+    """Memory-system probe (no method code): n_reads uniformly random, aligned reads of `gran`
+    bytes (32 / 64 / 128) over the first ws_bytes (a power of two) of the CUDA tensor `base`,
+    `per` independent reads per thread; `sink` (uint64, n_reads / (32 * per) + 1 words) keeps the
+    loads alive.  Enqueued on the current stream."""
+    import torch
+
+    assert base.is_cuda and sink.is_cuda and base.numel() * base.element_size() >= ws_bytes
+    assert sink.numel() * sink.element_size() >= 8 * (n_reads // (32 * per) + 1)
+    rc = lib().aibx_probe_random_reads(base.data_ptr(), ws_bytes, gran, per, n_reads, seed,
+                                       sink.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    if rc != 0:
+        raise RuntimeError("aibx_probe_random_reads -> %d" % rc)
