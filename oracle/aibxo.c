@@ -573,14 +573,24 @@ static int64_t tile_bytes(const aibxo_kv_layout_t* L) {
 }
 
 static int layout_ok(const aibxo_kv_layout_t* L) {
-  return L && (L->layout == 0 || L->layout == 1) && L->num_layers > 0 && L->num_kv_heads > 0 &&
+  return L && L->layout >= 0 && L->layout <= 2 && L->num_layers > 0 && L->num_kv_heads > 0 &&
          L->block_tokens > 0 && L->head_dim > 0 && L->elem_bytes > 0;
 }
 
-static int64_t pool_offset(const aibxo_kv_layout_t* L, uint32_t b, int32_t l) {
-  int64_t t = tile_bytes(L);
-  if (L->layout == 0) return ((int64_t)b * L->num_layers + l) * t;
-  return ((int64_t)l * L->num_blocks + b) * t;
+/* Where the K (kv = 0) or V (kv = 1) half of the tile of (block b, layer l) starts in the pool.
+ *   layout 0  [block][layer][K/V][head][token][dim]
+ *   layout 1  [layer][block][K/V][head][token][dim]
+ *   layout 2  [layer][K/V][block][head][token][dim]   (K and V of a layer are separate tensors) */
+static int64_t pool_offset(const aibxo_kv_layout_t* L, uint32_t b, int32_t l, int32_t kv) {
+  int64_t half = tile_bytes(L) / 2;
+  if (L->layout == 0) return (((int64_t)b * L->num_layers + l) * 2 + kv) * half;
+  if (L->layout == 1) return (((int64_t)l * L->num_blocks + b) * 2 + kv) * half;
+  return (((int64_t)l * 2 + kv) * L->num_blocks + b) * half;
+}
+
+/* The buffer is always [item][layer][K/V][head][token][dim]. */
+static int64_t buf_offset(const aibxo_kv_layout_t* L, int64_t i, int32_t l, int32_t kv) {
+  return ((i * L->num_layers + l) * 2 + kv) * (tile_bytes(L) / 2);
 }
 
 int32_t aibxo_kv_gather(const void* pool, const aibxo_kv_layout_t* L, const uint32_t* ids,
@@ -589,15 +599,15 @@ int32_t aibxo_kv_gather(const void* pool, const aibxo_kv_layout_t* L, const uint
   if (!layout_ok(L) || n < 0) return AIBXO_ERR_INVALID;
   if (n == 0) return AIBXO_OK;
   if (!pool || !ids || !buf) return AIBXO_ERR_INVALID;
-  int64_t t = tile_bytes(L);
+  int64_t half = tile_bytes(L) / 2;
   int64_t nbad = 0;
   for (int64_t i = 0; i < n; ++i) {
     if (ids[i] == AIBXO_NO_BLOCK) continue;
     if (ids[i] >= L->num_blocks) { ++nbad; continue; }
-    for (int32_t l = 0; l < L->num_layers; ++l) {
-      memcpy((uint8_t*)buf + (i * L->num_layers + l) * t,
-             (const uint8_t*)pool + pool_offset(L, ids[i], l), (size_t)t);
-    }
+    for (int32_t l = 0; l < L->num_layers; ++l)
+      for (int32_t kv = 0; kv < 2; ++kv)
+        memcpy((uint8_t*)buf + buf_offset(L, i, l, kv),
+               (const uint8_t*)pool + pool_offset(L, ids[i], l, kv), (size_t)half);
   }
   if (bad) *bad = nbad;
   return nbad ? AIBXO_ERR_RANGE : AIBXO_OK;
@@ -609,29 +619,28 @@ int32_t aibxo_kv_scatter(void* pool, const aibxo_kv_layout_t* L, const uint32_t*
   if (!layout_ok(L) || n < 0) return AIBXO_ERR_INVALID;
   if (n == 0) return AIBXO_OK;
   if (!pool || !ids || !buf) return AIBXO_ERR_INVALID;
-  int64_t t = tile_bytes(L);
+  int64_t half = tile_bytes(L) / 2;
   int64_t nbad = 0;
   for (int64_t i = 0; i < n; ++i) {
     if (ids[i] == AIBXO_NO_BLOCK) continue;
     if (ids[i] >= L->num_blocks) { ++nbad; continue; }
-    for (int32_t l = 0; l < L->num_layers; ++l) {
-      memcpy((uint8_t*)pool + pool_offset(L, ids[i], l),
-             (const uint8_t*)buf + (i * L->num_layers + l) * t, (size_t)t);
-    }
+    for (int32_t l = 0; l < L->num_layers; ++l)
+      for (int32_t kv = 0; kv < 2; ++kv)
+        memcpy((uint8_t*)pool + pool_offset(L, ids[i], l, kv),
+               (const uint8_t*)buf + buf_offset(L, i, l, kv), (size_t)half);
   }
   if (bad) *bad = nbad;
   return nbad ? AIBXO_ERR_RANGE : AIBXO_OK;
 }
 
 /* ------------------------------------------------------------------ inner-order change - */
-/* Offset of row (kv, head, token) inside a tile stored in the given inner order. */
+/* Offset of row (head, token) inside the K or V half of a tile stored in the given inner order. */
 
-static int64_t row_offset(const aibxo_kv_layout_t* L, int32_t inner, int32_t kv, int32_t head,
-                          int32_t token) {
+static int64_t row_offset(const aibxo_kv_layout_t* L, int32_t inner, int32_t head, int32_t token) {
   int64_t row = (int64_t)L->head_dim * L->elem_bytes;
   int64_t H = L->num_kv_heads, T = L->block_tokens;
-  if (inner == 0) return (((int64_t)kv * H + head) * T + token) * row;
-  return (((int64_t)kv * T + token) * H + head) * row;
+  if (inner == 0) return ((int64_t)head * T + token) * row;
+  return ((int64_t)token * H + head) * row;
 }
 
 static int32_t copy_inner(uint8_t* pool, const aibxo_kv_layout_t* L, int32_t pool_inner,
@@ -643,24 +652,23 @@ static int32_t copy_inner(uint8_t* pool, const aibxo_kv_layout_t* L, int32_t poo
     return AIBXO_ERR_INVALID;
   if (n == 0) return AIBXO_OK;
   if (!pool || !ids || !buf) return AIBXO_ERR_INVALID;
-  int64_t t = tile_bytes(L);
   int64_t row = (int64_t)L->head_dim * L->elem_bytes;
   int64_t nbad = 0;
   for (int64_t i = 0; i < n; ++i) {
     if (ids[i] == AIBXO_NO_BLOCK) continue;
     if (ids[i] >= L->num_blocks) { ++nbad; continue; }
-    for (int32_t l = 0; l < L->num_layers; ++l) {
-      uint8_t* ptile = pool + pool_offset(L, ids[i], l);
-      uint8_t* btile = buf + (i * L->num_layers + l) * t;
-      for (int32_t kv = 0; kv < 2; ++kv)
+    for (int32_t l = 0; l < L->num_layers; ++l)
+      for (int32_t kv = 0; kv < 2; ++kv) {
+        uint8_t* phalf = pool + pool_offset(L, ids[i], l, kv);
+        uint8_t* bhalf = buf + buf_offset(L, i, l, kv);
         for (int32_t h = 0; h < L->num_kv_heads; ++h)
           for (int32_t tok = 0; tok < L->block_tokens; ++tok) {
-            uint8_t* prow = ptile + row_offset(L, pool_inner, kv, h, tok);
-            uint8_t* brow = btile + row_offset(L, buf_inner, kv, h, tok);
+            uint8_t* prow = phalf + row_offset(L, pool_inner, h, tok);
+            uint8_t* brow = bhalf + row_offset(L, buf_inner, h, tok);
             if (to_pool) memcpy(prow, brow, (size_t)row);
             else memcpy(brow, prow, (size_t)row);
           }
-    }
+      }
   }
   if (bad) *bad = nbad;
   return nbad ? AIBXO_ERR_RANGE : AIBXO_OK;

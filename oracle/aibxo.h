@@ -132,7 +132,8 @@ int32_t aibxo_collect_blocks(const uint32_t* block_ids, int64_t n, uint32_t num_
 
 /* Paged-KV gather / scatter (Section 3.2.5 put/get data movement). */
 typedef struct {
-  int32_t layout; /* 0 block-major, 1 layer-major */
+  int32_t layout; /* 0 [block][layer][K/V]..., 1 [layer][block][K/V]..., 2 [layer][K/V][block]...
+                     (K and V of a layer as separate tensors) */
   int32_t num_layers;
   int32_t num_kv_heads;
   int32_t block_tokens;

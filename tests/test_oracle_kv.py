@@ -14,6 +14,77 @@ def _pool(rng, layout, L, nb, tile):
     return rng.integers(0, 256, shape, dtype=np.uint8)
 
 
+def _split_pool(rng, L, nb, half):
+    """Layout 2: K and V of a layer are separate tensors, [layer][K/V][block][half tile]."""
+    return rng.integers(0, 256, (L, 2, nb, half), dtype=np.uint8)
+
+
+def test_split_kv_gather_is_index_select_per_plane():
+    rng = np.random.default_rng(77)
+    L, H, Bt, D, E, nb = 3, 2, 4, 8, 2, 19
+    half = H * Bt * D * E
+    pool = _split_pool(rng, L, nb, half)
+    ids = rng.integers(0, nb, 13).astype(np.uint32)
+    lay = oracle.kv_layout(2, L, H, Bt, D, E, nb)
+    buf = np.zeros(13 * L * 2 * half, dtype=np.uint8)
+    before = pool.copy()
+    rc, bad = oracle.kv_gather(pool.reshape(-1), lay, ids, buf)
+    assert rc == oracle.OK and bad == 0 and np.array_equal(pool, before)
+    # library form: select the blocks on the block axis, then bring the item axis to the front
+    tp = torch.from_numpy(pool)
+    want = torch.index_select(tp, 2, torch.from_numpy(ids.astype(np.int64)))    # [L][2][n][half]
+    want = want.permute(2, 0, 1, 3).contiguous()                                # [n][L][2][half]
+    assert np.array_equal(buf, want.numpy().reshape(-1))
+    # the same content held layer-major gathers to the same buffer
+    lm = np.ascontiguousarray(pool.transpose(0, 2, 1, 3))                       # [L][nb][2][half]
+    buf1 = np.zeros_like(buf)
+    oracle.kv_gather(lm.reshape(-1), oracle.kv_layout(1, L, H, Bt, D, E, nb), ids, buf1)
+    assert np.array_equal(buf, buf1)
+
+
+def test_split_kv_hand_example_and_scatter():
+    # 2 layers, 3 blocks, half tile of 1 byte... a row must hold 1 head x 1 token x 1 dim x 1 byte
+    lay = oracle.kv_layout(2, 2, 1, 1, 1, 1, 3)
+    # pool bytes [layer][K/V][block]: K of layer 0 = 0,1,2  V of layer 0 = 3,4,5  K1 = 6,7,8  V1 = 9,10,11
+    pool = np.arange(12, dtype=np.uint8)
+    buf = np.zeros(8, dtype=np.uint8)
+    rc, _ = oracle.kv_gather(pool, lay, np.array([2, 0], np.uint32), buf)
+    assert rc == oracle.OK
+    # item 0 = block 2: (l0 K, l0 V, l1 K, l1 V) = 2, 5, 8, 11; item 1 = block 0: 0, 3, 6, 9
+    assert buf.tolist() == [2, 5, 8, 11, 0, 3, 6, 9]
+    out = np.full(12, 0xEE, dtype=np.uint8)
+    rc, _ = oracle.kv_scatter(out, lay, np.array([1, NO_BLOCK, 0], np.uint32),
+                              np.arange(100, 112, dtype=np.uint8))
+    # item 0 (100..103) -> block 1, item 2 (108..111) -> block 0, block 2 untouched
+    assert out.tolist() == [108, 100, 0xEE, 109, 101, 0xEE, 110, 102, 0xEE, 111, 103, 0xEE]
+
+
+def test_split_kv_round_trips_and_inner_order():
+    rng = np.random.default_rng(78)
+    L, H, Bt, D, E, nb = 2, 3, 4, 8, 1, 11
+    row = D * E
+    half = H * Bt * row
+    pool = _split_pool(rng, L, nb, half)
+    lay = oracle.kv_layout(2, L, H, Bt, D, E, nb)
+    ids = rng.permutation(nb)[:7].astype(np.uint32)
+    buf = np.zeros(7 * L * 2 * half, dtype=np.uint8)
+    oracle.kv_gather(pool.reshape(-1), lay, ids, buf)
+    fresh = np.zeros_like(pool)
+    oracle.kv_scatter(fresh.reshape(-1), lay, ids, buf)
+    assert np.array_equal(fresh[:, :, ids], pool[:, :, ids])
+    rest = np.setdiff1d(np.arange(nb), ids)
+    assert not fresh[:, :, rest].any()
+    # inner-order change: [head][token] rows of every plane become [token][head]
+    got = np.zeros_like(buf)
+    rc, _ = oracle.kv_gather_inner(pool.reshape(-1), lay, 0, 1, ids, got)
+    assert rc == oracle.OK
+    want = buf.reshape(7, L, 2, H, Bt, row).transpose(0, 1, 2, 4, 3, 5)
+    assert np.array_equal(got, np.ascontiguousarray(want).reshape(-1))
+    back = np.zeros_like(pool)
+    oracle.kv_scatter_inner(back.reshape(-1), lay, 0, 1, ids, got)
+    assert np.array_equal(back[:, :, ids], pool[:, :, ids])
+
+
 @pytest.mark.parametrize("layout", [0, 1])
 def test_gather_is_index_select(layout):
     rng = np.random.default_rng(layout)

@@ -100,16 +100,32 @@ MUTANTS = [
     ("prefix_policy_no_fallback", "test_oracle_policy.py",
      "if (arg == AIBXO_NO_POD) arg = lowest_ready(value, P, ready_mask);", "", 0),
     ("layer_major_as_block_major", "test_oracle_kv.py",
-     "return ((int64_t)l * L->num_blocks + b) * t;", "return ((int64_t)b * L->num_layers + l) * t;", 0),
+     "if (L->layout == 1) return (((int64_t)l * L->num_blocks + b) * 2 + kv) * half;",
+     "if (L->layout == 1) return (((int64_t)b * L->num_layers + l) * 2 + kv) * half;", 0),
+    ("split_kv_as_layer_major", "test_oracle_kv.py",
+     "return (((int64_t)l * 2 + kv) * L->num_blocks + b) * half;",
+     "return (((int64_t)l * L->num_blocks + b) * 2 + kv) * half;", 0),
+    ("split_kv_planes_swapped", "test_oracle_kv.py",
+     "return (((int64_t)l * 2 + kv) * L->num_blocks + b) * half;",
+     "return (((int64_t)l * 2 + (1 - kv)) * L->num_blocks + b) * half;", 0),
+    ("split_kv_layer_stride_of_one_plane", "test_oracle_kv.py",
+     "return (((int64_t)l * 2 + kv) * L->num_blocks + b) * half;",
+     "return (((int64_t)l + kv) * L->num_blocks + b) * half;", 0),
     ("buffer_layer_major", "test_oracle_kv.py",
-     "memcpy((uint8_t*)buf + (i * L->num_layers + l) * t,",
-     "memcpy((uint8_t*)buf + (i + l * n) * t,", 0),
+     "return ((i * L->num_layers + l) * 2 + kv) * (tile_bytes(L) / 2);",
+     "return ((l * L->num_blocks + i) * 2 + kv) * (tile_bytes(L) / 2);", 0),
+    ("buffer_kv_outermost", "test_oracle_kv.py",
+     "return ((i * L->num_layers + l) * 2 + kv) * (tile_bytes(L) / 2);",
+     "return ((i * 2 + kv) * L->num_layers + l) * (tile_bytes(L) / 2);", 0),
     ("no_block_counts_as_error", "test_oracle_kv.py",
-     "if (ids[i] == AIBXO_NO_BLOCK) continue;\n    if (ids[i] >= L->num_blocks) { ++nbad; continue; }\n    for (int32_t l = 0; l < L->num_layers; ++l) {\n      memcpy((uint8_t*)buf",
-     "if (ids[i] >= L->num_blocks) { ++nbad; continue; }\n    for (int32_t l = 0; l < L->num_layers; ++l) {\n      memcpy((uint8_t*)buf", 0),
+     "if (ids[i] == AIBXO_NO_BLOCK) continue;\n    if (ids[i] >= L->num_blocks) { ++nbad; continue; }\n    for (int32_t l = 0; l < L->num_layers; ++l)\n      for (int32_t kv = 0; kv < 2; ++kv)\n        memcpy((uint8_t*)buf",
+     "if (ids[i] >= L->num_blocks) { ++nbad; continue; }\n    for (int32_t l = 0; l < L->num_layers; ++l)\n      for (int32_t kv = 0; kv < 2; ++kv)\n        memcpy((uint8_t*)buf", 0),
     ("scatter_copies_wrong_way", "test_oracle_kv.py",
-     "memcpy((uint8_t*)pool + pool_offset(L, ids[i], l),\n             (const uint8_t*)buf + (i * L->num_layers + l) * t, (size_t)t);",
-     "memcpy((uint8_t*)buf + (i * L->num_layers + l) * t,\n             (const uint8_t*)pool + pool_offset(L, ids[i], l), (size_t)t);", 0),
+     "memcpy((uint8_t*)pool + pool_offset(L, ids[i], l, kv),\n               (const uint8_t*)buf + buf_offset(L, i, l, kv), (size_t)half);",
+     "memcpy((uint8_t*)buf + buf_offset(L, i, l, kv),\n               (const uint8_t*)pool + pool_offset(L, ids[i], l, kv), (size_t)half);", 0),
+    ("inner_order_ignored_on_the_buffer_side", "test_oracle_kv.py",
+     "uint8_t* brow = bhalf + row_offset(L, buf_inner, h, tok);",
+     "uint8_t* brow = bhalf + row_offset(L, pool_inner, h, tok);", 0),
 ]
 
 
