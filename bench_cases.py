@@ -791,6 +791,41 @@ def case_kv_sweep(args):
                       "status": aibx.status_fetch()}))
 
 
+def case_kv_layouts(args):
+    """Gather and scatter of the same block shapes out of pools laid out block-major (0),
+    layer-major (1) and layer-major with K and V of a layer as separate tensors (2): the three
+    should move bytes at the same rate (cfg2 shape: 1,600 x 2 MiB of a 4,096-block pool; cfg4
+    shape: 1,024 x 5 MiB of a 4,096-block pool; every launch moves more than L2 holds)."""
+    import torch
+
+    from paper_2504_03648_b200 import binding as aibx
+    from workloads import synth
+    import workloads as W
+
+    out = []
+    peak, kind = measured_peak_hbm()
+    for name, kv0, n in (("cfg2 shape", W.cfg2_kv(), 1600), ("cfg4 shape", W.cfg4_kv(), 1024)):
+        row = {"shape": name, "blocks": n}
+        for layout in (0, 1, 2):
+            kv = W.scaled(kv0, num_blocks=4096, layout=layout)
+            pool = torch.empty(kv.pool_bytes, dtype=torch.uint8, device="cuda")
+            synth.fill_pool(pool, kv)
+            ids = torch.from_numpy(W.distinct_ids(7, kv.num_blocks, n)).cuda()
+            buf = torch.empty(n * kv.block_bytes, dtype=torch.uint8, device="cuda")
+            lay = aibx.KVLayout(kv.layout, kv.num_layers, kv.num_kv_heads, kv.block_tokens,
+                                kv.head_dim, kv.elem_bytes, kv.num_blocks)
+            nbytes = 2 * n * kv.block_bytes
+            tg = statistics.median(_event_times(torch, lambda: aibx.kv_gather(pool, lay, ids, n, buf), 15, 3))
+            ts = statistics.median(_event_times(torch, lambda: aibx.kv_scatter(pool, lay, ids, n, buf), 15, 3))
+            row["layout%d_gather_GBps" % layout] = round(nbytes / (tg * 1e-3) / 1e9, 1)
+            row["layout%d_scatter_GBps" % layout] = round(nbytes / (ts * 1e-3) / 1e9, 1)
+            del pool, buf
+            torch.cuda.empty_cache()
+        out.append(row)
+    print(json.dumps({"case": "kv_layouts", "peak": peak, "peak_kind": kind, "results": out,
+                      "status": aibx.status_fetch()}))
+
+
 def case_index_ops(args):
     """Operational index calls on the routing-heavy index (2^20 entries in 2^21 slots, 64 pods):
     touch, pick_victims, export, rehash, and the sequential assignment of 4,096 requests."""
@@ -875,6 +910,6 @@ def case_kv_comparators(args):
 
 CASES = {"kv_comparators": case_kv_comparators, "index_ops": case_index_ops, "kv_inner": case_kv_inner, "kv_inner_small": case_kv_inner_small, "kv_sweep": case_kv_sweep, "hash_sweep": case_hash_sweep, "oracle_cfg": case_oracle_cfg, "kv_small": case_kv_small, "match_large": case_match_large, "match_cfg": case_match_cfg,
          "cfg4": case_cfg4, "cfg5": case_cfg5, "lookup_flat": case_lookup_flat,
-         "random_reads": case_random_reads}
+         "random_reads": case_random_reads, "kv_layouts": case_kv_layouts}
 
 

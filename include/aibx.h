@@ -347,7 +347,10 @@ uint32_t aibx_collect_static_max_blocks(void);
  *   block_bytes = num_layers * tile
  *   pool offset of (block b, layer l) = (b*num_layers + l)*tile      layout 0, block-major
  *                                     = (l*num_blocks + b)*tile      layout 1, layer-major
- *   buffer offset of (item i, layer l) = (i*num_layers + l)*tile     always block-major
+ *   layout 2, [layer][K/V][block][head][token][dim]: K and V of a layer are separate tensors (the
+ *   shape of a per-layer paged cache); the K (kv = 0) or V (kv = 1) half of (block b, layer l)
+ *   starts at ((l*2 + kv)*num_blocks + b) * tile/2, and tile/2 must be a multiple of 16 bytes
+ *   buffer offset of (item i, layer l) = (i*num_layers + l)*tile     always block-major, K then V
  * gather:  buffer item i <- pool block ids[i]   (ids may repeat)
  * scatter: pool block ids[i] <- buffer item i   (ids must be distinct; pool != buffer)
  * Bytes move verbatim.  An id equal to AIBX_NO_BLOCK is skipped silently; any other id
@@ -356,7 +359,7 @@ uint32_t aibx_collect_static_max_blocks(void);
  * aligned (INVALID otherwise).  n = 0 is a no-op.
  */
 typedef struct {
-  int32_t layout;        /* 0 block-major, 1 layer-major */
+  int32_t layout;        /* 0 block-major, 1 layer-major, 2 layer-major with split K and V */
   int32_t num_layers;
   int32_t num_kv_heads;
   int32_t block_tokens;

@@ -5,7 +5,8 @@
 // It is cut into fixed-size chunks; chunk c goes to CTA c mod grid, so at any moment the SMs
 // work on neighbouring addresses.  On the pool side a chunk is 1..4 "pieces": runs inside one
 // segment, where a segment is the longest contiguous run both sides share (the whole block for
-// a block-major pool, one layer's K/V tile for a layer-major pool).  Cutting the stream rather
+// a block-major pool, one layer's K/V tile for a layer-major pool, the K or the V half of it for
+// a pool that keeps K and V of a layer as separate tensors).  Cutting the stream rather
 // than the segments keeps every iteration at full size whatever the tile size is.
 //
 // Two copy engines, same chunk schedule:
@@ -415,7 +416,7 @@ inline int32_t launch_kv_copy(const void* pool, const aibx_kv_layout_t* L, const
                               int64_t n, const void* buf, int to_pool, cudaStream_t st,
                               const uint32_t* d_count = nullptr) {
   if (!L || n < 0) return AIBX_ERR_INVALID;
-  if ((L->layout != 0 && L->layout != 1) || L->num_layers <= 0 || L->num_kv_heads <= 0 ||
+  if (L->layout < 0 || L->layout > 2 || L->num_layers <= 0 || L->num_kv_heads <= 0 ||
       L->block_tokens <= 0 || L->head_dim <= 0 || L->elem_bytes <= 0)
     return AIBX_ERR_INVALID;
   if (n == 0) return AIBX_OK;
@@ -423,10 +424,13 @@ inline int32_t launch_kv_copy(const void* pool, const aibx_kv_layout_t* L, const
   if ((reinterpret_cast<uintptr_t>(pool) & 15) || (reinterpret_cast<uintptr_t>(buf) & 15))
     return AIBX_ERR_INVALID;
   const long long tile = 2LL * L->num_kv_heads * L->block_tokens * L->head_dim * L->elem_bytes;
-  if (tile % 16 != 0) return AIBX_ERR_UNSUPPORTED;
+  const long long half = tile / 2;
+  if (tile % 16 != 0 || (L->layout == 2 && half % 16 != 0)) return AIBX_ERR_UNSUPPORTED;
   const long long block_bytes = tile * L->num_layers;
-  const long long seg_bytes = L->layout == 0 ? block_bytes : tile;
-  const long long segs = L->layout == 0 ? 1 : L->num_layers;
+  // the longest run both sides share, how many of them make an item (in buffer order), and where
+  // consecutive ones lie in the pool: layout 2 keeps (layer l, K or V) at plane 2l + kv
+  const long long seg_bytes = L->layout == 0 ? block_bytes : L->layout == 1 ? tile : half;
+  const long long segs = L->layout == 0 ? 1 : L->layout == 1 ? L->num_layers : 2LL * L->num_layers;
   if (seg_bytes / 16 >= (1LL << 31) || block_bytes / 16 >= (1LL << 31)) return AIBX_ERR_UNSUPPORTED;
 
   const CopyTuning& tn = copy_tuning();
@@ -435,8 +439,8 @@ inline int32_t launch_kv_copy(const void* pool, const aibx_kv_layout_t* L, const
   pl.to_pool = to_pool;
   pl.segs_per_item = (unsigned int)segs;
   pl.seg_units = (unsigned int)(seg_bytes / 16);
-  pl.pool_item_stride = L->layout == 0 ? block_bytes : tile;
-  pl.pool_seg_stride = L->layout == 0 ? 0 : (long long)L->num_blocks * tile;
+  pl.pool_item_stride = seg_bytes;
+  pl.pool_seg_stride = L->layout == 0 ? 0 : (long long)L->num_blocks * seg_bytes;
   // chunk: the tuned size, or a whole number of segments when segments are shorter than that
   if (seg_bytes >= tn.chunk_bytes) {
     pl.chunk_units = (unsigned int)(tn.chunk_bytes / 16);

@@ -39,6 +39,7 @@ struct PermPlan {
   char* buf;
   long long pool_item_stride;    // bytes between consecutive block ids in the pool
   long long pool_layer_stride;   // bytes between consecutive layers of one block in the pool
+  long long pool_kv_stride;      // bytes from the K plane of a tile to its V plane in the pool
   long long plane_bytes;         // heads * tokens * row_bytes
   unsigned int num_layers;
   unsigned int rows_per_plane;   // heads * tokens
@@ -78,7 +79,7 @@ __device__ __forceinline__ PermChunk perm_chunk(const PermPlan& pl, unsigned int
     return ch;
   }
   char* pool_plane = pl.pool + (long long)id * pl.pool_item_stride +
-                     (long long)layer * pl.pool_layer_stride + (long long)kv * pl.plane_bytes;
+                     (long long)layer * pl.pool_layer_stride + (long long)kv * pl.pool_kv_stride;
   char* buf_plane = pl.buf + (long long)plane * pl.plane_bytes;
   const long long row_bytes = (long long)pl.vec_per_row * 16;
   if (pl.to_pool) {
@@ -237,8 +238,10 @@ struct TmaPermPlan {
   const char* buf;
   long long pool_item_stride;    // bytes between consecutive block ids in the pool
   long long pool_layer_stride;   // bytes between consecutive layers of one block in the pool
-  long long pool_item_planes;    // the same two strides in planes (tensor-map coordinate w)
+  long long pool_kv_stride;      // bytes from the K plane of a tile to its V plane in the pool
+  long long pool_item_planes;    // the same three strides in planes (tensor-map coordinate w)
   long long pool_layer_planes;
+  long long pool_kv_planes;
   long long plane_bytes;
   unsigned int row_bytes;
   unsigned int num_layers;
@@ -286,16 +289,17 @@ __device__ __forceinline__ TmaChunk tma_chunk(const TmaPermPlan& pl, unsigned in
                                                  : min(pl.box_b, pl.inner - b0);
   const long long row_off = ((long long)a0 * pl.inner + b0) * pl.row_bytes;
   const long long pool_plane = (long long)id * pl.pool_item_stride +
-                               (long long)layer * pl.pool_layer_stride + (long long)kv * pl.plane_bytes;
+                               (long long)layer * pl.pool_layer_stride + (long long)kv * pl.pool_kv_stride;
   const long long buf_plane = (long long)plane * pl.plane_bytes;
   const char* src = pl.to_pool ? pl.buf + buf_plane : pl.pool + pool_plane;
   ch.src0 = src + row_off;
-  if (pl.box_w == 2) ch.src1 = ch.src0 + pl.plane_bytes;
+  // the second plane of a two-plane box is the V plane of the same tile
+  if (pl.box_w == 2) ch.src1 = ch.src0 + (pl.to_pool ? pl.plane_bytes : pl.pool_kv_stride);
   ch.bytes = rows * pl.row_bytes;
   ch.y = (int)b0;
   ch.z = (int)a0;
   ch.w = pl.to_pool ? (int)((long long)id * pl.pool_item_planes +
-                            (long long)layer * pl.pool_layer_planes + kv)
+                            (long long)layer * pl.pool_layer_planes + kv * pl.pool_kv_planes)
                     : (int)plane;
   return ch;
 }
@@ -448,6 +452,25 @@ inline EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
+// Byte strides of a pool: from block to block, from layer to layer, from the K plane of a tile
+// to its V plane.
+inline void pool_strides(const aibx_kv_layout_t* L, long long tile, long long plane,
+                         long long& item, long long& layer, long long& kv) {
+  if (L->layout == 0) {            // [block][layer][K/V]...
+    item = tile * L->num_layers;
+    layer = tile;
+    kv = plane;
+  } else if (L->layout == 1) {     // [layer][block][K/V]...
+    item = tile;
+    layer = (long long)L->num_blocks * tile;
+    kv = plane;
+  } else {                         // [layer][K/V][block]...
+    item = plane;
+    layer = 2LL * L->num_blocks * plane;
+    kv = (long long)L->num_blocks * plane;
+  }
+}
+
 inline int& permute_engine() {
   static int engine = 0;        // 0 tensor store where the shape allows it, 1 storer warps,
                                 // 2 tensor store or UNSUPPORTED
@@ -481,14 +504,18 @@ inline int32_t launch_kv_permute_tma(const void* pool, const aibx_kv_layout_t* L
     if (box_a > 256) box_a = 256;
     if (box_a < 1) box_a = 1;
   }
-  const long long box_w = (box_a == outer && box_b == inner && 2 * plane <= kStageBytes) ? 2 : 1;
+  // two planes per box (K and V of a tile) only where the DESTINATION keeps them adjacent: the
+  // buffer always does, a pool with separate K and V tensors does not
+  const bool dst_kv_adjacent = !(to_pool && L->layout == 2);
+  const long long box_w =
+      (box_a == outer && box_b == inner && 2 * plane <= kStageBytes && dst_kv_adjacent) ? 2 : 1;
   pl.ids = d_ids;
   pl.pool = static_cast<const char*>(pool);
   pl.buf = static_cast<const char*>(buf);
-  pl.pool_item_stride = L->layout == 0 ? tile * L->num_layers : tile;
-  pl.pool_layer_stride = L->layout == 0 ? tile : (long long)L->num_blocks * tile;
+  pool_strides(L, tile, plane, pl.pool_item_stride, pl.pool_layer_stride, pl.pool_kv_stride);
   pl.pool_item_planes = pl.pool_item_stride / plane;
   pl.pool_layer_planes = pl.pool_layer_stride / plane;
+  pl.pool_kv_planes = pl.pool_kv_stride / plane;
   pl.plane_bytes = plane;
   pl.row_bytes = (unsigned int)row_bytes;
   pl.num_layers = (unsigned int)L->num_layers;
@@ -544,7 +571,7 @@ inline int32_t launch_kv_permute(const void* pool, const aibx_kv_layout_t* L, in
                                  int32_t buf_inner, const uint32_t* d_ids, int64_t n,
                                  const void* buf, int to_pool, cudaStream_t st) {
   if (!L || n < 0) return AIBX_ERR_INVALID;
-  if ((L->layout != 0 && L->layout != 1) || L->num_layers <= 0 || L->num_kv_heads <= 0 ||
+  if (L->layout < 0 || L->layout > 2 || L->num_layers <= 0 || L->num_kv_heads <= 0 ||
       L->block_tokens <= 0 || L->head_dim <= 0 || L->elem_bytes <= 0)
     return AIBX_ERR_INVALID;
   if ((pool_inner != 0 && pool_inner != 1) || (buf_inner != 0 && buf_inner != 1))
@@ -573,8 +600,7 @@ inline int32_t launch_kv_permute(const void* pool, const aibx_kv_layout_t* L, in
   pl.ids = d_ids;
   pl.pool = const_cast<char*>(static_cast<const char*>(pool));
   pl.buf = const_cast<char*>(static_cast<const char*>(buf));
-  pl.pool_item_stride = L->layout == 0 ? tile * L->num_layers : tile;
-  pl.pool_layer_stride = L->layout == 0 ? tile : (long long)L->num_blocks * tile;
+  pool_strides(L, tile, plane, pl.pool_item_stride, pl.pool_layer_stride, pl.pool_kv_stride);
   pl.plane_bytes = plane;
   pl.num_layers = (unsigned int)L->num_layers;
   pl.rows_per_plane = (unsigned int)rows;

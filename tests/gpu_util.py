@@ -104,7 +104,9 @@ def read_block(pool_t: torch.Tensor, kv: W.KVSpec, b: int) -> np.ndarray:
     """Logical bytes [layer][tile] of block b of a device pool, whatever its physical layout."""
     if kv.layout == 0:
         return host(pool_t.view(kv.num_blocks, kv.block_bytes)[b])
-    return host(pool_t.view(kv.num_layers, kv.num_blocks, kv.tile_bytes)[:, b].contiguous()).reshape(-1)
+    if kv.layout == 1:
+        return host(pool_t.view(kv.num_layers, kv.num_blocks, kv.tile_bytes)[:, b].contiguous()).reshape(-1)
+    return host(pool_t.view(kv.num_layers * 2, kv.num_blocks, kv.tile_bytes // 2)[:, b].contiguous()).reshape(-1)
 
 
 # ------------------------------------------------------------------------------------------
@@ -138,10 +140,7 @@ class PoolModel:
         if k and int(blocks[-1]) - int(blocks[0]) == k - 1 and (np.diff(blocks) == 1).all():
             mini = W.physical_blocks(kv, int(blocks[0]), int(blocks[0]) + k)
         else:
-            mini = W.logical_blocks(kv, blocks)
-            if kv.layout == 1:
-                t = mini.reshape(k, kv.num_layers, kv.tile_bytes)
-                mini = np.ascontiguousarray(t.transpose(1, 0, 2)).reshape(-1)
+            mini = W.to_physical(kv, W.logical_blocks(kv, blocks), k)
         lay = kv_layout_oracle(kv, num_blocks=k)
         for where, seed in self.history:
             pos = where[blocks]
@@ -242,8 +241,10 @@ def check_pool_full(model: PoolModel, pool_d: torch.Tensor, chunk_bytes=160 << 2
         b1 = min(b0 + per, kv.num_blocks)
         if kv.layout == 0:
             part = pool_d[b0 * bb: b1 * bb]
-        else:
+        elif kv.layout == 1:
             part = pool_d.view(kv.num_layers, kv.num_blocks, kv.tile_bytes)[:, b0:b1].contiguous().view(-1)
+        else:
+            part = pool_d.view(kv.num_layers * 2, kv.num_blocks, kv.tile_bytes // 2)[:, b0:b1].contiguous().view(-1)
         blocks = np.arange(b0, b1, dtype=np.int64)
         cmp.submit(part, (lambda bl: (lambda: model.mini_pool(bl)[0]))(blocks), ("blocks", b0, b1))
     return cmp.finish()

@@ -84,10 +84,11 @@ def test_cfg1_tiny(mode_args):
 
 
 @pytest.mark.parametrize("mode_args", MODES)
-@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("layout", [0, 1, 2])
 def test_shapes_with_ragged_chunks(layout, mode_args):
-    # tile = 2*3*5*24*1 = 720 bytes (not a multiple of any chunk size), 7 layers
-    kv = W.KVSpec("ragged", 5, layout, 7, 3, 5, 24, 1, 61)
+    # tile = 2*3*5*24*1 = 720 bytes (not a multiple of any chunk size), 7 layers; with K and V
+    # apart a half tile must be a multiple of 16 bytes: 2*3*5*32*1 = 960-byte tiles there
+    kv = W.KVSpec("ragged", 5, layout, 7, 3, 5, 24 if layout < 2 else 32, 1, 61)
     rng = np.random.default_rng(layout)
     ids_g = rng.integers(0, 61, 200).astype(np.uint32)               # repeats allowed
     ids_g[[3, 50]] = NO_BLOCK
@@ -141,10 +142,14 @@ def test_invalid_arguments():
     assert lib.aibx_kv_gather(pool.data_ptr(), None, ids.data_ptr(), 1, buf.data_ptr(), None) == -1
     assert lib.aibx_kv_gather(pool.data_ptr(), C.byref(lay), ids.data_ptr(), -1, buf.data_ptr(), None) == -1
     assert lib.aibx_kv_gather(pool.data_ptr() + 8, C.byref(lay), ids.data_ptr(), 1, buf.data_ptr(), None) == -1
-    bad = aibx.KVLayout(2, 2, 4, 16, 64, 2, 256)
+    bad = aibx.KVLayout(-1, 2, 4, 16, 64, 2, 256)
     assert lib.aibx_kv_scatter(pool.data_ptr(), C.byref(bad), ids.data_ptr(), 1, buf.data_ptr(), None) == -1
     odd = aibx.KVLayout(0, 2, 1, 1, 3, 1, 256)                      # 6-byte tiles
     assert lib.aibx_kv_gather(pool.data_ptr(), C.byref(odd), ids.data_ptr(), 1, buf.data_ptr(), None) == -5
+    split = aibx.KVLayout(2, 2, 1, 1, 24, 1, 256)                   # 48-byte tiles, 24-byte halves
+    assert lib.aibx_kv_gather(pool.data_ptr(), C.byref(split), ids.data_ptr(), 1, buf.data_ptr(), None) == -5
+    assert lib.aibx_kv_gather(pool.data_ptr(), C.byref(aibx.KVLayout(3, 2, 4, 16, 64, 2, 256)),
+                              ids.data_ptr(), 1, buf.data_ptr(), None) == -1
 
 
 # ------------------------------------------------------------------ large configurations
@@ -249,8 +254,37 @@ def test_cfg4_full_size_layer_major():
     print("cfg4 pool blocks used:", kv.num_blocks, "(shrunk)" if shrunk else "(full)")
 
 
+@pytest.mark.parametrize("which", ["cfg2", "cfg4"])
+def test_split_kv_pools_at_full_size(which):
+    """The Llama-3-8B and Llama-3-70B pools with K and V of every layer as separate tensors
+    ([layer][K/V][block]...): a put, a get of fresh content into other blocks, a put of those -
+    every byte of both buffers and of the whole pool against the oracle."""
+    kv0 = W.scaled(W.cfg2_kv() if which == "cfg2" else W.cfg4_kv(), layout=2)
+    n = 1660 if which == "cfg2" else 2048
+    kv, shrunk = _fit_blocks(kv0, n * kv0.block_bytes)
+    pool = empty(kv.pool_bytes, torch.uint8)
+    synth.fill_pool(pool, kv)
+    buf = empty(n * kv.block_bytes, torch.uint8)
+    lay = kv_layout_gpu(kv)
+    model = PoolModel(kv)
+    ids = W.distinct_ids(2000, kv.num_blocks, n)
+    aibx.kv_gather(pool, lay, dev(ids), n, buf)
+    assert aibx.status_fetch() == (0, 0)
+    assert check_gather_full(model, ids, buf) == []
+    ids2 = W.distinct_ids(2001, kv.num_blocks, n)
+    synth.fill_linear(buf, 6000)
+    aibx.kv_scatter(pool, lay, dev(ids2), n, buf)
+    model.scattered(ids2, 6000)
+    ids3 = np.concatenate([ids2[: n // 2], ids[: n - n // 2]])        # half of them just written
+    aibx.kv_gather(pool, lay, dev(ids3), n, buf)
+    assert aibx.status_fetch() == (0, 0)
+    assert check_gather_full(model, ids3, buf) == []
+    assert check_pool_full(model, pool) == []
+    print(which, "split-K/V pool blocks used:", kv.num_blocks, "(shrunk)" if shrunk else "(full)")
+
+
 @pytest.mark.parametrize("pinned", [True, False])
-@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("layout", [0, 1, 2])
 def test_host_side_put_and_get(layout, pinned):
     """gather_to_host / scatter_from_host: the far end of the transfer in host memory (pinned or
     pageable), byte for byte against the oracle's gather and scatter."""
@@ -369,7 +403,7 @@ def test_cfg5_full_size_fp8_mixed():
 
 
 @pytest.mark.parametrize("mode", [0, 1])
-@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("layout", [0, 1, 2])
 def test_counted_variants_stop_at_the_device_count(layout, mode):
     aibx.kv_set_tuning(mode, 16384, 4, 1)
     kv = W.KVSpec("counted", 9, layout, 3, 5, 16, 40, 2, 97)          # 38,400-byte blocks

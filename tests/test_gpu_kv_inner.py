@@ -35,7 +35,7 @@ def _default_engine_afterwards():
 
 @pytest.mark.parametrize("engine", ENGINES)
 @pytest.mark.parametrize("shape", SHAPES)
-@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("layout", [0, 1, 2])
 def test_inner_order_gather_and_scatter(layout, shape, engine):
     L, H, T, D, E, nb = shape
     if engine == 2 and D * E > 2048:
@@ -109,9 +109,11 @@ def test_inner_order_round_trip_and_invalid():
     assert aibx.status_fetch() == (0, 0)
 
 
-def test_inner_order_large_launch_bandwidth_shape():
-    """cfg2 block shape, 600 blocks out of a 2 GiB pool: sampled against the oracle."""
-    kv = W.scaled(W.cfg2_kv(), num_blocks=1000)
+@pytest.mark.parametrize("layout", [0, 2])
+def test_inner_order_large_launch_bandwidth_shape(layout):
+    """cfg2 block shape, 600 blocks out of a 2 GiB pool (block-major, and with K and V of a layer
+    as separate tensors): sampled against the oracle, engine against engine in full."""
+    kv = W.scaled(W.cfg2_kv(), num_blocks=1000, layout=layout)
     pool = empty(kv.pool_bytes, torch.uint8)
     synth.fill_pool(pool, kv)
     n = 600
@@ -188,7 +190,7 @@ def test_inner_order_random_shapes():
         D = int(rng.choice([16, 32, 64, 128, 256]))
         H = int(rng.integers(1, 20))
         T = int(rng.integers(1, 300 if rng.random() < 0.2 else 40))
-        L, layout = int(rng.integers(1, 4)), int(rng.integers(0, 2))
+        L, layout = int(rng.integers(1, 4)), int(rng.integers(0, 3))
         nb = int(rng.integers(2, 10))
         kv = W.KVSpec("rnd", seed, layout, L, H, T, D, E, nb)
         if kv.pool_bytes > (256 << 20):

@@ -11,14 +11,15 @@ from gpu_util import NO_BLOCK, PoolModel, check_gather_full, check_pool_full
 from workloads import build as synth_build
 
 
-@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("layout", [0, 1, 2])
 def test_model_follows_scatters_and_reports_a_flipped_byte(layout):
     synth_build.build()
     kv = W.KVSpec("pm", 21, layout, 3, 2, 4, 8, 1, 41)                 # 128-byte tiles, 384-byte blocks
     bb = kv.block_bytes
     pool = W.host_pool(kv).copy()
-    logical = (pool.reshape(41, 3, -1) if layout == 0
-               else pool.reshape(3, 41, -1).transpose(1, 0, 2)).reshape(41, bb).copy()
+    logical = {0: lambda: pool.reshape(41, 3, -1),
+               1: lambda: pool.reshape(3, 41, -1).transpose(1, 0, 2),
+               2: lambda: pool.reshape(3, 2, 41, -1).transpose(2, 0, 1, 3)}[layout]().reshape(41, bb).copy()
     model = PoolModel(kv)
     for seed, n in ((700, 9), (701, 17)):
         ids = W.distinct_ids(seed, 41, n)
@@ -28,8 +29,9 @@ def test_model_follows_scatters_and_reports_a_flipped_byte(layout):
             if b != NO_BLOCK:
                 logical[b] = content[i]
         model.scattered(ids, seed)
-    phys = logical.reshape(41, 3, -1)
-    phys = (phys if layout == 0 else phys.transpose(1, 0, 2)).reshape(-1).copy()
+    phys = {0: lambda: logical.reshape(41, 3, -1),
+            1: lambda: logical.reshape(41, 3, -1).transpose(1, 0, 2),
+            2: lambda: logical.reshape(41, 3, 2, -1).transpose(1, 2, 0, 3)}[layout]().reshape(-1).copy()
     pool_t = torch.from_numpy(phys)
     assert check_pool_full(model, pool_t, chunk_bytes=5 * bb) == []
     ids = np.concatenate([W.distinct_ids(5, 41, 30), [NO_BLOCK, 7, 7]]).astype(np.uint32)

@@ -90,6 +90,10 @@ def test_native_host_twin_equals_the_numpy_generator():
     p = W.physical_blocks(kv, 1, 4).reshape(3, 3, kv.tile_bytes)          # [layer][block][tile]
     whole = W.host_pool(kv).reshape(3, 5, kv.tile_bytes)
     assert np.array_equal(p, whole[:, 1:4])
+    kv2 = W.scaled(kv, layout=2)
+    p2 = W.physical_blocks(kv2, 1, 4).reshape(3, 2, 3, kv.tile_bytes // 2)   # [layer][K/V][block]
+    assert np.array_equal(p2.transpose(0, 2, 1, 3).reshape(3, 3, kv.tile_bytes), p)
+    assert np.array_equal(W.host_pool(kv2).reshape(3, 2, 5, -1)[:, :, 1:4], p2)
     kv0 = W.scaled(kv, layout=0)
     assert np.array_equal(W.physical_blocks(kv0, 1, 4), W.host_pool(kv0)[kv.block_bytes: 4 * kv.block_bytes])
 

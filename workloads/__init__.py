@@ -133,7 +133,7 @@ class KVSpec:
 
     name: str
     seed: int
-    layout: int                   # 0 block-major, 1 layer-major
+    layout: int                   # 0 block-major, 1 layer-major, 2 layer-major with split K and V
     num_layers: int
     num_kv_heads: int
     block_tokens: int
@@ -302,10 +302,19 @@ def host_pool(kv: KVSpec) -> np.ndarray:
         logical = bf16_normal_bits(kv.seed, kv.pool_bytes // 2).astype("<u2").view(np.uint8)
     else:
         logical = pool_bytes(kv.seed, 0, kv.pool_bytes)
+    return to_physical(kv, np.ascontiguousarray(logical), kv.num_blocks)
+
+
+def to_physical(kv: KVSpec, logical: np.ndarray, n: int) -> np.ndarray:
+    """Block-major bytes of n blocks ([block][layer][K half][V half]) placed as a pool of n blocks
+    in kv's physical layout.  Placement of generated content only."""
     if kv.layout == 0:
-        return np.ascontiguousarray(logical)
-    t = logical.reshape(kv.num_blocks, kv.num_layers, kv.tile_bytes)
-    return np.ascontiguousarray(t.transpose(1, 0, 2)).reshape(-1)
+        return logical
+    if kv.layout == 1:
+        t = logical.reshape(n, kv.num_layers, kv.tile_bytes)
+        return np.ascontiguousarray(t.transpose(1, 0, 2)).reshape(-1)
+    t = logical.reshape(n, kv.num_layers, 2, kv.tile_bytes // 2)
+    return np.ascontiguousarray(t.transpose(1, 2, 0, 3)).reshape(-1)       # [layer][K/V][block]
 
 
 def logical_blocks(kv: KVSpec, ids) -> np.ndarray:
@@ -328,10 +337,7 @@ def physical_blocks(kv: KVSpec, b0: int, b1: int) -> np.ndarray:
     n = b1 - b0
     logical = np.empty(n * kv.block_bytes, dtype=np.uint8)
     synth.fill_host(logical, kv.seed, b0 * kv.block_bytes)
-    if kv.layout == 0:
-        return logical
-    t = logical.reshape(n, kv.num_layers, kv.tile_bytes)
-    return np.ascontiguousarray(t.transpose(1, 0, 2)).reshape(-1)
+    return to_physical(kv, logical, n)
 
 
 def distinct_ids(seed: int, num_blocks: int, n: int) -> np.ndarray:

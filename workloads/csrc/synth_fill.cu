@@ -22,6 +22,7 @@ __host__ __device__ __forceinline__ unsigned long long mix64(unsigned long long 
 
 // layout 0: physical word == logical word (offset by first_word).
 // layout 1: physical [layer][block][tile] -> logical [block][layer][tile].
+// layout 2: physical [layer][K/V][block][half tile] -> logical [block][layer][K/V][half tile].
 __global__ void fill_kernel(unsigned long long* dst, unsigned long long n_words,
                             unsigned long long seed, unsigned long long first_word, int layout,
                             unsigned long long num_layers, unsigned long long num_blocks,
@@ -37,6 +38,14 @@ __global__ void fill_kernel(unsigned long long* dst, unsigned long long n_words,
       const unsigned long long b = rem / tile_words;
       const unsigned long long j = rem - b * tile_words;
       lw = (b * num_layers + l) * tile_words + j;
+    } else if (layout == 2) {
+      const unsigned long long half_words = tile_words / 2;
+      const unsigned long long per_plane = num_blocks * half_words;
+      const unsigned long long plane = pw / per_plane;            // 2 * layer + kv
+      const unsigned long long rem = pw - plane * per_plane;
+      const unsigned long long b = rem / half_words;
+      const unsigned long long j = rem - b * half_words;
+      lw = (b * 2 * num_layers + plane) * half_words + j;
     }
     dst[pw] = mix64(seed, lw);
   }
@@ -68,10 +77,12 @@ int32_t aibx_synth_fill_host(void* h_dst, uint64_t n_bytes, uint64_t seed, uint6
   return 0;
 }
 
-// Whole pool in its physical layout (0 block-major, 1 layer-major); tile_bytes multiple of 8.
+// Whole pool in its physical layout (0 block-major, 1 layer-major, 2 layer-major with the K and
+// V halves of the tiles in separate planes); tile_bytes multiple of 8 (16 for layout 2).
 int32_t aibx_synth_fill_pool(void* d_pool, uint64_t seed, int32_t layout, uint64_t num_layers,
                              uint64_t num_blocks, uint64_t tile_bytes, void* stream) {
-  if (!d_pool || (tile_bytes & 7) || (layout != 0 && layout != 1)) return -1;
+  if (!d_pool || (tile_bytes & 7) || layout < 0 || layout > 2) return -1;
+  if (layout == 2 && (tile_bytes & 15)) return -1;
   const unsigned long long n_words = num_layers * num_blocks * (tile_bytes / 8);
   if (n_words == 0) return 0;
   fill_kernel<<<148 * 16, 256, 0, static_cast<cudaStream_t>(stream)>>>(
