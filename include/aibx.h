@@ -22,9 +22,9 @@
  *     with aibx_status_fetch.  Nothing aborts, throws or traps.
  *   - All arithmetic is integer; results are defined bit-exactly.
  *   - Threads: calls on different indexes, pools and streams may come from different host
- *     threads, except that the FIRST call of any kind on a device performs a few one-time
- *     per-device settings (kernel attributes, the address of the status record) without locking:
- *     make it from one thread.  Calls on one index are ordered by the caller.
+ *     threads at any time (the few one-time per-device settings - kernel attributes, the address
+ *     of the status record - are made under a lock or as single atomic words).  Calls on one
+ *     index are ordered by the caller.
  */
 #ifndef AIBX_H_
 #define AIBX_H_
@@ -412,8 +412,8 @@ int32_t aibx_kv_scatter_counted(void* d_pool, const aibx_kv_layout_t* layout,
  * of head_dim elements move whole (head_dim * elem_bytes must be a multiple of 16 and at most
  * 32 KiB: UNSUPPORTED otherwise); everything else - layouts, ids, skipping, errors - is as in
  * aibx_kv_gather / aibx_kv_scatter, to which equal orders reduce.  The transposition goes
- * through shared memory so that global reads and writes both stay whole rows (see
- * aibx_kv_set_inner_engine for the two engines that write the destination).
+ * through shared memory so that global reads and writes both stay whole rows (aibx_tuning.h
+ * describes the two engines that write the destination).
  */
 #define AIBX_INNER_HEAD_TOKEN 0
 #define AIBX_INNER_TOKEN_HEAD 1
@@ -424,27 +424,6 @@ int32_t aibx_kv_scatter_inner(void* d_pool, const aibx_kv_layout_t* layout, int3
                               int32_t buf_inner, const uint32_t* d_block_ids, int64_t n,
                               const void* d_buf, void* stream);
 
-/* Launch shape of gather/scatter, process-wide; for measurement sweeps.  mode 0 = bulk-async
- * (TMA) ring through shared memory, 1 = 16-byte load/store loop.  chunk_bytes (multiple of 16,
- * 1 KiB..64 KiB) and stages (2..16) size the ring (chunk*stages <= 200 KiB; the stage count
- * bounds the loads in flight per CTA); ctas_per_sm 1..8.
- * Any argument <= 0 keeps its current value.  INVALID on an out-of-range value.
- */
-int32_t aibx_kv_set_tuning(int32_t mode, int32_t chunk_bytes, int32_t stages,
-                           int32_t ctas_per_sm);
-/* Which engine writes the destination of the _inner calls, process-wide; for measurement and
- * tests.  0 (default) = a tensor-map store (cp.async.bulk.tensor) whose strides are those of the
- * destination order, falling back to 1 for shapes it cannot take (rows of head_dim*elem_bytes
- * over 2 KiB); 1 = storer warps (shared memory read back, coalesced streaming stores);
- * 2 = the tensor-map store or AIBX_ERR_UNSUPPORTED, never the fallback.  INVALID otherwise.
- */
-int32_t aibx_kv_set_inner_engine(int32_t engine);
-
-
-/* Bulk ring only, process-wide: how many store groups may still be reading shared memory
- * before their stage is handed back to the loader (1..4; default 1).  INVALID otherwise.
- */
-int32_t aibx_kv_set_store_lag(int32_t lag);
 
 /* ---------------------------------------------------------------------------------------
  * Device status of the current device: the most severe (most negative) code recorded by any

@@ -110,6 +110,7 @@ def lib():
             "aibx_kv_scatter_inner": [vp, C.POINTER(KVLayout), i32, i32, vp, i64, vp, vp],
             "aibx_kv_set_tuning": [i32, i32, i32, i32],
             "aibx_kv_set_store_lag": [i32],
+            "aibx_kv_get_tuning": [vp, vp, vp, vp, vp],
             "aibx_kv_set_inner_engine": [i32],
             "aibx_selftest_bounded_wait": [u32, vp],
             "aibx_status_fetch": [vp, C.POINTER(i32), C.POINTER(i64)],
@@ -404,6 +405,13 @@ def kv_scatter_inner(pool, layout: KVLayout, pool_inner: int, buf_inner: int, bl
 def kv_set_tuning(mode: int = -1, chunk_bytes: int = 0, stages: int = 0,
                   ctas_per_sm: int = 0) -> None:
     _check("aibx_kv_set_tuning", lib().aibx_kv_set_tuning(mode, chunk_bytes, stages, ctas_per_sm))
+
+
+def kv_get_tuning():
+    """(mode, chunk_bytes, stages, ctas_per_sm, lag) as a copy call starting now would read them."""
+    v = [C.c_int32() for _ in range(5)]
+    _check("aibx_kv_get_tuning", lib().aibx_kv_get_tuning(*[C.addressof(x) for x in v]))
+    return tuple(x.value for x in v)
 
 
 def kv_set_inner_engine(engine: int = 0) -> None:

@@ -4,6 +4,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "aibx.h"
 
 namespace aibx {
@@ -53,21 +56,42 @@ __device__ __forceinline__ uint64_t shfl_up64(uint64_t v, int d) {
   return (uint64_t)lo | ((uint64_t)hi << 32);
 }
 
+// Result of the launches a call has just made.  cudaGetLastError, not Peek: the error is
+// reported once, by the call that caused it, and does not make every later call on this thread
+// fail.  (An error left behind by the caller's own earlier CUDA work is reported by the first
+// aibx call that checks - and cleared with it.)
 inline int32_t launch_status() {
-  return cudaPeekAtLastError() == cudaSuccess ? AIBX_OK : AIBX_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? AIBX_OK : AIBX_ERR_CUDA;
 }
 
+// The cached per-device values below are single atomic words: two threads that race on the
+// first call both compute the same value and store it.
 inline int sm_count() {
-  static int cached[64] = {0};
+  static std::atomic<int> cached[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-  if (cached[dev] == 0) {
-    int n = 0;
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
       n = 148;
-    cached[dev] = n;
+    cached[dev].store(n, std::memory_order_relaxed);
   }
-  return cached[dev];
+  return n;
+}
+
+// Raise a kernel's dynamic shared-memory limit to `bytes` once per device (the attribute lives
+// in the context); later calls with a smaller or equal size do nothing.  Under a lock, so that
+// concurrent first calls cannot leave the record ahead of the attribute.
+template <typename Kernel>
+inline bool ensure_dynamic_smem(Kernel kernel, size_t bytes, int dev, size_t (&configured)[64],
+                                std::mutex& lock) {
+  std::lock_guard<std::mutex> guard(lock);
+  if (bytes <= configured[dev]) return true;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) !=
+      cudaSuccess)
+    return false;
+  configured[dev] = bytes;
+  return true;
 }
 
 }  // namespace aibx

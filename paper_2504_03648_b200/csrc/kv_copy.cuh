@@ -407,10 +407,32 @@ struct CopyTuning {
   int lag = 1;             // store groups that may still read shared memory (1..4)
 };
 
-inline CopyTuning& copy_tuning() {
-  static CopyTuning t;
+// The process-wide launch shape lives in ONE atomic word, so that a call on one host thread
+// reads a whole setting while another thread replaces it.
+//   bits 0      mode            bits 1..13  chunk_bytes / 16 (64..4096)
+//   bits 14..18 stages (2..16)  bits 19..22 CTAs per SM (1..8)     bits 23..25 lag (1..4)
+inline unsigned long long pack_tuning(const CopyTuning& t) {
+  return (unsigned long long)(t.mode & 1) | ((unsigned long long)(t.chunk_bytes / 16) << 1) |
+         ((unsigned long long)t.stages << 14) | ((unsigned long long)t.ctas_per_sm << 19) |
+         ((unsigned long long)t.lag << 23);
+}
+
+inline CopyTuning unpack_tuning(unsigned long long w) {
+  CopyTuning t;
+  t.mode = (int)(w & 1);
+  t.chunk_bytes = (int)((w >> 1) & 0x1FFF) * 16;
+  t.stages = (int)((w >> 14) & 0x1F);
+  t.ctas_per_sm = (int)((w >> 19) & 0xF);
+  t.lag = (int)((w >> 23) & 0x7);
   return t;
 }
+
+inline std::atomic<unsigned long long>& tuning_word() {
+  static std::atomic<unsigned long long> w{pack_tuning(CopyTuning())};
+  return w;
+}
+
+inline CopyTuning copy_tuning() { return unpack_tuning(tuning_word().load(std::memory_order_acquire)); }
 
 inline int32_t launch_kv_copy(const void* pool, const aibx_kv_layout_t* L, const uint32_t* d_ids,
                               int64_t n, const void* buf, int to_pool, cudaStream_t st,
@@ -433,7 +455,7 @@ inline int32_t launch_kv_copy(const void* pool, const aibx_kv_layout_t* L, const
   const long long segs = L->layout == 0 ? 1 : L->layout == 1 ? L->num_layers : 2LL * L->num_layers;
   if (seg_bytes / 16 >= (1LL << 31) || block_bytes / 16 >= (1LL << 31)) return AIBX_ERR_UNSUPPORTED;
 
-  const CopyTuning& tn = copy_tuning();
+  const CopyTuning tn = copy_tuning();     // one read: the whole call uses this setting
   CopyPlan pl;
   pl.num_blocks = L->num_blocks;
   pl.to_pool = to_pool;
@@ -454,13 +476,9 @@ inline int32_t launch_kv_copy(const void* pool, const aibx_kv_layout_t* L, const
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AIBX_ERR_CUDA;
   const size_t smem = (size_t)tn.stages * tn.chunk_bytes;
   if (tn.mode == 0) {
-    static size_t configured[64] = {0};   // per device: the attribute lives in the context
-    if (smem > configured[dev]) {
-      if (cudaFuncSetAttribute(kv_copy_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               (int)smem) != cudaSuccess)
-        return AIBX_ERR_CUDA;
-      configured[dev] = smem;
-    }
+    static size_t configured[64] = {0};
+    static std::mutex lock;
+    if (!ensure_dynamic_smem(kv_copy_bulk_kernel, smem, dev, configured, lock)) return AIBX_ERR_CUDA;
   }
 
   // 32-bit stream offsets: one launch covers at most ~64 GiB; longer lists take several

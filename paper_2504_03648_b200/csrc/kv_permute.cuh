@@ -440,15 +440,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 inline EncodeTiledFn encode_tiled_fn() {
   static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  static std::once_flag once;
+  std::call_once(once, [] {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
         q == cudaDriverEntryPointSuccess)
       fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
+    else
+      cudaGetLastError();
+  });
   return fn;
 }
 
@@ -471,9 +472,9 @@ inline void pool_strides(const aibx_kv_layout_t* L, long long tile, long long pl
   }
 }
 
-inline int& permute_engine() {
-  static int engine = 0;        // 0 tensor store where the shape allows it, 1 storer warps,
-                                // 2 tensor store or UNSUPPORTED
+inline std::atomic<int>& permute_engine() {
+  static std::atomic<int> engine{0};   // 0 tensor store where the shape allows it, 1 storer
+                                       // warps, 2 tensor store or UNSUPPORTED
   return engine;
 }
 
@@ -553,13 +554,9 @@ inline int32_t launch_kv_permute_tma(const void* pool, const aibx_kv_layout_t* L
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AIBX_ERR_CUDA;
   const size_t smem = (size_t)kStages * kStageBytes;
-  static bool configured[64] = {false};
-  if (!configured[dev]) {
-    if (cudaFuncSetAttribute(kv_permute_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)smem) != cudaSuccess)
-      return AIBX_ERR_CUDA;
-    configured[dev] = true;
-  }
+  static size_t configured[64] = {0};
+  static std::mutex lock;
+  if (!ensure_dynamic_smem(kv_permute_tma_kernel, smem, dev, configured, lock)) return AIBX_ERR_CUDA;
   long long grid = sm_count();
   if (grid > total) grid = total;
   kv_permute_tma_kernel<<<(unsigned int)grid, kRoleThreads, smem, st>>>(map, pl, kStages,
@@ -588,9 +585,10 @@ inline int32_t launch_kv_permute(const void* pool, const aibx_kv_layout_t* L, in
   const long long tile = 2 * plane;
 
   const int src_order = to_pool ? buf_inner : pool_inner;     // 0: [head][token], 1: [token][head]
-  if (permute_engine() != 1) {
+  const int engine = permute_engine().load(std::memory_order_relaxed);   // one read per call
+  if (engine != 1) {
     const int32_t rc = launch_kv_permute_tma(pool, L, src_order, d_ids, n, buf, to_pool, st);
-    if (rc != AIBX_ERR_UNSUPPORTED || permute_engine() == 2) return rc;
+    if (rc != AIBX_ERR_UNSUPPORTED || engine == 2) return rc;
   }
 
   constexpr long long kStageBytes = 32768;
@@ -620,13 +618,9 @@ inline int32_t launch_kv_permute(const void* pool, const aibx_kv_layout_t* L, in
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return AIBX_ERR_CUDA;
   const size_t smem = (size_t)kStages * kStageBytes;
-  static bool configured[64] = {false};
-  if (!configured[dev]) {
-    if (cudaFuncSetAttribute(kv_permute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)smem) != cudaSuccess)
-      return AIBX_ERR_CUDA;
-    configured[dev] = true;
-  }
+  static size_t configured[64] = {0};
+  static std::mutex lock;
+  if (!ensure_dynamic_smem(kv_permute_kernel, smem, dev, configured, lock)) return AIBX_ERR_CUDA;
   long long grid = sm_count();
   if (grid > total) grid = total;
   kv_permute_kernel<<<(unsigned int)grid, kPermThreads, smem, st>>>(pl, kStages,

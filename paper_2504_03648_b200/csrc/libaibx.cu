@@ -5,6 +5,7 @@
 #include <new>
 
 #include "aibx.h"
+#include "aibx_tuning.h"
 #include "aibx_common.cuh"
 #include "collect_blocks.cuh"
 #include "hash_blocks.cuh"
@@ -45,10 +46,10 @@ inline unsigned int blocks_for(int64_t n, int threads) {
 // copy kernel's CTA waiting until the small kernel has drained (measured: the gather ended later
 // by the whole duration of whatever ran beside it).  Once per device.
 void prefer_copy_carveout() {
-  static bool done[64] = {false};
+  static std::once_flag once[64];
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 || done[dev]) return;
-  done[dev] = true;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return;
+  std::call_once(once[dev], [] {
   const void* side_kernels[] = {
       (const void*)hash_blocks_kernel<0>,      (const void*)hash_blocks_kernel<1>,
       (const void*)hash_blocks_kernel<2>,      (const void*)hash_blocks_kernel<4>,
@@ -60,19 +61,25 @@ void prefer_copy_carveout() {
     cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
                          cudaSharedmemCarveoutMaxShared);
   cudaGetLastError();   // a refused hint is not an error of the call that follows
+  });
 }
 
 // Device address of the status record of the current device.
 StatusRecord* status_ptr() {
-  static StatusRecord* cached[64] = {nullptr};
+  static std::atomic<StatusRecord*> cached[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  if (!cached[dev]) {
-    void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_status) != cudaSuccess) return nullptr;
-    cached[dev] = static_cast<StatusRecord*>(p);
+  StatusRecord* p = cached[dev].load(std::memory_order_acquire);
+  if (!p) {
+    void* q = nullptr;
+    if (cudaGetSymbolAddress(&q, g_status) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    p = static_cast<StatusRecord*>(q);
+    cached[dev].store(p, std::memory_order_release);
   }
-  return cached[dev];
+  return p;
 }
 
 // Built-in scratch of aibx_collect_blocks_static: a bitmap over block ids that lives in the
@@ -85,18 +92,18 @@ static __device__ __align__(256) unsigned int g_collect_bitmap[kStaticCollectMax
 // kernels must be given what cudaGetSymbolAddress returns.  Resolved once per device, with that
 // device current; returns nullptr when the runtime refuses.
 unsigned int* static_bitmap_ptr() {
-  static unsigned int* cached[64] = {nullptr};
+  static std::atomic<unsigned int*> cached[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  if (!cached[dev]) {
-    unsigned int* p = nullptr;
+  unsigned int* p = cached[dev].load(std::memory_order_acquire);
+  if (!p) {
     if (cudaGetSymbolAddress((void**)&p, g_collect_bitmap) != cudaSuccess) {
       cudaGetLastError();
       return nullptr;
     }
-    cached[dev] = p;
+    cached[dev].store(p, std::memory_order_release);
   }
-  return cached[dev];
+  return p;
 }
 
 }  // namespace
@@ -692,31 +699,51 @@ int32_t aibx_kv_scatter_inner(void* d_pool, const aibx_kv_layout_t* layout, int3
 
 int32_t aibx_kv_set_tuning(int32_t mode, int32_t chunk_bytes, int32_t stages,
                            int32_t ctas_per_sm) {
-  CopyTuning t = copy_tuning();
-  if (mode >= 0) t.mode = mode;
-  if (chunk_bytes > 0) t.chunk_bytes = chunk_bytes;
-  if (stages > 0) t.stages = stages;
-  if (ctas_per_sm > 0) t.ctas_per_sm = ctas_per_sm;
-  if (t.mode != 0 && t.mode != 1) return AIBX_ERR_INVALID;
-  if (t.chunk_bytes % 16 != 0 || t.chunk_bytes < 1024 || t.chunk_bytes > 65536)
-    return AIBX_ERR_INVALID;
-  if (t.stages < 2 || t.stages > kMaxStages) return AIBX_ERR_INVALID;
-  if (t.ctas_per_sm < 1 || t.ctas_per_sm > 8) return AIBX_ERR_INVALID;
-  if ((long long)t.chunk_bytes * t.stages * t.ctas_per_sm > 200 * 1024) return AIBX_ERR_INVALID;
-  copy_tuning() = t;
+  std::atomic<unsigned long long>& word = tuning_word();
+  unsigned long long seen = word.load(std::memory_order_acquire);
+  for (;;) {
+    CopyTuning t = unpack_tuning(seen);
+    if (mode >= 0) t.mode = mode;
+    if (chunk_bytes > 0) t.chunk_bytes = chunk_bytes;
+    if (stages > 0) t.stages = stages;
+    if (ctas_per_sm > 0) t.ctas_per_sm = ctas_per_sm;
+    if (t.mode != 0 && t.mode != 1) return AIBX_ERR_INVALID;
+    if (t.chunk_bytes % 16 != 0 || t.chunk_bytes < 1024 || t.chunk_bytes > 65536)
+      return AIBX_ERR_INVALID;
+    if (t.stages < 2 || t.stages > kMaxStages) return AIBX_ERR_INVALID;
+    if (t.ctas_per_sm < 1 || t.ctas_per_sm > 8) return AIBX_ERR_INVALID;
+    if ((long long)t.chunk_bytes * t.stages * t.ctas_per_sm > 200 * 1024) return AIBX_ERR_INVALID;
+    // the arguments left at "keep" come from the word just read: swap only if it is still that
+    if (word.compare_exchange_weak(seen, pack_tuning(t), std::memory_order_acq_rel)) return AIBX_OK;
+  }
+}
+
+int32_t aibx_kv_get_tuning(int32_t* mode, int32_t* chunk_bytes, int32_t* stages,
+                           int32_t* ctas_per_sm, int32_t* lag) {
+  const CopyTuning t = copy_tuning();
+  if (mode) *mode = t.mode;
+  if (chunk_bytes) *chunk_bytes = t.chunk_bytes;
+  if (stages) *stages = t.stages;
+  if (ctas_per_sm) *ctas_per_sm = t.ctas_per_sm;
+  if (lag) *lag = t.lag;
   return AIBX_OK;
 }
 
 int32_t aibx_kv_set_inner_engine(int32_t engine) {
   if (engine < 0 || engine > 2) return AIBX_ERR_INVALID;
-  permute_engine() = engine;
+  permute_engine().store(engine, std::memory_order_relaxed);
   return AIBX_OK;
 }
 
 int32_t aibx_kv_set_store_lag(int32_t lag) {
   if (lag < 1 || lag > 4) return AIBX_ERR_INVALID;
-  copy_tuning().lag = lag;
-  return AIBX_OK;
+  std::atomic<unsigned long long>& word = tuning_word();
+  unsigned long long seen = word.load(std::memory_order_acquire);
+  for (;;) {
+    CopyTuning t = unpack_tuning(seen);
+    t.lag = lag;
+    if (word.compare_exchange_weak(seen, pack_tuning(t), std::memory_order_acq_rel)) return AIBX_OK;
+  }
 }
 
 int32_t aibx_selftest_bounded_wait(uint32_t spins, void* stream) {
