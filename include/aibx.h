@@ -38,7 +38,7 @@ extern "C" {
 #define AIBX_OK               0
 #define AIBX_ERR_INVALID     (-1)  /* null pointer, negative count, bad parameter          */
 #define AIBX_ERR_RANGE       (-2)  /* a block id >= num_blocks (item skipped)               */
-#define AIBX_ERR_FULL        (-3)  /* index could not place a key within `capacity` probes  */
+#define AIBX_ERR_FULL        (-3)  /* more live entries than capacity, or no room near home */
 #define AIBX_ERR_CUDA        (-4)  /* a CUDA runtime call failed                            */
 #define AIBX_ERR_UNSUPPORTED (-5)  /* shape outside what the kernels handle                 */
 #define AIBX_ERR_NOMEM       (-6)  /* device allocation failed                              */
@@ -75,8 +75,12 @@ int32_t aibx_hash_blocks(const int32_t* d_tokens, const int64_t* d_tok_off,
  * where bit p of pod_mask says pod p holds the block and block_id names its slot in the KV
  * pool.  Keys 0 and ~0 are reserved: inserting them is a no-op, looking them up misses.
  *
- * create:  allocates capacity_slots (power of two, >= 8) slots of 32 bytes on the current
- *          device; num_pods in 1..64.  Syncs.  NOMEM if the allocation fails.
+ * create:  allocates a table for up to capacity_slots entries (power of two, >= 8) on the
+ *          current device: ceil(capacity_slots / 3) buckets of 64 bytes holding three entries
+ *          each, plus 4 bytes per entry for the eviction stamps (25.3 bytes per slot in all);
+ *          num_pods in 1..64.  Syncs.  NOMEM if the allocation fails.  Size it for a load of
+ *          about one half (capacity_slots = twice the entries expected): probes then end in
+ *          their first bucket 94 times out of 100.
  * destroy: frees it (syncs the device).     clear: empties it (async on stream).
  */
 int32_t aibx_index_create(aibx_index_t** out, uint64_t capacity_slots, int32_t num_pods);
@@ -86,9 +90,14 @@ int32_t aibx_index_clear(aibx_index_t* index, void* stream);
 /* insert: for every i < n (order-free): skip if key reserved or (mask & podmask(P)) == 0;
  *         absent key -> create (mask & podmask, id); present -> mask |= ..., id = min(id, new).
  *         AIBX_NO_BLOCK as id means "no id supplied" (identity of min).
- *         Device status FULL if a new key finds no free slot within `capacity` probes (all
- *         slots hold live entries); the index content is then unspecified until
- *         aibx_index_clear.  Slots freed by evict are reused.
+ *         Device status FULL (detail = number of entries refused or in excess) when the live
+ *         entries would exceed capacity_slots, or when a new key finds no free entry within
+ *         1,024 buckets (3,072 entries) of its home bucket - no entry is ever placed further
+ *         away, which bounds every later probe; tables up to a load of 0.9 stay far below that.  After FULL the index content is unspecified until aibx_index_clear or
+ *         aibx_index_rehash.  Entries removed by evict are reused by later inserts that pass
+ *         them, but a probe for an absent key only stops at a NEVER-used entry: under steady
+ *         publish/expire churn those run out, probes grow towards the 1,024-bucket bound, and
+ *         the table wants a rehash - aibx_index_stats2 says when.
  * evict:  batch-atomic.  First mask &= ~masks[i] for all present keys; then
  *         freed[i] = id if key i was present and its mask is now 0, else AIBX_NO_BLOCK
  *         (duplicates of a key all report the same value); then entries with mask 0 vanish.
@@ -96,6 +105,12 @@ int32_t aibx_index_clear(aibx_index_t* index, void* stream);
  * lookup: d_masks[i], d_block_ids[i] = entry of key i, or (0, AIBX_NO_BLOCK).  Either output
  *         may be null.
  * stats:  live entries and capacity.  Syncs the stream.
+ * stats2: the same plus what tells when aibx_index_rehash is due: `removed` = entries freed by
+ *         evict and not yet reused (live + removed, not live alone, is what the probe length
+ *         follows: rehash once it passes three quarters of capacity_slots), `longest_walk` = the
+ *         most buckets any insert has had to visit since the table was created, cleared or
+ *         rehashed (1 = every key so far went into its home bucket; a healthy table at a load of one
+ *         half stays below 10).  Any out-pointer may be null.  Syncs the stream.
  */
 int32_t aibx_index_insert(aibx_index_t* index, const uint64_t* d_keys,
                           const uint64_t* d_pod_masks, const uint32_t* d_block_ids,
@@ -107,6 +122,8 @@ int32_t aibx_index_lookup(const aibx_index_t* index, const uint64_t* d_keys,
                           uint64_t* d_masks, uint32_t* d_block_ids, int64_t n, void* stream);
 int32_t aibx_index_stats(const aibx_index_t* index, uint64_t* live, uint64_t* capacity,
                          void* stream);
+int32_t aibx_index_stats2(const aibx_index_t* index, uint64_t* live, uint64_t* removed,
+                          uint64_t* capacity, uint32_t* longest_walk, void* stream);
 
 /* Scan-resistant victim choice (Section 3.2.5 names a scan-resistant eviction policy without
  * describing it; the reading fixed here).  Every entry remembers the last epoch it was touched in
@@ -132,8 +149,9 @@ int32_t aibx_index_pick_victims(aibx_index_t* index, uint64_t k, uint64_t* d_key
  *         elements, in no particular order; *d_count (uint64, device) = number of live entries,
  *         which may exceed max_entries (the surplus is counted, not written).  Arrays may be
  *         null to only count.  Async on stream.
- * rehash: move the index into a table of new_capacity slots (power of two >= 8), dropping the
- *         slots freed by evict on the way; the way out of a FULL table.  FULL (and no change) if
+ * rehash: move the index into a fresh table of new_capacity slots (power of two >= 8; the same
+ *         size is fine), dropping the entries freed by evict on the way, so that probes are
+ *         short again; also the way out of a FULL table.  FULL (and no change) if
  *         the live entries do not fit, NOMEM if the new table cannot be allocated.  Syncs the
  *         device; the handle stays valid.
  */

@@ -83,6 +83,8 @@ def lib():
             "aibx_index_evict": [vp, vp, vp, vp, i64, vp],
             "aibx_index_lookup": [vp, vp, vp, vp, i64, vp],
             "aibx_index_stats": [vp, C.POINTER(u64), C.POINTER(u64), vp],
+            "aibx_index_stats2": [vp, C.POINTER(u64), C.POINTER(u64), C.POINTER(u64),
+                                  C.POINTER(u32), vp],
             "aibx_index_touch": [vp, vp, i64, u32, vp],
             "aibx_index_pick_victims": [vp, u64, vp, vp, vp, vp],
             "aibx_index_export": [vp, vp, vp, vp, u64, vp, vp],
@@ -207,6 +209,13 @@ class Index:
         _check("aibx_index_stats",
                lib().aibx_index_stats(self._h, C.byref(live), C.byref(cap), _stream()))
         return live.value, cap.value
+
+    def stats2(self):
+        """(live, removed, capacity, longest_walk)."""
+        live, removed, cap, walk = C.c_uint64(), C.c_uint64(), C.c_uint64(), C.c_uint32()
+        _check("aibx_index_stats2", lib().aibx_index_stats2(
+            self._h, C.byref(live), C.byref(removed), C.byref(cap), C.byref(walk), _stream()))
+        return live.value, removed.value, cap.value, walk.value
 
     def touch(self, keys, epoch: int) -> None:
         _check("aibx_index_touch", lib().aibx_index_touch(

@@ -26,6 +26,11 @@ __device__ __forceinline__ void raise_status(int code) {
   atomicAdd(&g_status.detail, 1ULL);
 }
 
+__device__ __forceinline__ void raise_status_n(int code, unsigned long long items) {
+  atomicMin(&g_status.code, code);
+  atomicAdd(&g_status.detail, items);
+}
+
 constexpr uint64_t kKeyEmpty = 0ULL;
 constexpr uint64_t kKeyTomb = ~0ULL;
 

@@ -1,5 +1,13 @@
-// GPU-resident residency index: open addressing with linear probing over 32-byte slots, so
-// that one probe touches exactly one DRAM sector holding key, pod mask and block id.
+// GPU-resident residency index: open addressing over 64-byte BUCKETS of three entries.
+//
+// What the memory system gives a random probe was measured on B200 before this layout was
+// chosen: an L2 miss always brings a whole 128-byte line from DRAM, whatever the load asked for,
+// and random reads of 32 and of 64 bytes run at the same rate.  So a probe may as well read 64
+// bytes, and the table should be as small as it can be so that more of it stays in L2.  A bucket
+// holds the keys, pod masks and block ids of three entries (the eviction stamps, which only the
+// touch and victim kernels need, live in a side array): 21.3 bytes per slot of capacity instead
+// of 32, and at a load of one half 94 % of the lookups end in their home bucket - one memory
+// round trip, two sectors.
 //
 //   insert / evict : one thread per item, atomics only (results are order-free by construction)
 //   lookup         : one thread per key
@@ -14,197 +22,235 @@
 
 namespace aibx {
 
-struct __align__(32) Slot {
-  unsigned long long key;    // 0 = never used, ~0 = removed (reusable by insert)
-  unsigned long long mask;   // pod residency bits; an entry with mask 0 is dead
-  unsigned int id;           // block id, min over inserts; AIBX_NO_BLOCK = none supplied
-  unsigned int stamp;        // reserved (recency stamp for eviction policies)
-  unsigned long long pad;
-};
-static_assert(sizeof(Slot) == 32, "one slot per 32-byte sector");
+constexpr int kBucketEntries = 3;
+constexpr unsigned int kMaxWalk = 1024;  // buckets a probe sequence may visit (3,072 entries)
 
+struct __align__(64) Bucket {
+  unsigned long long key[kBucketEntries];    // 0 = never used, ~0 = removed (reusable by insert)
+  unsigned long long mask[kBucketEntries];   // pod residency bits; an entry with mask 0 is dead
+  unsigned int id[kBucketEntries];           // block id, min over inserts; AIBX_NO_BLOCK = none
+  unsigned int spare;
+};
+static_assert(sizeof(Bucket) == 64, "one bucket per 64 bytes");
+
+// Entry e of the table is position e % 3 of bucket e / 3.
 struct IndexView {
-  Slot* slots;
-  unsigned long long cap_mask;   // capacity - 1
-  int shift;                     // 64 - log2(capacity)
+  Bucket* buckets;
+  unsigned int* stamps;          // [3 * nb] recency stamp of every entry (eviction policy)
+  unsigned long long nb;         // buckets: ceil(capacity / 3)
+  unsigned long long capacity;   // live entries the table accepts (FULL beyond)
+  unsigned int max_walk;         // min(nb, kMaxWalk): no entry lies further from its home bucket
   int num_pods;
-  unsigned long long* counters;  // [0] live entries, [1] removed slots
+  unsigned long long* counters;  // [0] live entries, [1] removed entries, [2] longest insert walk
 };
 
-__device__ __forceinline__ unsigned long long home_slot(const IndexView& ix, uint64_t key) {
-  return (key * 0x9E3779B97F4A7C15ULL) >> ix.shift;
+__device__ __forceinline__ unsigned long long num_entries(const IndexView& ix) {
+  return ix.nb * kBucketEntries;
 }
 
-// One 32-byte slot in one request: a 256-bit read-only load (slots are 32-byte aligned).
-__device__ __forceinline__ void load_slot(const Slot* p, unsigned long long& k,
-                                          unsigned long long& m, unsigned int& id) {
-  unsigned long long w2;
-  [[maybe_unused]] unsigned long long w3;       // stamp and padding: not needed by a probe
-  asm volatile("ld.global.nc.v4.u64 {%0,%1,%2,%3}, [%4];"
-               : "=l"(k), "=l"(m), "=l"(w2), "=l"(w3)
-               : "l"(p));
-  id = (unsigned int)w2;
+// Multiply-shift range reduction: any bucket count, no division.
+__device__ __forceinline__ unsigned long long home_bucket(const IndexView& ix, uint64_t key) {
+  return __umul64hi(key * 0x9E3779B97F4A7C15ULL, ix.nb);
 }
 
-// The same load with the third word (block id in its low half, stamp above) left as it arrives:
-// no instruction touches the result, so issuing it never waits for the data.
-__device__ __forceinline__ void load_slot_raw(const Slot* p, unsigned long long& k,
-                                              unsigned long long& m, unsigned long long& id_stamp) {
-  [[maybe_unused]] unsigned long long w3;
+__device__ __forceinline__ unsigned long long next_bucket(const IndexView& ix,
+                                                          unsigned long long b) {
+  return b + 1 == ix.nb ? 0ULL : b + 1;
+}
+
+// One whole bucket in two 256-bit read-only loads (the table is not modified meanwhile).
+struct BucketWords {
+  unsigned long long k0, k1, k2, m0, m1, m2, id01, id2;
+};
+
+__device__ __forceinline__ void load_bucket(const Bucket* b, BucketWords& w) {
+  const unsigned long long* p = reinterpret_cast<const unsigned long long*>(b);
   asm volatile("ld.global.nc.v4.u64 {%0,%1,%2,%3}, [%4];"
-               : "=l"(k), "=l"(m), "=l"(id_stamp), "=l"(w3)
+               : "=l"(w.k0), "=l"(w.k1), "=l"(w.k2), "=l"(w.m0)
                : "l"(p));
+  asm volatile("ld.global.nc.v4.u64 {%0,%1,%2,%3}, [%4];"
+               : "=l"(w.m1), "=l"(w.m2), "=l"(w.id01), "=l"(w.id2)
+               : "l"(p + 4));
 }
 
 __global__ void index_clear_kernel(IndexView ix) {
-  const unsigned long long n = ix.cap_mask + 1;
-  for (unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; i < n;
-       i += (unsigned long long)gridDim.x * blockDim.x) {
-    uint4* p = reinterpret_cast<uint4*>(ix.slots + i);
-    p[0] = make_uint4(0u, 0u, 0u, 0u);                      // key, mask
-    p[1] = make_uint4(AIBX_NO_BLOCK, 0u, 0u, 0u);           // id, stamp, pad
+  const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+  const unsigned long long t = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x;
+  // 16 bytes per thread and turn: words 0..2 of a bucket are keys and masks (zero), word 3
+  // holds the three ids and the spare word
+  for (unsigned long long i = t; i < ix.nb * 4; i += stride) {
+    uint4* p = reinterpret_cast<uint4*>(ix.buckets) + i;
+    *p = (i & 3) == 3 ? make_uint4(AIBX_NO_BLOCK, AIBX_NO_BLOCK, AIBX_NO_BLOCK, 0u)
+                      : make_uint4(0u, 0u, 0u, 0u);
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
-    ix.counters[0] = 0;
-    ix.counters[1] = 0;
-  }
+  for (unsigned long long i = t; i < num_entries(ix); i += stride) ix.stamps[i] = 0u;
+  if (t < 3) ix.counters[t] = 0;
 }
 
-// Read-only probe (index not modified while the kernel runs): the whole slot arrives with one
-// load, so a hit costs one memory round trip.
+// Read-only probe: a hit in the home bucket costs one memory round trip.  A bucket with a
+// never-used entry ends the walk: no key was ever placed beyond it.
 __device__ __forceinline__ bool probe_ro(const IndexView& ix, uint64_t key, uint64_t& mask,
                                          uint32_t& id) {
   mask = 0;
   id = AIBX_NO_BLOCK;
   if (key_reserved(key)) return false;
-  unsigned long long s = home_slot(ix, key);
-  for (unsigned long long n = 0; n <= ix.cap_mask; ++n) {
-    unsigned long long k, m;
-    unsigned int sid;
-    load_slot(ix.slots + s, k, m, sid);
-    if (k == key) {
-      if (m == 0) return false;
-      mask = m;
-      id = sid;
-      return true;
+  unsigned long long b = home_bucket(ix, key);
+  for (unsigned int n = 0; n < ix.max_walk; ++n) {
+    BucketWords w;
+    load_bucket(ix.buckets + b, w);
+    if (w.k0 == key) {
+      mask = w.m0;
+      id = (unsigned int)w.id01;
+    } else if (w.k1 == key) {
+      mask = w.m1;
+      id = (unsigned int)(w.id01 >> 32);
+    } else if (w.k2 == key) {
+      mask = w.m2;
+      id = (unsigned int)w.id2;
+    } else {
+      if (w.k0 == kKeyEmpty || w.k1 == kKeyEmpty || w.k2 == kKeyEmpty) return false;
+      b = next_bucket(ix, b);
+      continue;
     }
-    if (k == kKeyEmpty) return false;
-    s = (s + 1) & ix.cap_mask;
+    if (mask == 0) id = AIBX_NO_BLOCK;
+    return mask != 0;
   }
   return false;
 }
 
-// Keys of kWalk consecutive slots of a probe run, requested together (they usually share one
-// 128-byte line): a walk advances kWalk slots per memory round trip.  Volatile: other threads
-// may be claiming slots meanwhile.
-constexpr int kWalk = 2;
-__device__ __forceinline__ void load_keys(const IndexView& ix, unsigned long long s,
-                                           unsigned long long (&k)[kWalk]) {
+// The three keys of a bucket while other threads may be claiming entries.
+__device__ __forceinline__ void load_keys(const Bucket* b, unsigned long long (&k)[kBucketEntries]) {
 #pragma unroll
-  for (int j = 0; j < kWalk; ++j)
-    k[j] = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[(s + j) & ix.cap_mask].key);
+  for (int j = 0; j < kBucketEntries; ++j)
+    k[j] = *reinterpret_cast<const volatile unsigned long long*>(&b->key[j]);
 }
 
-// Probe while other threads may be claiming slots: returns the slot index or ~0.
-__device__ __forceinline__ unsigned long long find_slot_rw(const IndexView& ix, uint64_t key) {
-  unsigned long long s = home_slot(ix, key);
-  for (unsigned long long n = 0; n <= ix.cap_mask; n += kWalk) {
-    unsigned long long k[kWalk];
-    load_keys(ix, s, k);
+__device__ __forceinline__ unsigned long long* entry_key(const IndexView& ix, unsigned long long e) {
+  return &ix.buckets[e / kBucketEntries].key[e % kBucketEntries];
+}
+__device__ __forceinline__ unsigned long long* entry_mask(const IndexView& ix, unsigned long long e) {
+  return &ix.buckets[e / kBucketEntries].mask[e % kBucketEntries];
+}
+__device__ __forceinline__ unsigned int* entry_id(const IndexView& ix, unsigned long long e) {
+  return &ix.buckets[e / kBucketEntries].id[e % kBucketEntries];
+}
+
+// Probe while other threads may be claiming entries: returns the entry index or ~0.
+__device__ __forceinline__ unsigned long long find_entry_rw(const IndexView& ix, uint64_t key) {
+  unsigned long long b = home_bucket(ix, key);
+  for (unsigned int n = 0; n < ix.max_walk; ++n) {
+    unsigned long long k[kBucketEntries];
+    load_keys(ix.buckets + b, k);
 #pragma unroll
-    for (int j = 0; j < kWalk; ++j) {
-      if (k[j] == key) return (s + j) & ix.cap_mask;
+    for (int j = 0; j < kBucketEntries; ++j) {
+      if (k[j] == key) return b * kBucketEntries + j;
       if (k[j] == kKeyEmpty) return ~0ULL;
     }
-    s = (s + kWalk) & ix.cap_mask;
+    b = next_bucket(ix, b);
   }
   return ~0ULL;
 }
 
 // Insert or update one entry (mask already restricted to the table's pods, key not reserved).
-// Returns the slot, or ~0 when the table is full.
+// Returns the entry, or ~0 when no room is left within max_walk buckets of the key's home.
 //
-// One walk from the home slot to the first never-used slot: an existing entry anywhere on the
-// way wins; otherwise the first never-used or removed slot seen on the way is claimed.  An entry
-// may lie BEHIND a removed slot (it was placed when that slot was taken), hence the walk to the
-// end before claiming.  Every thread inserting this key walks the same path and tries the same
-// slots in the same order, and no slot turns reusable while inserts run, so the loser of a race
-// for a slot either finds the key there (another thread of the same key won) or starts over
-// and finds the key, or the next free slot, further on.
-// `added` / `reused` are raised when a slot was claimed / when that slot was a removed one: the
-// caller folds them into the table's counters once per CTA (one atomic per thread on the same
-// two words would serialise the whole kernel behind them).
+// One walk from the home bucket to the first bucket with a never-used entry: an existing entry
+// anywhere on the way wins; otherwise the first never-used or removed entry seen on the way is
+// claimed.  An entry may lie BEHIND a removed one (it was placed when that one was taken), hence
+// the walk to the end before claiming.  Every thread inserting this key walks the same path and
+// tries the same entries in the same order, and no entry turns reusable while inserts run, so
+// the loser of a race for an entry either finds the key there (another thread of the same key
+// won) or starts over and finds the key, or the next free entry, further on.  Inside a bucket
+// the never-used entries are always the last ones, which is what lets a reader stop at the
+// first bucket that has one.
+// `added` / `reused` are raised when an entry was claimed / when it was a removed one, `walked`
+// is the number of buckets visited: the caller folds them into the table's counters once per
+// CTA (one atomic per thread on the same words would serialise the whole kernel behind them).
 __device__ __forceinline__ unsigned long long insert_entry(const IndexView& ix, uint64_t key,
                                                            uint64_t m, uint32_t id,
-                                                           unsigned int& added,
-                                                           unsigned int& reused) {
-  unsigned long long slot = ~0ULL;
-  // a lost race costs one more walk; each one means some slot was taken, so the table bounds them
-  for (unsigned long long attempts = 0; attempts <= ix.cap_mask && slot == ~0ULL; ++attempts) {
-    unsigned long long s = home_slot(ix, key);
-    unsigned long long free_slot = ~0ULL, free_was = kKeyEmpty;
+                                                           unsigned int& added, unsigned int& reused,
+                                                           unsigned int& walked) {
+  unsigned long long entry = ~0ULL;
+  const unsigned int max_attempts = ix.max_walk * kBucketEntries + 1u;   // each lost race fills one
+  for (unsigned int attempts = 0; attempts < max_attempts && entry == ~0ULL; ++attempts) {
+    unsigned long long b = home_bucket(ix, key);
+    unsigned long long free_entry = ~0ULL, free_was = kKeyEmpty;
     bool at_end = false;
-    for (unsigned long long n = 0; n <= ix.cap_mask && slot == ~0ULL && !at_end; n += kWalk) {
-      unsigned long long k[kWalk];
-      load_keys(ix, s, k);
+    unsigned int n = 0;
+    for (; n < ix.max_walk && entry == ~0ULL && !at_end; ++n) {
+      unsigned long long k[kBucketEntries];
+      load_keys(ix.buckets + b, k);
 #pragma unroll
-      for (int j = 0; j < kWalk; ++j) {
-        if (slot != ~0ULL || at_end) continue;
-        const unsigned long long here = (s + j) & ix.cap_mask;
+      for (int j = 0; j < kBucketEntries; ++j) {
+        if (entry != ~0ULL || at_end) continue;
         if (k[j] == key) {
-          slot = here;
+          entry = b * kBucketEntries + j;
         } else if (k[j] == kKeyEmpty || k[j] == kKeyTomb) {
-          if (free_slot == ~0ULL) {
-            free_slot = here;
+          if (free_entry == ~0ULL) {
+            free_entry = b * kBucketEntries + j;
             free_was = k[j];
           }
           at_end = k[j] == kKeyEmpty;
         }
       }
-      s = (s + kWalk) & ix.cap_mask;
+      b = next_bucket(ix, b);
     }
-    if (slot != ~0ULL) break;
-    if (free_slot == ~0ULL) break;                      // no room anywhere on the path
+    walked = max(walked, n);
+    if (entry != ~0ULL) break;
+    if (free_entry == ~0ULL) break;                     // no room anywhere on the path
     const unsigned long long seen =
-        atomicCAS(&ix.slots[free_slot].key, free_was, (unsigned long long)key);
+        atomicCAS(entry_key(ix, free_entry), free_was, (unsigned long long)key);
     if (seen == free_was) {
       added += 1u;
       if (free_was == kKeyTomb) reused += 1u;
-      slot = free_slot;
+      entry = free_entry;
     } else if (seen == key) {
-      slot = free_slot;
+      entry = free_entry;
     }
   }
-  if (slot == ~0ULL) {
+  if (entry == ~0ULL) {
     raise_status(AIBX_ERR_FULL);
     return ~0ULL;
   }
-  atomicOr(&ix.slots[slot].mask, (unsigned long long)m);
-  atomicMin(&ix.slots[slot].id, id);
-  return slot;
+  atomicOr(entry_mask(ix, entry), (unsigned long long)m);
+  atomicMin(entry_id(ix, entry), id);
+  return entry;
 }
 
-// live += added - removed, freed-slot count += removed - reused: summed over the CTA in shared
-// memory, then one pair of atomics per CTA.  Every thread of the CTA must call it.
+// live += added - removed, removed-entry count += removed - reused, longest walk = max: summed
+// over the CTA in shared memory, then one atomic each per CTA.  Every thread of the CTA must
+// call it.  The CTA whose addition takes the live count past the table's capacity reports FULL
+// for the entries beyond it (the table has physical room for up to two more than `capacity`,
+// so the count, not the placement, is what keeps the limit exact).
 __device__ __forceinline__ void fold_counters(const IndexView& ix, unsigned int added,
-                                              unsigned int reused, unsigned int removed) {
-  __shared__ unsigned int s_cnt[3];
-  if (threadIdx.x < 3) s_cnt[threadIdx.x] = 0u;
+                                              unsigned int reused, unsigned int removed,
+                                              unsigned int walked) {
+  __shared__ unsigned int s_cnt[4];
+  if (threadIdx.x < 4) s_cnt[threadIdx.x] = 0u;
   __syncthreads();
   const unsigned int a = __reduce_add_sync(0xffffffffu, added);
   const unsigned int u = __reduce_add_sync(0xffffffffu, reused);
   const unsigned int d = __reduce_add_sync(0xffffffffu, removed);
-  if ((threadIdx.x & 31) == 0 && (a | u | d)) {
+  const unsigned int w = __reduce_max_sync(0xffffffffu, walked);
+  if ((threadIdx.x & 31) == 0 && (a | u | d | w)) {
     if (a) atomicAdd(&s_cnt[0], a);
     if (u) atomicAdd(&s_cnt[1], u);
     if (d) atomicAdd(&s_cnt[2], d);
+    if (w) atomicMax(&s_cnt[3], w);
   }
   __syncthreads();
   if (threadIdx.x == 0) {
     const unsigned long long live = (unsigned long long)s_cnt[0] - (unsigned long long)s_cnt[2];
     const unsigned long long tomb = (unsigned long long)s_cnt[2] - (unsigned long long)s_cnt[1];
-    if (live) atomicAdd(&ix.counters[0], live);       // two's complement: may be a decrease
+    if (live) {
+      const unsigned long long before = atomicAdd(&ix.counters[0], live);   // may be a decrease
+      if (s_cnt[0] > s_cnt[2] && before + live > ix.capacity) {
+        const unsigned long long over = before + live - ix.capacity;
+        raise_status_n(AIBX_ERR_FULL, over < live ? over : live);
+      }
+    }
     if (tomb) atomicAdd(&ix.counters[1], tomb);
+    if (s_cnt[3] > 1u) atomicMax(&ix.counters[2], (unsigned long long)s_cnt[3]);
   }
 }
 
@@ -212,13 +258,24 @@ __global__ void index_insert_kernel(IndexView ix, const uint64_t* __restrict__ k
                                     const uint64_t* __restrict__ masks,
                                     const uint32_t* __restrict__ ids, int64_t n) {
   const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-  unsigned int added = 0, reused = 0;
+  unsigned int added = 0, reused = 0, walked = 0;
   if (i < n) {
     const uint64_t key = keys[i];
     const uint64_t m = masks[i] & pod_all(ix.num_pods);
-    if (!key_reserved(key) && m != 0) insert_entry(ix, key, m, ids[i], added, reused);
+    if (!key_reserved(key) && m != 0) insert_entry(ix, key, m, ids[i], added, reused, walked);
   }
-  fold_counters(ix, added, reused, 0u);
+  fold_counters(ix, added, reused, 0u, walked);
+}
+
+// One entry as a scan sees it (entry-parallel kernels: export, move, victim choice).
+__device__ __forceinline__ bool load_entry(const IndexView& ix, unsigned long long e, uint64_t& key,
+                                           uint64_t& mask, uint32_t& id) {
+  const Bucket* b = ix.buckets + e / kBucketEntries;
+  const int j = (int)(e % kBucketEntries);
+  key = __ldg(&b->key[j]);
+  mask = __ldg(&b->mask[j]);
+  id = __ldg(&b->id[j]);
+  return !key_reserved(key) && mask != 0;
 }
 
 // Live entries of the table, in no particular order; *count ends as their number (entries
@@ -231,24 +288,16 @@ __global__ void index_export_kernel(IndexView ix, uint64_t* __restrict__ keys,
                                     unsigned long long* __restrict__ count) {
   __shared__ unsigned int s_warp[32];
   __shared__ unsigned long long s_base;
-  const unsigned long long n = ix.cap_mask + 1;
+  const unsigned long long n = num_entries(ix);
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int n_warps = blockDim.x >> 5;
   for (unsigned long long cta0 = blockIdx.x * (unsigned long long)blockDim.x; cta0 < n;
        cta0 += (unsigned long long)gridDim.x * blockDim.x) {
     const unsigned long long i = cta0 + threadIdx.x;
-    unsigned long long k = 0, m = 0;
+    uint64_t k = 0, m = 0;
     unsigned int id = AIBX_NO_BLOCK;
-    if (i < n) {
-      const uint4* p = reinterpret_cast<const uint4*>(ix.slots + i);
-      const uint4 a = __ldg(p);
-      const uint4 b = __ldg(p + 1);
-      k = (unsigned long long)a.x | ((unsigned long long)a.y << 32);
-      m = (unsigned long long)a.z | ((unsigned long long)a.w << 32);
-      id = b.x;
-    }
-    const bool live = i < n && !key_reserved(k) && m != 0;
+    const bool live = i < n && load_entry(ix, i, k, m, id);
     const unsigned int votes = __ballot_sync(0xffffffffu, live);
     if (lane == 0) s_warp[warp] = __popc(votes);
     __syncthreads();
@@ -276,21 +325,18 @@ __global__ void index_export_kernel(IndexView ix, uint64_t* __restrict__ keys,
 
 // Carry every live entry of one table over into another (larger or smaller) one.
 __global__ void index_move_kernel(IndexView from, IndexView to) {
-  const unsigned long long n = from.cap_mask + 1;
-  unsigned int added = 0, reused = 0;
+  const unsigned long long n = num_entries(from);
+  unsigned int added = 0, reused = 0, walked = 0;
   for (unsigned long long i = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x; i < n;
        i += (unsigned long long)gridDim.x * blockDim.x) {
-    const uint4* p = reinterpret_cast<const uint4*>(from.slots + i);
-    const uint4 a = __ldg(p);
-    const uint4 b = __ldg(p + 1);
-    const unsigned long long k = (unsigned long long)a.x | ((unsigned long long)a.y << 32);
-    const unsigned long long m = (unsigned long long)a.z | ((unsigned long long)a.w << 32);
-    if (!key_reserved(k) && m != 0) {
-      const unsigned long long s = insert_entry(to, k, m, b.x, added, reused);
-      if (s != ~0ULL) to.slots[s].stamp = b.y;          // the touch history moves along
+    uint64_t k, m;
+    uint32_t id;
+    if (load_entry(from, i, k, m, id)) {
+      const unsigned long long e = insert_entry(to, k, m, id, added, reused, walked);
+      if (e != ~0ULL) to.stamps[e] = from.stamps[i];    // the touch history moves along
     }
   }
-  fold_counters(to, added, reused, 0u);
+  fold_counters(to, added, reused, 0u, walked);
 }
 
 // evict, pass 1: clear the named pod bits
@@ -300,9 +346,9 @@ __global__ void index_evict_clear_kernel(IndexView ix, const uint64_t* __restric
   if (i >= n) return;
   const uint64_t key = keys[i];
   if (key_reserved(key)) return;
-  const unsigned long long s = find_slot_rw(ix, key);
-  if (s == ~0ULL) return;
-  atomicAnd(&ix.slots[s].mask, ~(unsigned long long)masks[i]);
+  const unsigned long long e = find_entry_rw(ix, key);
+  if (e == ~0ULL) return;
+  atomicAnd(entry_mask(ix, e), ~(unsigned long long)masks[i]);
 }
 
 // evict, pass 2: report ids of entries left without a pod (every duplicate sees the same state)
@@ -313,10 +359,10 @@ __global__ void index_evict_report_kernel(IndexView ix, const uint64_t* __restri
   const uint64_t key = keys[i];
   uint32_t out = AIBX_NO_BLOCK;
   if (!key_reserved(key)) {
-    const unsigned long long s = find_slot_rw(ix, key);
-    if (s != ~0ULL) {
-      const unsigned long long m = *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].mask);
-      if (m == 0) out = *reinterpret_cast<volatile unsigned int*>(&ix.slots[s].id);
+    const unsigned long long e = find_entry_rw(ix, key);
+    if (e != ~0ULL) {
+      const unsigned long long m = *reinterpret_cast<volatile unsigned long long*>(entry_mask(ix, e));
+      if (m == 0) out = *reinterpret_cast<volatile unsigned int*>(entry_id(ix, e));
     }
   }
   freed[i] = out;
@@ -329,16 +375,16 @@ __global__ void index_evict_remove_kernel(IndexView ix, const uint64_t* __restri
   unsigned int removed = 0;
   const uint64_t key = i < n ? keys[i] : kKeyEmpty;
   if (!key_reserved(key)) {
-    const unsigned long long s = find_slot_rw(ix, key);
-    if (s != ~0ULL &&
-        *reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].mask) == 0 &&
-        atomicCAS(&ix.slots[s].key, (unsigned long long)key, kKeyTomb) == key) {
-      ix.slots[s].id = AIBX_NO_BLOCK;      // ready for reuse by a later insert
-      ix.slots[s].stamp = 0u;
+    const unsigned long long e = find_entry_rw(ix, key);
+    if (e != ~0ULL &&
+        *reinterpret_cast<volatile unsigned long long*>(entry_mask(ix, e)) == 0 &&
+        atomicCAS(entry_key(ix, e), (unsigned long long)key, kKeyTomb) == key) {
+      *entry_id(ix, e) = AIBX_NO_BLOCK;    // ready for reuse by a later insert
+      ix.stamps[e] = 0u;
       removed = 1u;
     }
   }
-  fold_counters(ix, 0u, 0u, removed);     // live -= removed, freed slots += removed
+  fold_counters(ix, 0u, 0u, removed, 0u);   // live -= removed, removed entries += removed
 }
 
 __global__ void index_lookup_kernel(IndexView ix, const uint64_t* __restrict__ keys,
@@ -374,6 +420,14 @@ __device__ __forceinline__ void fold_chunk(PrefixFold& st, int lane, unsigned in
                                            uint32_t id, uint64_t all, unsigned int* ml,
                                            uint32_t* block_ids_at) {
   const bool valid = (unsigned int)lane < m;
+  // The common chunk changes nothing: every block of it is held by every pod still alive (so
+  // none is a total miss either).  One vote instead of the scan below.
+  if (st.alive != 0 &&
+      __all_sync(0xffffffffu, !valid || (mask & st.alive) == st.alive)) {
+    if (valid && block_ids_at) block_ids_at[st.pos + lane] = id;
+    st.pos += m;
+    return;
+  }
   const unsigned int none = __ballot_sync(0xffffffffu, valid && mask == 0);
   const unsigned int f = none ? (unsigned int)__ffs(none) - 1u : 32u;   // first total miss
   uint64_t pref = valid ? mask : all;
@@ -446,7 +500,7 @@ __device__ __forceinline__ void fold_finish(const PrefixFold& st, int lane, int 
 // are warps enough without splitting a request.  No barrier, no shared-memory atomics.
 constexpr int kMatchWarpKernelWarps = 4;
 
-__global__ void __launch_bounds__(kMatchWarpKernelWarps * 32, 16)
+__global__ void __launch_bounds__(kMatchWarpKernelWarps * 32, 12)
 match_prefix_warp_kernel(IndexView ix, const uint64_t* __restrict__ hashes,
                          const int64_t* __restrict__ blk_off, int R,
                          uint32_t* __restrict__ match_len, uint32_t* __restrict__ any_len,

@@ -64,6 +64,32 @@ void prefer_copy_carveout() {
   });
 }
 
+// Device storage of one table: buckets, stamps and counters in ONE allocation (64-byte aligned
+// parts), so that creating or dropping a table is one call into the allocator.
+int32_t alloc_view(uint64_t capacity, int num_pods, IndexView* out) {
+  const uint64_t nb = (capacity + kBucketEntries - 1) / kBucketEntries;
+  const size_t bucket_bytes = (size_t)nb * sizeof(Bucket);
+  const size_t stamp_bytes = ((size_t)nb * kBucketEntries * sizeof(unsigned int) + 63) & ~(size_t)63;
+  void* base = nullptr;
+  if (cudaMalloc(&base, bucket_bytes + stamp_bytes + 64) != cudaSuccess) {
+    cudaGetLastError();   // an allocation failure is not sticky; leave no error behind
+    return AIBX_ERR_NOMEM;
+  }
+  char* p = static_cast<char*>(base);
+  out->buckets = reinterpret_cast<Bucket*>(p);
+  out->stamps = reinterpret_cast<unsigned int*>(p + bucket_bytes);
+  out->counters = reinterpret_cast<unsigned long long*>(p + bucket_bytes + stamp_bytes);
+  out->nb = nb;
+  out->capacity = capacity;
+  out->max_walk = (unsigned int)(nb < kMaxWalk ? nb : kMaxWalk);
+  out->num_pods = num_pods;
+  return AIBX_OK;
+}
+
+void free_view(const IndexView& v) { cudaFree(v.buckets); }
+
+bool capacity_ok(uint64_t c) { return c >= 8 && (c & (c - 1)) == 0 && c <= (1ULL << 40); }
+
 // Device address of the status record of the current device.
 StatusRecord* status_ptr() {
   static std::atomic<StatusRecord*> cached[64];
@@ -126,37 +152,25 @@ int32_t aibx_index_create(aibx_index_t** out, uint64_t capacity_slots, int32_t n
   if (!out) return AIBX_ERR_INVALID;
   *out = nullptr;
   if (num_pods < 1 || num_pods > AIBX_MAX_PODS) return AIBX_ERR_INVALID;
-  if (capacity_slots < 8 || (capacity_slots & (capacity_slots - 1)) != 0) return AIBX_ERR_INVALID;
-  if (capacity_slots > (1ULL << 40)) return AIBX_ERR_INVALID;
+  if (!capacity_ok(capacity_slots)) return AIBX_ERR_INVALID;
   aibx_index* ix = new (std::nothrow) aibx_index();
   if (!ix) return AIBX_ERR_NOMEM;
-  int log2cap = 0;
-  while ((1ULL << log2cap) < capacity_slots) ++log2cap;
   if (cudaGetDevice(&ix->device) != cudaSuccess) {
     delete ix;
     return AIBX_ERR_CUDA;
   }
-  void* slots = nullptr;
-  void* counters = nullptr;
-  if (cudaMalloc(&slots, capacity_slots * sizeof(Slot)) != cudaSuccess ||
-      cudaMalloc(&counters, 2 * sizeof(unsigned long long)) != cudaSuccess) {
-    cudaGetLastError();   // clear the sticky-free allocation error
-    if (slots) cudaFree(slots);
+  const int32_t rc = alloc_view(capacity_slots, num_pods, &ix->view);
+  if (rc != AIBX_OK) {
     delete ix;
-    return AIBX_ERR_NOMEM;
+    return rc;
   }
   ix->capacity = capacity_slots;
   ix->migrating = false;
   ix->moved = nullptr;
-  ix->view.slots = static_cast<Slot*>(slots);
-  ix->view.cap_mask = capacity_slots - 1;
-  ix->view.shift = 64 - log2cap;
-  ix->view.num_pods = num_pods;
-  ix->view.counters = static_cast<unsigned long long*>(counters);
   index_clear_kernel<<<sm_count() * 8, 256>>>(ix->view);
   if (cudaDeviceSynchronize() != cudaSuccess) {
-    cudaFree(slots);
-    cudaFree(counters);
+    cudaGetLastError();
+    free_view(ix->view);
     delete ix;
     return AIBX_ERR_CUDA;
   }
@@ -167,13 +181,9 @@ int32_t aibx_index_create(aibx_index_t** out, uint64_t capacity_slots, int32_t n
 int32_t aibx_index_destroy(aibx_index_t* ix) {
   if (!ix) return AIBX_ERR_INVALID;
   cudaDeviceSynchronize();
-  if (ix->migrating) {
-    cudaFree(ix->pending.slots);
-    cudaFree(ix->pending.counters);
-  }
+  if (ix->migrating) free_view(ix->pending);
   if (ix->moved) cudaEventDestroy(ix->moved);
-  cudaFree(ix->view.slots);
-  cudaFree(ix->view.counters);
+  free_view(ix->view);
   if (ix->victim_scratch) cudaFree(ix->victim_scratch);
   delete ix;
   return AIBX_OK;
@@ -221,17 +231,26 @@ int32_t aibx_index_lookup(const aibx_index_t* ix, const uint64_t* d_keys, uint64
   return launch_status();
 }
 
-int32_t aibx_index_stats(const aibx_index_t* ix, uint64_t* live, uint64_t* capacity,
-                         void* stream) {
+int32_t aibx_index_stats2(const aibx_index_t* ix, uint64_t* live, uint64_t* removed,
+                          uint64_t* capacity, uint32_t* longest_walk, void* stream) {
   if (!ix) return AIBX_ERR_INVALID;
-  unsigned long long c[2] = {0, 0};
+  unsigned long long c[3] = {0, 0, 0};
   if (cudaMemcpyAsync(c, ix->view.counters, sizeof(c), cudaMemcpyDeviceToHost,
                       as_stream(stream)) != cudaSuccess ||
-      cudaStreamSynchronize(as_stream(stream)) != cudaSuccess)
+      cudaStreamSynchronize(as_stream(stream)) != cudaSuccess) {
+    cudaGetLastError();
     return AIBX_ERR_CUDA;
+  }
   if (live) *live = c[0];
+  if (removed) *removed = c[1];
   if (capacity) *capacity = ix->capacity;
+  if (longest_walk) *longest_walk = c[2] ? (uint32_t)c[2] : 1u;   // a walk visits at least one bucket
   return AIBX_OK;
+}
+
+int32_t aibx_index_stats(const aibx_index_t* ix, uint64_t* live, uint64_t* capacity,
+                         void* stream) {
+  return aibx_index_stats2(ix, live, nullptr, capacity, nullptr, stream);
 }
 
 int32_t aibx_index_touch(aibx_index_t* ix, const uint64_t* d_keys, int64_t n, uint32_t epoch,
@@ -286,32 +305,24 @@ int32_t aibx_index_export(const aibx_index_t* ix, uint64_t* d_keys, uint64_t* d_
 
 int32_t aibx_index_rehash(aibx_index_t* ix, uint64_t new_capacity) {
   if (!ix || ix->migrating) return AIBX_ERR_INVALID;
-  if (new_capacity < 8 || (new_capacity & (new_capacity - 1)) != 0 || new_capacity > (1ULL << 40))
-    return AIBX_ERR_INVALID;
+  if (!capacity_ok(new_capacity)) return AIBX_ERR_INVALID;
   if (cudaDeviceSynchronize() != cudaSuccess) return AIBX_ERR_CUDA;
-  unsigned long long c[2] = {0, 0};
-  if (cudaMemcpy(c, ix->view.counters, sizeof(c), cudaMemcpyDeviceToHost) != cudaSuccess)
+  unsigned long long live = 0;
+  if (cudaMemcpy(&live, ix->view.counters, sizeof(live), cudaMemcpyDeviceToHost) != cudaSuccess)
     return AIBX_ERR_CUDA;
-  if (c[0] > new_capacity) return AIBX_ERR_FULL;
-  void* slots = nullptr;
-  if (cudaMalloc(&slots, new_capacity * sizeof(Slot)) != cudaSuccess) {
-    cudaGetLastError();
-    return AIBX_ERR_NOMEM;
-  }
-  int log2cap = 0;
-  while ((1ULL << log2cap) < new_capacity) ++log2cap;
-  IndexView fresh = ix->view;
-  fresh.slots = static_cast<Slot*>(slots);
-  fresh.cap_mask = new_capacity - 1;
-  fresh.shift = 64 - log2cap;
+  if (live > new_capacity) return AIBX_ERR_FULL;
+  IndexView fresh;
+  const int32_t rc = alloc_view(new_capacity, ix->view.num_pods, &fresh);
+  if (rc != AIBX_OK) return rc;
   const IndexView old = ix->view;
-  index_clear_kernel<<<sm_count() * 8, 256>>>(fresh);          // also zeroes the shared counters
+  index_clear_kernel<<<sm_count() * 8, 256>>>(fresh);
   index_move_kernel<<<sm_count() * 8, 256>>>(old, fresh);      // re-counts the live entries
   if (cudaDeviceSynchronize() != cudaSuccess) {
-    cudaFree(slots);
+    cudaGetLastError();
+    free_view(fresh);
     return AIBX_ERR_CUDA;
   }
-  cudaFree(old.slots);
+  free_view(old);
   ix->view = fresh;
   ix->capacity = new_capacity;
   return AIBX_OK;
@@ -319,41 +330,28 @@ int32_t aibx_index_rehash(aibx_index_t* ix, uint64_t new_capacity) {
 
 int32_t aibx_index_rehash_begin(aibx_index_t* ix, uint64_t new_capacity, void* stream) {
   if (!ix || ix->migrating) return AIBX_ERR_INVALID;
-  if (new_capacity < 8 || (new_capacity & (new_capacity - 1)) != 0 || new_capacity > (1ULL << 40))
-    return AIBX_ERR_INVALID;
+  if (!capacity_ok(new_capacity)) return AIBX_ERR_INVALID;
   cudaStream_t st = as_stream(stream);
   // the live count as of `stream` (only this stream is waited for, not the device)
-  unsigned long long c[2] = {0, 0};
-  if (cudaMemcpyAsync(c, ix->view.counters, sizeof(c), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+  unsigned long long live = 0;
+  if (cudaMemcpyAsync(&live, ix->view.counters, sizeof(live), cudaMemcpyDeviceToHost, st) !=
+          cudaSuccess ||
       cudaStreamSynchronize(st) != cudaSuccess)
     return AIBX_ERR_CUDA;
-  if (c[0] > new_capacity) return AIBX_ERR_FULL;
+  if (live > new_capacity) return AIBX_ERR_FULL;
   if (!ix->moved &&
       cudaEventCreateWithFlags(&ix->moved, cudaEventDisableTiming) != cudaSuccess) {
     ix->moved = nullptr;
     return AIBX_ERR_CUDA;
   }
-  void* slots = nullptr;
-  void* counters = nullptr;
-  if (cudaMalloc(&slots, new_capacity * sizeof(Slot)) != cudaSuccess ||
-      cudaMalloc(&counters, 2 * sizeof(unsigned long long)) != cudaSuccess) {
-    cudaGetLastError();
-    if (slots) cudaFree(slots);
-    return AIBX_ERR_NOMEM;
-  }
-  int log2cap = 0;
-  while ((1ULL << log2cap) < new_capacity) ++log2cap;
-  IndexView fresh = ix->view;
-  fresh.slots = static_cast<Slot*>(slots);
-  fresh.counters = static_cast<unsigned long long*>(counters);   // its own: `view` stays intact
-  fresh.cap_mask = new_capacity - 1;
-  fresh.shift = 64 - log2cap;
+  IndexView fresh;                                       // its own storage: `view` stays intact
+  const int32_t rc = alloc_view(new_capacity, ix->view.num_pods, &fresh);
+  if (rc != AIBX_OK) return rc;
   index_clear_kernel<<<sm_count() * 8, 256, 0, st>>>(fresh);
   index_move_kernel<<<sm_count() * 8, 256, 0, st>>>(ix->view, fresh);
   if (cudaEventRecord(ix->moved, st) != cudaSuccess || launch_status() != AIBX_OK) {
     cudaStreamSynchronize(st);
-    cudaFree(slots);
-    cudaFree(counters);
+    free_view(fresh);
     return AIBX_ERR_CUDA;
   }
   ix->pending = fresh;
@@ -370,8 +368,7 @@ int32_t aibx_index_rehash_finish(aibx_index_t* ix) {
   ix->capacity = ix->pending_capacity;
   ix->migrating = false;
   // cudaFree waits for the work still using the old table (readers launched before the switch)
-  cudaFree(old.slots);
-  cudaFree(old.counters);
+  free_view(old);
   return AIBX_OK;
 }
 

@@ -1,6 +1,6 @@
 // Scan-resistant victim choice on the GPU-resident index.
 //
-// Every slot carries a 32-bit stamp: bits 0..29 the last epoch in which the entry was touched
+// Every entry has a 32-bit stamp (side array of the index): bits 0..29 the last epoch in which the entry was touched
 // (0 = never), bits 30..31 the number of distinct epochs it was touched in, saturating at 3.
 // priority = (touches >= 2 ? 2^30 : 0) + epoch: entries seen in fewer than two epochs - what a
 // single scan leaves behind - go first, oldest first.
@@ -47,10 +47,10 @@ __global__ void index_touch_kernel(IndexView ix, const uint64_t* __restrict__ ke
   if (i >= n) return;
   const uint64_t key = keys[i];
   if (key_reserved(key)) return;
-  const unsigned long long s = find_slot_rw(ix, key);
-  if (s == ~0ULL) return;
-  if (*reinterpret_cast<volatile unsigned long long*>(&ix.slots[s].mask) == 0) return;
-  unsigned int* stamp = &ix.slots[s].stamp;
+  const unsigned long long e = find_entry_rw(ix, key);
+  if (e == ~0ULL) return;
+  if (*reinterpret_cast<volatile unsigned long long*>(entry_mask(ix, e)) == 0) return;
+  unsigned int* stamp = &ix.stamps[e];
   unsigned int old = *reinterpret_cast<volatile unsigned int*>(stamp);
   // several touches of one key in one epoch count once, whoever gets there first
   for (int tries = 0; tries < 64; ++tries) {
@@ -63,16 +63,14 @@ __global__ void index_touch_kernel(IndexView ix, const uint64_t* __restrict__ ke
   }
 }
 
-// Reads one slot; returns whether it holds a live entry.
+// Reads one entry; returns whether it is live.
 __device__ __forceinline__ bool live_slot(const IndexView& ix, unsigned long long i, uint64_t& key,
                                           unsigned int& prio) {
-  const uint4* p = reinterpret_cast<const uint4*>(ix.slots + i);
-  const uint4 a = __ldg(p);
-  const uint4 b = __ldg(p + 1);
-  key = (uint64_t)a.x | ((uint64_t)a.y << 32);
-  const uint64_t m = (uint64_t)a.z | ((uint64_t)a.w << 32);
-  prio = stamp_priority(b.y);
-  return !key_reserved(key) && m != 0;
+  uint64_t m;
+  uint32_t id;
+  const bool live = load_entry(ix, i, key, m, id);
+  prio = live ? stamp_priority(__ldcg(ix.stamps + i)) : 0u;
+  return live;
 }
 
 // Histogram pass.  Priorities cluster (few distinct epochs), so (1) lanes of a warp that hit the
@@ -86,7 +84,7 @@ __global__ void __launch_bounds__(256)
 victims_hist_kernel(IndexView ix, VictimScratch* sc, int level) {
   __shared__ unsigned int s_bin[kHistCache];
   __shared__ unsigned int s_cnt[kHistCache];
-  const unsigned long long n = ix.cap_mask + 1;
+  const unsigned long long n = num_entries(ix);
   const unsigned int prefix = level == 2 ? sc->st.prefix : 0u;
   if (level == 2 && prefix == 0xFFFFFFFFu) return;       // everything is taken: no second level
   unsigned int* hist = level == 1 ? sc->hist1 : sc->hist2;
@@ -202,7 +200,7 @@ victims_collect_kernel(IndexView ix, VictimScratch* sc, uint64_t* __restrict__ o
                        uint32_t* __restrict__ out_prio) {
   __shared__ unsigned int s_eq[8], s_take[8];
   __shared__ unsigned long long s_eq_base, s_out_base;
-  const unsigned long long n = ix.cap_mask + 1;
+  const unsigned long long n = num_entries(ix);
   const unsigned int T = sc->st.threshold;
   const unsigned long long need_eq = sc->st.need_eq;
   const unsigned long long k = sc->st.k;

@@ -604,3 +604,59 @@ def test_index_duplicate_heavy_random_batches():
             checked += 1
         g.destroy()
     assert checked == 960
+
+
+def test_churn_fills_the_table_with_removed_entries_and_rehash_clears_them():
+    """Publish/expire churn in a 64-slot table: every batch inserts fresh keys and evicts them
+    again.  Live entries stay few, but never-used entries run out, so a probe for an absent key
+    has to walk further and further; stats2 shows it (removed count, longest insert walk), the
+    walk stays bounded, results stay those of the oracle, and a rehash to the same size brings
+    the probes back to one bucket."""
+    rng = np.random.default_rng(64)
+    g, o = aibx.Index(64, 4), oracle.Index(64, 4)
+    keep = rng.integers(1, 1 << 62, 10).astype(np.uint64)            # entries that stay
+    km, ki = np.full(10, 5, np.uint64), np.arange(10, dtype=np.uint32)
+    g.insert(dev(keep), dev(km), dev(ki)); o.insert(keep, km, ki)
+    probe = np.concatenate([keep, rng.integers(1, 1 << 62, 200).astype(np.uint64)])
+    ones = np.full(16, ALL, np.uint64)
+    for batch in range(12):
+        fresh = rng.integers(1, 1 << 62, 16).astype(np.uint64)
+        m, i = np.full(16, 3, np.uint64), rng.integers(0, 100, 16).astype(np.uint32)
+        g.insert(dev(fresh), dev(m), dev(i)); assert o.insert(fresh, m, i) == oracle.OK
+        d_f = empty(16, torch.uint32)
+        g.evict(dev(fresh), dev(ones), d_f)
+        rc, want = o.evict(fresh, ones)
+        assert np.array_equal(host(d_f), want)
+        d_m, d_i = empty(len(probe), torch.uint64), empty(len(probe), torch.uint32)
+        g.lookup(dev(probe), d_m, d_i)
+        wm, wi = o.lookup(probe)
+        assert np.array_equal(host(d_m), wm) and np.array_equal(host(d_i), wi)
+        assert aibx.status_fetch() == (0, 0)
+    live, removed, cap, walk = g.stats2()
+    assert (live, cap) == (10, 64) == (o.stats()[0], 64)
+    # 66 entries of physical room, 10 live: after 192 publish/expire pairs none was never used
+    assert 16 <= removed <= 56 and live + removed <= 66
+    assert 1 <= walk <= 22                                            # 22 buckets = the whole table
+    g.rehash(64)
+    live, removed, cap, walk = g.stats2()
+    assert (live, removed, cap) == (10, 0, 64) and walk <= 3
+    d_m, d_i = empty(len(probe), torch.uint64), empty(len(probe), torch.uint32)
+    g.lookup(dev(probe), d_m, d_i)
+    wm, wi = o.lookup(probe)
+    assert np.array_equal(host(d_m), wm) and np.array_equal(host(d_i), wi)
+    assert aibx.status_fetch() == (0, 0)
+
+
+def test_full_counts_the_entries_in_excess_of_capacity():
+    """capacity is a limit on live entries, kept by counting: 70 distinct keys into a 64-slot
+    table report FULL with detail 6, as the oracle does for the 65th key on."""
+    g, o = aibx.Index(64, 2), oracle.Index(64, 2)
+    keys = np.arange(1, 71, dtype=np.uint64) * np.uint64(0x9E3779B97F4A7C15)
+    m, i = np.ones(70, np.uint64), np.zeros(70, np.uint32)
+    assert o.insert(keys[:64], m[:64], i[:64]) == oracle.OK
+    g.insert(dev(keys[:64]), dev(m[:64]), dev(i[:64]))
+    assert aibx.status_fetch() == (0, 0) and g.stats() == (64, 64)
+    assert o.insert(keys[64:], m[64:], i[64:]) == oracle.ERR_FULL
+    g.insert(dev(keys[64:]), dev(m[64:]), dev(i[64:]))
+    st, detail = aibx.status_fetch()
+    assert st == aibx.ERR_FULL and detail == 6
