@@ -106,6 +106,12 @@ def case_kv_small(args):
                       "status": aibx.status_fetch()}))
 
 
+def index_table_bytes(slots: int) -> int:
+    """Bytes a probe can touch: ceil(slots / 3) buckets of 64 bytes (the 4-byte eviction stamps
+    per entry are a separate array that lookups never read)."""
+    return (slots + 2) // 3 * 64
+
+
 def _big_index(torch, aibx, W, log2cap, P, seed):
     """Index of 2^log2cap slots at load 0.5 filled with random keys (all pods resident)."""
     cap = 1 << log2cap
@@ -126,6 +132,7 @@ def _random_read_ceiling(torch, ws_bytes, gran, flush, t_flush, n=1 << 24):
     and 4 independent reads per thread)."""
     from workloads import synth
 
+    ws_bytes = (ws_bytes + 127) // 128 * 128
     base = torch.empty(ws_bytes // 8, dtype=torch.int64, device="cuda")
     base.zero_()
     best = 0.0
@@ -145,10 +152,12 @@ def _random_read_ceiling(torch, ws_bytes, gran, flush, t_flush, n=1 << 24):
 def measure_match_large(log2cap, Rs=(262144,), steps=7, with_ceiling=True):
     """Prefix match at a size where a bandwidth roofline means something: an index of 2^log2cap
     slots (load 0.5, 32 pods), R requests of 64 blocks, every block resident, so all 64 lookups
-    of a request are necessary.  Algorithmic bytes: 8 + 32 per lookup, 4*P + 4*64 + 4 out per
-    request.  L2 is evicted by a 256 MiB read before every launch (its time subtracted).  Two
-    denominators: the measured stream bandwidth, and the measured rate of random 32-byte reads
-    over a working set of the table's size (one read per lookup is the least the method needs)."""
+    of a request are necessary.  Algorithmic bytes: 8 (key) + 32 (key, mask and id of one entry,
+    rounded up to a sector) per lookup, 4*P + 4*64 + 4 out per request.  L2 is evicted by a
+    256 MiB read before every launch (its time subtracted).  Two denominators: the measured
+    stream bandwidth, and the measured rate of random 32-byte reads over a working set of the
+    table's own size (one read per lookup is the least the method needs; on this GPU a read that
+    misses L2 always moves a whole 128-byte line from DRAM, whatever it asked for)."""
     import torch
 
     from paper_2504_03648_b200 import binding as aibx
@@ -159,7 +168,8 @@ def measure_match_large(log2cap, Rs=(262144,), steps=7, with_ceiling=True):
     flush = torch.empty(64 << 20, dtype=torch.int32, device="cuda")
     t_flush = statistics.median(_event_times(torch, lambda: flush.sum(), max(steps, 5), 3))
     peak, kind = measured_peak_hbm()
-    ceiling = _random_read_ceiling(torch, 32 << log2cap, 32, flush, t_flush) if with_ceiling else None
+    table_bytes = index_table_bytes(1 << log2cap)
+    ceiling = _random_read_ceiling(torch, table_bytes, 32, flush, t_flush) if with_ceiling else None
     out = []
     for R in Rs:
         st = W.Stream(12, R)
@@ -187,7 +197,7 @@ def measure_match_large(log2cap, Rs=(262144,), steps=7, with_ceiling=True):
         del d_h, d_bo, d_ml, d_al, d_ids
     status = aibx.status_fetch()
     ix.destroy()
-    res = {"index_slots": 1 << log2cap, "table_MiB": (32 << log2cap) >> 20, "pods": P,
+    res = {"index_slots": 1 << log2cap, "table_MiB": round(table_bytes / 2 ** 20, 1), "pods": P,
            "blocks_per_request": nblk,
            "l2": "evicted before every launch (256 MiB read, its time subtracted)",
            "peak": peak, "peak_kind": kind, "results": out, "status": status}
@@ -212,7 +222,7 @@ def case_random_reads(args):
     t_flush = statistics.median(_event_times(torch, lambda: flush.sum(), 7, 3))
     peak, kind = measured_peak_hbm()
     rows = []
-    for ws_mib in (16, 64, 256, 1024, 4096):
+    for ws_mib in (11, 16, 43, 64, 171, 256, 1024, 4096):
         for gran in (32, 64, 128):
             g = _random_read_ceiling(torch, ws_mib << 20, gran, flush, t_flush)
             rows.append({"working_set_MiB": ws_mib, "read_bytes": gran, "Greads_per_s": round(g, 2),
@@ -506,7 +516,7 @@ def measure_lookup_flat(log2caps=(11, 19, 21, 23), reps=7, with_library=True):
         t_cold = statistics.median(_event_times(torch, cold, reps, 2)) - t_flush
         t_warm = statistics.median(_event_times(torch, lambda: ix.lookup(d_q, d_m, d_i), reps, 2))
         nbytes = n * (8 + 32 + 12)
-        row = {"slots": 1 << log2cap, "table_MiB": (32 << log2cap) >> 20,
+        row = {"slots": 1 << log2cap, "table_MiB": round(index_table_bytes(1 << log2cap) / 2 ** 20, 2),
                "cold_ms": round(t_cold, 4), "warm_ms": round(t_warm, 4),
                "cold_Glookups_per_s": round(n / (t_cold * 1e-3) / 1e9, 2),
                "warm_Glookups_per_s": round(n / (t_warm * 1e-3) / 1e9, 2),
@@ -515,7 +525,7 @@ def measure_lookup_flat(log2caps=(11, 19, 21, 23), reps=7, with_library=True):
                "cold_frac": round(nbytes / (t_cold * 1e-3) / 1e9 / peak, 4),
                "warm_frac": round(nbytes / (t_warm * 1e-3) / 1e9 / peak, 4)}
         if log2cap >= 12:
-            ceiling = _random_read_ceiling(torch, 32 << log2cap, 32, flush, t_flush)
+            ceiling = _random_read_ceiling(torch, index_table_bytes(1 << log2cap), 32, flush, t_flush)
             row["random_32B_read_ceiling_Greads_per_s"] = round(ceiling, 2)
             row["cold_frac_of_random_read_ceiling"] = round(n / (t_cold * 1e-3) / 1e9 / ceiling, 4)
         if with_library:
@@ -868,6 +878,58 @@ def case_index_ops(args):
     bs = torch.empty(R, dtype=torch.int64, device="cuda")
     ts = _event_times(torch, lambda: aibx.route_assign(ml, bo, P, load, (1 << 64) - 1, None, 1, bp, bs), 7, 2)
     res["route_assign_4096_requests_64_pods_us"] = round(statistics.median(ts) * 1e3, 1)
+    # matching alone against matching that also stamps the matched prefix (a new epoch per call,
+    # so every call writes its stamps), on the routing-heavy batch
+    w = W.build_routing(W.cfg3_routing())
+    s3 = w.spec
+    B, P3, R3 = s3.block_tokens, s3.num_pods, s3.R
+
+    def offsets(tok_off):
+        k = (tok_off[1:] - tok_off[:-1]) // B
+        o = np.zeros(len(tok_off), dtype=np.int64)
+        np.cumsum(k, out=o[1:])
+        return o
+
+    def dev(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+    bo3, sbo3 = offsets(w.tok_off), offsets(w.src_tok_off)
+    d_bo3 = dev(bo3)
+    d_h3 = torch.empty(int(bo3[-1]), dtype=torch.uint64, device="cuda")
+    d_sh3 = torch.empty(int(sbo3[-1]), dtype=torch.uint64, device="cuda")
+    aibx.hash_blocks(dev(w.tokens), dev(w.tok_off), d_bo3, B, 0, d_h3)
+    aibx.hash_blocks(dev(w.src_tokens), dev(w.src_tok_off), dev(sbo3), B, 0, d_sh3)
+    ix3 = aibx.Index(s3.capacity, P3)
+    ix3.insert(torch.cat([d_sh3, dev(w.filler_keys)]),
+               dev(np.concatenate([w.src_masks, w.filler_masks])),
+               dev(np.concatenate([w.src_ids, w.filler_ids])))
+    d_ml3 = torch.empty(R3 * P3, dtype=torch.uint32, device="cuda")
+    d_al3 = torch.empty(R3, dtype=torch.uint32, device="cuda")
+    d_id3 = torch.empty(int(bo3[-1]), dtype=torch.uint32, device="cuda")
+    epoch = [0]
+
+    def match_touch():
+        epoch[0] += 1
+        ix3.match_prefix_touch(d_h3, d_bo3, epoch[0], d_ml3, d_al3, d_id3)
+
+    t_m = statistics.median(_event_times(
+        torch, lambda: ix3.match_prefix(d_h3, d_bo3, d_ml3, d_al3, d_id3), 15, 3))
+    t_mt = statistics.median(_event_times(torch, match_touch, 15, 3))
+    hit = d_h3[:1]
+    keys_hit = torch.cat([d_h3[int(bo3[r]): int(bo3[r]) + int(a)]
+                          for r, a in enumerate(d_al3.cpu().numpy()) if a > 0] or [hit])
+
+    def separate():
+        epoch[0] += 1
+        ix3.match_prefix(d_h3, d_bo3, d_ml3, d_al3, d_id3)
+        ix3.touch(keys_hit, epoch[0])
+
+    t_sep = statistics.median(_event_times(torch, separate, 15, 3))
+    res["cfg3_match_us"] = round(t_m * 1e3, 1)
+    res["cfg3_match_touch_us"] = round(t_mt * 1e3, 1)
+    res["cfg3_match_then_touch_as_two_calls_us"] = round(t_sep * 1e3, 1)
+    res["cfg3_matched_blocks_stamped"] = int(keys_hit.numel())
+    res["cfg3_match_touch_over_match"] = round(t_mt / t_m, 3)
     print(json.dumps({"case": "index_ops", "entries": n, "results": res,
                       "status": aibx.status_fetch()}))
 

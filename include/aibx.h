@@ -191,6 +191,17 @@ int32_t aibx_match_prefix(const aibx_index_t* index, const uint64_t* d_hashes,
                           const int64_t* d_blk_off, int32_t R, uint32_t* d_match_len,
                           uint32_t* d_any_len, uint32_t* d_block_ids, void* stream);
 
+/* The same, and every entry of the matched prefix of every request (blocks below any_len[r])
+ * is marked as used in `epoch`, exactly as aibx_index_touch of those keys would (Section 3.2.5,
+ * scan-resistant eviction: what routing hits is what is hot).  The stamp is written while the
+ * probe still has the entry in hand, so matching and touching cost one pass over the index
+ * instead of two.  epoch in 1..2^30-1; INVALID otherwise and while a rehash is under way.
+ */
+int32_t aibx_match_prefix_touch(aibx_index_t* index, const uint64_t* d_hashes,
+                                const int64_t* d_blk_off, int32_t R, uint32_t epoch,
+                                uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
+                                void* stream);
+
 /* ---------------------------------------------------------------------------------------
  * Prefix-and-load route score (Section 3.2.2: prefix-cache-aware prefers instances whose
  * cache hit exceeds a threshold; least-request prefers the lowest number of admitted
@@ -258,6 +269,18 @@ int32_t aibx_route_head(const aibx_index_t* index, const int32_t* d_tokens,
                         uint64_t* d_hashes, uint32_t* d_match_len, uint32_t* d_any_len,
                         uint32_t* d_block_ids, int32_t* d_best_pod, int64_t* d_best_score,
                         uint32_t* d_hashed, uint64_t* d_next_seed, void* stream);
+
+/* aibx_route_head that also marks the entries of every request's matched prefix as used in
+ * `epoch` (see aibx_match_prefix_touch): the prober that has just found an entry stamps it.
+ */
+int32_t aibx_route_head_touch(aibx_index_t* index, const int32_t* d_tokens,
+                              const int64_t* d_tok_off, const int64_t* d_blk_off, int32_t R,
+                              int32_t block_tokens, uint64_t root_seed, const int32_t* d_pod_load,
+                              uint64_t ready_mask, const aibx_route_params_t* params,
+                              uint32_t epoch, uint64_t* d_hashes, uint32_t* d_match_len,
+                              uint32_t* d_any_len, uint32_t* d_block_ids, int32_t* d_best_pod,
+                              int64_t* d_best_score, uint32_t* d_hashed, uint64_t* d_next_seed,
+                              void* stream);
 int32_t aibx_hash_blocks_resume(const int32_t* d_tokens, const int64_t* d_tok_off,
                                 const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
                                 const uint32_t* d_hashed, const uint64_t* d_next_seed,

@@ -98,6 +98,9 @@ def lib():
             "aibx_route_assign": [vp, vp, i32, i32, vp, u64, C.POINTER(RouteParams), i32, vp, vp, vp],
             "aibx_route_head": [vp, vp, vp, vp, i32, i32, u64, vp, u64, C.POINTER(RouteParams),
                                 vp, vp, vp, vp, vp, vp, vp, vp, vp],
+            "aibx_route_head_touch": [vp, vp, vp, vp, i32, i32, u64, vp, u64, C.POINTER(RouteParams),
+                                      u32, vp, vp, vp, vp, vp, vp, vp, vp, vp],
+            "aibx_match_prefix_touch": [vp, vp, vp, i32, u32, vp, vp, vp, vp],
             "aibx_hash_blocks_resume": [vp, vp, vp, i32, i32, vp, vp, vp, vp],
             "aibx_route_policy": [i32, vp, vp, i32, i32, C.POINTER(PodMetrics), vp, u64, i32, vp, vp],
             "aibx_collect_blocks": [vp, i64, u32, vp, vp, vp, vp],
@@ -256,6 +259,15 @@ class Index:
             _ptr(match_len, torch.uint32), _ptr(any_len, torch.uint32),
             _ptr(block_ids, torch.uint32), _stream()))
 
+    def match_prefix_touch(self, hashes, blk_off, epoch: int, match_len, any_len=None,
+                           block_ids=None) -> None:
+        """match_prefix that also marks the entries of every matched prefix as used in `epoch`."""
+        R = blk_off.numel() - 1
+        _check("aibx_match_prefix_touch", lib().aibx_match_prefix_touch(
+            self._h, _ptr(hashes, torch.uint64), _ptr(blk_off, torch.int64), R, epoch,
+            _ptr(match_len, torch.uint32), _ptr(any_len, torch.uint32),
+            _ptr(block_ids, torch.uint32), _stream()))
+
 
 def route_score(match_len, blk_off, num_pods: int, pod_load, ready_mask: int, params,
                 best_pod, best_score, scores=None) -> None:
@@ -294,6 +306,21 @@ def route_head(index: Index, tokens, tok_off, blk_off, block_tokens: int, root_s
         _ptr(any_len, torch.uint32), _ptr(block_ids, torch.uint32), _ptr(best_pod, torch.int32),
         _ptr(best_score, torch.int64), _ptr(hashed, torch.uint32), _ptr(next_seed, torch.uint64),
         _stream()))
+
+
+def route_head_touch(index: Index, tokens, tok_off, blk_off, block_tokens: int, root_seed: int,
+                     pod_load, ready_mask: int, params, epoch: int, hashes, match_len, any_len,
+                     block_ids, best_pod, best_score, hashed, next_seed) -> None:
+    """route_head that also marks the entries of every matched prefix as used in `epoch`."""
+    R = tok_off.numel() - 1
+    prm = None if params is None else C.byref(RouteParams(*params))
+    _check("aibx_route_head_touch", lib().aibx_route_head_touch(
+        index._h, _ptr(tokens, torch.int32), _ptr(tok_off, torch.int64), _ptr(blk_off, torch.int64),
+        R, block_tokens, root_seed & (2**64 - 1), _ptr(pod_load, torch.int32),
+        ready_mask & (2**64 - 1), prm, epoch, _ptr(hashes, torch.uint64),
+        _ptr(match_len, torch.uint32), _ptr(any_len, torch.uint32), _ptr(block_ids, torch.uint32),
+        _ptr(best_pod, torch.int32), _ptr(best_score, torch.int64), _ptr(hashed, torch.uint32),
+        _ptr(next_seed, torch.uint64), _stream()))
 
 
 def hash_blocks_resume(tokens, tok_off, blk_off, block_tokens: int, hashed, next_seed,

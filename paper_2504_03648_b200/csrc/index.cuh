@@ -89,10 +89,12 @@ __global__ void index_clear_kernel(IndexView ix) {
 
 // Read-only probe: a hit in the home bucket costs one memory round trip.  A bucket with a
 // never-used entry ends the walk: no key was ever placed beyond it.
+// `entry` receives the entry's index (for its stamp) on a hit.
 __device__ __forceinline__ bool probe_ro(const IndexView& ix, uint64_t key, uint64_t& mask,
-                                         uint32_t& id) {
+                                         uint32_t& id, unsigned long long& entry) {
   mask = 0;
   id = AIBX_NO_BLOCK;
+  entry = ~0ULL;
   if (key_reserved(key)) return false;
   unsigned long long b = home_bucket(ix, key);
   for (unsigned int n = 0; n < ix.max_walk; ++n) {
@@ -101,12 +103,15 @@ __device__ __forceinline__ bool probe_ro(const IndexView& ix, uint64_t key, uint
     if (w.k0 == key) {
       mask = w.m0;
       id = (unsigned int)w.id01;
+      entry = b * kBucketEntries;
     } else if (w.k1 == key) {
       mask = w.m1;
       id = (unsigned int)(w.id01 >> 32);
+      entry = b * kBucketEntries + 1;
     } else if (w.k2 == key) {
       mask = w.m2;
       id = (unsigned int)w.id2;
+      entry = b * kBucketEntries + 2;
     } else {
       if (w.k0 == kKeyEmpty || w.k1 == kKeyEmpty || w.k2 == kKeyEmpty) return false;
       b = next_bucket(ix, b);
@@ -116,6 +121,31 @@ __device__ __forceinline__ bool probe_ro(const IndexView& ix, uint64_t key, uint
     return mask != 0;
   }
   return false;
+}
+
+__device__ __forceinline__ bool probe_ro(const IndexView& ix, uint64_t key, uint64_t& mask,
+                                         uint32_t& id) {
+  unsigned long long entry;
+  return probe_ro(ix, key, mask, id, entry);
+}
+
+// Recency stamp of an entry: bits 0..29 the last epoch in which it was touched (0 = never), bits
+// 30..31 the number of distinct epochs it was touched in, saturating at 3.  Several touches of
+// one entry in one epoch count once, whoever gets there first.
+constexpr unsigned int kEpochMask = (1u << 30) - 1u;
+
+__device__ __forceinline__ void touch_entry(const IndexView& ix, unsigned long long e,
+                                            unsigned int epoch) {
+  unsigned int* stamp = &ix.stamps[e];
+  unsigned int old = *reinterpret_cast<volatile unsigned int*>(stamp);
+  for (int tries = 0; tries < 64; ++tries) {
+    if ((old & kEpochMask) == epoch) return;
+    const unsigned int t = old >> 30;
+    const unsigned int fresh = ((t < 3u ? t + 1u : 3u) << 30) | epoch;
+    const unsigned int seen = atomicCAS(stamp, old, fresh);
+    if (seen == old) return;
+    old = seen;
+  }
 }
 
 // The three keys of a bucket while other threads may be claiming entries.
@@ -505,7 +535,8 @@ match_prefix_warp_kernel(IndexView ix, const uint64_t* __restrict__ hashes,
                          const int64_t* __restrict__ blk_off, int R,
                          uint32_t* __restrict__ match_len, uint32_t* __restrict__ any_len,
                          uint32_t* __restrict__ block_ids, ScoreParams sp,
-                         int32_t* __restrict__ best_pod, int64_t* __restrict__ best_score) {
+                         int32_t* __restrict__ best_pod, int64_t* __restrict__ best_score,
+                         unsigned int epoch) {
   __shared__ unsigned int s_ml[kMatchWarpKernelWarps][AIBX_MAX_PODS];
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
@@ -525,8 +556,12 @@ match_prefix_warp_kernel(IndexView ix, const uint64_t* __restrict__ hashes,
     const uint64_t key_next = nxt < n_r ? __ldg(hashes + off + nxt) : 0ULL;
     uint64_t mask = 0;
     uint32_t id = AIBX_NO_BLOCK;
-    if ((unsigned int)lane < m) probe_ro(ix, key, mask, id);
+    unsigned long long entry = ~0ULL;
+    if ((unsigned int)lane < m) probe_ro(ix, key, mask, id, entry);
+    const unsigned int first = st.pos;
     fold_chunk(st, lane, m, mask, id, all, s_ml[warp], block_ids ? block_ids + off : nullptr);
+    // the blocks of the matched prefix are marked as used, with the entry the probe just found
+    if (epoch && first + (unsigned int)lane < st.pos) touch_entry(ix, entry, epoch);
     key = key_next;
   }
   fold_finish(st, lane, P, r, n_r, off, s_ml[warp], match_len, any_len, block_ids, sp, best_pod,
@@ -550,7 +585,7 @@ __global__ void match_prefix_kernel(IndexView ix, const uint64_t* __restrict__ h
                                     uint32_t* __restrict__ any_len,
                                     uint32_t* __restrict__ block_ids, ScoreParams sp,
                                     int32_t* __restrict__ best_pod,
-                                    int64_t* __restrict__ best_score) {
+                                    int64_t* __restrict__ best_score, unsigned int epoch) {
   extern __shared__ MatchShared s_groups[];
   const int warps_per_cta = blockDim.x >> 5;
   const int groups_per_cta = warps_per_cta / wpr;
@@ -651,6 +686,17 @@ __global__ void match_prefix_kernel(IndexView ix, const uint64_t* __restrict__ h
     if (block_ids) {
       for (unsigned int i = a + tid_in_group; i < n_r; i += group_threads)
         block_ids[off + i] = AIBX_NO_BLOCK;
+    }
+    if (epoch) {
+      // Where the prefix ends is only known now that all warps of the request have met, so the
+      // stamps are set in a second walk over the matched blocks; their buckets were read a
+      // moment ago and are still in L2.
+      for (unsigned int i = tid_in_group; i < a; i += group_threads) {
+        uint64_t mask;
+        uint32_t id;
+        unsigned long long entry;
+        if (probe_ro(ix, __ldg(hashes + off + i), mask, id, entry)) touch_entry(ix, entry, epoch);
+      }
     }
   }
 }

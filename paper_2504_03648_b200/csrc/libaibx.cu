@@ -377,7 +377,7 @@ namespace {
 int32_t launch_match(const aibx_index_t* ix, const uint64_t* d_hashes, const int64_t* d_blk_off,
                      int32_t R, uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
                      const ScoreParams& sp, int32_t* d_best_pod, int64_t* d_best_score,
-                     cudaStream_t st);
+                     cudaStream_t st, unsigned int epoch = 0);
 
 }  // namespace
 
@@ -392,12 +392,24 @@ int32_t aibx_match_prefix(const aibx_index_t* ix, const uint64_t* d_hashes,
                       nullptr, nullptr, as_stream(stream));
 }
 
+int32_t aibx_match_prefix_touch(aibx_index_t* ix, const uint64_t* d_hashes,
+                                const int64_t* d_blk_off, int32_t R, uint32_t epoch,
+                                uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
+                                void* stream) {
+  if (!ix || R < 0 || epoch == 0 || epoch >= (1u << 30) || ix->migrating) return AIBX_ERR_INVALID;
+  if (R == 0) return AIBX_OK;
+  if (!d_hashes || !d_blk_off || !d_match_len) return AIBX_ERR_INVALID;
+  ScoreParams none = {nullptr, 0, 0, 0, 0};
+  return launch_match(ix, d_hashes, d_blk_off, R, d_match_len, d_any_len, d_block_ids, none,
+                      nullptr, nullptr, as_stream(stream), epoch);
+}
+
 namespace {
 
 int32_t launch_match(const aibx_index_t* ix, const uint64_t* d_hashes, const int64_t* d_blk_off,
                      int32_t R, uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
                      const ScoreParams& sp, int32_t* d_best_pod, int64_t* d_best_score,
-                     cudaStream_t st) {
+                     cudaStream_t st, unsigned int epoch) {
   // warps per request: aim at ~32 resident warps per SM; few requests get whole CTAs
   int wpr = 1;
   const long long target = (long long)sm_count() * 32;
@@ -406,7 +418,7 @@ int32_t launch_match(const aibx_index_t* ix, const uint64_t* d_hashes, const int
     // warps enough with one per request: the shape without barriers and shared-memory atomics
     match_prefix_warp_kernel<<<blocks_for(R, kMatchWarpKernelWarps), kMatchWarpKernelWarps * 32, 0,
                                st>>>(ix->view, d_hashes, d_blk_off, R, d_match_len, d_any_len,
-                                     d_block_ids, sp, d_best_pod, d_best_score);
+                                     d_block_ids, sp, d_best_pod, d_best_score, epoch);
     return launch_status();
   }
   const int warps_per_cta = wpr > kMatchWarpsMin ? wpr : kMatchWarpsMin;
@@ -415,7 +427,7 @@ int32_t launch_match(const aibx_index_t* ix, const uint64_t* d_hashes, const int
   const size_t smem = (size_t)groups * sizeof(MatchShared);
   match_prefix_kernel<<<grid, warps_per_cta * 32, smem, st>>>(
       ix->view, d_hashes, d_blk_off, R, wpr, d_match_len, d_any_len, d_block_ids, sp, d_best_pod,
-      d_best_score);
+      d_best_score, epoch);
   return launch_status();
 }
 
@@ -444,13 +456,15 @@ int32_t aibx_route_batch(const aibx_index_t* ix, const int32_t* d_tokens, const 
                       d_best_pod, d_best_score, st);
 }
 
-int32_t aibx_route_head(const aibx_index_t* ix, const int32_t* d_tokens, const int64_t* d_tok_off,
+namespace {
+
+int32_t route_head_impl(const aibx_index_t* ix, const int32_t* d_tokens, const int64_t* d_tok_off,
                         const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
                         uint64_t root_seed, const int32_t* d_pod_load, uint64_t ready_mask,
                         const aibx_route_params_t* params, uint64_t* d_hashes,
                         uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
                         int32_t* d_best_pod, int64_t* d_best_score, uint32_t* d_hashed,
-                        uint64_t* d_next_seed, void* stream) {
+                        uint64_t* d_next_seed, void* stream, unsigned int epoch) {
   if (!ix || R < 0 || block_tokens <= 0 || block_tokens % 8 != 0 || block_tokens > 1024)
     return AIBX_ERR_INVALID;
   if (R == 0) return AIBX_OK;
@@ -469,7 +483,7 @@ int32_t aibx_route_head(const aibx_index_t* ix, const int32_t* d_tokens, const i
   route_head_kernel<SPB><<<grid, 288, 0, st>>>(ix->view, d_tokens, d_tok_off, d_blk_off, R,      \
                                               root_seed, d_hashes, d_match_len, d_any_len,      \
                                               d_block_ids, sp, d_best_pod, d_best_score,        \
-                                              d_hashed, d_next_seed)
+                                              d_hashed, d_next_seed, epoch)
   if (spb == 1) {
     AIBX_HEAD_LAUNCH(1);
   } else if (spb == 2) {
@@ -484,13 +498,40 @@ int32_t aibx_route_head(const aibx_index_t* ix, const int32_t* d_tokens, const i
                                     d_hashes, st);
     if (rc != AIBX_OK) return rc;
     rc = launch_match(ix, d_hashes, d_blk_off, R, d_match_len, d_any_len, d_block_ids, sp,
-                      d_best_pod, d_best_score, st);
+                      d_best_pod, d_best_score, st, epoch);
     if (rc != AIBX_OK) return rc;
     route_head_state_full_kernel<<<blocks_for(R, 256), 256, 0, st>>>(d_blk_off, R, root_seed,
                                                                      d_hashes, d_hashed, d_next_seed);
   }
 #undef AIBX_HEAD_LAUNCH
   return launch_status();
+}
+
+}  // namespace
+
+int32_t aibx_route_head(const aibx_index_t* ix, const int32_t* d_tokens, const int64_t* d_tok_off,
+                        const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
+                        uint64_t root_seed, const int32_t* d_pod_load, uint64_t ready_mask,
+                        const aibx_route_params_t* params, uint64_t* d_hashes,
+                        uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
+                        int32_t* d_best_pod, int64_t* d_best_score, uint32_t* d_hashed,
+                        uint64_t* d_next_seed, void* stream) {
+  return route_head_impl(ix, d_tokens, d_tok_off, d_blk_off, R, block_tokens, root_seed, d_pod_load,
+                         ready_mask, params, d_hashes, d_match_len, d_any_len, d_block_ids,
+                         d_best_pod, d_best_score, d_hashed, d_next_seed, stream, 0u);
+}
+
+int32_t aibx_route_head_touch(aibx_index_t* ix, const int32_t* d_tokens, const int64_t* d_tok_off,
+                              const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
+                              uint64_t root_seed, const int32_t* d_pod_load, uint64_t ready_mask,
+                              const aibx_route_params_t* params, uint32_t epoch,
+                              uint64_t* d_hashes, uint32_t* d_match_len, uint32_t* d_any_len,
+                              uint32_t* d_block_ids, int32_t* d_best_pod, int64_t* d_best_score,
+                              uint32_t* d_hashed, uint64_t* d_next_seed, void* stream) {
+  if (!ix || epoch == 0 || epoch >= (1u << 30) || ix->migrating) return AIBX_ERR_INVALID;
+  return route_head_impl(ix, d_tokens, d_tok_off, d_blk_off, R, block_tokens, root_seed, d_pod_load,
+                         ready_mask, params, d_hashes, d_match_len, d_any_len, d_block_ids,
+                         d_best_pod, d_best_score, d_hashed, d_next_seed, stream, epoch);
 }
 
 int32_t aibx_hash_blocks_resume(const int32_t* d_tokens, const int64_t* d_tok_off,

@@ -86,7 +86,8 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
                   uint64_t root_seed, uint64_t* __restrict__ hashes, uint32_t* match_len,
                   uint32_t* __restrict__ any_len, uint32_t* __restrict__ block_ids, ScoreParams sp,
                   int32_t* __restrict__ best_pod, int64_t* __restrict__ best_score,
-                  uint32_t* __restrict__ hashed_out, uint64_t* __restrict__ seed_out) {
+                  uint32_t* __restrict__ hashed_out, uint64_t* __restrict__ seed_out,
+                  unsigned int epoch) {
   constexpr int BPG = kGroupStripes / SPB;             // blocks per group of 8 stripes
   __shared__ HeadShared sh;
   const int lane = threadIdx.x & 31;
@@ -223,15 +224,18 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
     const unsigned int m = min(32u, avail - st.pos);
     uint64_t mask = 0, key = 0;
     uint32_t id = AIBX_NO_BLOCK;
+    unsigned long long entry = ~0ULL;
     if ((unsigned int)lane < m) {
       key = *reinterpret_cast<volatile unsigned long long*>(
           &sh.ring[qi][(st.pos + lane) % kHeadRing]);
       hashes[out0 + st.pos + lane] = key;              // the keys leave the CTA through the prober
-      probe_ro(ix, key, mask, id);
+      probe_ro(ix, key, mask, id, entry);
     }
     written = st.pos + m;
     last_key = shfl64(0xffffffffu, key, (int)m - 1);
+    const unsigned int first = st.pos;
     fold_chunk(st, lane, m, mask, id, all, sh.match_len[qi], block_ids ? block_ids + out0 : nullptr);
+    if (epoch && first + (unsigned int)lane < st.pos) touch_entry(ix, entry, epoch);
     // Lets the hasher reuse the ring slots just read.  The keys read from them have been used
     // by now (every lane computed its probe address from its key), so the reads are complete
     // before this store is issued; a plain store is enough.

@@ -17,7 +17,6 @@
 
 namespace aibx {
 
-constexpr unsigned int kEpochMask = (1u << 30) - 1u;
 constexpr int kHist1Bins = 1 << 16;
 constexpr int kHist2Bins = 1 << 15;
 
@@ -50,17 +49,7 @@ __global__ void index_touch_kernel(IndexView ix, const uint64_t* __restrict__ ke
   const unsigned long long e = find_entry_rw(ix, key);
   if (e == ~0ULL) return;
   if (*reinterpret_cast<volatile unsigned long long*>(entry_mask(ix, e)) == 0) return;
-  unsigned int* stamp = &ix.stamps[e];
-  unsigned int old = *reinterpret_cast<volatile unsigned int*>(stamp);
-  // several touches of one key in one epoch count once, whoever gets there first
-  for (int tries = 0; tries < 64; ++tries) {
-    if ((old & kEpochMask) == epoch) return;
-    const unsigned int t = old >> 30;
-    const unsigned int fresh = ((t < 3u ? t + 1u : 3u) << 30) | epoch;
-    const unsigned int seen = atomicCAS(stamp, old, fresh);
-    if (seen == old) return;
-    old = seen;
-  }
+  touch_entry(ix, e, epoch);
 }
 
 // Reads one entry; returns whether it is live.

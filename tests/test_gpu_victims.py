@@ -7,8 +7,9 @@ import pytest
 import torch
 
 import oracle
-from gpu_util import dev, empty, host
+from gpu_util import dev, empty, fill_entries, gpu_hash, host
 from paper_2504_03648_b200 import binding as aibx
+import workloads as W
 
 pytestmark = pytest.mark.gpu
 ALL = (1 << 64) - 1
@@ -95,4 +96,63 @@ def test_random_traffic(n_keys, capacity):
     o.insert(np.concatenate([back, some]), np.ones(len(back) + 5, np.uint64),
              np.zeros(len(back) + 5, np.uint32))
     check_against_oracle(g, o, len(back) + 3)
+    assert aibx.status_fetch() == (0, 0)
+
+
+@pytest.mark.parametrize("R", [40, 3000])          # several warps per request / one warp per request
+def test_matching_stamps_the_matched_prefix(R):
+    """match_prefix_touch and route_head_touch against the oracle's match_prefix followed by
+    touch of the keys below any_len: same match results, and afterwards the same victims."""
+    spec = W.scaled(W.cfg3_routing(), R=R, capacity=1 << 16, n_entries=1 << 15, n_prompts=40,
+                    id_space=1 << 15, len_lo=64, len_hi=2048, len_mean=600.0, len_sd=300.0)
+    w = W.build_routing(spec)
+    B, P = spec.block_tokens, spec.num_pods
+    h, bo = gpu_hash(w.tokens, w.tok_off, B)
+    sh, _ = gpu_hash(w.src_tokens, w.src_tok_off, B)
+    keys, masks, ids = fill_entries(w, sh)
+    g, o = aibx.Index(spec.capacity, P), oracle.Index(spec.capacity, P)
+    g.insert(dev(keys), dev(masks), dev(ids)); assert o.insert(keys, masks, ids) == oracle.OK
+    d_h, d_bo = dev(h), dev(bo)
+    d_tok, d_toff = dev(w.tokens), dev(w.tok_off)
+    n_live = o.stats()[0]
+
+    def oracle_step(epoch, lo, hi):
+        sub_bo = bo[lo:hi + 1] - bo[lo]
+        sub_h = h[bo[lo]:bo[hi]]
+        ml, al, bid = o.match_prefix(sub_h, sub_bo)
+        hit = np.concatenate([sub_h[sub_bo[r]: sub_bo[r] + al[r]] for r in range(hi - lo)])
+        o.touch(hit, epoch)
+        return ml, al, bid
+
+    # epochs 1..3 over different slices of the batch through match_prefix_touch
+    cuts = [0, R // 2, (3 * R) // 4, R]
+    for epoch, (lo, hi) in enumerate(zip(cuts[:-1], cuts[1:]), start=1):
+        n = hi - lo
+        sub_bo = dev(bo[lo:hi + 1] - bo[lo])
+        sub_h = dev(h[bo[lo]:bo[hi]]) if bo[hi] > bo[lo] else empty(1, torch.uint64)
+        d_ml, d_al = empty(n * P, torch.uint32), empty(n, torch.uint32)
+        d_id = empty(max(int(bo[hi] - bo[lo]), 1), torch.uint32)
+        g.match_prefix_touch(sub_h, sub_bo, epoch, d_ml, d_al, d_id)
+        ml, al, bid = oracle_step(epoch, lo, hi)
+        assert np.array_equal(host(d_ml).reshape(n, P), ml) and np.array_equal(host(d_al), al)
+        assert np.array_equal(host(d_id)[: len(bid)], bid)
+        assert al.sum() > 0
+    for k in (1, n_live // 50 + 1, n_live // 2, n_live):
+        check_against_oracle(g, o, k)
+    # epoch 4 over the whole batch through route_head_touch
+    d_hh = torch.zeros(len(h), dtype=torch.uint64, device="cuda")
+    d_ml, d_al, d_id = empty(R * P, torch.uint32), empty(R, torch.uint32), empty(len(h), torch.uint32)
+    d_bp, d_bs = empty(R, torch.int32), empty(R, torch.int64)
+    d_dn, d_sd = empty(R, torch.uint32), empty(R, torch.uint64)
+    aibx.route_head_touch(g, d_tok, d_toff, d_bo, B, 0, dev(w.pod_load), w.ready_mask, None, 4, d_hh,
+                          d_ml, d_al, d_id, d_bp, d_bs, d_dn, d_sd)
+    ml, al, bid = oracle_step(4, 0, R)
+    assert np.array_equal(host(d_ml).reshape(R, P), ml) and np.array_equal(host(d_al), al)
+    for k in (1, n_live // 50 + 1, n_live // 2, n_live):
+        check_against_oracle(g, o, k)
+    # the plain calls leave the stamps alone
+    g.match_prefix(d_h, d_bo, d_ml, d_al, d_id)
+    check_against_oracle(g, o, n_live // 3)
+    with pytest.raises(aibx.AibxError):
+        g.match_prefix_touch(d_h, d_bo, 0, d_ml, d_al, d_id)
     assert aibx.status_fetch() == (0, 0)

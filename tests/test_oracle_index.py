@@ -209,3 +209,19 @@ def test_scan_resistant_victims_hand_example_and_model():
     assert list(zip(p.tolist(), k.tolist())) == want[:150]
     k, p = ix.pick_victims(10**6)
     assert len(k) == len(model)
+
+
+def test_match_then_touch_marks_the_matched_prefix_only():
+    """What the GPU's match-and-stamp calls are compared with: match_prefix followed by touch of
+    the keys below any_len.  Hand example: the index holds A, B, C; the request [A, B, X, C] is
+    cached up to B, so after the composition A and B carry the epoch and C, behind the hole, and
+    the never-requested D stay cold."""
+    A, B, Cc, D, X = 101, 202, 303, 404, 999
+    ix = oracle.Index(16, 2)
+    ix.insert(np.array([A, B, Cc, D], np.uint64), np.ones(4, np.uint64), np.arange(4, dtype=np.uint32))
+    req = np.array([A, B, X, Cc], np.uint64)
+    ml, al, ids = ix.match_prefix(req, np.array([0, 4], np.int64))
+    assert al.tolist() == [2]
+    ix.touch(req[: al[0]], 7)
+    keys, prio = ix.pick_victims(4)
+    assert dict(zip(keys.tolist(), prio.tolist())) == {Cc: 0, D: 0, A: 7, B: 7}

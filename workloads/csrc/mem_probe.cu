@@ -27,13 +27,14 @@ __device__ __forceinline__ unsigned long long load32(const unsigned long long* p
 // SECTORS 32-byte sectors per access (1, 2 or 4), PER independent accesses per thread.
 template <int SECTORS, int PER>
 __global__ void random_read_kernel(const unsigned long long* __restrict__ base,
-                                   unsigned long long unit_mask, unsigned long long n_reads,
+                                   unsigned long long units, unsigned long long n_reads,
                                    unsigned long long seed, unsigned long long* __restrict__ sink) {
   const unsigned long long t = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x;
   unsigned long long acc = 0;
   unsigned long long off[PER];
 #pragma unroll
-  for (int k = 0; k < PER; ++k) off[k] = (mix64(seed, t * PER + k) & unit_mask) * (4ULL * SECTORS);
+  for (int k = 0; k < PER; ++k)   // multiply-shift range reduction: any number of units
+    off[k] = __umul64hi(mix64(seed, t * PER + k), units) * (4ULL * SECTORS);
 #pragma unroll
   for (int k = 0; k < PER; ++k) {
     if (t * PER + k < n_reads) {
@@ -51,22 +52,22 @@ __global__ void random_read_kernel(const unsigned long long* __restrict__ base,
 
 extern "C" {
 
-// d_base: working set of `ws_bytes` (a power of two, >= 4 KiB), 32-byte aligned; every access
+// d_base: working set of `ws_bytes` (a multiple of 128, >= 4 KiB), 32-byte aligned; every access
 // reads `gran` bytes (32, 64 or 128) at a uniformly random gran-aligned offset; `per` accesses
 // per thread (1, 2 or 4) are independent; d_sink holds at least n_reads / (32 * per) + 1 words.
 int32_t aibx_probe_random_reads(const void* d_base, uint64_t ws_bytes, int32_t gran, int32_t per,
                                 uint64_t n_reads, uint64_t seed, void* d_sink, void* stream) {
-  if (!d_base || !d_sink || ws_bytes < 4096 || (ws_bytes & (ws_bytes - 1))) return -1;
+  if (!d_base || !d_sink || ws_bytes < 4096 || (ws_bytes & 127)) return -1;
   if (gran != 32 && gran != 64 && gran != 128) return -1;
   if (per != 1 && per != 2 && per != 4) return -1;
   if (n_reads == 0) return 0;
-  const unsigned long long unit_mask = ws_bytes / (unsigned long long)gran - 1ULL;
+  const unsigned long long units = ws_bytes / (unsigned long long)gran;
   const unsigned long long threads = (n_reads + per - 1) / per;
   const unsigned int grid = (unsigned int)((threads + 255) / 256);
   const unsigned long long* b = static_cast<const unsigned long long*>(d_base);
   unsigned long long* k = static_cast<unsigned long long*>(d_sink);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-#define PROBE(S, P) random_read_kernel<S, P><<<grid, 256, 0, st>>>(b, unit_mask, n_reads, seed, k)
+#define PROBE(S, P) random_read_kernel<S, P><<<grid, 256, 0, st>>>(b, units, n_reads, seed, k)
   if (gran == 32) {
     if (per == 1) PROBE(1, 1); else if (per == 2) PROBE(1, 2); else PROBE(1, 4);
   } else if (gran == 64) {

@@ -69,7 +69,7 @@ def fill_pool(pool, kv) -> None:
 
 def probe_random_reads(base, ws_bytes: int, gran: int, per: int, n_reads: int, seed, sink) -> None:
     """Memory-system probe (no method code): n_reads uniformly random, aligned reads of `gran`
-    bytes (32 / 64 / 128) over the first ws_bytes (a power of two) of the CUDA tensor `base`,
+    bytes (32 / 64 / 128) over the first ws_bytes (a multiple of 128) of the CUDA tensor `base`,
     `per` independent reads per thread; `sink` (uint64, n_reads / (32 * per) + 1 words) keeps the
     loads alive.  Enqueued on the current stream."""
     import torch
