@@ -45,7 +45,7 @@ METRIC = "kv_gather_scatter_GBps_whole_step"
 UNIT = "GB/s"
 WORKLOAD = "cfg2-llama3-8b: 64 requests (1k-8k tokens, 32 Zipf prompts), index 200k/2^19 x 16 pods, " \
            "pool 4096 x 2 MiB bf16 blocks, gather+scatter of all matched blocks"
-KERNELS_PER_STEP = 9    # head (hash+match+score), collect, gather, scatter, hash tail, insert, evict x3
+KERNELS_PER_STEP = 7    # head (hash+match+score), collect, gather, scatter, hash tail, insert, evict
 
 from bench_cases import CASES, cpu_model, measured_peak_hbm, ncu_traffic, routing_batch_times  # noqa: E402
 

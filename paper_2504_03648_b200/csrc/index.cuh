@@ -17,6 +17,8 @@
 //                    shared-memory minima and stop once an earlier total miss is known.
 #pragma once
 
+#include <cooperative_groups.h>
+
 #include "aibx_common.cuh"
 #include "route_score.cuh"
 
@@ -415,6 +417,60 @@ __global__ void index_evict_remove_kernel(IndexView ix, const uint64_t* __restri
     }
   }
   fold_counters(ix, 0u, 0u, removed, 0u);   // live -= removed, removed entries += removed
+}
+
+// The three passes of evict in ONE cooperative launch: every pass must see the whole batch's
+// previous pass finished, which a grid-wide barrier gives without going back to the host (three
+// launches cost about 10 us each for a batch that takes 3 us of work).  A thread that has a
+// single item keeps the entry it found in pass 1; with more items than threads the later passes
+// look their entries up again.  The launch is cooperative, so all CTAs are resident and the
+// barrier cannot wait for a CTA that has not started.
+__global__ void __launch_bounds__(256)
+index_evict_coop_kernel(IndexView ix, const uint64_t* __restrict__ keys,
+                        const uint64_t* __restrict__ masks, uint32_t* __restrict__ freed,
+                        int64_t n) {
+  cooperative_groups::grid_group grid = cooperative_groups::this_grid();
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  const bool single = n <= stride;
+  unsigned long long mine = ~0ULL;                       // entry of this thread's only item
+  for (int64_t i = t; i < n; i += stride) {
+    const uint64_t key = keys[i];
+    if (key_reserved(key)) continue;
+    const unsigned long long e = find_entry_rw(ix, key);
+    if (e != ~0ULL) atomicAnd(entry_mask(ix, e), ~(unsigned long long)masks[i]);
+    mine = e;
+  }
+  grid.sync();
+  if (freed) {
+    for (int64_t i = t; i < n; i += stride) {
+      const uint64_t key = keys[i];
+      uint32_t out = AIBX_NO_BLOCK;
+      if (!key_reserved(key)) {
+        const unsigned long long e = single ? mine : find_entry_rw(ix, key);
+        if (e != ~0ULL &&
+            *reinterpret_cast<volatile unsigned long long*>(entry_mask(ix, e)) == 0)
+          out = *reinterpret_cast<volatile unsigned int*>(entry_id(ix, e));
+      }
+      freed[i] = out;
+    }
+    grid.sync();
+  }
+  unsigned int removed = 0;
+  for (int64_t i = t; i < n; i += stride) {
+    const uint64_t key = keys[i];
+    if (key_reserved(key)) continue;
+    // an entry another thread of the same key has already removed no longer carries the key
+    const unsigned long long e = single ? mine : find_entry_rw(ix, key);
+    if (e != ~0ULL &&
+        *reinterpret_cast<volatile unsigned long long*>(entry_mask(ix, e)) == 0 &&
+        atomicCAS(entry_key(ix, e), (unsigned long long)key, kKeyTomb) == key) {
+      *entry_id(ix, e) = AIBX_NO_BLOCK;
+      ix.stamps[e] = 0u;
+      removed += 1u;
+    }
+  }
+  fold_counters(ix, 0u, 0u, removed, 0u);
 }
 
 __global__ void index_lookup_kernel(IndexView ix, const uint64_t* __restrict__ keys,

@@ -56,6 +56,7 @@ void prefer_copy_carveout() {
       (const void*)hash_blocks_kernel<8>,      (const void*)index_insert_kernel,
       (const void*)index_evict_clear_kernel,   (const void*)index_evict_report_kernel,
       (const void*)index_evict_remove_kernel,  (const void*)index_touch_kernel,
+      (const void*)index_evict_coop_kernel,
   };
   for (const void* f : side_kernels)
     cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -89,6 +90,31 @@ int32_t alloc_view(uint64_t capacity, int num_pods, IndexView* out) {
 void free_view(const IndexView& v) { cudaFree(v.buckets); }
 
 bool capacity_ok(uint64_t c) { return c >= 8 && (c & (c - 1)) == 0 && c <= (1ULL << 40); }
+
+// How many CTAs of the one-launch evict kernel the current device can hold at once (0: it
+// cannot launch kernels cooperatively, or the query failed).
+int evict_coop_ctas() {
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  int v = cached[dev].load(std::memory_order_relaxed);
+  if (v == 0) {
+    int coop = 0, per_sm = 0;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, index_evict_coop_kernel, 256, 0) !=
+            cudaSuccess ||
+        per_sm <= 0) {
+      cudaGetLastError();
+      v = -1;
+    } else {
+      // half of what fits: the kernel usually runs beside others, and every one of its CTAs
+      // must be resident before the first can pass the barrier
+      v = sm_count() * (per_sm > 1 ? per_sm / 2 : 1);
+    }
+    cached[dev].store(v, std::memory_order_relaxed);
+  }
+  return v > 0 ? v : 0;
+}
 
 // Device address of the status record of the current device.
 StatusRecord* status_ptr() {
@@ -214,6 +240,16 @@ int32_t aibx_index_evict(aibx_index_t* ix, const uint64_t* d_keys, const uint64_
   prefer_copy_carveout();
   cudaStream_t st = as_stream(stream);
   const unsigned int grid = blocks_for(n, 256);
+  const int coop = evict_coop_ctas();
+  if (coop > 0) {
+    IndexView view = ix->view;
+    void* args[] = {&view, &d_keys, &d_pod_masks, &d_freed_block_ids, &n};
+    const unsigned int g = grid < (unsigned int)coop ? grid : (unsigned int)coop;
+    if (cudaLaunchCooperativeKernel((const void*)index_evict_coop_kernel, dim3(g), dim3(256), args,
+                                    0, st) == cudaSuccess)
+      return AIBX_OK;
+    cudaGetLastError();       // fall back to the three plain launches
+  }
   index_evict_clear_kernel<<<grid, 256, 0, st>>>(ix->view, d_keys, d_pod_masks, n);
   if (d_freed_block_ids)
     index_evict_report_kernel<<<grid, 256, 0, st>>>(ix->view, d_keys, d_freed_block_ids, n);
