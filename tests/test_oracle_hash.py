@@ -42,7 +42,8 @@ def test_published_values():
 
 
 def test_block_sized_vectors():
-    """The sizes the path hashes (whole 32-byte stripes, no tail), values from the build plan."""
+    """The sizes the path hashes (whole 32-byte stripes, no tail): stored values that the
+    independent xxhash library gives for these inputs."""
     n_rows = 0
     for line in open(os.path.join(GOLDEN, "xxh64_block_sized.txt")):
         if line.startswith("#") or not line.strip():

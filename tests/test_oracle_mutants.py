@@ -171,3 +171,31 @@ def test_unmodified_copy_passes(tmp_path):
     name, rc, tail = _run_mutant((str(tmp_path), ("identity", "test_oracle_score.py",
                                                   "acc = rotl64(acc, 31);", "acc = rotl64(acc, 31);", 0)))
     assert rc == 0, tail
+
+
+def test_pins_pass_on_a_sanitizer_build_of_the_oracle(tmp_path):
+    """The unmodified oracle built with AddressSanitizer and UndefinedBehaviorSanitizer runs its
+    pin files clean: no out-of-bounds access, no signed overflow, no misaligned load behind the
+    results the GPU is compared with."""
+    import shutil
+
+    if shutil.which("gcc") is None:
+        return
+    lib = os.path.join(str(tmp_path), "libaibxo_san.so")
+    try:
+        subprocess.check_call(["gcc", "-std=c99", "-O1", "-g", "-fsanitize=address,undefined",
+                               "-fno-sanitize-recover=undefined", "-fPIC", "-shared", SRC, "-o", lib],
+                              stderr=subprocess.DEVNULL)
+        asan = subprocess.check_output(["gcc", "-print-file-name=libasan.so"]).decode().strip()
+    except (subprocess.CalledProcessError, OSError):
+        return                                       # no sanitizer runtime on this machine
+    if not os.path.isabs(asan) or not os.path.exists(asan):
+        return
+    env = dict(os.environ, AIBXO_LIB_OVERRIDE=lib, LD_PRELOAD=asan, PYTHONDONTWRITEBYTECODE="1",
+               ASAN_OPTIONS="detect_leaks=0:abort_on_error=1", OMP_NUM_THREADS="1")
+    files = ["test_oracle_hash.py", "test_oracle_index.py", "test_oracle_match.py",
+             "test_oracle_score.py", "test_oracle_kv.py", "test_oracle_policy.py"]
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider"] +
+                       [os.path.join(ROOT, "tests", f) for f in files],
+                       cwd=ROOT, env=env, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, timeout=900)
+    assert r.returncode == 0, r.stdout.decode()[-3000:]
