@@ -15,11 +15,16 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of kv_copy_bulk_kernel from the ncu
-# captures summarised under profiles/ (256 blocks of each shape, `--case kv_small --shape ...`),
-# valid only for the kernel source with this digest; scaled to a full launch by the bytes copied.
+# captures summarised under profiles/ (256 blocks of each shape, `--case kv_small --shape ...`,
+# mean of one gather and one scatter launch), valid only for the kernel source with this digest.
+# On all three shapes the DRAM traffic is the bytes copied minus about 50 MB: what the kernel
+# wrote last is still dirty in L2 when it ends.  That residue does not grow with the launch, so a
+# full launch is taken as its own algorithmic bytes minus the residue measured on the small one.
 NCU_TRAFFIC = {
-    "kv_copy_sha1": "8e2d19eba677",
-    "cfg2_shape": {"bytes_per_launch": 1026870016, "launch_algorithmic_bytes": 1073742848},
+    "kv_copy_sha1": "0ce289089085",
+    "cfg2_shape": {"bytes_per_launch": 1021574272, "launch_algorithmic_bytes": 1073742848},
+    "cfg4_shape": {"bytes_per_launch": 2634682112, "launch_algorithmic_bytes": 2684355584},
+    "cfg5_shape": {"bytes_per_launch": 417690368, "launch_algorithmic_bytes": 469763072},
 }
 
 
@@ -31,13 +36,14 @@ def kernel_digest() -> str:
 
 
 def ncu_traffic(shape: str, launch_bytes: int):
-    """DRAM bytes of one launch moving `launch_bytes`, scaled from the captured small case of
-    the same block shape; None when no capture exists for this shape or the kernel has changed
-    since the counters were taken."""
+    """DRAM bytes of one launch moving `launch_bytes`, from the captured small case of the same
+    block shape; None when no capture exists for this shape or the kernel has changed since the
+    counters were taken."""
     rec = NCU_TRAFFIC.get(shape)
     if not rec or NCU_TRAFFIC["kv_copy_sha1"] != kernel_digest():
         return None
-    return rec["bytes_per_launch"] * launch_bytes / rec["launch_algorithmic_bytes"]
+    residue = rec["launch_algorithmic_bytes"] - rec["bytes_per_launch"]
+    return float(max(launch_bytes - residue, 0))
 
 
 def measured_peak_hbm():
