@@ -112,10 +112,10 @@ def case_kv_small(args):
                       "status": aibx.status_fetch()}))
 
 
-def index_table_bytes(slots: int) -> int:
-    """Bytes a probe can touch: ceil(slots / 3) buckets of 64 bytes (the 4-byte eviction stamps
-    per entry are a separate array that lookups never read)."""
-    return (slots + 2) // 3 * 64
+def index_table_bytes(slots: int, pods: int = 32) -> int:
+    """Bytes a probe can touch: 16 bytes per slot with up to 32 pods, 32 bytes with more (the
+    4-byte eviction stamps per entry are a separate array that lookups never read)."""
+    return slots * (16 if pods <= 32 else 32)
 
 
 def _big_index(torch, aibx, W, log2cap, P, seed):

@@ -76,11 +76,11 @@ int32_t aibx_hash_blocks(const int32_t* d_tokens, const int64_t* d_tok_off,
  * pool.  Keys 0 and ~0 are reserved: inserting them is a no-op, looking them up misses.
  *
  * create:  allocates a table for up to capacity_slots entries (power of two, >= 8) on the
- *          current device: ceil(capacity_slots / 3) buckets of 64 bytes holding three entries
- *          each, plus 4 bytes per entry for the eviction stamps (25.3 bytes per slot in all);
- *          num_pods in 1..64.  Syncs.  NOMEM if the allocation fails.  Size it for a load of
- *          about one half (capacity_slots = twice the entries expected): probes then end in
- *          their first bucket 94 times out of 100.
+ *          current device; num_pods in 1..64.  The table is an array of 32-byte sectors probed
+ *          linearly: with up to 32 pods a sector holds two entries (key, 32-bit pod mask, block
+ *          id: 16 bytes per slot), with more pods one entry (32 bytes per slot); 4 more bytes
+ *          per slot hold the eviction stamps.  Syncs.  NOMEM if the allocation fails.  Size it
+ *          for a load of about one half (capacity_slots = twice the entries expected).
  * destroy: frees it (syncs the device).     clear: empties it (async on stream).
  */
 int32_t aibx_index_create(aibx_index_t** out, uint64_t capacity_slots, int32_t num_pods);
@@ -92,11 +92,11 @@ int32_t aibx_index_clear(aibx_index_t* index, void* stream);
  *         AIBX_NO_BLOCK as id means "no id supplied" (identity of min).
  *         Device status FULL (detail = number of entries refused or in excess) when the live
  *         entries would exceed capacity_slots, or when a new key finds no free entry within
- *         1,024 buckets (3,072 entries) of its home bucket - no entry is ever placed further
- *         away, which bounds every later probe; tables up to a load of 0.9 stay far below that.  After FULL the index content is unspecified until aibx_index_clear or
+ *         4,096 entries of its home sector - no entry is ever placed further away, which bounds
+ *         every later probe; tables up to a load of 0.9 stay far below that.  After FULL the index content is unspecified until aibx_index_clear or
  *         aibx_index_rehash.  Entries removed by evict are reused by later inserts that pass
  *         them, but a probe for an absent key only stops at a NEVER-used entry: under steady
- *         publish/expire churn those run out, probes grow towards the 1,024-bucket bound, and
+ *         publish/expire churn those run out, probes grow towards the 4,096-entry bound, and
  *         the table wants a rehash - aibx_index_stats2 says when.
  * evict:  batch-atomic.  First mask &= ~masks[i] for all present keys; then
  *         freed[i] = id if key i was present and its mask is now 0, else AIBX_NO_BLOCK
@@ -108,9 +108,9 @@ int32_t aibx_index_clear(aibx_index_t* index, void* stream);
  * stats2: the same plus what tells when aibx_index_rehash is due: `removed` = entries freed by
  *         evict and not yet reused (live + removed, not live alone, is what the probe length
  *         follows: rehash once it passes three quarters of capacity_slots), `longest_walk` = the
- *         most buckets any insert has had to visit since the table was created, cleared or
- *         rehashed (1 = every key so far went into its home bucket; a healthy table at a load of one
- *         half stays below 10).  Any out-pointer may be null.  Syncs the stream.
+ *         most sectors any insert has had to visit since the table was created, cleared or
+ *         rehashed (1 = every key so far went into its home sector; a healthy table at a load
+ *         of one half stays below 20).  Any out-pointer may be null.  Syncs the stream.
  */
 int32_t aibx_index_insert(aibx_index_t* index, const uint64_t* d_keys,
                           const uint64_t* d_pod_masks, const uint32_t* d_block_ids,

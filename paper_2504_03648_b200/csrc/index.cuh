@@ -1,13 +1,16 @@
-// GPU-resident residency index: open addressing over 64-byte BUCKETS of three entries.
+// GPU-resident residency index: open addressing with linear probing over 32-byte SECTORS, in
+// two entry widths.
 //
 // What the memory system gives a random probe was measured on B200 before this layout was
-// chosen: an L2 miss always brings a whole 128-byte line from DRAM, whatever the load asked for,
-// and random reads of 32 and of 64 bytes run at the same rate.  So a probe may as well read 64
-// bytes, and the table should be as small as it can be so that more of it stays in L2.  A bucket
-// holds the keys, pod masks and block ids of three entries (the eviction stamps, which only the
-// touch and victim kernels need, live in a side array): 21.3 bytes per slot of capacity instead
-// of 32, and at a load of one half 94 % of the lookups end in their home bucket - one memory
-// round trip, two sectors.
+// chosen.  (1) An L2 miss always brings a whole 128-byte line from DRAM, whatever the load asked
+// for, so the smaller the table, the more of it stays in L2 and the fewer lines a lookup costs.
+// (2) Inside an SM the limit is the L1 data stage: a load whose 32 lanes go to 32 different lines
+// costs 32 passes, so a lookup should be ONE 32-byte load, not two.  Hence:
+//   narrow (tables of up to 32 pods): a sector holds TWO entries, {key0, key1, mask0|id0<<32,
+//       mask1|id1<<32}: 16 bytes per slot of capacity, and at a load of one half nine lookups in
+//       ten end with the first load;
+//   wide (33 to 64 pods): a sector holds ONE entry, {key, mask, id, unused}.
+// The eviction stamps, which only the touch and victim kernels need, live in a side array.
 //
 //   insert / evict : one thread per item, atomics only (results are order-free by construction)
 //   lookup         : one thread per key
@@ -24,105 +27,115 @@
 
 namespace aibx {
 
-constexpr int kBucketEntries = 3;
-constexpr unsigned int kMaxWalk = 1024;  // buckets a probe sequence may visit (3,072 entries)
+constexpr unsigned int kMaxWalkEntries = 4096;   // entries a probe sequence may pass
 
-struct __align__(64) Bucket {
-  unsigned long long key[kBucketEntries];    // 0 = never used, ~0 = removed (reusable by insert)
-  unsigned long long mask[kBucketEntries];   // pod residency bits; an entry with mask 0 is dead
-  unsigned int id[kBucketEntries];           // block id, min over inserts; AIBX_NO_BLOCK = none
-  unsigned int spare;
-};
-static_assert(sizeof(Bucket) == 64, "one bucket per 64 bytes");
-
-// Entry e of the table is position e % 3 of bucket e / 3.
+// Entry e of the table is position e % per_sector of sector e / per_sector.
 struct IndexView {
-  Bucket* buckets;
-  unsigned int* stamps;          // [3 * nb] recency stamp of every entry (eviction policy)
-  unsigned long long nb;         // buckets: ceil(capacity / 3)
+  unsigned long long* words;     // nb sectors of four 64-bit words
+  unsigned int* stamps;          // one recency stamp per entry (eviction policy)
+  unsigned long long nb;         // sectors: capacity / 2 (narrow) or capacity (wide)
   unsigned long long capacity;   // live entries the table accepts (FULL beyond)
-  unsigned int max_walk;         // min(nb, kMaxWalk): no entry lies further from its home bucket
+  unsigned int max_walk;         // sectors a probe may visit: no entry lies further from home
   int num_pods;
+  int narrow;                    // 1: two 16-byte entries per sector, 0: one 32-byte entry
   unsigned long long* counters;  // [0] live entries, [1] removed entries, [2] longest insert walk
 };
 
+__device__ __forceinline__ int per_sector(const IndexView& ix) { return ix.narrow ? 2 : 1; }
+
 __device__ __forceinline__ unsigned long long num_entries(const IndexView& ix) {
-  return ix.nb * kBucketEntries;
+  return ix.narrow ? ix.nb * 2 : ix.nb;
 }
 
-// Multiply-shift range reduction: any bucket count, no division.
-__device__ __forceinline__ unsigned long long home_bucket(const IndexView& ix, uint64_t key) {
+// Multiply-shift range reduction: any sector count, no division.
+__device__ __forceinline__ unsigned long long home_sector(const IndexView& ix, uint64_t key) {
   return __umul64hi(key * 0x9E3779B97F4A7C15ULL, ix.nb);
 }
 
-__device__ __forceinline__ unsigned long long next_bucket(const IndexView& ix,
-                                                          unsigned long long b) {
-  return b + 1 == ix.nb ? 0ULL : b + 1;
+__device__ __forceinline__ unsigned long long next_sector(const IndexView& ix,
+                                                          unsigned long long s) {
+  return s + 1 == ix.nb ? 0ULL : s + 1;
 }
 
-// One whole bucket in two 256-bit read-only loads (the table is not modified meanwhile).
-struct BucketWords {
-  unsigned long long k0, k1, k2, m0, m1, m2, id01, id2;
-};
-
-__device__ __forceinline__ void load_bucket(const Bucket* b, BucketWords& w) {
-  const unsigned long long* p = reinterpret_cast<const unsigned long long*>(b);
+// One whole sector in one 256-bit read-only load (the table is not modified meanwhile).
+__device__ __forceinline__ void load_sector(const unsigned long long* p, unsigned long long& w0,
+                                            unsigned long long& w1, unsigned long long& w2,
+                                            unsigned long long& w3) {
   asm volatile("ld.global.nc.v4.u64 {%0,%1,%2,%3}, [%4];"
-               : "=l"(w.k0), "=l"(w.k1), "=l"(w.k2), "=l"(w.m0)
+               : "=l"(w0), "=l"(w1), "=l"(w2), "=l"(w3)
                : "l"(p));
-  asm volatile("ld.global.nc.v4.u64 {%0,%1,%2,%3}, [%4];"
-               : "=l"(w.m1), "=l"(w.m2), "=l"(w.id01), "=l"(w.id2)
-               : "l"(p + 4));
 }
+
+constexpr unsigned long long kNarrowEmptyValue = 0xFFFFFFFF00000000ULL;   // mask 0, id NO_BLOCK
 
 __global__ void index_clear_kernel(IndexView ix) {
   const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
   const unsigned long long t = blockIdx.x * (unsigned long long)blockDim.x + threadIdx.x;
-  // 16 bytes per thread and turn: words 0..2 of a bucket are keys and masks (zero), word 3
-  // holds the three ids and the spare word
-  for (unsigned long long i = t; i < ix.nb * 4; i += stride) {
-    uint4* p = reinterpret_cast<uint4*>(ix.buckets) + i;
-    *p = (i & 3) == 3 ? make_uint4(AIBX_NO_BLOCK, AIBX_NO_BLOCK, AIBX_NO_BLOCK, 0u)
-                      : make_uint4(0u, 0u, 0u, 0u);
+  // 16 bytes per thread and turn: the first half of a sector (keys, or key and mask) is zero,
+  // the second half holds the "no id" patterns
+  for (unsigned long long i = t; i < ix.nb * 2; i += stride) {
+    uint4* p = reinterpret_cast<uint4*>(ix.words) + i;
+    if ((i & 1) == 0) {
+      *p = make_uint4(0u, 0u, 0u, 0u);
+    } else if (ix.narrow) {
+      *p = make_uint4(0u, AIBX_NO_BLOCK, 0u, AIBX_NO_BLOCK);
+    } else {
+      *p = make_uint4(AIBX_NO_BLOCK, 0u, 0u, 0u);
+    }
   }
   for (unsigned long long i = t; i < num_entries(ix); i += stride) ix.stamps[i] = 0u;
   if (t < 3) ix.counters[t] = 0;
 }
 
-// Read-only probe: a hit in the home bucket costs one memory round trip.  A bucket with a
-// never-used entry ends the walk: no key was ever placed beyond it.
-// `entry` receives the entry's index (for its stamp) on a hit.
-__device__ __forceinline__ bool probe_ro(const IndexView& ix, uint64_t key, uint64_t& mask,
-                                         uint32_t& id, unsigned long long& entry) {
+// Read-only probe: a hit in the home sector costs one memory round trip.  A sector with a
+// never-used entry ends the walk: no key was ever placed beyond it.  `entry` receives the
+// entry's index (for its stamp) on a hit.
+template <bool NARROW>
+__device__ __forceinline__ bool probe_ro_w(const IndexView& ix, uint64_t key, uint64_t& mask,
+                                           uint32_t& id, unsigned long long& entry) {
   mask = 0;
   id = AIBX_NO_BLOCK;
   entry = ~0ULL;
   if (key_reserved(key)) return false;
-  unsigned long long b = home_bucket(ix, key);
+  unsigned long long s = home_sector(ix, key);
   for (unsigned int n = 0; n < ix.max_walk; ++n) {
-    BucketWords w;
-    load_bucket(ix.buckets + b, w);
-    if (w.k0 == key) {
-      mask = w.m0;
-      id = (unsigned int)w.id01;
-      entry = b * kBucketEntries;
-    } else if (w.k1 == key) {
-      mask = w.m1;
-      id = (unsigned int)(w.id01 >> 32);
-      entry = b * kBucketEntries + 1;
-    } else if (w.k2 == key) {
-      mask = w.m2;
-      id = (unsigned int)w.id2;
-      entry = b * kBucketEntries + 2;
+    unsigned long long w0, w1, w2, w3;
+    load_sector(ix.words + 4 * s, w0, w1, w2, w3);
+    if (NARROW) {
+      unsigned long long v;
+      if (w0 == key) {
+        v = w2;
+        entry = 2 * s;
+      } else if (w1 == key) {
+        v = w3;
+        entry = 2 * s + 1;
+      } else {
+        if (w0 == kKeyEmpty || w1 == kKeyEmpty) return false;
+        s = next_sector(ix, s);
+        continue;
+      }
+      mask = (unsigned int)v;
+      id = (unsigned int)(v >> 32);
     } else {
-      if (w.k0 == kKeyEmpty || w.k1 == kKeyEmpty || w.k2 == kKeyEmpty) return false;
-      b = next_bucket(ix, b);
-      continue;
+      if (w0 != key) {
+        if (w0 == kKeyEmpty) return false;
+        s = next_sector(ix, s);
+        continue;
+      }
+      mask = w1;
+      id = (unsigned int)w2;
+      entry = s;
     }
     if (mask == 0) id = AIBX_NO_BLOCK;
     return mask != 0;
   }
   return false;
+}
+
+__device__ __forceinline__ bool probe_ro(const IndexView& ix, uint64_t key, uint64_t& mask,
+                                         uint32_t& id, unsigned long long& entry) {
+  return ix.narrow ? probe_ro_w<true>(ix, key, mask, id, entry)
+                   : probe_ro_w<false>(ix, key, mask, id, entry);
 }
 
 __device__ __forceinline__ bool probe_ro(const IndexView& ix, uint64_t key, uint64_t& mask,
@@ -150,82 +163,99 @@ __device__ __forceinline__ void touch_entry(const IndexView& ix, unsigned long l
   }
 }
 
-// The three keys of a bucket while other threads may be claiming entries.
-__device__ __forceinline__ void load_keys(const Bucket* b, unsigned long long (&k)[kBucketEntries]) {
-#pragma unroll
-  for (int j = 0; j < kBucketEntries; ++j)
-    k[j] = *reinterpret_cast<const volatile unsigned long long*>(&b->key[j]);
-}
-
+// Where the parts of entry e live (both widths).
 __device__ __forceinline__ unsigned long long* entry_key(const IndexView& ix, unsigned long long e) {
-  return &ix.buckets[e / kBucketEntries].key[e % kBucketEntries];
+  return ix.narrow ? ix.words + 4 * (e >> 1) + (e & 1) : ix.words + 4 * e;
 }
-__device__ __forceinline__ unsigned long long* entry_mask(const IndexView& ix, unsigned long long e) {
-  return &ix.buckets[e / kBucketEntries].mask[e % kBucketEntries];
+__device__ __forceinline__ unsigned int* narrow_value(const IndexView& ix, unsigned long long e) {
+  return reinterpret_cast<unsigned int*>(ix.words + 4 * (e >> 1) + 2 + (e & 1));   // {mask, id}
 }
 __device__ __forceinline__ unsigned int* entry_id(const IndexView& ix, unsigned long long e) {
-  return &ix.buckets[e / kBucketEntries].id[e % kBucketEntries];
+  return ix.narrow ? narrow_value(ix, e) + 1 : reinterpret_cast<unsigned int*>(ix.words + 4 * e + 2);
+}
+__device__ __forceinline__ unsigned long long entry_mask_now(const IndexView& ix,
+                                                             unsigned long long e) {
+  if (ix.narrow) return *reinterpret_cast<volatile unsigned int*>(narrow_value(ix, e));
+  return *reinterpret_cast<volatile unsigned long long*>(ix.words + 4 * e + 1);
+}
+__device__ __forceinline__ void entry_mask_or(const IndexView& ix, unsigned long long e,
+                                              unsigned long long m) {
+  if (ix.narrow) atomicOr(narrow_value(ix, e), (unsigned int)m);
+  else atomicOr(ix.words + 4 * e + 1, m);
+}
+__device__ __forceinline__ void entry_mask_clear(const IndexView& ix, unsigned long long e,
+                                                 unsigned long long bits) {
+  if (ix.narrow) atomicAnd(narrow_value(ix, e), ~(unsigned int)bits);
+  else atomicAnd(ix.words + 4 * e + 1, ~bits);
+}
+
+// The keys of a sector while other threads may be claiming entries (k[1] only when narrow).
+__device__ __forceinline__ void load_keys(const IndexView& ix, unsigned long long s,
+                                          unsigned long long (&k)[2]) {
+  const volatile unsigned long long* p = ix.words + 4 * s;
+  k[0] = p[0];
+  k[1] = ix.narrow ? p[1] : 1ULL;      // wide: a value that is neither a key's match nor free
 }
 
 // Probe while other threads may be claiming entries: returns the entry index or ~0.
 __device__ __forceinline__ unsigned long long find_entry_rw(const IndexView& ix, uint64_t key) {
-  unsigned long long b = home_bucket(ix, key);
+  const int E = per_sector(ix);
+  unsigned long long s = home_sector(ix, key);
   for (unsigned int n = 0; n < ix.max_walk; ++n) {
-    unsigned long long k[kBucketEntries];
-    load_keys(ix.buckets + b, k);
-#pragma unroll
-    for (int j = 0; j < kBucketEntries; ++j) {
-      if (k[j] == key) return b * kBucketEntries + j;
+    unsigned long long k[2];
+    load_keys(ix, s, k);
+    for (int j = 0; j < E; ++j) {
+      if (k[j] == key) return s * E + j;
       if (k[j] == kKeyEmpty) return ~0ULL;
     }
-    b = next_bucket(ix, b);
+    s = next_sector(ix, s);
   }
   return ~0ULL;
 }
 
 // Insert or update one entry (mask already restricted to the table's pods, key not reserved).
-// Returns the entry, or ~0 when no room is left within max_walk buckets of the key's home.
+// Returns the entry, or ~0 when no room is left within max_walk sectors of the key's home.
 //
-// One walk from the home bucket to the first bucket with a never-used entry: an existing entry
+// One walk from the home sector to the first sector with a never-used entry: an existing entry
 // anywhere on the way wins; otherwise the first never-used or removed entry seen on the way is
 // claimed.  An entry may lie BEHIND a removed one (it was placed when that one was taken), hence
 // the walk to the end before claiming.  Every thread inserting this key walks the same path and
 // tries the same entries in the same order, and no entry turns reusable while inserts run, so
 // the loser of a race for an entry either finds the key there (another thread of the same key
-// won) or starts over and finds the key, or the next free entry, further on.  Inside a bucket
-// the never-used entries are always the last ones, which is what lets a reader stop at the
-// first bucket that has one.
+// won) or starts over and finds the key, or the next free entry, further on.  Inside a sector
+// a never-used entry is always the last one, which is what lets a reader stop at the first
+// sector that has one.
 // `added` / `reused` are raised when an entry was claimed / when it was a removed one, `walked`
-// is the number of buckets visited: the caller folds them into the table's counters once per
+// is the number of sectors visited: the caller folds them into the table's counters once per
 // CTA (one atomic per thread on the same words would serialise the whole kernel behind them).
 __device__ __forceinline__ unsigned long long insert_entry(const IndexView& ix, uint64_t key,
                                                            uint64_t m, uint32_t id,
                                                            unsigned int& added, unsigned int& reused,
                                                            unsigned int& walked) {
+  const int E = per_sector(ix);
   unsigned long long entry = ~0ULL;
-  const unsigned int max_attempts = ix.max_walk * kBucketEntries + 1u;   // each lost race fills one
+  const unsigned int max_attempts = ix.max_walk * 2u + 1u;   // each lost race fills one entry
   for (unsigned int attempts = 0; attempts < max_attempts && entry == ~0ULL; ++attempts) {
-    unsigned long long b = home_bucket(ix, key);
+    unsigned long long s = home_sector(ix, key);
     unsigned long long free_entry = ~0ULL, free_was = kKeyEmpty;
     bool at_end = false;
     unsigned int n = 0;
     for (; n < ix.max_walk && entry == ~0ULL && !at_end; ++n) {
-      unsigned long long k[kBucketEntries];
-      load_keys(ix.buckets + b, k);
-#pragma unroll
-      for (int j = 0; j < kBucketEntries; ++j) {
+      unsigned long long k[2];
+      load_keys(ix, s, k);
+      for (int j = 0; j < E; ++j) {
         if (entry != ~0ULL || at_end) continue;
         if (k[j] == key) {
-          entry = b * kBucketEntries + j;
+          entry = s * E + j;
         } else if (k[j] == kKeyEmpty || k[j] == kKeyTomb) {
           if (free_entry == ~0ULL) {
-            free_entry = b * kBucketEntries + j;
+            free_entry = s * E + j;
             free_was = k[j];
           }
           at_end = k[j] == kKeyEmpty;
         }
       }
-      b = next_bucket(ix, b);
+      s = next_sector(ix, s);
     }
     walked = max(walked, n);
     if (entry != ~0ULL) break;
@@ -244,7 +274,7 @@ __device__ __forceinline__ unsigned long long insert_entry(const IndexView& ix, 
     raise_status(AIBX_ERR_FULL);
     return ~0ULL;
   }
-  atomicOr(entry_mask(ix, entry), (unsigned long long)m);
+  entry_mask_or(ix, entry, m);
   atomicMin(entry_id(ix, entry), id);
   return entry;
 }
@@ -252,8 +282,7 @@ __device__ __forceinline__ unsigned long long insert_entry(const IndexView& ix, 
 // live += added - removed, removed-entry count += removed - reused, longest walk = max: summed
 // over the CTA in shared memory, then one atomic each per CTA.  Every thread of the CTA must
 // call it.  The CTA whose addition takes the live count past the table's capacity reports FULL
-// for the entries beyond it (the table has physical room for up to two more than `capacity`,
-// so the count, not the placement, is what keeps the limit exact).
+// for the entries beyond it (the count, not the placement, is what keeps the limit exact).
 __device__ __forceinline__ void fold_counters(const IndexView& ix, unsigned int added,
                                               unsigned int reused, unsigned int removed,
                                               unsigned int walked) {
@@ -302,11 +331,18 @@ __global__ void index_insert_kernel(IndexView ix, const uint64_t* __restrict__ k
 // One entry as a scan sees it (entry-parallel kernels: export, move, victim choice).
 __device__ __forceinline__ bool load_entry(const IndexView& ix, unsigned long long e, uint64_t& key,
                                            uint64_t& mask, uint32_t& id) {
-  const Bucket* b = ix.buckets + e / kBucketEntries;
-  const int j = (int)(e % kBucketEntries);
-  key = __ldg(&b->key[j]);
-  mask = __ldg(&b->mask[j]);
-  id = __ldg(&b->id[j]);
+  if (ix.narrow) {
+    const unsigned long long* p = ix.words + 4 * (e >> 1);
+    key = __ldg(p + (e & 1));
+    const unsigned long long v = __ldg(p + 2 + (e & 1));
+    mask = (unsigned int)v;
+    id = (unsigned int)(v >> 32);
+  } else {
+    const unsigned long long* p = ix.words + 4 * e;
+    key = __ldg(p);
+    mask = __ldg(p + 1);
+    id = (unsigned int)__ldg(p + 2);
+  }
   return !key_reserved(key) && mask != 0;
 }
 
@@ -380,7 +416,7 @@ __global__ void index_evict_clear_kernel(IndexView ix, const uint64_t* __restric
   if (key_reserved(key)) return;
   const unsigned long long e = find_entry_rw(ix, key);
   if (e == ~0ULL) return;
-  atomicAnd(entry_mask(ix, e), ~(unsigned long long)masks[i]);
+  entry_mask_clear(ix, e, masks[i]);
 }
 
 // evict, pass 2: report ids of entries left without a pod (every duplicate sees the same state)
@@ -393,8 +429,7 @@ __global__ void index_evict_report_kernel(IndexView ix, const uint64_t* __restri
   if (!key_reserved(key)) {
     const unsigned long long e = find_entry_rw(ix, key);
     if (e != ~0ULL) {
-      const unsigned long long m = *reinterpret_cast<volatile unsigned long long*>(entry_mask(ix, e));
-      if (m == 0) out = *reinterpret_cast<volatile unsigned int*>(entry_id(ix, e));
+      if (entry_mask_now(ix, e) == 0) out = *reinterpret_cast<volatile unsigned int*>(entry_id(ix, e));
     }
   }
   freed[i] = out;
@@ -409,7 +444,7 @@ __global__ void index_evict_remove_kernel(IndexView ix, const uint64_t* __restri
   if (!key_reserved(key)) {
     const unsigned long long e = find_entry_rw(ix, key);
     if (e != ~0ULL &&
-        *reinterpret_cast<volatile unsigned long long*>(entry_mask(ix, e)) == 0 &&
+        entry_mask_now(ix, e) == 0 &&
         atomicCAS(entry_key(ix, e), (unsigned long long)key, kKeyTomb) == key) {
       *entry_id(ix, e) = AIBX_NO_BLOCK;    // ready for reuse by a later insert
       ix.stamps[e] = 0u;
@@ -438,7 +473,7 @@ index_evict_coop_kernel(IndexView ix, const uint64_t* __restrict__ keys,
     const uint64_t key = keys[i];
     if (key_reserved(key)) continue;
     const unsigned long long e = find_entry_rw(ix, key);
-    if (e != ~0ULL) atomicAnd(entry_mask(ix, e), ~(unsigned long long)masks[i]);
+    if (e != ~0ULL) entry_mask_clear(ix, e, masks[i]);
     mine = e;
   }
   grid.sync();
@@ -448,8 +483,7 @@ index_evict_coop_kernel(IndexView ix, const uint64_t* __restrict__ keys,
       uint32_t out = AIBX_NO_BLOCK;
       if (!key_reserved(key)) {
         const unsigned long long e = single ? mine : find_entry_rw(ix, key);
-        if (e != ~0ULL &&
-            *reinterpret_cast<volatile unsigned long long*>(entry_mask(ix, e)) == 0)
+        if (e != ~0ULL && entry_mask_now(ix, e) == 0)
           out = *reinterpret_cast<volatile unsigned int*>(entry_id(ix, e));
       }
       freed[i] = out;
@@ -463,7 +497,7 @@ index_evict_coop_kernel(IndexView ix, const uint64_t* __restrict__ keys,
     // an entry another thread of the same key has already removed no longer carries the key
     const unsigned long long e = single ? mine : find_entry_rw(ix, key);
     if (e != ~0ULL &&
-        *reinterpret_cast<volatile unsigned long long*>(entry_mask(ix, e)) == 0 &&
+        entry_mask_now(ix, e) == 0 &&
         atomicCAS(entry_key(ix, e), (unsigned long long)key, kKeyTomb) == key) {
       *entry_id(ix, e) = AIBX_NO_BLOCK;
       ix.stamps[e] = 0u;
@@ -586,7 +620,8 @@ __device__ __forceinline__ void fold_finish(const PrefixFold& st, int lane, int 
 // are warps enough without splitting a request.  No barrier, no shared-memory atomics.
 constexpr int kMatchWarpKernelWarps = 4;
 
-__global__ void __launch_bounds__(kMatchWarpKernelWarps * 32, 12)
+template <bool NARROW>
+__global__ void __launch_bounds__(kMatchWarpKernelWarps * 32, 16)
 match_prefix_warp_kernel(IndexView ix, const uint64_t* __restrict__ hashes,
                          const int64_t* __restrict__ blk_off, int R,
                          uint32_t* __restrict__ match_len, uint32_t* __restrict__ any_len,
@@ -613,7 +648,7 @@ match_prefix_warp_kernel(IndexView ix, const uint64_t* __restrict__ hashes,
     uint64_t mask = 0;
     uint32_t id = AIBX_NO_BLOCK;
     unsigned long long entry = ~0ULL;
-    if ((unsigned int)lane < m) probe_ro(ix, key, mask, id, entry);
+    if ((unsigned int)lane < m) probe_ro_w<NARROW>(ix, key, mask, id, entry);
     const unsigned int first = st.pos;
     fold_chunk(st, lane, m, mask, id, all, s_ml[warp], block_ids ? block_ids + off : nullptr);
     // the blocks of the matched prefix are marked as used, with the entry the probe just found
@@ -745,7 +780,7 @@ __global__ void match_prefix_kernel(IndexView ix, const uint64_t* __restrict__ h
     }
     if (epoch) {
       // Where the prefix ends is only known now that all warps of the request have met, so the
-      // stamps are set in a second walk over the matched blocks; their buckets were read a
+      // stamps are set in a second walk over the matched blocks; their sectors were read a
       // moment ago and are still in L2.
       for (unsigned int i = tid_in_group; i < a; i += group_threads) {
         uint64_t mask;

@@ -65,29 +65,33 @@ void prefer_copy_carveout() {
   });
 }
 
-// Device storage of one table: buckets, stamps and counters in ONE allocation (64-byte aligned
-// parts), so that creating or dropping a table is one call into the allocator.
+// Device storage of one table: sectors, stamps and counters in ONE allocation (64-byte aligned
+// parts), so that creating or dropping a table is one call into the allocator.  Tables of up to
+// 32 pods take the narrow entry (two per 32-byte sector), the others the wide one.
 int32_t alloc_view(uint64_t capacity, int num_pods, IndexView* out) {
-  const uint64_t nb = (capacity + kBucketEntries - 1) / kBucketEntries;
-  const size_t bucket_bytes = (size_t)nb * sizeof(Bucket);
-  const size_t stamp_bytes = ((size_t)nb * kBucketEntries * sizeof(unsigned int) + 63) & ~(size_t)63;
+  const int narrow = num_pods <= 32 ? 1 : 0;
+  const uint64_t nb = narrow ? capacity / 2 : capacity;
+  const size_t sector_bytes = (size_t)nb * 32;
+  const size_t stamp_bytes = ((size_t)capacity * sizeof(unsigned int) + 63) & ~(size_t)63;
   void* base = nullptr;
-  if (cudaMalloc(&base, bucket_bytes + stamp_bytes + 64) != cudaSuccess) {
+  if (cudaMalloc(&base, sector_bytes + stamp_bytes + 64) != cudaSuccess) {
     cudaGetLastError();   // an allocation failure is not sticky; leave no error behind
     return AIBX_ERR_NOMEM;
   }
   char* p = static_cast<char*>(base);
-  out->buckets = reinterpret_cast<Bucket*>(p);
-  out->stamps = reinterpret_cast<unsigned int*>(p + bucket_bytes);
-  out->counters = reinterpret_cast<unsigned long long*>(p + bucket_bytes + stamp_bytes);
+  out->words = reinterpret_cast<unsigned long long*>(p);
+  out->stamps = reinterpret_cast<unsigned int*>(p + sector_bytes);
+  out->counters = reinterpret_cast<unsigned long long*>(p + sector_bytes + stamp_bytes);
   out->nb = nb;
   out->capacity = capacity;
-  out->max_walk = (unsigned int)(nb < kMaxWalk ? nb : kMaxWalk);
+  const uint64_t walk = narrow ? kMaxWalkEntries / 2 : kMaxWalkEntries;
+  out->max_walk = (unsigned int)(nb < walk ? nb : walk);
   out->num_pods = num_pods;
+  out->narrow = narrow;
   return AIBX_OK;
 }
 
-void free_view(const IndexView& v) { cudaFree(v.buckets); }
+void free_view(const IndexView& v) { cudaFree(v.words); }
 
 bool capacity_ok(uint64_t c) { return c >= 8 && (c & (c - 1)) == 0 && c <= (1ULL << 40); }
 
@@ -452,9 +456,15 @@ int32_t launch_match(const aibx_index_t* ix, const uint64_t* d_hashes, const int
   while (wpr < 32 && (long long)R * wpr * 2 <= target) wpr *= 2;
   if (wpr == 1) {
     // warps enough with one per request: the shape without barriers and shared-memory atomics
-    match_prefix_warp_kernel<<<blocks_for(R, kMatchWarpKernelWarps), kMatchWarpKernelWarps * 32, 0,
-                               st>>>(ix->view, d_hashes, d_blk_off, R, d_match_len, d_any_len,
-                                     d_block_ids, sp, d_best_pod, d_best_score, epoch);
+    const unsigned int grid = blocks_for(R, kMatchWarpKernelWarps);
+    if (ix->view.narrow)
+      match_prefix_warp_kernel<true><<<grid, kMatchWarpKernelWarps * 32, 0, st>>>(
+          ix->view, d_hashes, d_blk_off, R, d_match_len, d_any_len, d_block_ids, sp, d_best_pod,
+          d_best_score, epoch);
+    else
+      match_prefix_warp_kernel<false><<<grid, kMatchWarpKernelWarps * 32, 0, st>>>(
+          ix->view, d_hashes, d_blk_off, R, d_match_len, d_any_len, d_block_ids, sp, d_best_pod,
+          d_best_score, epoch);
     return launch_status();
   }
   const int warps_per_cta = wpr > kMatchWarpsMin ? wpr : kMatchWarpsMin;

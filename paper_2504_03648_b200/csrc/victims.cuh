@@ -48,7 +48,7 @@ __global__ void index_touch_kernel(IndexView ix, const uint64_t* __restrict__ ke
   if (key_reserved(key)) return;
   const unsigned long long e = find_entry_rw(ix, key);
   if (e == ~0ULL) return;
-  if (*reinterpret_cast<volatile unsigned long long*>(entry_mask(ix, e)) == 0) return;
+  if (entry_mask_now(ix, e) == 0) return;
   touch_entry(ix, e, epoch);
 }
 

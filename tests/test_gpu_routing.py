@@ -634,9 +634,9 @@ def test_churn_fills_the_table_with_removed_entries_and_rehash_clears_them():
         assert aibx.status_fetch() == (0, 0)
     live, removed, cap, walk = g.stats2()
     assert (live, cap) == (10, 64) == (o.stats()[0], 64)
-    # 66 entries of physical room, 10 live: after 192 publish/expire pairs none was never used
-    assert 16 <= removed <= 56 and live + removed <= 66
-    assert 1 <= walk <= 22                                            # 22 buckets = the whole table
+    # 64 entries of room, 10 live, 192 publish/expire pairs
+    assert 16 <= removed <= 54 and live + removed <= 64
+    assert 1 <= walk <= 32                                            # 32 sectors = the whole table
     g.rehash(64)
     live, removed, cap, walk = g.stats2()
     assert (live, removed, cap) == (10, 0, 64) and walk <= 3
