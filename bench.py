@@ -713,6 +713,9 @@ def main():
     ap.add_argument("--case", default=None, choices=sorted(CASES),
                     help="run one small single-kernel case instead of the bench step")
     ap.add_argument("--log2cap", type=int, default=23)
+    ap.add_argument("--ws-mib", type=int, default=0, help="random_reads: one working-set size")
+    ap.add_argument("--read-bytes", type=int, default=0, choices=[0, 32, 64, 128],
+                    help="random_reads: one read size")
     ap.add_argument("--shape", default="cfg2", choices=["cfg2", "cfg4", "cfg5"],
                     help="block shape of the kv_small case")
     ap.add_argument("--gpus", type=int, default=1)

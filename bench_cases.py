@@ -228,8 +228,9 @@ def case_random_reads(args):
     t_flush = statistics.median(_event_times(torch, lambda: flush.sum(), 7, 3))
     peak, kind = measured_peak_hbm()
     rows = []
-    for ws_mib in (11, 16, 43, 64, 171, 256, 1024, 4096):
-        for gran in (32, 64, 128):
+    sizes = (args.ws_mib,) if args.ws_mib else (11, 16, 43, 64, 128, 171, 256, 1024, 4096)
+    for ws_mib in sizes:
+        for gran in ((args.read_bytes,) if args.read_bytes else (32, 64, 128)):
             g = _random_read_ceiling(torch, ws_mib << 20, gran, flush, t_flush)
             rows.append({"working_set_MiB": ws_mib, "read_bytes": gran, "Greads_per_s": round(g, 2),
                          "GBps": round(g * gran, 1), "frac_of_stream": round(g * gran / peak, 4)})
