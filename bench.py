@@ -45,7 +45,7 @@ METRIC = "kv_gather_scatter_GBps_whole_step"
 UNIT = "GB/s"
 WORKLOAD = "cfg2-llama3-8b: 64 requests (1k-8k tokens, 32 Zipf prompts), index 200k/2^19 x 16 pods, " \
            "pool 4096 x 2 MiB bf16 blocks, gather+scatter of all matched blocks"
-KERNELS_PER_STEP = 7    # head (hash+match+score), collect, gather, scatter, hash tail, insert, evict
+KERNELS_PER_STEP = 6    # head (hash+match+score+matched-block set), gather, scatter, hash tail, insert, evict
 
 from bench_cases import CASES, cpu_model, measured_peak_hbm, ncu_traffic, routing_batch_times  # noqa: E402
 
@@ -175,7 +175,7 @@ class GpuJob:
         self.d_hashed = torch.empty(R, dtype=torch.uint32, device="cuda")
         self.d_next_seed = torch.empty(R, dtype=torch.uint64, device="cuda")
         self.d_pod_load = dev(w.pod_load)
-        self.d_scratch = torch.empty(aibx.collect_scratch_bytes(kv.num_blocks) // 4 + 1,
+        self.d_scratch = torch.empty(aibx.route_collect_scratch_bytes(kv.num_blocks) // 4 + 1,
                                      dtype=torch.int32, device="cuda")
         self.d_unique = torch.empty(self.nb, dtype=torch.uint32, device="cuda")
         self.d_count = torch.empty(1, dtype=torch.uint32, device="cuda")
@@ -207,15 +207,15 @@ class GpuJob:
     # -- pieces of a step ------------------------------------------------------------------
     def routing_async(self) -> None:
         """Routing half of a step, enqueued only: the block count stays on the device.  Only
-        the part of every chain that matching needs is hashed here (aibx_route_head); the rest
+        the part of every chain that matching needs is hashed here (aibx_route_head_collect, which
+        also leaves the set of matched blocks); the rest
         is hashed by hash_tail() off the critical path."""
         aibx = self.aibx
-        aibx.route_head(self.index, self.d_tokens, self.d_tok_off, self.d_blk_off, self.B, 0,
-                        self.d_pod_load, self.w.ready_mask, None, self.d_hashes, self.d_match_len,
-                        self.d_any_len, self.d_block_ids, self.d_best_pod, self.d_best_score,
-                        self.d_hashed, self.d_next_seed)
-        aibx.collect_blocks(self.d_block_ids, self.kv.num_blocks, self.d_scratch, self.d_unique,
-                            self.d_count)
+        aibx.route_head_collect(self.index, self.d_tokens, self.d_tok_off, self.d_blk_off, self.B, 0,
+                                self.d_pod_load, self.w.ready_mask, None, 0, self.d_hashes,
+                                self.d_match_len, self.d_any_len, self.d_block_ids, self.d_best_pod,
+                                self.d_best_score, self.d_hashed, self.d_next_seed,
+                                self.kv.num_blocks, self.d_scratch, self.d_unique, self.d_count)
 
     def hash_tail(self) -> None:
         """The rest of every chain (the keys of the blocks that will be published)."""
@@ -241,7 +241,7 @@ class GpuJob:
 
     def step(self, record_copy_events=False):
         """One pass of the whole path, enqueued without any host round trip: the number of
-        matched blocks goes from aibx_collect_blocks to the copies on the device; the tail of
+        matched blocks goes from the routing kernel to the copies on the device; the tail of
         the hash chains and the index publish/expire batch (both independent of the copies) run
         beside them on a second stream."""
         torch, aibx = self.torch, self.aibx
@@ -335,6 +335,7 @@ class GpuJob:
                 self.d_pod_load, self.w.ready_mask, None, self.d_hashes, self.d_match_len,
                 self.d_any_len, self.d_block_ids, self.d_best_pod, self.d_best_score,
                 self.d_hashed, self.d_next_seed),
+            "route_head_collect": self.routing_async,
             "hash_tail": self.hash_tail,
             "match_prefix": lambda: self.index.match_prefix(self.d_hashes, self.d_blk_off,
                                                             self.d_match_len, self.d_any_len,

@@ -281,6 +281,29 @@ int32_t aibx_route_head_touch(aibx_index_t* index, const int32_t* d_tokens,
                               uint32_t* d_any_len, uint32_t* d_block_ids, int32_t* d_best_pod,
                               int64_t* d_best_score, uint32_t* d_hashed, uint64_t* d_next_seed,
                               void* stream);
+/* aibx_route_head that also makes the set of matched blocks (what aibx_collect_blocks gives for
+ * d_block_ids: ascending distinct valid ids of all matched prefixes in d_unique_ids [blk_off[R]],
+ * padded with AIBX_NO_BLOCK, their number in *d_count) without a further launch: the probers
+ * mark the ids in a bitmap and the last one to finish turns it into the list, so the copies can
+ * follow the routing kernel directly (Section 3.2.5: a block shared by several requests moves
+ * once).  epoch = 0: no stamping; otherwise as aibx_route_head_touch.  d_scratch: device memory
+ * of aibx_route_collect_scratch_bytes(num_blocks) bytes, 4-byte aligned, contents irrelevant
+ * (cleared by the call).  d_block_ids is required.  Pools of more than 262,144 blocks and block
+ * sizes other than 8, 16, 32, 64 tokens take the routing call followed by the collect kernels
+ * (same results; the list length is read on the device, so there is still no host round trip).
+ * Ids >= num_blocks other than AIBX_NO_BLOCK raise device status RANGE and are left out.
+ */
+uint64_t aibx_route_collect_scratch_bytes(uint32_t num_blocks);
+int32_t aibx_route_head_collect(aibx_index_t* index, const int32_t* d_tokens,
+                                const int64_t* d_tok_off, const int64_t* d_blk_off, int32_t R,
+                                int32_t block_tokens, uint64_t root_seed,
+                                const int32_t* d_pod_load, uint64_t ready_mask,
+                                const aibx_route_params_t* params, uint32_t epoch,
+                                uint64_t* d_hashes, uint32_t* d_match_len, uint32_t* d_any_len,
+                                uint32_t* d_block_ids, int32_t* d_best_pod, int64_t* d_best_score,
+                                uint32_t* d_hashed, uint64_t* d_next_seed, uint32_t num_blocks,
+                                void* d_scratch, uint32_t* d_unique_ids, uint32_t* d_count,
+                                void* stream);
 int32_t aibx_hash_blocks_resume(const int32_t* d_tokens, const int64_t* d_tok_off,
                                 const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
                                 const uint32_t* d_hashed, const uint64_t* d_next_seed,

@@ -100,6 +100,8 @@ def lib():
                                 vp, vp, vp, vp, vp, vp, vp, vp, vp],
             "aibx_route_head_touch": [vp, vp, vp, vp, i32, i32, u64, vp, u64, C.POINTER(RouteParams),
                                       u32, vp, vp, vp, vp, vp, vp, vp, vp, vp],
+            "aibx_route_head_collect": [vp, vp, vp, vp, i32, i32, u64, vp, u64, C.POINTER(RouteParams),
+                                        u32, vp, vp, vp, vp, vp, vp, vp, vp, u32, vp, vp, vp, vp],
             "aibx_match_prefix_touch": [vp, vp, vp, i32, u32, vp, vp, vp, vp],
             "aibx_hash_blocks_resume": [vp, vp, vp, i32, i32, vp, vp, vp, vp],
             "aibx_route_policy": [i32, vp, vp, i32, i32, C.POINTER(PodMetrics), vp, u64, i32, vp, vp],
@@ -126,6 +128,8 @@ def lib():
             fn.restype = i32
         L.aibx_collect_scratch_bytes.argtypes = [u32]
         L.aibx_collect_scratch_bytes.restype = u64
+        L.aibx_route_collect_scratch_bytes.argtypes = [u32]
+        L.aibx_route_collect_scratch_bytes.restype = u64
         L.aibx_collect_static_max_blocks.argtypes = []
         L.aibx_collect_static_max_blocks.restype = u32
         L.aibx_strerror.argtypes = [i32]
@@ -321,6 +325,28 @@ def route_head_touch(index: Index, tokens, tok_off, blk_off, block_tokens: int, 
         _ptr(match_len, torch.uint32), _ptr(any_len, torch.uint32), _ptr(block_ids, torch.uint32),
         _ptr(best_pod, torch.int32), _ptr(best_score, torch.int64), _ptr(hashed, torch.uint32),
         _ptr(next_seed, torch.uint64), _stream()))
+
+
+def route_collect_scratch_bytes(num_blocks: int) -> int:
+    return int(lib().aibx_route_collect_scratch_bytes(num_blocks))
+
+
+def route_head_collect(index: Index, tokens, tok_off, blk_off, block_tokens: int, root_seed: int,
+                       pod_load, ready_mask: int, params, epoch: int, hashes, match_len, any_len,
+                       block_ids, best_pod, best_score, hashed, next_seed, num_blocks: int,
+                       scratch, unique_ids, count) -> None:
+    """route_head (+ stamping when epoch > 0) that also leaves the set of matched blocks in
+    unique_ids / count, without a further launch."""
+    R = tok_off.numel() - 1
+    prm = None if params is None else C.byref(RouteParams(*params))
+    _check("aibx_route_head_collect", lib().aibx_route_head_collect(
+        index._h, _ptr(tokens, torch.int32), _ptr(tok_off, torch.int64), _ptr(blk_off, torch.int64),
+        R, block_tokens, root_seed & (2**64 - 1), _ptr(pod_load, torch.int32),
+        ready_mask & (2**64 - 1), prm, epoch, _ptr(hashes, torch.uint64),
+        _ptr(match_len, torch.uint32), _ptr(any_len, torch.uint32), _ptr(block_ids, torch.uint32),
+        _ptr(best_pod, torch.int32), _ptr(best_score, torch.int64), _ptr(hashed, torch.uint32),
+        _ptr(next_seed, torch.uint64), num_blocks, _ptr(scratch), _ptr(unique_ids, torch.uint32),
+        _ptr(count, torch.uint32), _stream()))
 
 
 def hash_blocks_resume(tokens, tok_off, blk_off, block_tokens: int, hashed, next_seed,

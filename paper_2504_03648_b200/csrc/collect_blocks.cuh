@@ -10,23 +10,30 @@ namespace aibx {
 
 constexpr int kCollectThreads = 1024;
 
+// `n_dev` (nullable): the list's length read on the device instead of `n` (the grid then
+// strides over it).
 __global__ void collect_mark_kernel(const uint32_t* __restrict__ ids, int64_t n,
-                                    uint32_t num_blocks, unsigned int* __restrict__ bitmap) {
-  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const uint32_t id = ids[i];
-  if (id < num_blocks) {
-    atomicOr(&bitmap[id >> 5], 1u << (id & 31u));
-  } else if (id != AIBX_NO_BLOCK) {
-    raise_status(AIBX_ERR_RANGE);
+                                    const int64_t* __restrict__ n_dev, uint32_t num_blocks,
+                                    unsigned int* __restrict__ bitmap) {
+  if (n_dev) n = *n_dev;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    const uint32_t id = ids[i];
+    if (id < num_blocks) {
+      atomicOr(&bitmap[id >> 5], 1u << (id & 31u));
+    } else if (id != AIBX_NO_BLOCK) {
+      raise_status(AIBX_ERR_RANGE);
+    }
   }
 }
 
 __global__ void __launch_bounds__(kCollectThreads)
 collect_compact_kernel(const unsigned int* __restrict__ bitmap, uint32_t num_blocks, int64_t n,
-                       uint32_t* __restrict__ out, uint32_t* __restrict__ count) {
+                       const int64_t* __restrict__ n_dev, uint32_t* __restrict__ out,
+                       uint32_t* __restrict__ count) {
   __shared__ unsigned int s_warp[32];
   __shared__ unsigned int s_base;
+  if (n_dev) n = *n_dev;
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const int warp = tid >> 5;

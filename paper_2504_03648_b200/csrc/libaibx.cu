@@ -510,7 +510,8 @@ int32_t route_head_impl(const aibx_index_t* ix, const int32_t* d_tokens, const i
                         const aibx_route_params_t* params, uint64_t* d_hashes,
                         uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
                         int32_t* d_best_pod, int64_t* d_best_score, uint32_t* d_hashed,
-                        uint64_t* d_next_seed, void* stream, unsigned int epoch) {
+                        uint64_t* d_next_seed, void* stream, unsigned int epoch,
+                        HeadCollect hc = HeadCollect{nullptr, nullptr, nullptr, nullptr, 0u}) {
   if (!ix || R < 0 || block_tokens <= 0 || block_tokens % 8 != 0 || block_tokens > 1024)
     return AIBX_ERR_INVALID;
   if (R == 0) return AIBX_OK;
@@ -529,7 +530,7 @@ int32_t route_head_impl(const aibx_index_t* ix, const int32_t* d_tokens, const i
   route_head_kernel<SPB><<<grid, 288, 0, st>>>(ix->view, d_tokens, d_tok_off, d_blk_off, R,      \
                                               root_seed, d_hashes, d_match_len, d_any_len,      \
                                               d_block_ids, sp, d_best_pod, d_best_score,        \
-                                              d_hashed, d_next_seed, epoch)
+                                              d_hashed, d_next_seed, epoch, hc)
   if (spb == 1) {
     AIBX_HEAD_LAUNCH(1);
   } else if (spb == 2) {
@@ -578,6 +579,61 @@ int32_t aibx_route_head_touch(aibx_index_t* ix, const int32_t* d_tokens, const i
   return route_head_impl(ix, d_tokens, d_tok_off, d_blk_off, R, block_tokens, root_seed, d_pod_load,
                          ready_mask, params, d_hashes, d_match_len, d_any_len, d_block_ids,
                          d_best_pod, d_best_score, d_hashed, d_next_seed, stream, epoch);
+}
+
+uint64_t aibx_route_collect_scratch_bytes(uint32_t num_blocks) {
+  return aibx_collect_scratch_bytes(num_blocks) + 64;    // the bitmap, then the arrival counter
+}
+
+int32_t aibx_route_head_collect(aibx_index_t* ix, const int32_t* d_tokens, const int64_t* d_tok_off,
+                                const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
+                                uint64_t root_seed, const int32_t* d_pod_load, uint64_t ready_mask,
+                                const aibx_route_params_t* params, uint32_t epoch,
+                                uint64_t* d_hashes, uint32_t* d_match_len, uint32_t* d_any_len,
+                                uint32_t* d_block_ids, int32_t* d_best_pod, int64_t* d_best_score,
+                                uint32_t* d_hashed, uint64_t* d_next_seed, uint32_t num_blocks,
+                                void* d_scratch, uint32_t* d_unique_ids, uint32_t* d_count,
+                                void* stream) {
+  if (!ix || epoch >= (1u << 30) || (epoch && ix->migrating)) return AIBX_ERR_INVALID;
+  if (!d_count || !d_scratch || (reinterpret_cast<uintptr_t>(d_scratch) & 3)) return AIBX_ERR_INVALID;
+  if (R > 0 && (!d_block_ids || !d_unique_ids)) return AIBX_ERR_INVALID;
+  cudaStream_t st = as_stream(stream);
+  const int spb = block_tokens / 8;
+  const bool head_path = block_tokens > 0 && block_tokens % 8 == 0 &&
+                         (spb == 1 || spb == 2 || spb == 4 || spb == 8);
+  const uint32_t n_words = (num_blocks + 31u) / 32u;
+  if (R <= 0 || !head_path || n_words > kCollectSmallWords) {
+    // nothing to fuse into (no requests, another block size, a pool too large for one warp to
+    // compact): the plain call, then the set from its block ids
+    const int32_t rc = route_head_impl(ix, d_tokens, d_tok_off, d_blk_off, R, block_tokens,
+                                       root_seed, d_pod_load, ready_mask, params, d_hashes,
+                                       d_match_len, d_any_len, d_block_ids, d_best_pod,
+                                       d_best_score, d_hashed, d_next_seed, stream, epoch);
+    if (rc != AIBX_OK) return rc;
+    if (R <= 0) return cudaMemsetAsync(d_count, 0, sizeof(uint32_t), st) == cudaSuccess
+                           ? AIBX_OK : AIBX_ERR_CUDA;
+    // the list's length, blk_off[R], is read on the device: no host round trip here either
+    unsigned int* bitmap = static_cast<unsigned int*>(d_scratch);
+    if (num_blocks > 0 &&
+        cudaMemsetAsync(bitmap, 0, aibx_collect_scratch_bytes(num_blocks), st) != cudaSuccess)
+      return AIBX_ERR_CUDA;
+    collect_mark_kernel<<<sm_count() * 8, 256, 0, st>>>(d_block_ids, 0, d_blk_off + R, num_blocks,
+                                                        bitmap);
+    collect_compact_kernel<<<1, kCollectThreads, 0, st>>>(bitmap, num_blocks, 0, d_blk_off + R,
+                                                          d_unique_ids, d_count);
+    return launch_status();
+  }
+  const size_t bitmap_bytes = (size_t)aibx_collect_scratch_bytes(num_blocks);
+  if (cudaMemsetAsync(d_scratch, 0, bitmap_bytes + 64, st) != cudaSuccess) return AIBX_ERR_CUDA;
+  HeadCollect hc;
+  hc.bitmap = static_cast<unsigned int*>(d_scratch);
+  hc.arrived = reinterpret_cast<unsigned int*>(static_cast<char*>(d_scratch) + bitmap_bytes);
+  hc.unique = d_unique_ids;
+  hc.count = d_count;
+  hc.num_blocks = num_blocks;
+  return route_head_impl(ix, d_tokens, d_tok_off, d_blk_off, R, block_tokens, root_seed, d_pod_load,
+                         ready_mask, params, d_hashes, d_match_len, d_any_len, d_block_ids,
+                         d_best_pod, d_best_score, d_hashed, d_next_seed, stream, epoch, hc);
 }
 
 int32_t aibx_hash_blocks_resume(const int32_t* d_tokens, const int64_t* d_tok_off,
@@ -684,9 +740,10 @@ int32_t aibx_collect_blocks(const uint32_t* d_block_ids, int64_t n, uint32_t num
       cudaMemsetAsync(bitmap, 0, aibx_collect_scratch_bytes(num_blocks), st) != cudaSuccess)
     return AIBX_ERR_CUDA;
   if (n > 0)
-    collect_mark_kernel<<<blocks_for(n, 256), 256, 0, st>>>(d_block_ids, n, num_blocks, bitmap);
-  collect_compact_kernel<<<1, kCollectThreads, 0, st>>>(bitmap, num_blocks, n, d_unique_ids,
-                                                        d_count);
+    collect_mark_kernel<<<blocks_for(n, 256), 256, 0, st>>>(d_block_ids, n, nullptr, num_blocks,
+                                                            bitmap);
+  collect_compact_kernel<<<1, kCollectThreads, 0, st>>>(bitmap, num_blocks, n, nullptr,
+                                                        d_unique_ids, d_count);
   return launch_status();
 }
 
@@ -703,9 +760,10 @@ int32_t aibx_collect_blocks_static(const uint32_t* d_block_ids, int64_t n, uint3
       cudaMemsetAsync(bitmap, 0, aibx_collect_scratch_bytes(num_blocks), st) != cudaSuccess)
     return AIBX_ERR_CUDA;
   if (n > 0)
-    collect_mark_kernel<<<blocks_for(n, 256), 256, 0, st>>>(d_block_ids, n, num_blocks, bitmap);
-  collect_compact_kernel<<<1, kCollectThreads, 0, st>>>(bitmap, num_blocks, n, d_unique_ids,
-                                                        d_count);
+    collect_mark_kernel<<<blocks_for(n, 256), 256, 0, st>>>(d_block_ids, n, nullptr, num_blocks,
+                                                            bitmap);
+  collect_compact_kernel<<<1, kCollectThreads, 0, st>>>(bitmap, num_blocks, n, nullptr,
+                                                        d_unique_ids, d_count);
   return launch_status();
 }
 

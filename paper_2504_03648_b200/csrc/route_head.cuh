@@ -79,6 +79,46 @@ __device__ __noinline__ bool head_wait_for_room(const unsigned int* word, unsign
   return false;
 }
 
+// The set of matched blocks made by the head kernel itself (no further launch): the probers mark
+// the ids of every matched prefix in a bitmap over block ids; every prober fills its own
+// request's part of the output with AIBX_NO_BLOCK, counts itself in, and the warp that counts in
+// last - all marks are in the bitmap by then - turns it into the ascending list.  Nobody waits:
+// the last arriver does the work.  bitmap == nullptr: no set is made.
+struct HeadCollect {
+  unsigned int* bitmap;      // zeroed before the launch, (num_blocks + 31) / 32 words
+  unsigned int* arrived;     // zeroed before the launch
+  uint32_t* unique;          // [blk_off[R]] ascending distinct ids, then AIBX_NO_BLOCK
+  uint32_t* count;
+  uint32_t num_blocks;
+};
+
+// One warp turns the bitmap into the ascending id list (at most kCollectSmallWords words: the
+// host only fuses the set into the head kernel for pools of that size).
+__device__ __forceinline__ void head_compact(const HeadCollect& hc, int lane, int64_t n_total) {
+  const uint32_t n_words = (hc.num_blocks + 31u) / 32u;
+  unsigned int base = 0;
+  for (uint32_t w0 = 0; w0 < n_words; w0 += 32) {
+    const uint32_t w = w0 + lane;
+    unsigned int bits = w < n_words ? __ldcg(hc.bitmap + w) : 0u;
+    const unsigned int c = __popc(bits);
+    unsigned int inc = c;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const unsigned int o = __shfl_up_sync(0xffffffffu, inc, d);
+      if (lane >= d) inc += o;
+    }
+    unsigned int pos = base + inc - c;
+    while (bits) {
+      const int b = __ffs(bits) - 1;
+      bits &= bits - 1;
+      if ((int64_t)pos < n_total) hc.unique[pos] = w * 32u + (uint32_t)b;
+      ++pos;
+    }
+    base += __shfl_sync(0xffffffffu, inc, 31);
+  }
+  if (lane == 0) *hc.count = base;
+}
+
 template <int SPB>   // stripes of 32 bytes per block: 1, 2, 4 or 8
 __global__ void __launch_bounds__(288)
 route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
@@ -87,7 +127,7 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
                   uint32_t* __restrict__ any_len, uint32_t* __restrict__ block_ids, ScoreParams sp,
                   int32_t* __restrict__ best_pod, int64_t* __restrict__ best_score,
                   uint32_t* __restrict__ hashed_out, uint64_t* __restrict__ seed_out,
-                  unsigned int epoch) {
+                  unsigned int epoch, HeadCollect hc) {
   constexpr int BPG = kGroupStripes / SPB;             // blocks per group of 8 stripes
   __shared__ HeadShared sh;
   const int lane = threadIdx.x & 31;
@@ -235,7 +275,12 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
     last_key = shfl64(0xffffffffu, key, (int)m - 1);
     const unsigned int first = st.pos;
     fold_chunk(st, lane, m, mask, id, all, sh.match_len[qi], block_ids ? block_ids + out0 : nullptr);
-    if (epoch && first + (unsigned int)lane < st.pos) touch_entry(ix, entry, epoch);
+    const bool matched = first + (unsigned int)lane < st.pos;
+    if (epoch && matched) touch_entry(ix, entry, epoch);
+    if (hc.bitmap && matched) {
+      if (id < hc.num_blocks) atomicOr(&hc.bitmap[id >> 5], 1u << (id & 31u));
+      else if (id != AIBX_NO_BLOCK) raise_status(AIBX_ERR_RANGE);
+    }
     // Lets the hasher reuse the ring slots just read.  The keys read from them have been used
     // by now (every lane computed its probe address from its key), so the reads are complete
     // before this store is issued; a plain store is enough.
@@ -248,6 +293,17 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
   if (lane == 0) {
     hashed_out[r] = written;                           // keys the hasher made beyond these are dropped
     seed_out[r] = last_key;
+  }
+  if (hc.bitmap) {
+    for (unsigned int i = lane; i < n_r; i += 32) hc.unique[out0 + i] = AIBX_NO_BLOCK;
+    __threadfence();                                   // marks and padding before the count
+    unsigned int before = 0;
+    if (lane == 0) before = atomicAdd(hc.arrived, 1u);
+    before = __shfl_sync(0xffffffffu, before, 0);
+    if (before == (unsigned int)R - 1u) {              // every other request has counted in
+      __threadfence();
+      head_compact(hc, lane, blk_off[R]);
+    }
   }
 }
 

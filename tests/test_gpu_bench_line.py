@@ -38,7 +38,7 @@ def test_bench_line_contract():
     e = d["e2e"]
     assert e["unit"] == d["unit"] and 0 < e["value"] < d["value"]
     assert e["h2d_bytes_per_step"] > moved // 4 and e["d2h_bytes_per_step"] > moved // 4
-    assert d["gpu_launches"] == 7 * d["steps"]
+    assert d["gpu_launches"] == 6 * d["steps"]
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and c["unit"] == d["unit"]
     assert c["cpu"] and c["all_cores"]["cores"] == c["cores_available"] >= 1

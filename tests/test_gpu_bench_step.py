@@ -1,5 +1,5 @@
 """The step that bench.py times, at the benchmark's full size and in its launch configuration
-(route_head, collect, device-counted gather and scatter; the tail of the hash chains and the index
+(route_head_collect, device-counted gather and scatter; the tail of the hash chains and the index
 publish/expire on a second stream), checked against the oracle: routing outputs element by element, the gathered buffer
 and the pool byte for byte, and the index back in its start state."""
 import os

@@ -198,3 +198,52 @@ def test_resume_from_any_block(B):
         assert (got[lo: lo + start[r]] == 0x7E7E7E7E7E7E7E7E).all(), r
         assert np.array_equal(got[lo + start[r]: hi], want[lo + start[r]: hi]), r
     assert aibx.status_fetch() == (0, 0)
+
+
+@pytest.mark.parametrize("mk,num_blocks", [(W.cfg1_routing, None), (W.cfg2_routing, None),
+                                           (W.cfg3_routing, None), (W.cfg5_routing, None),
+                                           (W.cfg2_routing, 3000), (W.cfg1_routing, 300000)])
+def test_route_head_collect_makes_the_matched_block_set(mk, num_blocks):
+    """route_head_collect against the oracle's match_prefix + collect_blocks: same routing
+    results and the same ascending set of matched blocks, twice in a row on the same scratch
+    (filled with garbage first: the call clears it).  num_blocks 3000 puts some ids of the cfg2
+    entries out of range (dropped, RANGE); 300,000 is a pool too large for the fused form, which
+    takes the separate collect kernels with the list length read on the device."""
+    w = W.build_routing(mk())
+    s = w.spec
+    B, P, R = s.block_tokens, s.num_pods, s.R
+    nblk = s.id_space if num_blocks is None else num_blocks
+    o = routing_oracle(w)
+    h, bo = o["hashes"], o["blk_off"]
+    rc, want_u, want_c = oracle.collect_blocks(o["block_ids"], nblk)
+    keys, masks, ids = fill_entries(w, o["src_hashes"])
+    g = aibx.Index(s.capacity, P)
+    g.insert(dev(keys), dev(masks), dev(ids))
+    nb = max(len(h), 1)
+    d_tok, d_toff, d_bo = dev(w.tokens), dev(w.tok_off), dev(bo)
+    scratch = torch.full((aibx.route_collect_scratch_bytes(nblk) // 4,), -1, dtype=torch.int32,
+                         device="cuda")
+    for rep in range(2):
+        d_h = torch.zeros(nb, dtype=torch.uint64, device="cuda")
+        d_ml, d_al, d_id = empty(R * P, torch.uint32), empty(R, torch.uint32), empty(nb, torch.uint32)
+        d_bp, d_bs = empty(R, torch.int32), empty(R, torch.int64)
+        d_dn, d_sd = empty(R, torch.uint32), empty(R, torch.uint64)
+        d_un = torch.full((nb,), 0x55, dtype=torch.uint32, device="cuda")
+        d_cnt = torch.full((1,), 0x55, dtype=torch.uint32, device="cuda")
+        aibx.route_head_collect(g, d_tok, d_toff, d_bo, B, 0, dev(w.pod_load), w.ready_mask, None,
+                                0, d_h, d_ml, d_al, d_id, d_bp, d_bs, d_dn, d_sd, nblk, scratch,
+                                d_un, d_cnt)
+        st = aibx.status_fetch()
+        assert np.array_equal(host(d_ml).reshape(R, P), o["match_len"])
+        assert np.array_equal(host(d_al), o["any_len"])
+        assert np.array_equal(host(d_id)[: len(h)], o["block_ids"])
+        assert np.array_equal(host(d_bp), o["best_pod"]) and np.array_equal(host(d_bs), o["best_score"])
+        assert int(host(d_cnt)[0]) == want_c
+        assert np.array_equal(host(d_un)[: len(h)], want_u)
+        if rc == oracle.ERR_RANGE:
+            assert st[0] == aibx.ERR_RANGE and st[1] > 0
+        else:
+            assert st == (0, 0)
+        aibx.hash_blocks_resume(d_tok, d_toff, d_bo, B, d_dn, d_sd, d_h)
+        assert np.array_equal(host(d_h)[: len(h)], h)
+    assert want_c > 0
