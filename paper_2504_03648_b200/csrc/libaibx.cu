@@ -284,7 +284,7 @@ int32_t aibx_index_stats2(const aibx_index_t* ix, uint64_t* live, uint64_t* remo
   if (live) *live = c[0];
   if (removed) *removed = c[1];
   if (capacity) *capacity = ix->capacity;
-  if (longest_walk) *longest_walk = c[2] ? (uint32_t)c[2] : 1u;   // a walk visits at least one bucket
+  if (longest_walk) *longest_walk = c[2] ? (uint32_t)c[2] : 1u;   // a walk visits at least one sector
   return AIBX_OK;
 }
 

@@ -611,7 +611,7 @@ def test_churn_fills_the_table_with_removed_entries_and_rehash_clears_them():
     again.  Live entries stay few, but never-used entries run out, so a probe for an absent key
     has to walk further and further; stats2 shows it (removed count, longest insert walk), the
     walk stays bounded, results stay those of the oracle, and a rehash to the same size brings
-    the probes back to one bucket."""
+    the probes back to one sector."""
     rng = np.random.default_rng(64)
     g, o = aibx.Index(64, 4), oracle.Index(64, 4)
     keep = rng.integers(1, 1 << 62, 10).astype(np.uint64)            # entries that stay
