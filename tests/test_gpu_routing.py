@@ -214,11 +214,13 @@ def test_match_hand_example():
     assert host(bp).tolist() == [aibx.NO_POD] and host(bs).tolist() == [-(1 << 63)]
 
 
+@pytest.mark.parametrize("wide", [False, True])
 @pytest.mark.parametrize("R", [1, 3, 40, 200, 700, 1500, 5000])
-def test_match_group_shapes_and_holes(R):
-    """Every warps-per-request choice (R picks it), requests of 0..600 blocks, random holes."""
-    rng = np.random.default_rng(R)
-    P = int(rng.integers(1, 65))
+def test_match_group_shapes_and_holes(R, wide):
+    """Every warps-per-request choice (R picks it) on both entry widths of the index (up to 32
+    pods / more), requests of 0..600 blocks, random holes."""
+    rng = np.random.default_rng(R + 100 * wide)
+    P = int(rng.integers(33, 65)) if wide else int(rng.integers(1, 33))
     lens = rng.integers(0, 600 if R < 100 else 80, R)
     lens[rng.random(R) < 0.1] = 0
     bo = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
