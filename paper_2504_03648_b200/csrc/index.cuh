@@ -536,6 +536,7 @@ struct PrefixFold {
 // block and records them in ml[pod] (each pod at most once over the whole request).  The pods
 // still there at the first total miss, or at the end of the request, are NOT recorded here:
 // they all get the same value (any_len, or the request's length) from fold_finish, in parallel.
+// `ml` must be all zeros when the request's first chunk is folded.
 __device__ __forceinline__ void fold_chunk(PrefixFold& st, int lane, unsigned int m, uint64_t mask,
                                            uint32_t id, uint64_t all, unsigned int* ml,
                                            uint32_t* block_ids_at) {
@@ -561,6 +562,10 @@ __device__ __forceinline__ void fold_chunk(PrefixFold& st, int lane, unsigned in
   const uint64_t before = lane == 0 ? st.alive : prev;
   uint64_t drops = valid ? (before & ~pref) : 0ULL;
   if ((unsigned int)lane == f) drops = 0;
+  // The pods that lack the request's very first block - in a large fleet most of them - would
+  // all be recorded by this one lane, one after the other; their length is 0, which is what the
+  // caller's scratch starts as.
+  if (st.pos == 0u && lane == 0) drops = 0;
   while (drops) {
     const int q = __ffsll((long long)drops) - 1;
     drops &= drops - 1;
@@ -638,6 +643,9 @@ match_prefix_warp_kernel(IndexView ix, const uint64_t* __restrict__ hashes,
   const int64_t off = blk_off[r];
   const unsigned int n_r = (unsigned int)(blk_off[r + 1] - off);
   PrefixFold st = {all, 0u, false};
+  s_ml[warp][lane] = 0u;
+  s_ml[warp][lane + 32] = 0u;
+  __syncwarp();
   // the keys of the next chunk are requested before this chunk is probed: if the request goes
   // on, they are there by then (one memory round trip less per further chunk)
   uint64_t key = (unsigned int)lane < n_r ? __ldg(hashes + off + lane) : 0ULL;

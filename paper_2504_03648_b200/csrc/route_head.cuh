@@ -244,6 +244,9 @@ route_head_kernel(IndexView ix, const int32_t* __restrict__ tokens,
   const int P = ix.num_pods;
   const uint64_t all = pod_all(P);
   PrefixFold st = {all, 0u, false};                    // see index.cuh
+  sh.match_len[qi][lane] = 0u;                         // fold_chunk wants its scratch zeroed
+  sh.match_len[qi][lane + 32] = 0u;
+  __syncwarp();
   unsigned int idle = 0;
   unsigned int written = 0;                            // keys of this request written to `hashes`
   uint64_t last_key = root_seed;                       // the last of them: the seed to resume from
