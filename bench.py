@@ -508,6 +508,8 @@ def run_gpu(args):
             "match_requests_per_s": cfg3["match_requests_per_s"], "match_us": cfg3["match_us"],
             "match_requests_per_s_back_to_back": cfg3["match_requests_per_s_back_to_back"],
             "match_us_back_to_back": cfg3["match_us_back_to_back"],
+            "match_us_in_a_graph": cfg3.get("match_us_in_a_graph"),
+            "match_requests_per_s_in_a_graph": cfg3.get("match_requests_per_s_in_a_graph"),
             "hash_us": cfg3["hash_us"], "route_head_us": cfg3["route_head_us"],
             "decisions_per_s_via_route_head": round(cfg3["R"] / (cfg3["route_head_us"] * 1e-6), 0),
             "match_algorithmic_GBps": cfg3["match_algorithmic_GBps"]},
