@@ -169,6 +169,7 @@ extern "C" {
 int32_t aibx_hash_blocks(const int32_t* d_tokens, const int64_t* d_tok_off,
                          const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
                          uint64_t root_seed, uint64_t* d_hashes, void* stream) {
+  AIBX_CALL_RANGE();
   if (R < 0 || block_tokens <= 0 || block_tokens % 8 != 0 || block_tokens > 1024)
     return AIBX_ERR_INVALID;
   if (R == 0) return AIBX_OK;
@@ -179,6 +180,7 @@ int32_t aibx_hash_blocks(const int32_t* d_tokens, const int64_t* d_tok_off,
 }
 
 int32_t aibx_index_create(aibx_index_t** out, uint64_t capacity_slots, int32_t num_pods) {
+  AIBX_CALL_RANGE();
   if (!out) return AIBX_ERR_INVALID;
   *out = nullptr;
   if (num_pods < 1 || num_pods > AIBX_MAX_PODS) return AIBX_ERR_INVALID;
@@ -209,6 +211,7 @@ int32_t aibx_index_create(aibx_index_t** out, uint64_t capacity_slots, int32_t n
 }
 
 int32_t aibx_index_destroy(aibx_index_t* ix) {
+  AIBX_CALL_RANGE();
   if (!ix) return AIBX_ERR_INVALID;
   cudaDeviceSynchronize();
   if (ix->migrating) free_view(ix->pending);
@@ -220,6 +223,7 @@ int32_t aibx_index_destroy(aibx_index_t* ix) {
 }
 
 int32_t aibx_index_clear(aibx_index_t* ix, void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || ix->migrating) return AIBX_ERR_INVALID;
   index_clear_kernel<<<sm_count() * 8, 256, 0, as_stream(stream)>>>(ix->view);
   return launch_status();
@@ -227,6 +231,7 @@ int32_t aibx_index_clear(aibx_index_t* ix, void* stream) {
 
 int32_t aibx_index_insert(aibx_index_t* ix, const uint64_t* d_keys, const uint64_t* d_pod_masks,
                           const uint32_t* d_block_ids, int64_t n, void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || n < 0 || ix->migrating) return AIBX_ERR_INVALID;
   if (n == 0) return AIBX_OK;
   if (!d_keys || !d_pod_masks || !d_block_ids) return AIBX_ERR_INVALID;
@@ -238,6 +243,7 @@ int32_t aibx_index_insert(aibx_index_t* ix, const uint64_t* d_keys, const uint64
 
 int32_t aibx_index_evict(aibx_index_t* ix, const uint64_t* d_keys, const uint64_t* d_pod_masks,
                          uint32_t* d_freed_block_ids, int64_t n, void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || n < 0 || ix->migrating) return AIBX_ERR_INVALID;
   if (n == 0) return AIBX_OK;
   if (!d_keys || !d_pod_masks) return AIBX_ERR_INVALID;
@@ -263,6 +269,7 @@ int32_t aibx_index_evict(aibx_index_t* ix, const uint64_t* d_keys, const uint64_
 
 int32_t aibx_index_lookup(const aibx_index_t* ix, const uint64_t* d_keys, uint64_t* d_masks,
                           uint32_t* d_block_ids, int64_t n, void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || n < 0) return AIBX_ERR_INVALID;
   if (n == 0) return AIBX_OK;
   if (!d_keys) return AIBX_ERR_INVALID;
@@ -273,6 +280,7 @@ int32_t aibx_index_lookup(const aibx_index_t* ix, const uint64_t* d_keys, uint64
 
 int32_t aibx_index_stats2(const aibx_index_t* ix, uint64_t* live, uint64_t* removed,
                           uint64_t* capacity, uint32_t* longest_walk, void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix) return AIBX_ERR_INVALID;
   unsigned long long c[3] = {0, 0, 0};
   if (cudaMemcpyAsync(c, ix->view.counters, sizeof(c), cudaMemcpyDeviceToHost,
@@ -290,11 +298,13 @@ int32_t aibx_index_stats2(const aibx_index_t* ix, uint64_t* live, uint64_t* remo
 
 int32_t aibx_index_stats(const aibx_index_t* ix, uint64_t* live, uint64_t* capacity,
                          void* stream) {
+  AIBX_CALL_RANGE();
   return aibx_index_stats2(ix, live, nullptr, capacity, nullptr, stream);
 }
 
 int32_t aibx_index_touch(aibx_index_t* ix, const uint64_t* d_keys, int64_t n, uint32_t epoch,
                          void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || n < 0 || epoch == 0 || epoch >= (1u << 30) || ix->migrating) return AIBX_ERR_INVALID;
   if (n == 0) return AIBX_OK;
   if (!d_keys) return AIBX_ERR_INVALID;
@@ -304,6 +314,7 @@ int32_t aibx_index_touch(aibx_index_t* ix, const uint64_t* d_keys, int64_t n, ui
 
 int32_t aibx_index_pick_victims(aibx_index_t* ix, uint64_t k, uint64_t* d_keys,
                                 uint32_t* d_priorities, uint64_t* d_count, void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || !d_count) return AIBX_ERR_INVALID;
   cudaStream_t st = as_stream(stream);
   if (!ix->victim_scratch) {
@@ -334,6 +345,7 @@ int32_t aibx_index_pick_victims(aibx_index_t* ix, uint64_t k, uint64_t* d_keys,
 int32_t aibx_index_export(const aibx_index_t* ix, uint64_t* d_keys, uint64_t* d_masks,
                           uint32_t* d_block_ids, uint64_t max_entries, uint64_t* d_count,
                           void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || !d_count) return AIBX_ERR_INVALID;
   cudaStream_t st = as_stream(stream);
   if (cudaMemsetAsync(d_count, 0, sizeof(uint64_t), st) != cudaSuccess) return AIBX_ERR_CUDA;
@@ -344,6 +356,7 @@ int32_t aibx_index_export(const aibx_index_t* ix, uint64_t* d_keys, uint64_t* d_
 }
 
 int32_t aibx_index_rehash(aibx_index_t* ix, uint64_t new_capacity) {
+  AIBX_CALL_RANGE();
   if (!ix || ix->migrating) return AIBX_ERR_INVALID;
   if (!capacity_ok(new_capacity)) return AIBX_ERR_INVALID;
   if (cudaDeviceSynchronize() != cudaSuccess) return AIBX_ERR_CUDA;
@@ -369,6 +382,7 @@ int32_t aibx_index_rehash(aibx_index_t* ix, uint64_t new_capacity) {
 }
 
 int32_t aibx_index_rehash_begin(aibx_index_t* ix, uint64_t new_capacity, void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || ix->migrating) return AIBX_ERR_INVALID;
   if (!capacity_ok(new_capacity)) return AIBX_ERR_INVALID;
   cudaStream_t st = as_stream(stream);
@@ -401,6 +415,7 @@ int32_t aibx_index_rehash_begin(aibx_index_t* ix, uint64_t new_capacity, void* s
 }
 
 int32_t aibx_index_rehash_finish(aibx_index_t* ix) {
+  AIBX_CALL_RANGE();
   if (!ix || !ix->migrating) return AIBX_ERR_INVALID;
   if (cudaEventSynchronize(ix->moved) != cudaSuccess) return AIBX_ERR_CUDA;
   const IndexView old = ix->view;
@@ -424,6 +439,7 @@ int32_t launch_match(const aibx_index_t* ix, const uint64_t* d_hashes, const int
 int32_t aibx_match_prefix(const aibx_index_t* ix, const uint64_t* d_hashes,
                           const int64_t* d_blk_off, int32_t R, uint32_t* d_match_len,
                           uint32_t* d_any_len, uint32_t* d_block_ids, void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || R < 0) return AIBX_ERR_INVALID;
   if (R == 0) return AIBX_OK;
   if (!d_hashes || !d_blk_off || !d_match_len) return AIBX_ERR_INVALID;
@@ -436,6 +452,7 @@ int32_t aibx_match_prefix_touch(aibx_index_t* ix, const uint64_t* d_hashes,
                                 const int64_t* d_blk_off, int32_t R, uint32_t epoch,
                                 uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
                                 void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || R < 0 || epoch == 0 || epoch >= (1u << 30) || ix->migrating) return AIBX_ERR_INVALID;
   if (R == 0) return AIBX_OK;
   if (!d_hashes || !d_blk_off || !d_match_len) return AIBX_ERR_INVALID;
@@ -485,6 +502,7 @@ int32_t aibx_route_batch(const aibx_index_t* ix, const int32_t* d_tokens, const 
                          const aibx_route_params_t* params, uint64_t* d_hashes,
                          uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
                          int32_t* d_best_pod, int64_t* d_best_score, void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || R < 0 || block_tokens <= 0 || block_tokens % 8 != 0 || block_tokens > 1024)
     return AIBX_ERR_INVALID;
   if (R == 0) return AIBX_OK;
@@ -563,6 +581,7 @@ int32_t aibx_route_head(const aibx_index_t* ix, const int32_t* d_tokens, const i
                         uint32_t* d_match_len, uint32_t* d_any_len, uint32_t* d_block_ids,
                         int32_t* d_best_pod, int64_t* d_best_score, uint32_t* d_hashed,
                         uint64_t* d_next_seed, void* stream) {
+  AIBX_CALL_RANGE();
   return route_head_impl(ix, d_tokens, d_tok_off, d_blk_off, R, block_tokens, root_seed, d_pod_load,
                          ready_mask, params, d_hashes, d_match_len, d_any_len, d_block_ids,
                          d_best_pod, d_best_score, d_hashed, d_next_seed, stream, 0u);
@@ -575,6 +594,7 @@ int32_t aibx_route_head_touch(aibx_index_t* ix, const int32_t* d_tokens, const i
                               uint64_t* d_hashes, uint32_t* d_match_len, uint32_t* d_any_len,
                               uint32_t* d_block_ids, int32_t* d_best_pod, int64_t* d_best_score,
                               uint32_t* d_hashed, uint64_t* d_next_seed, void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || epoch == 0 || epoch >= (1u << 30) || ix->migrating) return AIBX_ERR_INVALID;
   return route_head_impl(ix, d_tokens, d_tok_off, d_blk_off, R, block_tokens, root_seed, d_pod_load,
                          ready_mask, params, d_hashes, d_match_len, d_any_len, d_block_ids,
@@ -594,6 +614,7 @@ int32_t aibx_route_head_collect(aibx_index_t* ix, const int32_t* d_tokens, const
                                 uint32_t* d_hashed, uint64_t* d_next_seed, uint32_t num_blocks,
                                 void* d_scratch, uint32_t* d_unique_ids, uint32_t* d_count,
                                 void* stream) {
+  AIBX_CALL_RANGE();
   if (!ix || epoch >= (1u << 30) || (epoch && ix->migrating)) return AIBX_ERR_INVALID;
   if (!d_count || !d_scratch || (reinterpret_cast<uintptr_t>(d_scratch) & 3)) return AIBX_ERR_INVALID;
   if (R > 0 && (!d_block_ids || !d_unique_ids)) return AIBX_ERR_INVALID;
@@ -640,6 +661,7 @@ int32_t aibx_hash_blocks_resume(const int32_t* d_tokens, const int64_t* d_tok_of
                                 const int64_t* d_blk_off, int32_t R, int32_t block_tokens,
                                 const uint32_t* d_hashed, const uint64_t* d_next_seed,
                                 uint64_t* d_hashes, void* stream) {
+  AIBX_CALL_RANGE();
   if (R < 0 || block_tokens <= 0 || block_tokens % 8 != 0 || block_tokens > 1024)
     return AIBX_ERR_INVALID;
   if (R == 0) return AIBX_OK;
@@ -654,6 +676,7 @@ int32_t aibx_route_assign(const uint32_t* d_match_len, const int64_t* d_blk_off,
                           int32_t num_pods, int32_t* d_pod_load, uint64_t ready_mask,
                           const aibx_route_params_t* params, int32_t load_increment,
                           int32_t* d_best_pod, int64_t* d_best_score, void* stream) {
+  AIBX_CALL_RANGE();
   if (R < 0 || num_pods < 1 || num_pods > AIBX_MAX_PODS) return AIBX_ERR_INVALID;
   if (R == 0) return AIBX_OK;
   if (!d_match_len || !d_blk_off || !d_pod_load || !d_best_pod || !d_best_score)
@@ -670,6 +693,7 @@ int32_t aibx_route_score(const uint32_t* d_match_len, const int64_t* d_blk_off, 
                          int32_t num_pods, const int32_t* d_pod_load, uint64_t ready_mask,
                          const aibx_route_params_t* params, int32_t* d_best_pod,
                          int64_t* d_best_score, int64_t* d_scores, void* stream) {
+  AIBX_CALL_RANGE();
   if (R < 0 || num_pods < 1 || num_pods > AIBX_MAX_PODS) return AIBX_ERR_INVALID;
   if (R == 0) return AIBX_OK;
   if (!d_match_len || !d_blk_off || !d_pod_load || !d_best_pod || !d_best_score)
@@ -686,6 +710,7 @@ int32_t aibx_route_policy(int32_t policy, const uint32_t* d_match_len, const int
                           int32_t R, int32_t num_pods, const aibx_pod_metrics_t* metrics,
                           const uint64_t* d_draws, uint64_t ready_mask, int32_t threshold_pct,
                           int32_t* d_best_pod, void* stream) {
+  AIBX_CALL_RANGE();
   if (R < 0 || num_pods < 1 || num_pods > AIBX_MAX_PODS || policy < AIBX_POLICY_RANDOM ||
       policy > AIBX_POLICY_PREFIX_CACHE_AWARE)
     return AIBX_ERR_INVALID;
@@ -724,6 +749,7 @@ uint64_t aibx_collect_scratch_bytes(uint32_t num_blocks) {
 int32_t aibx_collect_blocks(const uint32_t* d_block_ids, int64_t n, uint32_t num_blocks,
                             void* d_scratch, uint32_t* d_unique_ids, uint32_t* d_count,
                             void* stream) {
+  AIBX_CALL_RANGE();
   if (n < 0 || !d_count) return AIBX_ERR_INVALID;
   if (n > 0 && (!d_block_ids || !d_unique_ids)) return AIBX_ERR_INVALID;
   if (num_blocks > 0 && !d_scratch) return AIBX_ERR_INVALID;
@@ -749,6 +775,7 @@ int32_t aibx_collect_blocks(const uint32_t* d_block_ids, int64_t n, uint32_t num
 
 int32_t aibx_collect_blocks_static(const uint32_t* d_block_ids, int64_t n, uint32_t num_blocks,
                                    uint32_t* d_unique_ids, uint32_t* d_count, void* stream) {
+  AIBX_CALL_RANGE();
   if (n < 0 || !d_count) return AIBX_ERR_INVALID;
   if (n > 0 && (!d_block_ids || !d_unique_ids)) return AIBX_ERR_INVALID;
   if (num_blocks > kStaticCollectMaxBlocks) return AIBX_ERR_UNSUPPORTED;
@@ -771,18 +798,21 @@ uint32_t aibx_collect_static_max_blocks(void) { return kStaticCollectMaxBlocks; 
 
 int32_t aibx_kv_gather(const void* d_pool, const aibx_kv_layout_t* layout,
                        const uint32_t* d_block_ids, int64_t n, void* d_buf, void* stream) {
+  AIBX_CALL_RANGE();
   return launch_kv_copy(d_pool, layout, d_block_ids, n, d_buf, 0, as_stream(stream));
 }
 
 int32_t aibx_kv_scatter(void* d_pool, const aibx_kv_layout_t* layout,
                         const uint32_t* d_block_ids, int64_t n, const void* d_buf,
                         void* stream) {
+  AIBX_CALL_RANGE();
   return launch_kv_copy(d_pool, layout, d_block_ids, n, d_buf, 1, as_stream(stream));
 }
 
 int32_t aibx_kv_gather_to_host(const void* d_pool, const aibx_kv_layout_t* layout,
                                const uint32_t* d_block_ids, int64_t n, void* d_staging,
                                void* h_buf, void* stream) {
+  AIBX_CALL_RANGE();
   if (n > 0 && !h_buf) return AIBX_ERR_INVALID;
   const int32_t rc = launch_kv_copy(d_pool, layout, d_block_ids, n, d_staging, 0, as_stream(stream));
   if (rc != AIBX_OK || n == 0) return rc;
@@ -797,6 +827,7 @@ int32_t aibx_kv_gather_to_host(const void* d_pool, const aibx_kv_layout_t* layou
 int32_t aibx_kv_scatter_from_host(void* d_pool, const aibx_kv_layout_t* layout,
                                   const uint32_t* d_block_ids, int64_t n, void* d_staging,
                                   const void* h_buf, void* stream) {
+  AIBX_CALL_RANGE();
   if (!layout || n < 0) return AIBX_ERR_INVALID;
   if (n == 0) return AIBX_OK;
   if (!h_buf || !d_staging) return AIBX_ERR_INVALID;
@@ -814,6 +845,7 @@ int32_t aibx_kv_scatter_from_host(void* d_pool, const aibx_kv_layout_t* layout,
 int32_t aibx_kv_gather_counted(const void* d_pool, const aibx_kv_layout_t* layout,
                                const uint32_t* d_block_ids, int64_t n_max, const uint32_t* d_count,
                                void* d_buf, void* stream) {
+  AIBX_CALL_RANGE();
   if (!d_count) return AIBX_ERR_INVALID;
   return launch_kv_copy(d_pool, layout, d_block_ids, n_max, d_buf, 0, as_stream(stream), d_count);
 }
@@ -821,6 +853,7 @@ int32_t aibx_kv_gather_counted(const void* d_pool, const aibx_kv_layout_t* layou
 int32_t aibx_kv_scatter_counted(void* d_pool, const aibx_kv_layout_t* layout,
                                 const uint32_t* d_block_ids, int64_t n_max,
                                 const uint32_t* d_count, const void* d_buf, void* stream) {
+  AIBX_CALL_RANGE();
   if (!d_count) return AIBX_ERR_INVALID;
   return launch_kv_copy(d_pool, layout, d_block_ids, n_max, d_buf, 1, as_stream(stream), d_count);
 }
@@ -828,6 +861,7 @@ int32_t aibx_kv_scatter_counted(void* d_pool, const aibx_kv_layout_t* layout,
 int32_t aibx_kv_gather_inner(const void* d_pool, const aibx_kv_layout_t* layout, int32_t pool_inner,
                              int32_t buf_inner, const uint32_t* d_block_ids, int64_t n,
                              void* d_buf, void* stream) {
+  AIBX_CALL_RANGE();
   return launch_kv_permute(d_pool, layout, pool_inner, buf_inner, d_block_ids, n, d_buf, 0,
                            as_stream(stream));
 }
@@ -835,6 +869,7 @@ int32_t aibx_kv_gather_inner(const void* d_pool, const aibx_kv_layout_t* layout,
 int32_t aibx_kv_scatter_inner(void* d_pool, const aibx_kv_layout_t* layout, int32_t pool_inner,
                               int32_t buf_inner, const uint32_t* d_block_ids, int64_t n,
                               const void* d_buf, void* stream) {
+  AIBX_CALL_RANGE();
   return launch_kv_permute(d_pool, layout, pool_inner, buf_inner, d_block_ids, n, d_buf, 1,
                            as_stream(stream));
 }
@@ -889,12 +924,14 @@ int32_t aibx_kv_set_store_lag(int32_t lag) {
 }
 
 int32_t aibx_selftest_bounded_wait(uint32_t spins, void* stream) {
+  AIBX_CALL_RANGE();
   if (spins == 0 || spins > (1u << 20)) return AIBX_ERR_INVALID;
   bounded_wait_probe_kernel<<<1, 32, 0, as_stream(stream)>>>(spins);
   return launch_status();
 }
 
 int32_t aibx_status_fetch(void* stream, int32_t* status, int64_t* detail) {
+  AIBX_CALL_RANGE();
   StatusRecord* dev = status_ptr();
   if (!dev) return AIBX_ERR_CUDA;
   cudaStream_t st = as_stream(stream);
