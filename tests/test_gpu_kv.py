@@ -457,3 +457,61 @@ def test_a_wait_that_runs_out_becomes_a_status_not_a_hang():
     check_gather_scatter(kv, W.distinct_ids(0, 256, 64), W.distinct_ids(100, 256, 64), (0, 32768, 3, 1, 1))
     with pytest.raises(aibx.AibxError):
         aibx.selftest_bounded_wait(0)
+
+
+def test_calls_from_several_host_threads_while_the_launch_shape_changes():
+    """Two host threads gather and scatter on their own streams and pools while a third keeps
+    switching the process-wide launch shape: every call reads one whole setting, so every result
+    is the oracle's whatever shape each launch happened to get."""
+    import threading
+
+    kv = W.KVSpec("mt", 41, 1, 4, 2, 16, 64, 2, 200)                  # 8 KiB tiles, layer-major
+    lay_g, lay_o = kv_layout_gpu(kv), kv_layout_oracle(kv)
+    pool_h = W.host_pool(kv)
+    stop = threading.Event()
+    errors = []
+
+    def switcher():
+        shapes = [(0, 32768, 3, 1), (0, 4096, 12, 2), (1, 16384, 2, 1), (0, 16384, 6, 1)]
+        i = 0
+        while not stop.is_set():
+            aibx.kv_set_tuning(*shapes[i % len(shapes)])
+            aibx.kv_set_store_lag(1 + i % 3)
+            i += 1
+
+    def worker(seed):
+        try:
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                pool_d = dev(pool_h)
+                want_pool = pool_h.copy()
+                for it in range(12):
+                    ids = W.distinct_ids(seed * 100 + it, kv.num_blocks, 50)
+                    buf = torch.zeros(50 * kv.block_bytes, dtype=torch.uint8, device="cuda")
+                    aibx.kv_gather(pool_d, lay_g, dev(ids), 50, buf)
+                    want = np.zeros(50 * kv.block_bytes, dtype=np.uint8)
+                    oracle.kv_gather(want_pool, lay_o, ids, want)
+                    stream.synchronize()
+                    if not np.array_equal(host(buf), want):
+                        errors.append(("gather", seed, it))
+                    dst = W.distinct_ids(seed * 100 + it + 50, kv.num_blocks, 50)
+                    aibx.kv_scatter(pool_d, lay_g, dev(dst), 50, buf)
+                    oracle.kv_scatter(want_pool, lay_o, dst, want)
+                stream.synchronize()
+                if not np.array_equal(host(pool_d), want_pool):
+                    errors.append(("pool", seed))
+        except Exception as e:                                        # pragma: no cover
+            errors.append(("exception", seed, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(s,)) for s in (1, 2)]
+    sw = threading.Thread(target=switcher)
+    sw.start()
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    stop.set()
+    sw.join()
+    torch.cuda.synchronize()
+    assert errors == []
+    assert aibx.status_fetch() == (0, 0)
