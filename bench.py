@@ -146,7 +146,6 @@ class GpuJob:
         blk_off = offsets(w.tok_off)
         self.nb = int(blk_off[-1])
         self.d_blk_off = dev(blk_off)
-        self.d_hashes = torch.empty(self.nb, dtype=torch.uint64, device="cuda")
 
         # index content: the prompts' own chains (hashed on the GPU) plus filler entries
         src_off = offsets(w.src_tok_off)
@@ -165,20 +164,28 @@ class GpuJob:
         self.d_all_ones = dev(np.full(self.nb, 0xFFFFFFFFFFFFFFFF, dtype=np.uint64))
         self.d_freed = torch.empty(self.nb, dtype=torch.uint32, device="cuda")
 
-        # routing outputs
+        # routing outputs: two sets, used by alternate steps, so that the routing of the next
+        # batch can run while the copies of this one still read this one's block list
         R, P = self.R, self.P
-        self.d_match_len = torch.empty(R * P, dtype=torch.uint32, device="cuda")
-        self.d_any_len = torch.empty(R, dtype=torch.uint32, device="cuda")
-        self.d_block_ids = torch.empty(self.nb, dtype=torch.uint32, device="cuda")
-        self.d_best_pod = torch.empty(R, dtype=torch.int32, device="cuda")
-        self.d_best_score = torch.empty(R, dtype=torch.int64, device="cuda")
-        self.d_hashed = torch.empty(R, dtype=torch.uint32, device="cuda")
-        self.d_next_seed = torch.empty(R, dtype=torch.uint64, device="cuda")
         self.d_pod_load = dev(w.pod_load)
-        self.d_scratch = torch.empty(aibx.route_collect_scratch_bytes(kv.num_blocks) // 4 + 1,
-                                     dtype=torch.int32, device="cuda")
-        self.d_unique = torch.empty(self.nb, dtype=torch.uint32, device="cuda")
-        self.d_count = torch.empty(1, dtype=torch.uint32, device="cuda")
+
+        def routing_outputs():
+            return dict(
+                d_hashes=torch.empty(self.nb, dtype=torch.uint64, device="cuda"),
+                d_match_len=torch.empty(R * P, dtype=torch.uint32, device="cuda"),
+                d_any_len=torch.empty(R, dtype=torch.uint32, device="cuda"),
+                d_block_ids=torch.empty(self.nb, dtype=torch.uint32, device="cuda"),
+                d_best_pod=torch.empty(R, dtype=torch.int32, device="cuda"),
+                d_best_score=torch.empty(R, dtype=torch.int64, device="cuda"),
+                d_hashed=torch.empty(R, dtype=torch.uint32, device="cuda"),
+                d_next_seed=torch.empty(R, dtype=torch.uint64, device="cuda"),
+                d_scratch=torch.empty(aibx.route_collect_scratch_bytes(kv.num_blocks) // 4 + 1,
+                                      dtype=torch.int32, device="cuda"),
+                d_unique=torch.empty(self.nb, dtype=torch.uint32, device="cuda"),
+                d_count=torch.empty(1, dtype=torch.uint32, device="cuda"))
+
+        self._slots = [routing_outputs(), routing_outputs()]
+        self._use(0)
         self.h_count = torch.empty(1, dtype=torch.uint32).pin_memory()
         self.h_best_pod = torch.empty(R, dtype=torch.int32).pin_memory()
         self.h_any_len = torch.empty(R, dtype=torch.uint32).pin_memory()
@@ -196,6 +203,12 @@ class GpuJob:
         self.copy_events = []
         st_code = aibx.status_fetch()
         assert st_code == (0, 0), st_code
+
+    def _use(self, slot: int) -> None:
+        """Make the routing outputs of one of the two sets the current ones (self.d_hashes ...)."""
+        self._slot = slot
+        for name, t in self._slots[slot].items():
+            setattr(self, name, t)
 
     def release(self) -> None:
         """Give the device memory back (the index through its own destroy call)."""
@@ -243,16 +256,29 @@ class GpuJob:
         """One pass of the whole path, enqueued without any host round trip: the number of
         matched blocks goes from the routing kernel to the copies on the device; the tail of
         the hash chains and the index publish/expire batch (both independent of the copies) run
-        beside them on a second stream."""
+        beside them on a second stream; and as soon as the index is back in its start state the
+        routing of the NEXT batch is enqueued on a third stream, beside this batch's copies
+        (its outputs go to the other of two sets of buffers).  Every batch still goes through
+        every stage in order; consecutive batches overlap as in any pipeline."""
         torch, aibx = self.torch, self.aibx
         main = torch.cuda.current_stream()
         if self.side is None:
             self.side = torch.cuda.Stream()
-            self.ev_routed = torch.cuda.Event()
+            self.route = torch.cuda.Stream()
+            self.ev_routed = [torch.cuda.Event(), torch.cuda.Event()]
+            self.ev_copied = [torch.cuda.Event(), torch.cuda.Event()]
             self.ev_index = torch.cuda.Event()
-        self.routing_async()
-        self.ev_routed.record(main)
-        self.side.wait_event(self.ev_routed)
+            self._routed_ahead = None
+        if self._routed_ahead is not None:
+            self._use(self._routed_ahead)                 # this batch was routed during the last step
+        slot = self._slot
+        if self._routed_ahead != slot:                    # first step: nothing was routed ahead
+            self.route.wait_stream(main)
+            with torch.cuda.stream(self.route):
+                self.routing_async()
+                self.ev_routed[slot].record(self.route)
+        main.wait_event(self.ev_routed[slot])
+        self.side.wait_event(self.ev_routed[slot])
         with torch.cuda.stream(self.side):
             self.hash_tail()
             self.publish_expire()
@@ -269,7 +295,19 @@ class GpuJob:
         if record_copy_events:
             e[2].record()
             self.copy_events.append(e)
-        main.wait_event(self.ev_index)                    # the next step matches the restored index
+        self.ev_copied[slot].record(main)
+        main.wait_event(self.ev_index)                    # the index is back in its start state
+        # the next batch's routing: needs the restored index and the other set of buffers, whose
+        # last reader was the previous step's scatter
+        nxt = 1 - slot
+        self.route.wait_event(self.ev_index)
+        self.route.wait_event(self.ev_copied[nxt])
+        self._use(nxt)
+        with torch.cuda.stream(self.route):
+            self.routing_async()
+            self.ev_routed[nxt].record(self.route)
+        self._routed_ahead = nxt
+        self._use(slot)                                   # results of the step just enqueued
 
     def step_e2e(self, pieces=32):
         """Same step with host buffers on both sides of every transfer: tokens come from pinned
@@ -489,7 +527,7 @@ def run_gpu(args):
         "config": {"workload": WORKLOAD, "blocks_moved_per_step": count,
                    "bytes_moved_per_step": step_bytes, "parallelism": "replicas only" if world > 1 else "1 gpu",
                    "l2": "inputs larger than L2: 6.5 GB of KV traffic per step evicts it between steps",
-                   "overlap": "hash chains past the first uncached block and index publish/expire on a second stream beside the copies; no host sync inside a step",
+                   "overlap": "hash chains past the first uncached block and index publish/expire on a second stream beside the copies; the next batch's routing on a third stream beside them once the index is restored (two sets of routing outputs); no host sync inside a step",
                    "kv_tuning": "bulk ring, loader + storer warp, 32 KiB x 3 stages, 1 CTA/SM",
                    "sibling_records": "kv_cfg4 (largest configuration), kv_cfg5, prefix_match_large_index, index_lookup_flat: measured at n_gpus = 1 only"},
         "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},

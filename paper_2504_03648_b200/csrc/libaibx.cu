@@ -56,7 +56,9 @@ void prefer_copy_carveout() {
       (const void*)hash_blocks_kernel<8>,      (const void*)index_insert_kernel,
       (const void*)index_evict_clear_kernel,   (const void*)index_evict_report_kernel,
       (const void*)index_evict_remove_kernel,  (const void*)index_touch_kernel,
-      (const void*)index_evict_coop_kernel,
+      (const void*)index_evict_coop_kernel,    (const void*)route_head_kernel<1>,
+      (const void*)route_head_kernel<2>,       (const void*)route_head_kernel<4>,
+      (const void*)route_head_kernel<8>,
   };
   for (const void* f : side_kernels)
     cudaFuncSetAttribute(f, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -540,6 +542,7 @@ int32_t route_head_impl(const aibx_index_t* ix, const int32_t* d_tokens, const i
   if (d_best_pod && !d_pod_load) return AIBX_ERR_INVALID;
   aibx_route_params_t prm = {4, 1, 50};
   if (params) prm = *params;
+  prefer_copy_carveout();      // the routing of the next batch may run beside this batch's copies
   cudaStream_t st = as_stream(stream);
   ScoreParams sp = {d_pod_load, ready_mask, prm.w_prefix, prm.w_load, prm.threshold_pct};
   const int spb = block_tokens / 8;
