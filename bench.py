@@ -5,7 +5,8 @@ One step = one pass of the whole path over one batch of the Llama-3-8B-shaped wo
 hash the 64 requests as far as matching needs, longest cached prefix against a 200k-entry index
 and route score (one kernel) -> set of matched blocks -> gather them from the 8 GiB paged pool
 into the transfer buffer -> scatter them back; beside the copies, on a second stream: the rest
-of the hash chains, then publish and expire one batch of new index entries.
+of the hash chains, then publish and expire one batch of new index entries; and on a third
+stream, once the index is back in its start state, the routing of the next batch.
 
 `value` is gather+scatter bytes (read + written) per second over the whole step, inputs
 resident in HBM.  `e2e` is the same with host buffers: tokens come from pinned host memory,
