@@ -515,3 +515,51 @@ def test_calls_from_several_host_threads_while_the_launch_shape_changes():
     torch.cuda.synchronize()
     assert errors == []
     assert aibx.status_fetch() == (0, 0)
+
+
+def test_plain_copy_random_shapes_all_layouts():
+    """Ninety random shapes (element size, head dim, heads, tokens, layers, pool size; tiles from
+    32 bytes to 200 KiB) on the three pool layouts and two launch shapes: gather with repeats,
+    skips and out-of-range ids, scatter to distinct ids, every byte against the oracle."""
+    done = 0
+    for seed in range(90):
+        rng = np.random.default_rng(7000 + seed)
+        layout = seed % 3
+        E = int(rng.choice([1, 2, 4]))
+        D = int(rng.choice([16, 32, 64, 128, 256]))
+        H = int(rng.integers(1, 9))
+        T = int(rng.integers(1, 65))
+        L = int(rng.integers(1, 6))
+        nb = int(rng.integers(3, 40))
+        kv = W.KVSpec("rnd", 300 + seed, layout, L, H, T, D, E, nb)
+        half = kv.tile_bytes // 2
+        if kv.pool_bytes > (64 << 20) or (layout == 2 and half % 16) or kv.tile_bytes % 16:
+            continue
+        n = int(rng.integers(1, 3 * nb))
+        ids_g = rng.integers(0, nb, n).astype(np.uint32)
+        if n > 4:
+            ids_g[int(rng.integers(0, n))] = NO_BLOCK
+            ids_g[int(rng.integers(0, n))] = nb + int(rng.integers(0, 5))
+        m = int(rng.integers(1, nb + 1))
+        ids_s = rng.permutation(nb)[:m].astype(np.uint32)
+        mode_args = (0, 32768, 3, 1, 1) if seed % 2 == 0 else (0, int(rng.choice([1024, 4096, 16384])),
+                                                              int(rng.integers(2, 9)), 1, 1)
+        aibx.kv_set_tuning(*mode_args[:4])
+        lay_g, lay_o = kv_layout_gpu(kv), kv_layout_oracle(kv)
+        pool_h = W.host_pool(kv)
+        pool_d = dev(pool_h)
+        buf_w, buf_d = guarded(n * kv.block_bytes, 0xEE)
+        aibx.kv_gather(pool_d, lay_g, dev(ids_g), n, buf_d)
+        want = np.full(n * kv.block_bytes, 0xEE, dtype=np.uint8)
+        rc, bad = oracle.kv_gather(pool_h, lay_o, ids_g, want)
+        assert np.array_equal(host(buf_d), want), (seed, "gather")
+        assert aibx.status_fetch() == ((aibx.ERR_RANGE, bad) if bad else (0, 0)), seed
+        assert guards_intact(buf_w, n * kv.block_bytes, 0xEE)
+        src = dev(W.pool_bytes(900 + seed, 0, (m * kv.block_bytes + 7) // 8 * 8)[: m * kv.block_bytes])
+        aibx.kv_scatter(pool_d, lay_g, dev(ids_s), m, src)
+        pool_want = pool_h.copy()
+        oracle.kv_scatter(pool_want, lay_o, ids_s, host(src).copy())
+        assert np.array_equal(host(pool_d), pool_want), (seed, "scatter")
+        assert aibx.status_fetch() == (0, 0)
+        done += 1
+    assert done >= 60
