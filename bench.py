@@ -755,6 +755,8 @@ def main():
     ap.add_argument("--case", default=None, choices=sorted(CASES),
                     help="run one small single-kernel case instead of the bench step")
     ap.add_argument("--log2cap", type=int, default=23)
+    ap.add_argument("--pods", type=int, default=32, help="match_large: pods of the index (up to 32: "
+                    "16-byte entries, beyond: 32-byte entries)")
     ap.add_argument("--ws-mib", type=int, default=0, help="random_reads: one working-set size")
     ap.add_argument("--read-bytes", type=int, default=0, choices=[0, 32, 64, 128],
                     help="random_reads: one read size")

@@ -155,7 +155,7 @@ def _random_read_ceiling(torch, ws_bytes, gran, flush, t_flush, n=1 << 24):
     return best
 
 
-def measure_match_large(log2cap, Rs=(262144,), steps=7, with_ceiling=True):
+def measure_match_large(log2cap, Rs=(262144,), steps=7, with_ceiling=True, P=32):
     """Prefix match at a size where a bandwidth roofline means something: an index of 2^log2cap
     slots (load 0.5, 32 pods), R requests of 64 blocks, every block resident, so all 64 lookups
     of a request are necessary.  Algorithmic bytes: 8 (key) + 32 (key, mask and id of one entry,
@@ -169,12 +169,12 @@ def measure_match_large(log2cap, Rs=(262144,), steps=7, with_ceiling=True):
     from paper_2504_03648_b200 import binding as aibx
     import workloads as W
 
-    P, nblk = 32, 64
+    nblk = 64
     ix, keys = _big_index(torch, aibx, W, log2cap, P, 11)
     flush = torch.empty(64 << 20, dtype=torch.int32, device="cuda")
     t_flush = statistics.median(_event_times(torch, lambda: flush.sum(), max(steps, 5), 3))
     peak, kind = measured_peak_hbm()
-    table_bytes = index_table_bytes(1 << log2cap)
+    table_bytes = index_table_bytes(1 << log2cap, P)
     ceiling = _random_read_ceiling(torch, table_bytes, 32, flush, t_flush) if with_ceiling else None
     out = []
     for R in Rs:
@@ -213,7 +213,7 @@ def measure_match_large(log2cap, Rs=(262144,), steps=7, with_ceiling=True):
 
 
 def case_match_large(args):
-    out = measure_match_large(args.log2cap, Rs=(4096, 32768, 262144), steps=args.steps)
+    out = measure_match_large(args.log2cap, Rs=(4096, 32768, 262144), steps=args.steps, P=args.pods)
     out["case"] = "match_large"
     print(json.dumps(out))
 
