@@ -61,12 +61,18 @@ def measured_peak_hbm():
 # small single-kernel cases (profiling targets and microbenchmarks; not the bench line)
 
 
-def _event_times(torch, fn, reps, warm):
+def _event_times(torch, fn, reps, warm, before=None):
+    """Event-timed calls of fn; `before` (an L2 eviction, say) runs ahead of every call on the
+    same stream, outside the timed pair of events."""
     for _ in range(warm):
+        if before:
+            before()
         fn()
     ts = []
     for _ in range(reps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if before:
+            before()
         a.record()
         fn()
         b.record()
@@ -132,7 +138,7 @@ def _big_index(torch, aibx, W, log2cap, P, seed):
     return ix, keys
 
 
-def _random_read_ceiling(torch, ws_bytes, gran, flush, t_flush, n=1 << 24):
+def _random_read_ceiling(torch, ws_bytes, gran, flush, n=1 << 24):
     """Measured ceiling for this access pattern: G reads/s of uniformly random, aligned reads of
     `gran` bytes over a working set of ws_bytes, L2 evicted before every launch (best of 1, 2
     and 4 independent reads per thread)."""
@@ -146,10 +152,9 @@ def _random_read_ceiling(torch, ws_bytes, gran, flush, t_flush, n=1 << 24):
         sink = torch.empty(n // (32 * per) + 1, dtype=torch.int64, device="cuda")
 
         def run():
-            flush.sum()
             synth.probe_random_reads(base, ws_bytes, gran, per, n, 17 + per, sink)
 
-        t = statistics.median(_event_times(torch, run, 7, 2)) - t_flush
+        t = statistics.median(_event_times(torch, run, 7, 2, before=flush.sum))
         best = max(best, n / (t * 1e-3) / 1e9)
     del base
     return best
@@ -160,7 +165,7 @@ def measure_match_large(log2cap, Rs=(262144,), steps=7, with_ceiling=True, P=32)
     slots (load 0.5, 32 pods), R requests of 64 blocks, every block resident, so all 64 lookups
     of a request are necessary.  Algorithmic bytes: 8 (key) + 32 (key, mask and id of one entry,
     rounded up to a sector) per lookup, 4*P + 4*64 + 4 out per request.  L2 is evicted by a
-    256 MiB read before every launch (its time subtracted).  Two denominators: the measured
+    256 MiB read before every launch (outside the timed events).  Two denominators: the measured
     stream bandwidth, and the measured rate of random 32-byte reads over a working set of the
     table's own size (one read per lookup is the least the method needs; on this GPU a read that
     misses L2 always moves a whole 128-byte line from DRAM, whatever it asked for)."""
@@ -172,10 +177,9 @@ def measure_match_large(log2cap, Rs=(262144,), steps=7, with_ceiling=True, P=32)
     nblk = 64
     ix, keys = _big_index(torch, aibx, W, log2cap, P, 11)
     flush = torch.empty(64 << 20, dtype=torch.int32, device="cuda")
-    t_flush = statistics.median(_event_times(torch, lambda: flush.sum(), max(steps, 5), 3))
     peak, kind = measured_peak_hbm()
     table_bytes = index_table_bytes(1 << log2cap, P)
-    ceiling = _random_read_ceiling(torch, table_bytes, 32, flush, t_flush) if with_ceiling else None
+    ceiling = _random_read_ceiling(torch, table_bytes, 32, flush) if with_ceiling else None
     out = []
     for R in Rs:
         st = W.Stream(12, R)
@@ -187,10 +191,10 @@ def measure_match_large(log2cap, Rs=(262144,), steps=7, with_ceiling=True, P=32)
         d_ids = torch.empty(R * nblk, dtype=torch.uint32, device="cuda")
 
         def run():
-            flush.sum()                         # a 256 MiB read evicts the table from L2
             ix.match_prefix(d_h, d_bo, d_ml, d_al, d_ids)
 
-        ms = statistics.median(_event_times(torch, run, max(steps, 5), 3)) - t_flush
+        # a 256 MiB read evicts the table from L2 before every timed call
+        ms = statistics.median(_event_times(torch, run, max(steps, 5), 3, before=flush.sum))
         assert int(d_al.cpu().numpy().min()) == nblk
         nbytes = R * nblk * 40 + R * (4 * P + 4 * nblk + 4)
         gbs = nbytes / (ms * 1e-3) / 1e9
@@ -205,7 +209,7 @@ def measure_match_large(log2cap, Rs=(262144,), steps=7, with_ceiling=True, P=32)
     ix.destroy()
     res = {"index_slots": 1 << log2cap, "table_MiB": round(table_bytes / 2 ** 20, 1), "pods": P,
            "blocks_per_request": nblk,
-           "l2": "evicted before every launch (256 MiB read, its time subtracted)",
+           "l2": "evicted before every launch (256 MiB read, outside the timed events)",
            "peak": peak, "peak_kind": kind, "results": out, "status": status}
     if ceiling:
         res["random_32B_read_ceiling_Greads_per_s"] = round(ceiling, 2)
@@ -225,13 +229,12 @@ def case_random_reads(args):
     import torch
 
     flush = torch.empty(64 << 20, dtype=torch.int32, device="cuda")
-    t_flush = statistics.median(_event_times(torch, lambda: flush.sum(), 7, 3))
     peak, kind = measured_peak_hbm()
     rows = []
     sizes = (args.ws_mib,) if args.ws_mib else (11, 16, 43, 64, 128, 171, 256, 1024, 4096)
     for ws_mib in sizes:
         for gran in ((args.read_bytes,) if args.read_bytes else (32, 64, 128)):
-            g = _random_read_ceiling(torch, ws_mib << 20, gran, flush, t_flush)
+            g = _random_read_ceiling(torch, ws_mib << 20, gran, flush)
             rows.append({"working_set_MiB": ws_mib, "read_bytes": gran, "Greads_per_s": round(g, 2),
                          "GBps": round(g * gran, 1), "frac_of_stream": round(g * gran / peak, 4)})
     print(json.dumps({"case": "random_reads", "reads_per_launch": 1 << 24, "peak": peak,
@@ -521,7 +524,6 @@ def measure_lookup_flat(log2caps=(11, 19, 21, 23), reps=7, with_library=True):
     n = 1 << 24
     peak, kind = measured_peak_hbm()
     flush = torch.empty(64 << 20, dtype=torch.int32, device="cuda")
-    t_flush = statistics.median(_event_times(torch, lambda: flush.sum(), reps, 2))
     out = []
     for log2cap in log2caps:
         ix, keys = _big_index(torch, aibx, W, log2cap, 32, 20 + log2cap)
@@ -535,10 +537,9 @@ def measure_lookup_flat(log2caps=(11, 19, 21, 23), reps=7, with_library=True):
         d_i = torch.empty(n, dtype=torch.uint32, device="cuda")
 
         def cold():
-            flush.sum()
             ix.lookup(d_q, d_m, d_i)
 
-        t_cold = statistics.median(_event_times(torch, cold, reps, 2)) - t_flush
+        t_cold = statistics.median(_event_times(torch, cold, reps, 2, before=flush.sum))
         t_warm = statistics.median(_event_times(torch, lambda: ix.lookup(d_q, d_m, d_i), reps, 2))
         nbytes = n * (8 + 32 + 12)
         row = {"slots": 1 << log2cap, "table_MiB": round(index_table_bytes(1 << log2cap) / 2 ** 20, 2),
@@ -550,7 +551,7 @@ def measure_lookup_flat(log2caps=(11, 19, 21, 23), reps=7, with_library=True):
                "cold_frac": round(nbytes / (t_cold * 1e-3) / 1e9 / peak, 4),
                "warm_frac": round(nbytes / (t_warm * 1e-3) / 1e9 / peak, 4)}
         if log2cap >= 12:
-            ceiling = _random_read_ceiling(torch, index_table_bytes(1 << log2cap), 32, flush, t_flush)
+            ceiling = _random_read_ceiling(torch, index_table_bytes(1 << log2cap), 32, flush)
             row["random_32B_read_ceiling_Greads_per_s"] = round(ceiling, 2)
             row["cold_frac_of_random_read_ceiling"] = round(n / (t_cold * 1e-3) / 1e9 / ceiling, 4)
         if with_library:
@@ -789,7 +790,6 @@ def case_kv_sweep(args):
 
     out = []
     flush = torch.empty(64 << 20, dtype=torch.int32, device="cuda")
-    t_flush = statistics.median(_event_times(torch, lambda: flush.sum(), 15, 3))
     for name, kv in (("cfg2 shape (2 MiB blocks, block-major)", W.scaled(W.cfg2_kv(), num_blocks=4096)),
                      ("cfg4 shape (5 MiB blocks, layer-major)", W.scaled(W.cfg4_kv(), num_blocks=4096)),
                      ("cfg5 shape (896 KiB blocks, block-major)", W.scaled(W.cfg5_kv(), num_blocks=4096))):
@@ -804,15 +804,13 @@ def case_kv_sweep(args):
             ids = all_ids[:n].contiguous()
 
             def g():
-                flush.sum()
                 aibx.kv_gather(pool, lay, ids, n, buf)
 
             def sc():
-                flush.sum()
                 aibx.kv_scatter(pool, lay, ids, n, buf)
 
-            tg = statistics.median(_event_times(torch, g, 15, 3)) - t_flush
-            ts = statistics.median(_event_times(torch, sc, 15, 3)) - t_flush
+            tg = statistics.median(_event_times(torch, g, 15, 3, before=flush.sum))
+            ts = statistics.median(_event_times(torch, sc, 15, 3, before=flush.sum))
             nbytes = 2 * n * kv.block_bytes
             rows.append({"n": n, "MB_moved": round(nbytes / 1e6, 1),
                          "gather_us": round(tg * 1e3, 1), "scatter_us": round(ts * 1e3, 1),
